@@ -1,0 +1,435 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, invariants, brute force.
+
+Every check here compares the oracle with something other than itself, so that a dropped
+term, a wrong sign, a wrong bit order or a transposed index in the oracle fails a test.
+No GPU and no product code is involved.
+"""
+import numpy as np
+import pytest
+
+import datagen
+import oracle
+
+
+def bits_lsb_first(bits):
+    return sum(int(b) << i for i, b in enumerate(bits))
+
+
+# --- Fig. 4: pdep ---------------------------------------------------------------------
+def test_pdep_fig4_example(golden):
+    g = golden("pdep_fig4.txt")
+    mask = bits_lsb_first(g["mask"][0])
+    a = bits_lsb_first(g["a"][0])
+    dst = bits_lsb_first(g["dst"][0])
+    assert (mask, a, dst) == (0x4D, 0x0D, 0x49)
+    assert oracle.pdep32(a, mask) == dst
+
+
+def test_pdep_identities_and_bruteforce():
+    rng = np.random.default_rng(1)
+    for _ in range(300):
+        a, mask = (int(v) for v in rng.integers(0, 2**32, 2, dtype=np.uint64))
+        # independent construction: list the set positions, hand the source bits out in order
+        pos = [i for i in range(32) if (mask >> i) & 1]
+        want = sum(((a >> j) & 1) << p for j, p in enumerate(pos))
+        assert oracle.pdep32(a, mask) == want
+        assert oracle.pdep32(a, 0xFFFFFFFF) == a
+        assert oracle.pdep32(a, 0) == 0
+        assert oracle.pdep32(0xFFFFFFFF, mask) == mask
+        assert oracle.pdep32(a, mask) & ~mask == 0
+
+
+# --- Section II-C: the column example, Eq. 2 and the byte arithmetic ---------------------
+def test_column_example(golden):
+    g = golden("column_example_sec2c.txt")
+    values = np.array([int(v) for v in g["values"][0]], np.int8)
+    p = [int(v) for v in g["p"][0]]
+    n = [int(v) for v in g["n"][0]]
+    stored = [int(v) for v in g["stored_signs"][0]]
+    bitmap, signs, nnz = oracle.stream_pack(values)
+    assert bitmap[0] == int(g["bitmap_hex"][0][0], 16) == 0xDF
+    assert nnz == 7 == sum(p)
+    assert signs[0] == bits_lsb_first(stored) == 0x30
+    # recovering n from the stored bits is the deposit
+    assert oracle.pdep32(int(signs[0]), int(bitmap[0])) == bits_lsb_first(n) == 0x50
+    # Eq. 2 returns the column
+    assert [oracle.ternary_from_pn(pi, ni) for pi, ni in zip(p, n)] == list(values)
+    # byte arithmetic
+    P, T, W = oracle.avx2_bytes(p, n)
+    assert [f"{v:02X}" for v in P] == g["P_bytes"][0]
+    assert [f"{v:02X}" for v in T] == g["T_bytes"][0]
+    assert [f"{v:02X}" for v in W] == g["W_bytes"][0]
+    assert list(W.view(np.int8)) == list(values)
+    # the sign of row 6 is the sixth stored bit (index 5), not the seventh
+    assert stored[5] == 1 and n[6] == 1
+    for dec in ("bits", "pdep", "lut"):
+        out, end = oracle.stream_unpack(bitmap, signs, 8, dec)
+        assert list(out) == list(values) and end == 7
+
+
+def test_eq2_truth_table():
+    assert oracle.ternary_from_pn(0, 0) == 0
+    assert oracle.ternary_from_pn(1, 0) == 1
+    assert oracle.ternary_from_pn(1, 1) == -1
+
+
+# --- Section II-D: the lookup table ---------------------------------------------------------
+def test_lut_printed_entries(golden):
+    g = golden("lut_entries_sec2d.txt")
+    for key in ("B6", "66"):
+        row = g[key][0]
+        k = int(key, 16)
+        c, used = oracle.lut_entry(k >> 4, k & 0xF)
+        assert list(c) == [int(v) for v in row[:4]]
+        assert used == int(row[4])
+    assert int(g["entries"][0][0]) == 256
+
+
+def test_lut_is_a_four_bit_deposit():
+    live = set()
+    for m in range(16):
+        for s in range(16):
+            c, used = oracle.lut_entry(m, s)
+            n = oracle.pdep32(s, m)
+            want = [((m >> i) & 1) - 2 * ((n >> i) & 1) for i in range(4)]
+            assert list(c) == want
+            assert used == bin(m).count("1")
+            live.add((m, s & ((1 << used) - 1)))
+    # sum over m of 2^popcount(m) = 3^4 distinct (mask, consumed sign bits) pairs
+    assert len(live) == 81
+
+
+# --- Section II-A: sizes -------------------------------------------------------------------
+def test_8x8_example_bits(golden):
+    g = golden("layout_8x8_fig2.txt")
+    n, zeros = int(g["weights"][0][0]), int(g["zeros"][0][0])
+    rng = np.random.default_rng(2)
+    for _ in range(5):
+        sym = np.zeros(n, np.int8)
+        nz = rng.choice(n, n - zeros, replace=False)
+        sym[nz] = rng.choice([-1, 1], n - zeros)
+        bitmap, signs, nnz = oracle.stream_pack(sym)
+        assert bitmap.size * 32 == int(g["presence_bits"][0][0])
+        assert nnz == int(g["sign_bits"][0][0])
+        bpw = (bitmap.size * 32 + nnz) / n
+        assert round(bpw, 3) == float(g["bits_per_weight"][0][0])
+        assert round(zeros / n, 3) == float(g["z"][0][0])
+        for dec in ("bits", "pdep", "lut"):
+            out, end = oracle.stream_unpack(bitmap, signs, n, dec)
+            assert np.array_equal(out, sym) and end == nnz
+
+
+def exact_density_matrix(M, K, z_percent, seed):
+    n = M * K
+    zeros = int(round(z_percent / 100.0 * n))
+    rng = np.random.default_rng(seed)
+    flat = rng.choice([-1, 1], n).astype(np.int8)
+    flat[rng.choice(n, zeros, replace=False)] = 0
+    return flat.reshape(M, K), zeros
+
+
+def test_table1_rates(golden):
+    g = golden("table1_rows.txt")
+    M, K = 64, 6400                      # 409600 weights: 1/n is far below the table's rounding
+    for i, (model, row) in enumerate(g.items()):
+        zp, sym_b, bc_s, b2_s, red2, t5_s, red5 = (float(v) for v in row[0])
+        W, zeros = exact_density_matrix(M, K, zp, 10 + i)
+        pk = oracle.bitcos_pack(W)
+        z_hat = zeros / (M * K)
+        assert pk.nnz == M * K - zeros
+        assert pk.bits_per_weight() == pytest.approx(2.0 - z_hat, abs=1e-12)          # Eq. 1
+        assert abs(pk.bits_per_weight() - sym_b) <= 0.00051, model
+        scale_bits = 16 * M * (K // 128)
+        bitcos_total = (pk.bitmap.size * 32 + pk.nnz + scale_bits) / (M * K)
+        assert abs(bitcos_total - bc_s) <= 0.00051, model
+        t5_total = (oracle.trit5_pack(W).size * 32 + scale_bits) / (M * K)
+        b2_total = (oracle.bit2_pack(W).size * 32 + scale_bits) / (M * K)
+        assert t5_total == t5_s == 1.75 and b2_total == b2_s == 2.125
+        assert abs(b2_total / bitcos_total - red2) <= 0.0051, model
+        assert abs(t5_total / bitcos_total - red5) <= 0.0051, model
+
+
+def test_break_even_and_bytes_per_32_weights():
+    # five-trit break-even at z = 0.375; always below 2 bits
+    M, K = 32, 1280
+    W, zeros = exact_density_matrix(M, K, 37.5, 3)
+    pk = oracle.bitcos_pack(W)
+    assert pk.bits_per_weight() == 1.625 == oracle.trit5_pack(W).size * 32 / (M * K)
+    # bytes read per 32 weights with a 16-bit scale per 128: 4 + 4(1-z) + 0.5 = 8.5 - 4z; 6.9 at z = 0.4
+    W, zeros = exact_density_matrix(M, K, 40.0, 4)
+    pk = oracle.bitcos_pack(W)
+    per32 = (pk.bitmap.size * 4 + pk.nnz / 8 + 2 * M * (K // 128)) / (M * K / 32)
+    assert per32 == pytest.approx(6.9, abs=1e-9)
+
+
+# --- matrix layout: tensor order, entry offsets, decoders ---------------------------------------
+@pytest.mark.parametrize("M,K", [(32, 128), (64, 256), (33, 128), (100, 384), (1, 128)])
+def test_tile_order_is_a_bijection(M, K):
+    Mp = oracle.padded_rows(M)
+    assert Mp % 32 == 0 and 0 <= Mp - M < 32
+    seen = np.zeros(Mp * K, bool)
+    for m in range(Mp):
+        for k in range(0, K, 7):
+            seen[oracle.tile_order_pos(M, K, m, k)] = True
+    pos = np.array([[oracle.tile_order_pos(M, K, m, k) for k in range(K)] for m in range(min(M, 40))])
+    assert len(np.unique(pos)) == pos.size and pos.max() < Mp * K
+    # inside a tile: row major, k ascending; tiles: row block major, group minor
+    assert oracle.tile_order_pos(M, K, 0, 0) == 0
+    assert oracle.tile_order_pos(M, K, 0, 127) == 127
+    if Mp >= 2:
+        assert oracle.tile_order_pos(M, K, 1, 0) == 128
+    if K >= 256:
+        assert oracle.tile_order_pos(M, K, 0, 128) == 32 * 128
+    if Mp >= 64:
+        assert oracle.tile_order_pos(M, K, 32, 0) == 32 * K
+
+
+@pytest.mark.parametrize("M,K,z", [(32, 128, 0.42), (96, 512, 0.3), (40, 256, 0.515), (7, 128, 0.47)])
+def test_round_trip_all_decoders(M, K, z):
+    W = datagen.trits(5, M, K, z)
+    pk = oracle.bitcos_pack(W)
+    assert pk.nnz == np.count_nonzero(W)
+    # offsets are the running number of nonzeros at each tile boundary
+    Mp, G = oracle.padded_rows(M), K // 128
+    Wp = np.zeros((Mp, K), np.int8)
+    Wp[:M] = W
+    per_tile = [np.count_nonzero(Wp[rb * 32:(rb + 1) * 32, g * 128:(g + 1) * 128])
+                for rb in range(Mp // 32) for g in range(G)]
+    assert list(pk.tile_off) == list(np.concatenate([[0], np.cumsum(per_tile)]))
+    for dec in ("bits", "pdep", "lut", "tiles"):
+        assert np.array_equal(oracle.bitcos_unpack(pk.bitmap, pk.signs, pk.tile_off, M, K, dec), W), dec
+    # padding bits and slack words are zero
+    assert pk.signs.size == oracle.sign_words(pk.nnz)
+    assert pk.signs.size * 32 >= pk.nnz + 256 and pk.signs.size % 4 == 0
+    tail = pk.nnz
+    assert (int(pk.signs[tail // 32]) >> (tail % 32)) == 0 and not pk.signs[tail // 32 + 1:].any()
+
+
+def test_first_weight_of_row_r_takes_the_right_sign():
+    # one nonzero per row at k = 5, alternating sign: sign bit j belongs to row j of the tile
+    M, K = 32, 128
+    W = np.zeros((M, K), np.int8)
+    W[:, 5] = np.where(np.arange(M) % 3 == 0, -1, 1)
+    pk = oracle.bitcos_pack(W)
+    assert pk.nnz == 32
+    assert int(pk.signs[0]) == bits_lsb_first([1 if r % 3 == 0 else 0 for r in range(32)])
+    assert all(int(pk.bitmap[4 * r]) == 1 << 5 for r in range(32))
+
+
+def test_special_cases():
+    M, K = 32, 256
+    for fill, nnz in ((0, 0), (1, M * K), (-1, M * K)):
+        W = np.full((M, K), fill, np.int8)
+        pk = oracle.bitcos_pack(W)
+        assert pk.nnz == nnz
+        assert pk.bits_per_weight() == (2.0 if fill else 1.0)     # z = 0 -> 2 b/w, z = 1 -> 1 b/w
+        if fill == -1:
+            assert (pk.signs[:nnz // 32] == 0xFFFFFFFF).all()
+        if fill == 1:
+            assert not pk.signs.any()
+        for dec in ("bits", "pdep", "lut", "tiles"):
+            assert np.array_equal(oracle.bitcos_unpack(pk.bitmap, pk.signs, pk.tile_off, M, K, dec), W)
+    for k in (0, 31, 32, 127, 128, K - 1):
+        W = np.zeros((M, K), np.int8)
+        W[3, k] = -1
+        pk = oracle.bitcos_pack(W)
+        word = (((0 * 2 + k // 128) * 32 + 3) * 128 + k % 128) // 32
+        assert pk.bitmap[word] == 1 << (k % 32) and np.count_nonzero(pk.bitmap) == 1
+        assert pk.signs[0] == 1 and pk.nnz == 1
+
+
+def test_invalid_symbol_rejected():
+    W = np.zeros((32, 128), np.int8)
+    W[0, 0] = 2
+    with pytest.raises(oracle.OracleError):
+        oracle.bitcos_pack(W)
+    with pytest.raises(oracle.OracleError):
+        oracle.trit5_pack(W)
+    with pytest.raises(oracle.OracleError):
+        oracle.bit2_pack(W)
+
+
+# --- five-trit and 2-bit ------------------------------------------------------------------------
+def test_trit5_block_bytes():
+    t = np.zeros(128, np.int8)
+    assert list(oracle.trit5_block_encode(t)) == [121] * 26          # 1 + 3 + 9 + 27 + 81
+    assert oracle.trit5_block_encode(t).size == 26                    # ceil(128 / 5)
+    t[:] = -1
+    b = oracle.trit5_block_encode(t)
+    assert list(b[:25]) == [0] * 25 and b[25] == 27 + 81              # trits 125..127 = -1 (digit 0), digits 3, 4 = 1
+    t[:] = 1
+    b = oracle.trit5_block_encode(t)
+    assert list(b[:25]) == [242] * 25 and b[25] == 2 + 6 + 18 + 27 + 81
+    t[:] = 0
+    t[0] = 1
+    assert oracle.trit5_block_encode(t)[0] == 122
+    t[:] = 0
+    t[4] = 1
+    assert oracle.trit5_block_encode(t)[0] == 1 + 3 + 9 + 27 + 162
+    t[:] = 0
+    t[127] = -1
+    assert oracle.trit5_block_encode(t)[25] == 1 + 3 + 0 + 27 + 81
+
+
+def test_trit5_all_byte_values_round_trip():
+    # a block whose first 25 bytes walk through base-3 values; all 243 values appear over 10 blocks
+    seen = set()
+    for start in range(0, 243, 25):
+        t = np.zeros(128, np.int8)
+        for j in range(25):
+            v = (start + j) % 243
+            for i in range(5):
+                t[5 * j + i] = v % 3 - 1
+                v //= 3
+        b = oracle.trit5_block_encode(t)
+        seen.update(int(x) for x in b[:25])
+        assert np.array_equal(oracle.trit5_block_decode(b), t)
+    assert seen == set(range(243))
+    bad = np.full(26, 121, np.uint8)
+    bad[3] = 243
+    with pytest.raises(oracle.OracleError):
+        oracle.trit5_block_decode(bad)
+
+
+def test_bit2_code_positions():
+    M, K = 32, 128
+
+    def word0(i, val):
+        W = np.zeros((M, K), np.int8)
+        W[0, i] = val
+        return int(oracle.bit2_pack(W)[0])
+
+    assert word0(0, 0) == 0x55555555
+    assert word0(0, 1) == 0x55555556
+    assert word0(0, -1) == 0x55555554
+    assert word0(1, 1) == 0x55555655
+    assert word0(4, 1) == 0x55555559
+    assert word0(15, 1) == 0x95555555
+
+
+@pytest.mark.parametrize("M,K", [(32, 128), (64, 384), (45, 256)])
+def test_trit5_bit2_round_trip_and_sizes(M, K):
+    W = datagen.trits(6, M, K, 0.4)
+    Mp = oracle.padded_rows(M)
+    t5 = oracle.trit5_pack(W)
+    b2 = oracle.bit2_pack(W)
+    assert t5.size * 4 == Mp * ((26 * (K // 128) + 3) // 4) * 4
+    if (K // 128) % 2 == 0:
+        assert t5.size * 4 == Mp * 26 * (K // 128)                    # 26 bytes per 128 weights
+    assert b2.size * 32 == Mp * K * 2
+    assert np.array_equal(oracle.trit5_unpack(t5, M, K), W)
+    assert np.array_equal(oracle.bit2_unpack(b2, M, K), W)
+    # row interleave: word 0 of row r of block 0 is at index r (five-trit) / 4r (2-bit)
+    W2 = np.zeros((M, K), np.int8)
+    W2[5, :5] = [1, 1, 1, 1, 1]
+    assert oracle.trit5_pack(W2)[5] & 0xFF == 242
+    W2[5, :] = 0
+    W2[5, 0] = 1
+    assert oracle.bit2_pack(W2)[4 * 5] == 0x55555556
+
+
+# --- the product ------------------------------------------------------------------------------------
+def test_dense_product_bruteforce_tiny():
+    rng = np.random.default_rng(7)
+    for M, K, B in ((3, 128, 1), (3, 256, 3), (5, 384, 2)):
+        W = rng.integers(-1, 2, (M, K)).astype(np.int8)
+        x = rng.integers(-128, 128, (B, K)).astype(np.int8)
+        xs = rng.uniform(0.01, 0.04, B).astype(np.float32)
+        S = datagen.scales(8, M, K)
+        acc, y, mag = oracle.gemv_dense(W, S, x, xs)
+        Sf = datagen.bf16_bits_to_f32(S).astype(np.float64)
+        for b in range(B):
+            for m in range(M):
+                tot = 0.0
+                for g in range(K // 128):
+                    a = sum(int(W[m, k]) * int(x[b, k]) for k in range(128 * g, 128 * g + 128))
+                    assert acc[b, m, g] == a
+                    tot += Sf[m, g] * a
+                assert y[b, m] == pytest.approx(float(xs[b]) * tot, rel=1e-14, abs=1e-300)
+                assert mag[b, m] >= abs(y[b, m]) * (1 - 1e-12)
+
+
+def test_dense_product_closed_forms():
+    M, K = 4, 256
+    x, xs = datagen.activations(9, 2, K)
+    ones = np.full((M, K // 128), 0x3F80, np.uint16)                  # bf16 1.0
+    for fill in (1, -1, 0):
+        W = np.full((M, K), fill, np.int8)
+        acc, y, _ = oracle.gemv_dense(W, ones, x, np.ones(2, np.float32))
+        want = fill * x.astype(np.int64).reshape(2, 2, 128).sum(-1)
+        assert np.array_equal(acc, np.broadcast_to(want[:, None, :], acc.shape))
+        assert np.array_equal(y, np.broadcast_to(want.sum(-1)[:, None].astype(np.float64), y.shape))
+    for k in (0, 127, 128, 255):
+        W = np.zeros((M, K), np.int8)
+        W[2, k] = -1
+        acc, y, _ = oracle.gemv_dense(W, ones, x, np.ones(2, np.float32))
+        assert acc[0, 2, k // 128] == -int(x[0, k]) and np.count_nonzero(acc[0]) == (x[0, k] != 0)
+    # linearity in x (no int8 overflow: halves)
+    W = datagen.trits(10, M, K, 0.4)
+    x1 = (x // 2).astype(np.int8)
+    x2 = (x - x1).astype(np.int8)
+    a, _, _ = oracle.gemv_dense(W, ones, x, np.ones(2, np.float32))
+    a1, _, _ = oracle.gemv_dense(W, ones, x1, np.ones(2, np.float32))
+    a2, _, _ = oracle.gemv_dense(W, ones, x2, np.ones(2, np.float32))
+    assert np.array_equal(a, a1 + a2)
+    # x = -128 is accepted
+    xm = np.full((1, K), -128, np.int8)
+    a, _, _ = oracle.gemv_dense(np.ones((M, K), np.int8), ones, xm, np.ones(1, np.float32))
+    assert (a == -128 * 128).all()
+    # the activation scale multiplies the whole output
+    S = datagen.scales(11, M, K)
+    _, y1, _ = oracle.gemv_dense(W, S, x, np.array([1.0, 1.0], np.float32))
+    _, y2, _ = oracle.gemv_dense(W, S, x, np.array([0.5, 2.0], np.float32))
+    assert np.array_equal(y2[0], 0.5 * y1[0]) and np.array_equal(y2[1], 2.0 * y1[1])
+
+
+@pytest.mark.parametrize("M,K,B,z", [(256, 512, 1, 0.42), (40, 384, 3, 0.33)])
+def test_packed_formats_agree_with_dense(M, K, B, z):
+    W = datagen.trits(12, M, K, z)
+    S = datagen.scales(12, M, K)
+    x, xs = datagen.activations(12, B, K)
+    acc, y, mag = oracle.gemv_dense(W, S, x, xs)
+    pk = oracle.bitcos_pack(W)
+    for fmt, payload, signs, off in ((oracle.FORMAT_BITCOS, pk.bitmap, pk.signs, pk.tile_off),
+                                     (oracle.FORMAT_TRIT5, oracle.trit5_pack(W), None, None),
+                                     (oracle.FORMAT_BIT2, oracle.bit2_pack(W), None, None)):
+        a2, y2, m2 = oracle.gemv_packed(fmt, payload, signs, off, S, x, xs, M, K)
+        assert np.array_equal(a2, acc) and np.array_equal(y2, y) and np.array_equal(m2, mag)
+
+
+def test_scales_tile_order():
+    M, K = 40, 384
+    S = datagen.scales(13, M, K)
+    T = oracle.scales_to_tile_order(S, M, K)
+    G = K // 128
+    assert T.size == 64 * G
+    for m in (0, 1, 31, 32, 39):
+        for g in range(G):
+            assert T[((m // 32) * G + g) * 32 + m % 32] == S[m, g]
+    assert T.reshape(2, G, 32)[1, :, 8:].sum() == 0
+
+
+def test_grouped_equals_independent_calls():
+    E, M, K = 4, 32, 128
+    Ws = [datagen.trits(20 + e, M, K, 0.33) for e in range(E)]
+    Ss = [datagen.scales(20 + e, M, K) for e in range(E)]
+    x, xs = datagen.activations(14, 3, K)
+    pe, pr = [0, 2, 2, 3], [0, 0, 1, 2]
+    acc, y, mag = oracle.grouped_dense(Ws, Ss, pe, pr, x, xs)
+    for i, (e, r) in enumerate(zip(pe, pr)):
+        a1, y1, _ = oracle.gemv_dense(Ws[e], Ss[e], x[r:r + 1], xs[r:r + 1])
+        assert np.array_equal(acc[i], a1[0]) and np.array_equal(y[i], y1[0])
+
+
+def test_generator_is_counter_based_and_has_the_stated_distribution():
+    a = datagen.uniform(1, 0, 0, 1000)
+    b = datagen.uniform(1, 0, 500, 10)
+    assert np.array_equal(a[500:510], b) and (a >= 0).all() and (a < 1).all()
+    W = datagen.trits(2, 512, 1024, 0.42)
+    assert abs((W == 0).mean() - 0.42) < 0.005 and abs((W == 1).mean() - 0.29) < 0.005
+    S = datagen.bf16_bits_to_f32(datagen.scales(2, 64, 1024))
+    assert S.min() >= 0.0099 and S.max() <= 0.0501
+    x, xs = datagen.activations(2, 4, 4096)
+    assert x.min() >= -127 and x.max() <= 127 and (xs > 0).all()
+    ids = datagen.expert_choices(2, 16, 128, 8)
+    assert all(len(set(r)) == 8 for r in ids) and ids.min() >= 0 and ids.max() < 128
