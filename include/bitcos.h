@@ -1,0 +1,198 @@
+/*
+ * bitcos.h -- C ABI of the BITCOS ternary GEMV library for NVIDIA B200 (sm_100a).
+ *
+ * The library stores a ternary weight matrix W in {-1,0,+1}^{M x K} (M output rows, K
+ * reduction length, one bf16 scale per row and group of 128 reduction elements) in three
+ * formats and multiplies it with int8 activations:
+ *
+ *   BITCOS     presence bitmap (1 bit per weight) + compacted sign vector (1 bit per
+ *              non-zero weight, same order) + entry offsets: 2 - z bits per weight at zero
+ *              density z (paper Section II-A, Eq. 1).
+ *   five-trit  five ternary digits per byte, 26 bytes per 128 weights (paper Section I).
+ *   2-bit      two bits per weight (the paper's baseline format, Section IV).
+ *
+ *     acc[b][m][g] = sum_{k in group g} W[m][k] * x[b][k]                    (int32, exact)
+ *     y[b][m]      = x_scale[b] * sum_g float(scale[m][g]) * float(acc[b][m][g])   (fp32)
+ *
+ * (integer path of Section II-C: w = p - 2n, Eq. 2; int32 accumulation per group; the
+ * group scale applied once per group).  Batch b = 0 .. batch-1, 1 <= batch <= 16; the
+ * packed weights are read once per call, not once per token.
+ *
+ * Conventions
+ *   - Every function returns a bitcos_status.  Nothing throws, prints or allocates.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA device memory of
+ *     the current device, owned by the caller, 16-byte aligned.
+ *   - Device entry points enqueue work on the given stream (a cudaStream_t passed as
+ *     void*, NULL = default stream) and return without synchronising.  They never call
+ *     cudaMalloc / cudaFree.
+ *   - K must be a multiple of 128 (the only group size); any M >= 1.
+ *
+ * Storage order ("tensor order").  The paper leaves the order of weights inside the
+ * bitmap open and itself interleaves 32 output rows (Fig. 2, Section II-D).  Here rows are
+ * taken in blocks of 32 (Mp = M rounded up to 32; padding rows hold zero weights) and the
+ * reduction in groups of 128.  A tile = (row block rb, group g), numbered
+ * t = rb * (K/128) + g.  Inside a tile: row r = 0..31, then k ascending.  Hence
+ *   bitmap    uint32[Mp*K/32]; word (t*32 + r)*4 + j holds k = 128g + 32j .. +31 of row
+ *             32rb + r, bit i <-> k = 128g + 32j + i (LSB first);
+ *   signs     uint32[]; bit q of the sign vector is bit (q & 31) of word q >> 5; the q-th
+ *             sign bit belongs to the q-th set bit of the bitmap; 1 = negative (Eq. 4);
+ *   tile_off  uint32[n_tiles + 1]; tile_off[t] = index of tile t's first sign bit,
+ *             tile_off[n_tiles] = number of non-zero weights;
+ *   scales    uint16[Mp*K/128] bf16 bit patterns, scale of (row 32rb + r, group g) at
+ *             t*32 + r (padding rows +0).
+ */
+#ifndef BITCOS_H
+#define BITCOS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BITCOS_GROUP 128
+#define BITCOS_TILE_ROWS 32
+#define BITCOS_MAX_BATCH 16
+
+typedef enum bitcos_status {
+    BITCOS_OK = 0,
+    BITCOS_ERR_NULL = 1,      /* a required pointer is NULL */
+    BITCOS_ERR_SHAPE = 2,     /* M < 1, K < 128, K % 128 != 0, batch outside 1..16, bad list */
+    BITCOS_ERR_ALIGN = 3,     /* a device pointer is not 16-byte aligned */
+    BITCOS_ERR_TRIT = 4,      /* a weight outside {-1,0,+1} / an invalid packed code */
+    BITCOS_ERR_SCALE = 5,     /* a scale that is NaN, Inf or has its sign bit set */
+    BITCOS_ERR_CAPACITY = 6,  /* an output or workspace buffer is too small */
+    BITCOS_ERR_OVERFLOW = 7,  /* more than 2^32 - 1 non-zero weights */
+    BITCOS_ERR_CUDA = 8       /* a CUDA runtime call failed; see bitcos_last_cuda_error() */
+} bitcos_status;
+
+/* Static string naming a status value. */
+const char *bitcos_status_string(int status);
+/* cudaError_t value of the last failed CUDA call made by this library in this thread. */
+int bitcos_last_cuda_error(void);
+
+/* ---------------------------------------------------------------------------------------
+ * Host side: packers (paper Section II-A for BITCOS; Section I for five-trit; the 2-bit
+ * format of Section IV).  Synchronous, deterministic; every padding bit and byte written
+ * is zero so that packed buffers can be compared with memcmp.
+ * ------------------------------------------------------------------------------------- */
+
+/* Sizes in bytes of the four BITCOS buffers for an M x K matrix with nnz non-zero weights.
+ * sign_bytes = ceil(nnz/8) rounded up to 16, plus 32 bytes of zero slack (a decoder may
+ * fetch a fixed-size aligned window at the last cursor).  Any output pointer may be NULL. */
+int bitcos_pack_sizes(int64_t M, int64_t K, uint64_t nnz, size_t *bitmap_bytes, size_t *sign_bytes,
+                      size_t *tile_off_bytes, size_t *scale_bytes);
+
+/* Counts the non-zero weights of trits[M][K] (host, row major); ERR_TRIT on a bad value. */
+int bitcos_count_nnz(const int8_t *trits, int64_t M, int64_t K, uint64_t *nnz);
+
+/* Packs trits[M][K] (host, row major, values -1/0/+1) and scales_bf16[M][K/128] (host, row
+ * major, bf16 bit patterns, finite and non-negative) into the four caller-provided host
+ * buffers sized by bitcos_pack_sizes.  sign_capacity_bytes is the size of `signs`.
+ * nnz_out (optional) receives the number of sign bits. */
+int bitcos_pack(const int8_t *trits, const uint16_t *scales_bf16, int64_t M, int64_t K,
+                uint32_t *bitmap, uint32_t *signs, size_t sign_capacity_bytes, uint32_t *tile_off,
+                uint16_t *scales_tiled, uint64_t *nnz_out);
+
+/* Inverse of bitcos_pack: trits_out[M][K] (host).  ERR_TRIT if the offsets do not match the
+ * bitmap's population counts. */
+int bitcos_unpack(const uint32_t *bitmap, const uint32_t *signs, const uint32_t *tile_off,
+                  int64_t M, int64_t K, int8_t *trits_out);
+
+/* Reorders row-major scales[M][K/128] into the tile order described above (and back). */
+int bitcos_scales_tile(const uint16_t *scales_bf16, int64_t M, int64_t K, uint16_t *scales_tiled);
+int bitcos_scales_untile(const uint16_t *scales_tiled, int64_t M, int64_t K, uint16_t *scales_bf16);
+
+/* Five-trit: byte j of a 128-weight block = sum_{i<5} (t[5j+i] + 1) * 3^i; byte 25 carries
+ * trits 125..127 and digit 1 in its two unused places; 26 bytes per block.  A row's K/128
+ * blocks are concatenated, zero padded to a multiple of 4 bytes, and read as little-endian
+ * 32-bit words; word q of row 32rb + r is stored at index (rb*WPR + q)*32 + r, where
+ * WPR = ceil(26*(K/128)/4).  *bytes = Mp * WPR * 4. */
+int trit5_pack_sizes(int64_t M, int64_t K, size_t *bytes);
+int trit5_pack(const int8_t *trits, int64_t M, int64_t K, uint32_t *words);
+int trit5_unpack(const uint32_t *words, int64_t M, int64_t K, int8_t *trits_out);
+
+/* 2-bit: code = t + 1; 16 weights per 32-bit word, weight i at bits [8*(i%4) + 2*(i/4), +2);
+ * a row is K/16 words; word j of 16-byte chunk c of row 32rb + r is stored at index
+ * ((rb*(K/64) + c)*32 + r)*4 + j.  *bytes = Mp * K / 4. */
+int bit2_pack_sizes(int64_t M, int64_t K, size_t *bytes);
+int bit2_pack(const int8_t *trits, int64_t M, int64_t K, uint32_t *words);
+int bit2_unpack(const uint32_t *words, int64_t M, int64_t K, int8_t *trits_out);
+
+/* ---------------------------------------------------------------------------------------
+ * Device side: the products.
+ * ------------------------------------------------------------------------------------- */
+
+/* A packed BITCOS matrix in device memory (layout above). */
+typedef struct bitcos_weights {
+    const uint32_t *bitmap;
+    const uint32_t *signs;
+    const uint32_t *tile_off;
+    const uint16_t *scales;   /* tile order */
+    int64_t M;
+    int64_t K;
+} bitcos_weights;
+
+/* Scratch memory the three GEMV entry points need for an M x K matrix (the same value for
+ * all formats and batches): partial row sums of reduction segments that were spread over
+ * several thread blocks, and one arrival counter per row block.  The caller allocates it
+ * on the device, fills it with zeros ONCE (bitcos_workspace_init), and may reuse it for
+ * any later call whose requirement is not larger: every call leaves the counters zero.
+ * Two calls that may run at the same time must not share a workspace. */
+size_t bitcos_gemv_workspace_bytes(int64_t M, int64_t K);
+int bitcos_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* y[b][m] for b < batch, m < M from a BITCOS matrix (steps of Section II-B..II-D on the GPU:
+ * entry offset + running population count locate each row's sign window, a 256-entry
+ * (presence nibble, sign nibble) table as in Eq. 4 rebuilds four weights at a time as int8,
+ * dp4a accumulates int32 per group, the bf16 group scale and the per-token scale are applied
+ * in fp32).
+ *   W            host struct holding device pointers
+ *   x            device int8 [batch][K], row major
+ *   x_scale      device float [batch]
+ *   y            device float [batch][M], overwritten
+ *   acc_debug    NULL, or device int32 [batch][M][K/128] receiving every group accumulator
+ *   workspace    device scratch of at least bitcos_gemv_workspace_bytes(M, K) bytes */
+int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
+                int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Host-buffer form of bitcos_gemv for callers whose activations live in host memory: copies
+ * x_host[batch][K] and x_scale_host[batch] into `staging`, runs bitcos_gemv, copies
+ * y[batch][M] back to y_host and waits for the stream, so y_host is valid on return.  The
+ * weights stay resident on the device.  Pinned host buffers make the copies asynchronous
+ * until the final wait.  staging: device scratch of bitcos_gemv_host_staging_bytes bytes. */
+size_t bitcos_gemv_host_staging_bytes(int64_t M, int64_t K, int batch);
+int bitcos_gemv_host(const bitcos_weights *W, const int8_t *x_host, const float *x_scale_host, int batch,
+                     float *y_host, void *staging, size_t staging_bytes, void *workspace,
+                     size_t workspace_bytes, void *cuda_stream);
+
+/* The same product from the five-trit and 2-bit layouts (device pointers; scales in tile order). */
+int trit5_gemv(const uint32_t *words, const uint16_t *scales_tiled, int64_t M, int64_t K, const int8_t *x,
+               const float *x_scale, int batch, float *y, int32_t *acc_debug, void *workspace,
+               size_t workspace_bytes, void *cuda_stream);
+int bit2_gemv(const uint32_t *words, const uint16_t *scales_tiled, int64_t M, int64_t K, const int8_t *x,
+              const float *x_scale, int batch, float *y, int32_t *acc_debug, void *workspace,
+              size_t workspace_bytes, void *cuda_stream);
+
+/* Grouped product over selected experts of a mixture-of-experts layer (all experts M x K).
+ * The caller lists the P (token, expert) pairs grouped by expert: group i covers pairs
+ * group_begin[i] .. group_begin[i+1]-1 (at most 16 per group), all using expert
+ * group_expert[i]; pair p reads activation row pair_xrow[p] of x[R][K] and writes y[p][M].
+ * Each listed expert's packed bytes are read once.  No activation function, routing weight
+ * or sum over experts is applied.
+ *   experts       device array of bitcos_weights (device pointers inside), n_experts entries
+ *   group_expert  device int32 [n_groups];  group_begin  device int32 [n_groups + 1]
+ *   pair_xrow     device int32 [P];  x device int8 [R][K];  x_scale device float [R]
+ *   y             device float [P][M];  acc_debug NULL or device int32 [P][M][K/128]
+ *   workspace     at least n_groups * bitcos_gemv_workspace_bytes(M, K) bytes, zero filled once */
+int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K,
+                        const int32_t *group_expert, const int32_t *group_begin, int n_groups,
+                        const int32_t *pair_xrow, int n_pairs, int max_group_size, const int8_t *x,
+                        const float *x_scale, float *y, int32_t *acc_debug, void *workspace,
+                        size_t workspace_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITCOS_H */

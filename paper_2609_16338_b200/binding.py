@@ -1,0 +1,360 @@
+"""ctypes binding of libbitcos.so: same names as the C ABI, argument marshalling only.
+
+Host packers take and return numpy arrays.  Device entry points take torch CUDA tensors
+(used here only as owners of device memory) and enqueue on torch's current stream.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+
+GROUP = 128
+TILE_ROWS = 32
+MAX_BATCH = 16
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libbitcos.so")
+
+EXPORTED_SYMBOLS = [
+    "bitcos_status_string", "bitcos_last_cuda_error", "bitcos_pack_sizes", "bitcos_count_nnz", "bitcos_pack",
+    "bitcos_unpack", "bitcos_scales_tile", "bitcos_scales_untile", "trit5_pack_sizes", "trit5_pack",
+    "trit5_unpack", "bit2_pack_sizes", "bit2_pack", "bit2_unpack", "bitcos_gemv_workspace_bytes",
+    "bitcos_workspace_init", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
+    "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host",
+]
+
+
+class BitcosError(RuntimeError):
+    def __init__(self, status: int, what: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({detail})")
+
+
+class _Weights(C.Structure):
+    _fields_ = [("bitmap", C.c_void_p), ("signs", C.c_void_p), ("tile_off", C.c_void_p), ("scales", C.c_void_p),
+                ("M", C.c_int64), ("K", C.c_int64)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Loads libbitcos.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise BitcosError(-1, "load_library", f"{_LIB_PATH} is missing: run `python -m paper_2609_16338_b200.build`")
+    L = C.CDLL(_LIB_PATH)
+    vp, i64, sz, u64 = C.c_void_p, C.c_int64, C.c_size_t, C.c_uint64
+    psz = C.POINTER(C.c_size_t)
+    L.bitcos_status_string.restype = C.c_char_p
+    L.bitcos_status_string.argtypes = [C.c_int]
+    L.bitcos_last_cuda_error.restype = C.c_int
+    L.bitcos_last_cuda_error.argtypes = []
+    L.bitcos_pack_sizes.argtypes = [i64, i64, u64, psz, psz, psz, psz]
+    L.bitcos_count_nnz.argtypes = [vp, i64, i64, C.POINTER(u64)]
+    L.bitcos_pack.argtypes = [vp, vp, i64, i64, vp, vp, sz, vp, vp, C.POINTER(u64)]
+    L.bitcos_unpack.argtypes = [vp, vp, vp, i64, i64, vp]
+    L.bitcos_scales_tile.argtypes = [vp, i64, i64, vp]
+    L.bitcos_scales_untile.argtypes = [vp, i64, i64, vp]
+    for name in ("trit5", "bit2"):
+        getattr(L, name + "_pack_sizes").argtypes = [i64, i64, psz]
+        getattr(L, name + "_pack").argtypes = [vp, i64, i64, vp]
+        getattr(L, name + "_unpack").argtypes = [vp, i64, i64, vp]
+    L.bitcos_gemv_workspace_bytes.restype = sz
+    L.bitcos_gemv_workspace_bytes.argtypes = [i64, i64]
+    L.bitcos_workspace_init.argtypes = [vp, sz, vp]
+    L.bitcos_gemv.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, vp, sz, vp]
+    for name in ("trit5_gemv", "bit2_gemv"):
+        getattr(L, name).argtypes = [vp, vp, i64, i64, vp, vp, C.c_int, vp, vp, vp, sz, vp]
+    L.bitcos_gemv_grouped.argtypes = [vp, C.c_int, i64, i64, vp, vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp, vp,
+                                      vp, sz, vp]
+    L.bitcos_gemv_host_staging_bytes.restype = sz
+    L.bitcos_gemv_host_staging_bytes.argtypes = [i64, i64, C.c_int]
+    L.bitcos_gemv_host.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, sz, vp, sz, vp]
+    _lib = L
+    return L
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        L = load_library()
+        detail = L.bitcos_status_string(status).decode()
+        if status == 8:
+            detail += f", cudaError {L.bitcos_last_cuda_error()}"
+        raise BitcosError(status, what, detail)
+
+
+def _np(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _ptr(a: np.ndarray):
+    return C.c_void_p(a.ctypes.data)
+
+
+# ---------------------------------------------------------------------------------------------
+# host packers
+# ---------------------------------------------------------------------------------------------
+@dataclass
+class PackedBitcos:
+    M: int
+    K: int
+    nnz: int
+    bitmap: np.ndarray      # uint32
+    signs: np.ndarray       # uint32, zero slack included
+    tile_off: np.ndarray    # uint32 [n_tiles + 1]
+    scales: np.ndarray      # uint16, tile order
+
+    def payload_bytes(self) -> int:
+        """Bytes a GEMV has to read: bitmap, the sign bits (not the slack), offsets, scales."""
+        return self.bitmap.nbytes + (self.nnz + 7) // 8 + self.tile_off.nbytes + self.scales.nbytes
+
+    def to_device(self, device="cuda"):
+        import torch
+        t = [torch.from_numpy(a.view(np.int32) if a.dtype == np.uint32 else a.view(np.int16)).to(device)
+             for a in (self.bitmap, self.signs, self.tile_off, self.scales)]
+        return DeviceBitcos(self.M, self.K, self.nnz, *t)
+
+
+class DeviceBitcos:
+    """A BITCOS matrix resident in device memory (tensors only own the bytes)."""
+
+    def __init__(self, M, K, nnz, bitmap, signs, tile_off, scales):
+        self.M, self.K, self.nnz = M, K, nnz
+        self.bitmap, self.signs, self.tile_off, self.scales = bitmap, signs, tile_off, scales
+        self.desc = _Weights(bitmap.data_ptr(), signs.data_ptr(), tile_off.data_ptr(), scales.data_ptr(), M, K)
+
+    def clone(self):
+        return DeviceBitcos(self.M, self.K, self.nnz, self.bitmap.clone(), self.signs.clone(),
+                            self.tile_off.clone(), self.scales.clone())
+
+    def payload_bytes(self) -> int:
+        return self.bitmap.numel() * 4 + (self.nnz + 7) // 8 + self.tile_off.numel() * 4 + self.scales.numel() * 2
+
+
+class DevicePlain:
+    """A five-trit or 2-bit matrix in device memory: payload words + scales in tile order."""
+
+    def __init__(self, M, K, words, scales):
+        self.M, self.K, self.words, self.scales = M, K, words, scales
+
+    def clone(self):
+        return DevicePlain(self.M, self.K, self.words.clone(), self.scales.clone())
+
+    def payload_bytes(self) -> int:
+        return self.words.numel() * 4 + self.scales.numel() * 2
+
+
+def bitcos_pack(trits, scales_bf16) -> PackedBitcos:
+    L = load_library()
+    t = _np(trits, np.int8)
+    M, K = t.shape
+    s = _np(scales_bf16, np.uint16)
+    nnz = C.c_uint64(0)
+    _check(L.bitcos_count_nnz(_ptr(t), M, K, C.byref(nnz)), "bitcos_count_nnz")
+    sizes = [C.c_size_t(0) for _ in range(4)]
+    _check(L.bitcos_pack_sizes(M, K, nnz.value, *[C.byref(v) for v in sizes]), "bitcos_pack_sizes")
+    bitmap = np.zeros(sizes[0].value // 4, np.uint32)
+    signs = np.zeros(sizes[1].value // 4, np.uint32)
+    tile_off = np.zeros(sizes[2].value // 4, np.uint32)
+    scales = np.zeros(sizes[3].value // 2, np.uint16)
+    out = C.c_uint64(0)
+    _check(L.bitcos_pack(_ptr(t), _ptr(s), M, K, _ptr(bitmap), _ptr(signs), signs.nbytes, _ptr(tile_off),
+                         _ptr(scales), C.byref(out)), "bitcos_pack")
+    return PackedBitcos(M, K, int(out.value), bitmap, signs, tile_off, scales)
+
+
+def bitcos_unpack(p: PackedBitcos) -> np.ndarray:
+    out = np.zeros((p.M, p.K), np.int8)
+    _check(load_library().bitcos_unpack(_ptr(p.bitmap), _ptr(p.signs), _ptr(p.tile_off), p.M, p.K, _ptr(out)),
+           "bitcos_unpack")
+    return out
+
+
+def scales_tile(scales_bf16, M, K) -> np.ndarray:
+    s = _np(scales_bf16, np.uint16)
+    Mp = (M + TILE_ROWS - 1) // TILE_ROWS * TILE_ROWS
+    out = np.zeros(Mp * (K // GROUP), np.uint16)
+    _check(load_library().bitcos_scales_tile(_ptr(s), M, K, _ptr(out)), "bitcos_scales_tile")
+    return out
+
+
+def scales_untile(tiled, M, K) -> np.ndarray:
+    t = _np(tiled, np.uint16)
+    out = np.zeros((M, K // GROUP), np.uint16)
+    _check(load_library().bitcos_scales_untile(_ptr(t), M, K, _ptr(out)), "bitcos_scales_untile")
+    return out
+
+
+def _plain_pack(name, trits):
+    L = load_library()
+    t = _np(trits, np.int8)
+    M, K = t.shape
+    n = C.c_size_t(0)
+    _check(getattr(L, name + "_pack_sizes")(M, K, C.byref(n)), name + "_pack_sizes")
+    words = np.zeros(n.value // 4, np.uint32)
+    _check(getattr(L, name + "_pack")(_ptr(t), M, K, _ptr(words)), name + "_pack")
+    return words
+
+
+def _plain_unpack(name, words, M, K):
+    w = _np(words, np.uint32)
+    out = np.zeros((M, K), np.int8)
+    _check(getattr(load_library(), name + "_unpack")(_ptr(w), M, K, _ptr(out)), name + "_unpack")
+    return out
+
+
+def trit5_pack(trits) -> np.ndarray:
+    return _plain_pack("trit5", trits)
+
+
+def trit5_unpack(words, M, K) -> np.ndarray:
+    return _plain_unpack("trit5", words, M, K)
+
+
+def bit2_pack(trits) -> np.ndarray:
+    return _plain_pack("bit2", trits)
+
+
+def bit2_unpack(words, M, K) -> np.ndarray:
+    return _plain_unpack("bit2", words, M, K)
+
+
+def plain_to_device(words, scales_tiled, M, K, device="cuda") -> DevicePlain:
+    import torch
+    return DevicePlain(M, K, torch.from_numpy(_np(words, np.uint32).view(np.int32)).to(device),
+                       torch.from_numpy(_np(scales_tiled, np.uint16).view(np.int16)).to(device))
+
+
+# ---------------------------------------------------------------------------------------------
+# device entry points
+# ---------------------------------------------------------------------------------------------
+def bitcos_gemv_workspace_bytes(M: int, K: int) -> int:
+    return int(load_library().bitcos_gemv_workspace_bytes(M, K))
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_workspace(M: int, K: int, device="cuda", copies: int = 1):
+    """Device scratch for the GEMV entry points, zero filled through bitcos_workspace_init."""
+    import torch
+    n = bitcos_gemv_workspace_bytes(M, K) * copies
+    ws = torch.empty(max(n, 256), dtype=torch.uint8, device=device)
+    _check(load_library().bitcos_workspace_init(C.c_void_p(ws.data_ptr()), ws.numel(), _stream()),
+           "bitcos_workspace_init")
+    return ws
+
+
+def _outputs(M, K, batch, y, acc_debug, device):
+    import torch
+    if y is None:
+        y = torch.empty((batch, M), dtype=torch.float32, device=device)
+    acc = None
+    if acc_debug is True:
+        acc = torch.empty((batch, M, K // GROUP), dtype=torch.int32, device=device)
+    elif acc_debug is not None and acc_debug is not False:
+        acc = acc_debug
+    return y, acc
+
+
+def bitcos_gemv(W: DeviceBitcos, x, x_scale, y=None, acc_debug=None, workspace=None):
+    """y[b][m] = x_scale[b] * sum_g scale[m][g] * sum_{k in g} W[m][k] x[b][k]; returns (y, acc or None)."""
+    batch = x.shape[0]
+    if workspace is None:
+        workspace = make_workspace(W.M, W.K, x.device)
+    y, acc = _outputs(W.M, W.K, batch, y, acc_debug, x.device)
+    _check(load_library().bitcos_gemv(C.byref(W.desc), x.data_ptr(), x_scale.data_ptr(), batch, y.data_ptr(),
+                                      acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
+                                      workspace.numel(), _stream()), "bitcos_gemv")
+    return y, acc
+
+
+def _plain_gemv(name, W: DevicePlain, x, x_scale, y, acc_debug, workspace):
+    batch = x.shape[0]
+    if workspace is None:
+        workspace = make_workspace(W.M, W.K, x.device)
+    y, acc = _outputs(W.M, W.K, batch, y, acc_debug, x.device)
+    _check(getattr(load_library(), name)(W.words.data_ptr(), W.scales.data_ptr(), W.M, W.K, x.data_ptr(),
+                                         x_scale.data_ptr(), batch, y.data_ptr(),
+                                         acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
+                                         workspace.numel(), _stream()), name)
+    return y, acc
+
+
+def trit5_gemv(W: DevicePlain, x, x_scale, y=None, acc_debug=None, workspace=None):
+    return _plain_gemv("trit5_gemv", W, x, x_scale, y, acc_debug, workspace)
+
+
+def bit2_gemv(W: DevicePlain, x, x_scale, y=None, acc_debug=None, workspace=None):
+    return _plain_gemv("bit2_gemv", W, x, x_scale, y, acc_debug, workspace)
+
+
+class DeviceExperts:
+    """Descriptors of E same-shaped BITCOS matrices, copied to the device once."""
+
+    def __init__(self, experts: list[DeviceBitcos]):
+        import torch
+        self.experts = experts
+        self.M, self.K = experts[0].M, experts[0].K
+        arr = (_Weights * len(experts))(*[e.desc for e in experts])
+        raw = np.frombuffer(bytes(arr), dtype=np.uint8).copy()
+        self.table = torch.from_numpy(raw).to(experts[0].bitmap.device)
+
+
+def group_pairs(pair_expert, pair_xrow):
+    """Sorts (expert, activation row) pairs by expert.  Returns (order, group_expert, group_begin,
+    xrow_sorted, max_group_size): pair i of the sorted list is input pair order[i]."""
+    pe = np.asarray(pair_expert, np.int32)
+    pr = np.asarray(pair_xrow, np.int32)
+    order = np.argsort(pe, kind="stable")
+    pe_s, pr_s = pe[order], pr[order]
+    ge, first = np.unique(pe_s, return_index=True)
+    begin = np.concatenate([first, [len(pe_s)]]).astype(np.int32)
+    return order, ge.astype(np.int32), begin, pr_s, int(np.diff(begin).max())
+
+
+def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale,
+                        y=None, acc_debug=None, workspace=None):
+    """Grouped product: pairs listed per expert (device int32 tensors); y is [P, M] in list order."""
+    import torch
+    n_groups, n_pairs = group_expert.numel(), pair_xrow.numel()
+    if workspace is None:
+        workspace = make_workspace(E.M, E.K, x.device, copies=n_groups)
+    if y is None:
+        y = torch.empty((n_pairs, E.M), dtype=torch.float32, device=x.device)
+    acc = None
+    if acc_debug is True:
+        acc = torch.empty((n_pairs, E.M, E.K // GROUP), dtype=torch.int32, device=x.device)
+    _check(load_library().bitcos_gemv_grouped(E.table.data_ptr(), len(E.experts), E.M, E.K, group_expert.data_ptr(),
+                                              group_begin.data_ptr(), n_groups, pair_xrow.data_ptr(), n_pairs,
+                                              max_group_size, x.data_ptr(), x_scale.data_ptr(), y.data_ptr(),
+                                              acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
+                                              workspace.numel(), _stream()), "bitcos_gemv_grouped")
+    return y, acc
+
+
+def bitcos_gemv_host_staging_bytes(M: int, K: int, batch: int) -> int:
+    return int(load_library().bitcos_gemv_host_staging_bytes(M, K, batch))
+
+
+def bitcos_gemv_host(W: DeviceBitcos, x_host: np.ndarray, x_scale_host: np.ndarray, y_host: np.ndarray, staging,
+                     workspace):
+    """Host-buffer form: copies x and x_scale to the device, multiplies, copies y back and
+    waits for the stream.  x_host int8 [B, K], x_scale_host float32 [B], y_host float32 [B, M]."""
+    batch = x_host.shape[0]
+    _check(load_library().bitcos_gemv_host(C.byref(W.desc), x_host.ctypes.data, x_scale_host.ctypes.data, batch,
+                                           y_host.ctypes.data, staging.data_ptr(), staging.numel(),
+                                           workspace.data_ptr(), workspace.numel(), _stream()), "bitcos_gemv_host")
+    return y_host

@@ -1,0 +1,191 @@
+"""GPU parity: every device entry point of the C ABI against the CPU oracle, element by
+element, on the same seeded inputs.
+
+Bar: int32 group accumulators bit-exact; fp32 outputs within 1e-5 of sum|terms|
+(|y - y_ref| <= 1e-5 * mag, and exactly 0 where mag is 0).
+"""
+import numpy as np
+import pytest
+
+import datagen
+import oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+REL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def bc():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_16338_b200 as m
+    from paper_2609_16338_b200 import build
+    build.build()
+    m.load_library()
+    return m
+
+
+def dev(a):
+    if a.dtype == np.uint32:
+        a = a.view(np.int32)
+    if a.dtype == np.uint16:
+        a = a.view(np.int16)
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def check(y, acc, acc_ref, y_ref, mag, what):
+    torch.cuda.synchronize()
+    if acc is not None:
+        assert np.array_equal(acc.cpu().numpy(), acc_ref), f"{what}: int32 accumulators differ"
+    yv = y.cpu().numpy().astype(np.float64)
+    err = np.abs(yv - y_ref)
+    bad = err > REL * mag
+    assert not bad.any(), f"{what}: {bad.sum()} outputs off, worst {np.max(err / np.maximum(mag, 1e-300)):.3e}"
+    assert (yv[mag == 0] == 0).all()
+
+
+def run_all_formats(bc, W, S, x, xs, what, formats=("bitcos", "trit5", "bit2"), debug=True):
+    M, K = W.shape
+    acc_ref, y_ref, mag = oracle.gemv_dense(W, S, x, xs)
+    xd, xsd = dev(x), dev(xs)
+    ws = bc.make_workspace(M, K)
+    st = bc.scales_tile(S, M, K)
+    for fmt in formats:
+        if fmt == "bitcos":
+            Wd = bc.bitcos_pack(W, S).to_device()
+            f = bc.bitcos_gemv
+        elif fmt == "trit5":
+            Wd = bc.plain_to_device(bc.trit5_pack(W), st, M, K)
+            f = bc.trit5_gemv
+        else:
+            Wd = bc.plain_to_device(bc.bit2_pack(W), st, M, K)
+            f = bc.bit2_gemv
+        for rep in range(2):                          # twice: the workspace must come back clean
+            y, acc = f(Wd, xd, xsd, acc_debug=debug if rep == 0 else None, workspace=ws)
+            check(y, acc, acc_ref, y_ref, mag, f"{what} {fmt} rep{rep}")
+    return acc_ref, y_ref, mag
+
+
+def test_config0_tiny(bc):
+    M, K, z = 256, 512, 0.42
+    s = datagen.config_seed(0, 0)
+    W, S = datagen.trits(s, M, K, z), datagen.scales(s, M, K)
+    x, xs = datagen.activations(s, 1, K)
+    run_all_formats(bc, W, S, x, xs, "config0")
+
+
+@pytest.mark.parametrize("M,K,B", [
+    (32, 128, 1), (1, 128, 1), (33, 256, 2), (100, 384, 3), (640, 2560, 1), (96, 6912, 1), (64, 2176, 5),
+    (256, 512, 16), (50, 1280, 8), (2560, 2560, 1), (160, 25600, 2), (320, 8192, 1),
+])
+def test_shapes_and_batches(bc, M, K, B):
+    W, S = datagen.trits(100 + M, M, K, 0.42), datagen.scales(100 + M, M, K)
+    x, xs = datagen.activations(100 + K, B, K)
+    run_all_formats(bc, W, S, x, xs, f"{M}x{K} B{B}")
+
+
+def test_degenerate_weights_and_activations(bc):
+    M, K = 96, 512
+    S = datagen.scales(7, M, K)
+    x, xs = datagen.activations(7, 2, K)
+    x[0, :] = -128                                       # the int8 minimum is accepted
+    x[1, ::2] = 127
+    for fill in (0, 1, -1):
+        run_all_formats(bc, np.full((M, K), fill, np.int8), S, x, xs, f"fill {fill}")
+    W = np.zeros((M, K), np.int8)
+    for k in (0, 31, 32, 127, 128, K - 1):
+        W[:] = 0
+        W[5, k] = -1
+        W[37, k] = 1
+        run_all_formats(bc, W, S, x, xs, f"single nonzero k={k}")
+    # all scales one, activation scale one: y is an exact integer
+    ones = np.full((M, K // 128), 0x3F80, np.uint16)
+    W = datagen.trits(8, M, K, 0.3)
+    acc_ref, y_ref, _ = run_all_formats(bc, W, ones, x, np.ones(2, np.float32), "unit scales")
+    assert np.array_equal(y_ref, acc_ref.sum(-1).astype(np.float64))
+    # dense rows next to empty rows (sign cursors far apart inside one tile)
+    W = np.zeros((M, K), np.int8)
+    W[::2] = datagen.trits(9, M // 2, K, 0.0)
+    run_all_formats(bc, W, S, x, xs, "alternating dense / empty rows")
+
+
+@pytest.mark.parametrize("z", [0.30, 0.375, 0.42, 0.47, 0.515])
+def test_density_sweep_small(bc, z):
+    M, K = 384, 1536
+    W, S = datagen.trits(11, M, K, z), datagen.scales(11, M, K)
+    x, xs = datagen.activations(11, 1, K)
+    run_all_formats(bc, W, S, x, xs, f"z={z}")
+
+
+def test_grouped_experts(bc):
+    E, M, K, top_k = 16, 768, 2048, 4
+    z = 0.3288
+    Ws = [datagen.trits(200 + e, M, K, z) for e in range(E)]
+    Ss = [datagen.scales(200 + e, M, K) for e in range(E)]
+    experts = bc.DeviceExperts([bc.bitcos_pack(Ws[e], Ss[e]).to_device() for e in range(E)])
+    for tokens in (1, 3, 16):
+        x, xs = datagen.activations(300 + tokens, tokens, K)
+        ids = datagen.expert_choices(300 + tokens, tokens, E, top_k)
+        pair_expert = ids.reshape(-1)
+        pair_xrow = np.repeat(np.arange(tokens, dtype=np.int32), top_k)
+        order, ge, gb, xr, mx = bc.group_pairs(pair_expert, pair_xrow)
+        acc_ref, y_ref, mag = oracle.grouped_dense(Ws, Ss, pair_expert[order], pair_xrow[order], x, xs)
+        ws = bc.make_workspace(M, K, copies=len(ge))
+        for rep in range(2):
+            y, acc = bc.bitcos_gemv_grouped(experts, dev(ge), dev(gb), dev(xr), mx, dev(x), dev(xs),
+                                            acc_debug=True, workspace=ws)
+            check(y, acc, acc_ref, y_ref, mag, f"grouped tokens={tokens} rep{rep}")
+
+
+def test_grouped_down_projection_shape(bc):
+    # K = 768 (six groups), per-pair activation rows
+    E, M, K = 4, 2048, 768
+    Ws = [datagen.trits(400 + e, M, K, 0.3288) for e in range(E)]
+    Ss = [datagen.scales(400 + e, M, K) for e in range(E)]
+    experts = bc.DeviceExperts([bc.bitcos_pack(Ws[e], Ss[e]).to_device() for e in range(E)])
+    pair_expert = np.array([3, 0, 3, 1, 0, 3], np.int32)
+    pair_xrow = np.arange(6, dtype=np.int32)
+    x, xs = datagen.activations(401, 6, K)
+    order, ge, gb, xr, mx = bc.group_pairs(pair_expert, pair_xrow)
+    acc_ref, y_ref, mag = oracle.grouped_dense(Ws, Ss, pair_expert[order], pair_xrow[order], x, xs)
+    y, acc = bc.bitcos_gemv_grouped(experts, dev(ge), dev(gb), dev(xr), mx, dev(x), dev(xs), acc_debug=True)
+    check(y, acc, acc_ref, y_ref, mag, "grouped down")
+
+
+def test_host_buffer_entry_point(bc):
+    M, K, B = 640, 2560, 4
+    W, S = datagen.trits(21, M, K, 0.4219), datagen.scales(21, M, K)
+    x, xs = datagen.activations(21, B, K)
+    acc_ref, y_ref, mag = oracle.gemv_dense(W, S, x, xs)
+    Wd = bc.bitcos_pack(W, S).to_device()
+    staging = torch.empty(bc.bitcos_gemv_host_staging_bytes(M, K, B), dtype=torch.uint8, device="cuda")
+    ws = bc.make_workspace(M, K)
+    xh = torch.from_numpy(x).pin_memory()
+    xsh = torch.from_numpy(xs).pin_memory()
+    yh = torch.empty((B, M), dtype=torch.float32).pin_memory()
+    bc.bitcos_gemv_host(Wd, xh.numpy(), xsh.numpy(), yh.numpy(), staging, ws)
+    err = np.abs(yh.numpy().astype(np.float64) - y_ref)
+    assert (err <= REL * mag).all()
+
+
+def test_sampled_outputs_at_full_size(bc):
+    """The largest layer shapes of the benchmark configurations, in the launch configuration
+    the benchmark times; the oracle checks a sample of rows it computes one by one."""
+    for (M, K, z, B) in ((6912, 2560, 0.4219, 1), (2560, 6912, 0.4219, 1), (5120, 25600, 0.4711, 2)):
+        W, S = datagen.trits(500 + M, M, K, z), datagen.scales(500 + M, M, K)
+        x, xs = datagen.activations(500 + M, B, K)
+        rows = np.unique(np.concatenate([np.arange(0, M, max(1, M // 97)), [M - 1, M - 32, 31, 32]]))
+        acc_ref, y_ref, mag = oracle.gemv_dense(W[rows], S[rows], x, xs)
+        xd, xsd = dev(x), dev(xs)
+        ws = bc.make_workspace(M, K)
+        st = bc.scales_tile(S, M, K)
+        for fmt, Wd, f in (("bitcos", bc.bitcos_pack(W, S).to_device(), bc.bitcos_gemv),
+                           ("trit5", bc.plain_to_device(bc.trit5_pack(W), st, M, K), bc.trit5_gemv),
+                           ("bit2", bc.plain_to_device(bc.bit2_pack(W), st, M, K), bc.bit2_gemv)):
+            y, acc = f(Wd, xd, xsd, acc_debug=True, workspace=ws)
+            torch.cuda.synchronize()
+            assert np.array_equal(acc.cpu().numpy()[:, rows], acc_ref), fmt
+            err = np.abs(y.cpu().numpy().astype(np.float64)[:, rows] - y_ref)
+            assert (err <= REL * mag).all(), fmt
