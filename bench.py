@@ -1,0 +1,452 @@
+#!/usr/bin/env python
+"""Benchmark of the BITCOS GEMV hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Workload (N = 1): one decode token (batch 1) through the seven ternary GEMVs of one
+BitNet-b1.58-2B-shaped decoder layer -- q/o 2560x2560, k/v 640x2560, gate/up 6912x2560,
+down 2560x6912 -- zero density 0.4219, group 128, bf16 group scales, int8 activations.
+A "step" is that whole layer pass: seven bitcos_gemv launches.  Inputs are seeded synthetic
+tensors; the packed layer is replicated so that consecutive steps never find their weights
+in L2 (rotation set > 4x L2).
+
+Prints one JSON line.  `value` is microseconds per token with everything resident in HBM;
+`e2e` is the same through the host-buffer entry point with the host<->device copies of the
+activations and outputs inside the timed region; `roofline` is the achieved algorithmic
+bytes per second of the bitcos_gemv kernel against the measured HBM peak; `cpu_baseline` is
+the CPU oracle timed on this machine's host cores.  With --gpus N every rank runs its own
+replica of the workload (the path has no cross-GPU exchange).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import datagen  # noqa: E402
+
+METRIC = "bitcos_gemv_us_per_token"
+UNIT = "us"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+def layer_config():
+    cfg = datagen.CONFIG_BITNET_2B
+    return cfg, "bitnet-b1.58-2B decoder layer, 7 GEMVs, batch 1, z=0.4219, group 128"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def generate_layer(cfg, config_index=1):
+    """Seeded trits, scales and activations for every matrix of the layer (host numpy)."""
+    out = []
+    for i, (name, M, K) in enumerate(cfg["shapes"]):
+        seed = datagen.config_seed(config_index, i)
+        W = datagen.trits(seed, M, K, cfg["z"])
+        S = datagen.scales(seed, M, K)
+        x, xs = datagen.activations(seed, 1, K)
+        out.append({"name": name, "M": M, "K": K, "W": W, "S": S, "x": x, "xs": xs})
+    return out
+
+
+def algorithmic_bytes(M, K, nnz, batch, fmt="bitcos"):
+    """Bytes one GEMV must move: packed weights + scales + offsets + activations + outputs."""
+    Mp = (M + 31) // 32 * 32
+    G = K // 128
+    scales = 2 * Mp * G
+    io = batch * (K + 4) + 4 * batch * M
+    if fmt == "bitcos":
+        return Mp * K // 8 + (nnz + 7) // 8 + scales + 4 * (Mp // 32 * G + 1) + io
+    if fmt == "trit5":
+        return Mp * ((26 * G + 3) // 4) * 4 + scales + io
+    return Mp * K // 4 + scales + io
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# ---------------------------------------------------------------------------------------------
+def oracle_layer_pass(layer, packed):
+    import oracle
+    for m, p in zip(layer, packed):
+        oracle.gemv_packed(oracle.FORMAT_BITCOS, p.bitmap, p.signs, p.tile_off, m["S"], m["x"], m["xs"], m["M"], m["K"])
+
+
+def oracle_pack_layer(layer):
+    import oracle
+    return [oracle.bitcos_pack(m["W"]) for m in layer]
+
+
+def run_reference(args):
+    """Times the oracle on the host cores.  Each step is a bounded sample of the layer pass: the
+    first rows of every matrix (a multiple of 32), sized from one calibration pass so that the
+    whole run stays within about two minutes; the reported time is scaled to the full layer."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, workload = layer_config()
+    layer = generate_layer(cfg)
+    packed = oracle_pack_layer(layer)
+    cores = oracle.threads()
+    t0 = time.perf_counter()
+    oracle_layer_pass(layer, packed)
+    full_pass = time.perf_counter() - t0
+    frac = min(1.0, 120.0 / (full_pass * (args.steps + args.warmup)))
+    sample = []
+    for m in layer:
+        rows = min(m["M"], max(32, int(m["M"] * frac) // 32 * 32))
+        sample.append({**m, "M": rows, "W": m["W"][:rows], "S": m["S"][:rows]})
+    frac = sum(s["M"] * s["K"] for s in sample) / sum(m["M"] * m["K"] for m in layer)
+    spacked = oracle_pack_layer(sample)
+    for _ in range(args.warmup):
+        oracle_layer_pass(sample, spacked)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_layer_pass(sample, spacked)
+    dt = time.perf_counter() - t0
+    us = dt / args.steps * 1e6 / frac
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": workload, "batch": 1},
+        "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"each step = the first {frac:.4f} of every matrix's rows (whole layer = 69.5 M "
+                                   "weights), time scaled to the full layer: BITCOS decode bit by bit, dense int32 "
+                                   "dot per group, double scale-and-sum"},
+        "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import paper_2609_16338_b200 as bc
+    from paper_2609_16338_b200 import build as lib_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        lib_build.build()
+    if dist is not None:
+        dist.barrier()
+    bc.load_library()
+    L = bc.load_library()
+
+    cfg, workload = layer_config()
+    layer = generate_layer(cfg)
+    host_packed = [bc.bitcos_pack(m["W"], m["S"]) for m in layer]
+    layer_bytes = sum(algorithmic_bytes(m["M"], m["K"], p.nnz, 1) for m, p in zip(layer, host_packed))
+    packed_bytes = sum(p.payload_bytes() for p in host_packed)
+    copies = max(2, int(np.ceil(4.2 * L2_BYTES / packed_bytes)))
+
+    base = [p.to_device() for p in host_packed]
+    replicas = [base] + [[w.clone() for w in base] for _ in range(copies - 1)]
+    xs_dev = [(torch.from_numpy(m["x"]).cuda(), torch.from_numpy(m["xs"]).cuda()) for m in layer]
+    ys = [torch.empty((1, m["M"]), dtype=torch.float32, device="cuda") for m in layer]
+    wss = [bc.make_workspace(m["M"], m["K"]) for m in layer]
+
+    def step(i):
+        rep = replicas[i % copies]
+        for j in range(len(layer)):
+            bc.bitcos_gemv(rep[j], xs_dev[j][0], xs_dev[j][1], y=ys[j], workspace=wss[j])
+
+    # parity spot check of what is being timed (first replica, against the oracle, rank 0)
+    step(0)
+    torch.cuda.synchronize()
+    if rank == 0:
+        import oracle
+        m = layer[1]
+        _, y_ref, mag = oracle.gemv_dense(m["W"], m["S"], m["x"], m["xs"])
+        err = np.abs(ys[1].cpu().numpy().astype(np.float64) - y_ref)
+        assert (err <= 1e-5 * mag).all(), "bench: bitcos_gemv disagrees with the oracle"
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+
+    # Capture the rotation as CUDA graphs so that the host's launch cost is not what is timed.
+    stream = torch.cuda.Stream()
+    graphs = {}
+
+    def capture(n_steps, first):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(n_steps):
+                    step(first + i)
+        return g
+
+    full, rem = divmod(args.steps, copies)
+    with torch.cuda.stream(stream):
+        if full:
+            graphs["full"] = capture(copies, 0)
+        if rem:
+            graphs["rem"] = capture(rem, 0)
+        for _ in range(2):
+            for g in graphs.values():
+                g.replay()
+        stream.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(full):
+            graphs["full"].replay()
+        if rem:
+            graphs["rem"].replay()
+        e1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    # keep the GPU busy a little longer so that the clock sampler sees it under load
+    t_end = time.time() + 0.6
+    with torch.cuda.stream(stream):
+        while time.time() < t_end:
+            (graphs.get("full") or graphs["rem"]).replay()
+            stream.synchronize()
+    clocks = sampler.stop()
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # ---- end to end: host buffers through bitcos_gemv_host, copies inside the timed region ----
+    stagings = [torch.empty(bc.bitcos_gemv_host_staging_bytes(m["M"], m["K"], 1), dtype=torch.uint8, device="cuda")
+                for m in layer]
+    xh = [torch.from_numpy(m["x"]).pin_memory() for m in layer]
+    xsh = [torch.from_numpy(m["xs"]).pin_memory() for m in layer]
+    yh = [torch.empty((1, m["M"]), dtype=torch.float32).pin_memory() for m in layer]
+    xh_np, xsh_np, yh_np = [t.numpy() for t in xh], [t.numpy() for t in xsh], [t.numpy() for t in yh]
+
+    def e2e_step(i):
+        rep = replicas[i % copies]
+        for j in range(len(layer)):
+            bc.bitcos_gemv_host(rep[j], xh_np[j], xsh_np[j], yh_np[j], stagings[j], wss[j])
+
+    e2e_steps = min(args.steps, 200)
+    for i in range(3):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_us = (time.perf_counter() - t0) / e2e_steps * 1e6
+    if dist is not None:
+        t = torch.tensor([e2e_us], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_us = float(t.item())
+    h2d = sum(m["K"] + 4 for m in layer)
+    d2h = sum(4 * m["M"] for m in layer)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-shape detail: each format on each shape, rotated copies, CUDA graph of 64 launches ----
+    detail = shape_detail(bc, torch, layer, host_packed, stream) if not args.no_detail else None
+
+    # ---- CPU baseline: the oracle on the host cores, bounded sample ----
+    import oracle
+    o_packed = oracle_pack_layer(layer)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        oracle_layer_pass(layer, o_packed)
+        reps += 1
+        if time.perf_counter() - t0 > 10.0 or reps >= 20:
+            break
+    cpu_us = (time.perf_counter() - t0) / reps * 1e6
+
+    peak, which = measured_peaks()
+    us_per_step = ms * 1e3 / args.steps
+    n_launch = 7 * args.steps
+    achieved = layer_bytes * args.steps / (ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": us_per_step / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": us_per_step / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": workload, "batch": 1, "weights": int(sum(m["M"] * m["K"] for m in layer)),
+                   "packed_bytes_per_step": int(packed_bytes), "algorithmic_bytes_per_step": int(layer_bytes),
+                   "l2_policy": f"{copies} rotated copies of the packed layer ({copies * packed_bytes / 2**20:.0f} MiB)"
+                                " so no step finds its weights in L2",
+                   "launch": "CUDA graphs of the rotation, replayed on one stream", "replicas": world},
+        "achieved_gbs": achieved,
+        "frac_of_8tbs": achieved / 8000.0,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_source": f"{which} (STREAM-style copy)",
+                     "kernel": "gemv_kernel<bitcos, 1 token>", "launches": n_launch,
+                     "avg_launch_us": ms * 1e3 / n_launch,
+                     "algorithmic_bytes_per_launch": layer_bytes / 7.0},
+        "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                         "sample": f"{reps} full layer passes (7 GEMVs, 69.5 M weights each): BITCOS decode bit by "
+                                   "bit, dense int32 dot per group, double scale-and-sum"},
+        "e2e": {"value": e2e_us / world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "path": "bitcos_gemv_host per GEMV: pinned x -> device, kernel, y -> pinned host, "
+                                            "stream wait"},
+        "gpu_launches": n_launch,
+        "clocks": clocks,
+    }
+    if detail is not None:
+        line["shapes"] = detail
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def shape_detail(bc, torch, layer, host_packed, stream, launches=64):
+    """Per distinct shape: microseconds and GB/s of bitcos / trit5 / bit2 on identical weights."""
+    peak, _ = measured_peaks()
+    seen, out = set(), []
+    for m, p in zip(layer, host_packed):
+        key = (m["M"], m["K"])
+        if key in seen:
+            continue
+        seen.add(key)
+        M, K = key
+        st = bc.scales_tile(m["S"], M, K)
+        fmts = {"bitcos": (p.to_device(), bc.bitcos_gemv), "trit5": (bc.plain_to_device(bc.trit5_pack(m["W"]), st, M, K), bc.trit5_gemv),
+                "bit2": (bc.plain_to_device(bc.bit2_pack(m["W"]), st, M, K), bc.bit2_gemv)}
+        x, xs = torch.from_numpy(m["x"]).cuda(), torch.from_numpy(m["xs"]).cuda()
+        y = torch.empty((1, M), dtype=torch.float32, device="cuda")
+        ws = bc.make_workspace(M, K)
+        row = {"name": m["name"], "M": M, "K": K}
+        for name, (Wd, f) in fmts.items():
+            nbytes = algorithmic_bytes(M, K, p.nnz, 1, name)
+            n_copies = max(2, int(np.ceil(4.2 * L2_BYTES / Wd.payload_bytes())))
+            reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
+            f(reps[0], x, xs, y=y, workspace=ws)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                with torch.cuda.graph(g, stream=stream):
+                    for i in range(launches):
+                        f(reps[i % n_copies], x, xs, y=y, workspace=ws)
+                g.replay()
+                stream.synchronize()
+                times = []
+                for _ in range(5):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    g.replay()
+                    e1.record(stream)
+                    stream.synchronize()
+                    times.append(e0.elapsed_time(e1) * 1e3 / launches)
+            us = float(np.median(times))
+            row[name] = {"us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak, "bytes": int(nbytes)}
+            del reps, g
+        row["speedup_vs_trit5"] = row["trit5"]["us"] / row["bitcos"]["us"]
+        row["byte_ratio_trit5"] = row["trit5"]["bytes"] / row["bitcos"]["bytes"]
+        row["speedup_vs_bit2"] = row["bit2"]["us"] / row["bitcos"]["us"]
+        row["byte_ratio_bit2"] = row["bit2"]["bytes"] / row["bitcos"]["bytes"]
+        out.append(row)
+        torch.cuda.empty_cache()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-detail", action="store_true", help="skip the per-shape / per-format table")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps is None:
+            args.steps = 3
+        run_reference(args)
+    else:
+        if args.steps is None:
+            args.steps = 2000
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -499,18 +499,35 @@ size_t smem_bytes(int fmt, int nw, int nb) {
     return (fmt == kBit2 ? 0 : kLutBytes) + static_cast<size_t>(nw) * nb * kRows * sizeof(float);
 }
 
-template <typename Kernel>
-int grid_for(Kernel kernel, int threads, size_t smem, int64_t units, int *grid) {
-    int dev = 0, sms = 0, per_sm = 0;
+// Number of thread blocks to launch: min(units, SMs x resident blocks per SM).  The
+// occupancy query and the opt-in to large dynamic shared memory are done on the first call
+// for a given kernel (one cache per kernel instantiation), block size and device, and remembered (so that first call must not
+// happen during stream capture; later calls only read the cache).
+template <auto kernel>
+int grid_for(int threads, size_t smem, int64_t units, int *grid) {
+    constexpr int kMaxDev = 32;
+    static int cache[kMaxDev][kMaxWarps + 1][2];      // [device][warps][0: blocks per SM, 1: SMs]; 0 = unknown
+    int dev = 0;
     int rc = check_cuda(cudaGetDevice(&dev));
     if (rc) return rc;
-    rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    if (rc) return rc;
-    rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    if (rc) return rc;
-    rc = check_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
-    if (rc) return rc;
-    if (per_sm < 1) per_sm = 1;
+    const int nw = threads / 32;
+    int per_sm = 0, sms = 0;
+    if (dev < kMaxDev && cache[dev][nw][0] > 0) {
+        per_sm = cache[dev][nw][0];
+        sms = cache[dev][nw][1];
+    } else {
+        rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        if (rc) return rc;
+        rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes + 32 * 1024));
+        if (rc) return rc;
+        rc = check_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
+        if (rc) return rc;
+        if (per_sm < 1) per_sm = 1;
+        if (dev < kMaxDev) {
+            cache[dev][nw][1] = sms;
+            cache[dev][nw][0] = per_sm;
+        }
+    }
     const int64_t cap = static_cast<int64_t>(sms) * per_sm;
     *grid = static_cast<int>(units < cap ? units : cap);
     return BITCOS_OK;
@@ -520,7 +537,7 @@ template <int FMT, int NB>
 int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
     const size_t smem = smem_bytes(FMT, pl.NW, NB);
     int grid = 1;
-    int rc = grid_for(gemv_kernel<FMT, NB>, pl.NW * 32, smem, pl.units, &grid);
+    int rc = grid_for<gemv_kernel<FMT, NB>>(pl.NW * 32, smem, pl.units, &grid);
     if (rc) return rc;
     gemv_kernel<FMT, NB><<<grid, pl.NW * 32, smem, stream>>>(pr, pl);
     return check_cuda(cudaGetLastError());
@@ -539,7 +556,7 @@ template <int NB>
 int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int n_groups, cudaStream_t stream) {
     const size_t smem = smem_bytes(kBitcos, pl.NW, NB);
     int grid = 1;
-    int rc = grid_for(gemv_grouped_kernel<NB>, pl.NW * 32, smem, pl.units, &grid);
+    int rc = grid_for<gemv_grouped_kernel<NB>>(pl.NW * 32, smem, pl.units, &grid);
     if (rc) return rc;
     // the grid's x extent is shared by all groups: spread the machine over them
     int gx = (grid + n_groups - 1) / n_groups;
