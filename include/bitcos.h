@@ -134,14 +134,21 @@ typedef struct bitcos_weights {
     int64_t K;
 } bitcos_weights;
 
-/* Scratch memory the three GEMV entry points need for an M x K matrix (the same value for
- * all formats and batches): partial row sums of reduction segments that were spread over
- * several thread blocks, and one arrival counter per row block.  The caller allocates it
- * on the device, fills it with zeros ONCE (bitcos_workspace_init), and may reuse it for
- * any later call whose requirement is not larger: every call leaves the counters zero.
- * Two calls that may run at the same time must not share a workspace. */
+/* Scratch memory the GEMV entry points need for an M x K matrix (the same value for all
+ * formats and batches): a 256-byte header (word 0 = status), one arrival counter per row
+ * block, and the partial row sums of reduction segments that were spread over several
+ * thread blocks.  The caller allocates it on the device, fills it with zeros ONCE
+ * (bitcos_workspace_init), and may reuse it for any later call whose requirement is not
+ * larger: every call leaves the counters zero.  Two calls that may run at the same time
+ * must not share a workspace. */
 size_t bitcos_gemv_workspace_bytes(int64_t M, int64_t K);
 int bitcos_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Every wait inside the kernels (on the arrival of an asynchronous copy) is bounded; if one
+ * ever runs out, the thread block stops working on the call and sets the workspace's status
+ * word to 1 instead of hanging.  This call copies that word back (it waits for the stream):
+ * *status == 0 means every call that used the workspace so far completed normally. */
+int bitcos_workspace_status(const void *workspace, void *cuda_stream, int *status);
 
 /* y[b][m] for b < batch, m < M from a BITCOS matrix (steps of Section II-B..II-D on the GPU:
  * entry offset + running population count locate each row's sign window, a 256-entry

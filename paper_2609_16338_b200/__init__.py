@@ -32,5 +32,6 @@ from .binding import (  # noqa: F401
     trit5_gemv,
     trit5_pack,
     trit5_unpack,
+    workspace_status,
     EXPORTED_SYMBOLS,
 )

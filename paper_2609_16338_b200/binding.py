@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_status_string", "bitcos_last_cuda_error", "bitcos_pack_sizes", "bitcos_count_nnz", "bitcos_pack",
     "bitcos_unpack", "bitcos_scales_tile", "bitcos_scales_untile", "trit5_pack_sizes", "trit5_pack",
     "trit5_unpack", "bit2_pack_sizes", "bit2_pack", "bit2_unpack", "bitcos_gemv_workspace_bytes",
-    "bitcos_workspace_init", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
+    "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host",
 ]
 
@@ -72,6 +72,7 @@ def load_library():
     L.bitcos_gemv_workspace_bytes.restype = sz
     L.bitcos_gemv_workspace_bytes.argtypes = [i64, i64]
     L.bitcos_workspace_init.argtypes = [vp, sz, vp]
+    L.bitcos_workspace_status.argtypes = [vp, vp, C.POINTER(C.c_int)]
     L.bitcos_gemv.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, vp, sz, vp]
     for name in ("trit5_gemv", "bit2_gemv"):
         getattr(L, name).argtypes = [vp, vp, i64, i64, vp, vp, C.c_int, vp, vp, vp, sz, vp]
@@ -255,6 +256,14 @@ def make_workspace(M: int, K: int, device="cuda", copies: int = 1):
     _check(load_library().bitcos_workspace_init(C.c_void_p(ws.data_ptr()), ws.numel(), _stream()),
            "bitcos_workspace_init")
     return ws
+
+
+def workspace_status(workspace) -> int:
+    """0 if every call that used this workspace completed normally (waits for the stream)."""
+    v = C.c_int(0)
+    _check(load_library().bitcos_workspace_status(C.c_void_p(workspace.data_ptr()), _stream(), C.byref(v)),
+           "bitcos_workspace_status")
+    return int(v.value)
 
 
 def _outputs(M, K, batch, y, acc_debug, device):

@@ -1,22 +1,28 @@
 // Device side of the BITCOS library: ternary GEMV kernels for sm_100a and their C entry
-// points (bitcos_gemv, trit5_gemv, bit2_gemv, bitcos_gemv_grouped).
+// points (bitcos_gemv, trit5_gemv, bit2_gemv, bitcos_gemv_grouped, bitcos_gemv_host).
 //
 // Work decomposition (all formats).  Rows are handled 32 at a time (a "row block"), one
 // row per lane, so that the activations a warp needs are the same for all of its lanes
-// and arrive by broadcast loads; the reduction is cut into groups of 128.  A warp runs over
-// `gpw` consecutive groups of one row block, keeping one fp32 partial sum per lane and
-// token.  The S = (K/128)/gpw runs of a row block are spread over SC warps of one thread
-// block and, if S > SC, over CS thread blocks; partial sums are added in a fixed order
-// (shared memory inside a block, then a scratch buffer and an arrival counter across
-// blocks), so results do not depend on scheduling.
+// and arrive by broadcast reads; the reduction is cut into groups of 128.  A tile is one
+// group of one row block (32 x 128 weights); one warp decodes one tile at a time.  An
+// "item" is a run of up to 20 consecutive tiles -- CG groups of one row block, or several
+// whole row blocks when a row has few groups -- and is what one thread block processes per
+// pipeline stage: because tiles are stored in that order, an item's bitmap words, sign bits
+// and scales are three contiguous byte ranges, fetched with three bulk asynchronous copies
+// (cp.async.bulk + mbarrier) into a ring of shared-memory stages while earlier stages are
+// being decoded.  Thread blocks are persistent and walk the item list with a fixed stride.
+// Row sums are formed in a fixed order (groups ascending inside a block through shared
+// memory; column blocks ascending through a scratch buffer and an arrival counter), so
+// results do not depend on scheduling.
 //
 // BITCOS decode (paper Section II-D, Eq. 4, adapted): the GPU has no bit-deposit
 // instruction, so four weights at a time are rebuilt from a (presence nibble, next four
 // sign bits) key through a 256-entry table held in shared memory, replicated once per lane
 // so that lookups never conflict.  Entries are the four weights as int8 (w = p - 2n, Eq. 2)
 // and feed dp4a directly.  A lane's position in the sign vector is the tile's entry offset
-// plus a warp prefix sum over the rows' population counts; inside a row the window is
-// shifted by the number of sign bits each nibble consumed.
+// plus a warp prefix sum over the rows' population counts; the four 32-bit presence words of
+// a lane's row are decoded as four independent chains, each shifting its own sign window by
+// the number of sign bits a nibble consumed.
 #include "bitcos.h"
 
 #include <cuda_runtime.h>
@@ -27,8 +33,10 @@ namespace {
 
 constexpr int kGroup = BITCOS_GROUP;
 constexpr int kRows = BITCOS_TILE_ROWS;
-constexpr int kMaxWarps = 16;           // warps per thread block
-constexpr int kLutBytes = 64 * 1024;    // replicated lookup tables (BITCOS, five-trit)
+constexpr int kMaxWarps = 20;             // warps per thread block = tiles per item
+constexpr int kStages = 3;                // shared-memory ring depth
+constexpr int kLutBytes = 64 * 1024;      // replicated lookup tables (BITCOS, five-trit)
+constexpr uint32_t kSpinLimit = 1u << 22; // bound on mbarrier polls before giving up
 
 enum Format { kBitcos = 0, kTrit5 = 1, kBit2 = 2 };
 
@@ -80,20 +88,51 @@ constexpr Lut256x2 make_trit5_lut() {
     return t;
 }
 
-__constant__ Lut256 c_nibble_lut = make_nibble_lut();
-__constant__ Lut256x2 c_trit5_lut = make_trit5_lut();
+// The tables as they sit in shared memory, replicated once per lane (32 copies) so that a warp's
+// 32 lookups always fall into 32 different banks.  They live in global memory in that final
+// form and each thread block fetches its copy with one bulk asynchronous copy.
+struct LutBig {
+    uint32_t v[kLutBytes / 4];
+};
+
+// BITCOS: byte address = key * 256 + sub * 128 + lane * 4;
+//   sub 0 ("even" nibbles): key = (s << 4) | m;  sub 1 ("odd" nibbles): key = (m << 4) | s,
+// so that a presence BYTE placed in address bits 8..15 needs only its other nibble replaced
+// by the four sign bits.
+constexpr LutBig make_bitcos_lut() {
+    const Lut256 base = make_nibble_lut();
+    LutBig t{};
+    for (int idx = 0; idx < kLutBytes / 4; ++idx) {
+        const int key = idx >> 6, sub = (idx >> 5) & 1;
+        const int src = sub ? (((key & 15) << 4) | (key >> 4)) : key;
+        t.v[idx] = base.v[src];
+    }
+    return t;
+}
+
+// Five-trit: byte address = byte value * 256 + lane * 8 (lo word, hi word).
+constexpr LutBig make_trit5_big() {
+    const Lut256x2 base = make_trit5_lut();
+    LutBig t{};
+    for (int idx = 0; idx < kLutBytes / 4; ++idx) {
+        const int key = idx >> 6;
+        t.v[idx] = (idx & 1) ? base.hi[key] : base.lo[key];
+    }
+    return t;
+}
+
+__device__ __align__(128) const LutBig g_bitcos_lut = make_bitcos_lut();
+__device__ __align__(128) const LutBig g_trit5_lut = make_trit5_big();
 
 // ---------------------------------------------------------------------------------------------
-// Launch plan.
+// Launch plan and problem description.
 // ---------------------------------------------------------------------------------------------
 struct Plan {
-    int gpw;        // groups per warp run
-    int S;          // runs per row block
-    int SC;         // runs of a row block inside one thread block
-    int CS;         // thread blocks per row block
-    int RBC;        // row blocks per thread block (> 1 only if CS == 1)
-    int NW;         // warps per thread block
-    int64_t units;  // work units
+    int CG;          // groups per column block
+    int CS;          // column blocks per row
+    int RBC;         // row blocks per item (1 unless CS == 1)
+    int NW;          // warps per thread block = CG * RBC
+    int64_t items;   // ceil(RB / RBC) * CS
 };
 
 struct Problem {
@@ -108,6 +147,7 @@ struct Problem {
     int32_t *acc_debug;
     float *partial;
     unsigned int *counters;
+    unsigned int *status;      // device word set to 1 if an mbarrier wait ran out
     int64_t M, K;
     int G, RB;
     int nb;                    // tokens in this call / group
@@ -127,57 +167,79 @@ inline int64_t padded_rows(int64_t M) { return (M + kRows - 1) / kRows * kRows; 
 Plan make_plan(int64_t M, int64_t K) {
     const int G = static_cast<int>(K / kGroup);
     const int64_t RB = padded_rows(M) / kRows;
-    const int64_t target = 148 * 32;
-    // Longest run that still yields enough warps to fill the machine; else one group per warp.
-    int best = 1;
-    for (int d = 1; d <= G; ++d) {
-        if (G % d) continue;
-        if (RB * (G / d) >= target) best = d;
-    }
     Plan p{};
-    auto derive = [&](int d) {
-        p.gpw = d;
-        p.S = G / d;
-        if (p.S <= kMaxWarps) {
-            p.SC = p.S;
-            p.CS = 1;
-            int64_t r = kMaxWarps / p.S;
-            if (r > RB) r = RB;
-            if (r < 1) r = 1;
-            p.RBC = static_cast<int>(r);
-        } else {
-            int sc = 1;
-            for (int c = 1; c <= kMaxWarps; ++c)
-                if (p.S % c == 0) sc = c;
-            p.SC = sc;
-            p.CS = p.S / sc;
-            p.RBC = 1;
-        }
-        p.NW = p.SC * p.RBC;
-    };
-    derive(best);
-    if (p.NW < 4) {
-        // S has no useful divisor: fall back to the divisor of G giving the fullest block
-        int pick = best, pick_nw = p.NW;
-        for (int d = 1; d <= G; ++d) {
-            if (G % d) continue;
-            derive(d);
-            if (p.NW > pick_nw) { pick = d; pick_nw = p.NW; }
-        }
-        derive(pick);
+    const int blocks = (G + kMaxWarps - 1) / kMaxWarps;
+    p.CG = (G + blocks - 1) / blocks;
+    p.CS = (G + p.CG - 1) / p.CG;
+    p.RBC = 1;
+    if (p.CS == 1) {
+        int64_t r = kMaxWarps / p.CG;
+        if (r > RB) r = RB;
+        if (r < 1) r = 1;
+        p.RBC = static_cast<int>(r);
     }
-    p.units = ((RB + p.RBC - 1) / p.RBC) * p.CS;
+    p.NW = p.CG * p.RBC;
+    p.items = ((RB + p.RBC - 1) / p.RBC) * p.CS;
     return p;
 }
 
+// workspace: [0, 256) header (word 0 = status), arrival counters, partial sums
+constexpr size_t kHeaderBytes = 256;
 size_t counters_bytes(int64_t RB) { return static_cast<size_t>((RB * 4 + 255) / 256 * 256); }
 
 size_t workspace_bytes_for(int64_t M, int64_t K) {
     const Plan p = make_plan(M, K);
     const int64_t RB = padded_rows(M) / kRows;
-    size_t b = counters_bytes(RB);
+    size_t b = kHeaderBytes + counters_bytes(RB);
     if (p.CS > 1) b += static_cast<size_t>(RB) * p.CS * BITCOS_MAX_BATCH * kRows * sizeof(float);
     return b;
+}
+
+// Shared-memory layout of a thread block (byte offsets).
+struct SmemLayout {
+    uint32_t lut;        // lookup tables (0 bytes for 2-bit)
+    uint32_t stage;      // stage 0
+    uint32_t stage_bytes;
+    uint32_t payload_cap, sign_cap, scale_cap;   // per-stage capacities
+    uint32_t x;          // activations of the block's groups, [nb][CG * 128]
+    uint32_t red;        // [NW][NB][32] floats
+    uint32_t bar;        // kStages mbarriers, then (at +64) per-stage sign base words
+    uint32_t total;
+};
+
+__host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+__host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G, int nbmax) {
+    SmemLayout L{};
+    uint32_t off = 0;
+    L.lut = off;
+    off += (fmt == kBit2) ? 0 : kLutBytes;
+    const uint32_t tiles = static_cast<uint32_t>(pl.NW);
+    if (fmt == kBitcos) {
+        L.payload_cap = tiles * 512;
+        L.sign_cap = tiles * 512 + 64;
+    } else if (fmt == kTrit5) {
+        const uint32_t WPR = (26u * static_cast<uint32_t>(G) + 3) / 4;
+        // whole rows when CS == 1, else at most CG groups (+1 shared word) of one row block
+        L.payload_cap = (pl.CS == 1) ? static_cast<uint32_t>(pl.RBC) * WPR * 128
+                                     : ((26u * static_cast<uint32_t>(pl.CG) + 3) / 4 + 1) * 128;
+        L.sign_cap = 0;
+    } else {
+        L.payload_cap = tiles * 1024;
+        L.sign_cap = 0;
+    }
+    L.scale_cap = tiles * 64;
+    L.stage = off;
+    L.stage_bytes = align_up(L.payload_cap + L.sign_cap + L.scale_cap, 128);
+    off += L.stage_bytes * kStages;
+    L.x = off;
+    off += align_up(static_cast<uint32_t>(nbmax) * static_cast<uint32_t>(pl.CG) * kGroup, 128);
+    L.red = off;
+    off += tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
+    L.bar = off;
+    off += 128;
+    L.total = off;
+    return L;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -197,102 +259,106 @@ __device__ __forceinline__ int dp4a_us(uint32_t a, int b, int c) {
 }
 __device__ __forceinline__ float bf16_to_float(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
 
-// Replicated table layout, byte address = key * 256 + sub * 128 + lane * 4:
-//   sub 0 ("even" nibbles): key = (s << 4) | m;  sub 1 ("odd" nibbles): key = (m << 4) | s.
-// so that a presence BYTE placed in address bits 8..15 needs only its other nibble replaced
-// by the four sign bits.
-__device__ __forceinline__ void build_bitcos_lut(uint8_t *smem) {
-    uint32_t *lut = reinterpret_cast<uint32_t *>(smem);
-    for (int idx = threadIdx.x; idx < kLutBytes / 4; idx += blockDim.x) {
-        const int key = idx >> 6, sub = (idx >> 5) & 1;
-        const int src = sub ? (((key & 15) << 4) | (key >> 4)) : key;
-        lut[idx] = c_nibble_lut.v[src];
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bulk asynchronous copy global -> shared; size and both addresses are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// Waits for the given phase parity with a bounded number of polls; false if it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
     }
+    return false;
 }
 
-// byte address = byte value * 256 + lane * 8 (lo, hi)
-__device__ __forceinline__ void build_trit5_lut(uint8_t *smem) {
-    uint32_t *lut = reinterpret_cast<uint32_t *>(smem);
-    for (int idx = threadIdx.x; idx < kLutBytes / 4; idx += blockDim.x) {
-        const int key = idx >> 6;
-        lut[idx] = (idx & 1) ? c_trit5_lut.hi[key] : c_trit5_lut.lo[key];
-    }
+// d = (a & c) | (b & ~c): one LOP3
+__device__ __forceinline__ uint32_t bit_select(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xE4;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
 }
 
-// One 32-bit presence word: eight (nibble, sign window) lookups.  `sw` holds the sign bits
-// of this word's non-zeros from bit 0 upwards.  lane4 = lane * 4.
-__device__ __forceinline__ void bitcos_decode_word(uint32_t P, uint32_t sw, const uint8_t *lut, uint32_t lane4,
-                                                   int *w) {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        // address bits 0..6 = lane * 4, bits 8..15 = presence byte k
-        const uint32_t R = __byte_perm(P, lane4, 0x6504 | (k << 4));
-        uint32_t off = ((sw << 12) & 0xF000u) | (R & 0x0FFFu);
-        int e = static_cast<int>(lds32(lut, off));
-        w[2 * k] = e;
-        sw >>= __dp4a(e, e, 0);                      // number of non-zeros = sign bits consumed
-        off = ((sw << 8) & 0x0F00u) | (R & 0xF0FFu);
-        e = static_cast<int>(lds32(lut + 128, off));
-        w[2 * k + 1] = e;
-        sw >>= __dp4a(e, e, 0);
-    }
-}
+// ---------------------------------------------------------------------------------------------
+// Tile decoders.  For the lane's row they produce either the int32 accumulator against one
+// token (FUSED: decode fused with dp4a) or the 32 int8x4 words of the row.
+// ---------------------------------------------------------------------------------------------
 
-// Decodes tile t (32 rows x 128 k) of a BITCOS matrix: lane = row.  w[i] = weights 4i..4i+3 as int8.
-__device__ __forceinline__ void bitcos_decode_tile(const Problem &pr, int64_t t, int lane, const uint8_t *lut,
-                                                   int (&w)[32]) {
-    const uint4 bm = __ldcs(reinterpret_cast<const uint4 *>(pr.payload) + t * kRows + lane);
-    const int c0 = __popc(bm.x), c1 = __popc(bm.y), c2 = __popc(bm.z), c3 = __popc(bm.w);
-    const int c = c0 + c1 + c2 + c3;
-    int incl = c;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-        if (lane >= d) incl += v;
-    }
-    const uint32_t cursor = __ldg(pr.tile_off + t) + static_cast<uint32_t>(incl - c);
-    const uint32_t *sp = pr.signs + (cursor >> 5);
-    const uint32_t s0 = __ldg(sp), s1 = __ldg(sp + 1), s2 = __ldg(sp + 2), s3 = __ldg(sp + 3), s4 = __ldg(sp + 4);
-    const uint32_t sh = cursor & 31u;
+// BITCOS: bm = the row's four presence words, sp = the stage's sign words at the word holding the
+// row's first sign bit, sh = bit offset inside that word.
+template <bool FUSED>
+__device__ __forceinline__ int bitcos_decode_row(const uint4 bm, const uint32_t *sp, uint32_t sh, const uint8_t *lut,
+                                                 uint32_t lane4, const int4 *xg, int (&w)[32]) {
+    const int c0 = __popc(bm.x), c1 = __popc(bm.y), c2 = __popc(bm.z);
+    const uint32_t s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3], s4 = sp[4];
     uint32_t a0 = __funnelshift_r(s0, s1, sh), a1 = __funnelshift_r(s1, s2, sh);
     uint32_t a2 = __funnelshift_r(s2, s3, sh), a3 = __funnelshift_r(s3, s4, sh);
-    const uint32_t lane4 = static_cast<uint32_t>(lane) * 4u;
-    bitcos_decode_word(bm.x, a0, lut, lane4, w);
+    uint32_t S[4];
+    S[0] = a0;
     a0 = __funnelshift_rc(a0, a1, c0);
     a1 = __funnelshift_rc(a1, a2, c0);
     a2 = __funnelshift_rc(a2, a3, c0);
-    bitcos_decode_word(bm.y, a0, lut, lane4, w + 8);
+    S[1] = a0;
     a0 = __funnelshift_rc(a0, a1, c1);
     a1 = __funnelshift_rc(a1, a2, c1);
-    bitcos_decode_word(bm.z, a0, lut, lane4, w + 16);
-    a0 = __funnelshift_rc(a0, a1, c2);
-    bitcos_decode_word(bm.w, a0, lut, lane4, w + 24);
+    S[2] = a0;
+    S[3] = __funnelshift_rc(a0, a1, c2);
+    const uint32_t P[4] = {bm.x, bm.y, bm.z, bm.w};
+    int acc[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        int4 xq[4];
+        if (FUSED) {
+            // activation words 8j + 2k and 8j + 2k + 1 for the four chains j
+#pragma unroll
+            for (int j = 0; j < 4; ++j) xq[j] = xg[2 * j + (k >> 1)];
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            // address bits 0..6 = lane * 4, bits 8..15 = presence byte k of word j (bits 16.. are 0)
+            const uint32_t R = __byte_perm(P[j], lane4, 0x6504 | (k << 4));
+            uint32_t off = bit_select(S[j] << 12, R, 0xF000u);     // sign nibble over the odd presence nibble
+            int e = static_cast<int>(lds32(lut, off));
+            if (FUSED) acc[j] = __dp4a(e, (k & 1) ? xq[j].z : xq[j].x, acc[j]);
+            else w[8 * j + 2 * k] = e;
+            S[j] >>= __dp4a(e, e, 0);                    // non-zeros in the nibble = sign bits consumed
+            off = bit_select(S[j] << 8, R, 0x0F00u);               // sign nibble over the even presence nibble
+            e = static_cast<int>(lds32(lut + 128, off));
+            if (FUSED) acc[j] = __dp4a(e, (k & 1) ? xq[j].w : xq[j].y, acc[j]);
+            else w[8 * j + 2 * k + 1] = e;
+            S[j] >>= __dp4a(e, e, 0);
+        }
+    }
+    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
 }
 
-// Five-trit tile: the 26 bytes of group g of the lane's row start at byte 26g of the row
-// string, i.e. at word (26g)/4 with byte offset 0 (g even) or 2 (g odd): seven words.
-__device__ __forceinline__ void trit5_decode_tile(const Problem &pr, int64_t rb, int g, int lane, const uint8_t *lut,
-                                                  int (&w)[32]) {
-    const int64_t WPR = (26 * static_cast<int64_t>(pr.G) + 3) / 4;
-    const int q0 = (26 * g) >> 2;
-    const uint32_t *src = pr.payload + (rb * WPR + q0) * kRows + lane;
-    uint32_t wd[7];
-#pragma unroll
-    for (int i = 0; i < 7; ++i) {
-        // row strings are padded to whole words, so word q0 + 6 always exists
-        wd[i] = __ldcs(src + static_cast<int64_t>(i) * kRows);
-    }
-    const uint32_t lane8 = static_cast<uint32_t>(lane) * 8u;
-    const int odd = g & 1;
+// Five-trit: wd = the seven words that hold the row's 26 bytes, odd = byte offset 2 (odd group).
+__device__ __forceinline__ void trit5_decode_row(const uint32_t (&wd)[7], int odd, const uint8_t *lut, uint32_t lane8,
+                                                 int (&w)[32]) {
     uint32_t lo[26], hi[26];
 #pragma unroll
     for (int j = 0; j < 26; ++j) {
-        // byte j of the block = byte (j + 2*odd) of the seven loaded words
         const int be = j, bo = j + 2;
-        const uint32_t we = wd[be >> 2], wo = wd[bo >> 2];
-        const uint32_t word = odd ? wo : we;
+        const uint32_t word = odd ? wd[bo >> 2] : wd[be >> 2];
         const uint32_t sel = odd ? (0x6504u | ((bo & 3) << 4)) : (0x6504u | ((be & 3) << 4));
-        const uint32_t off = __byte_perm(word, lane8, sel);   // byte * 256 + lane * 8
+        const uint32_t off = __byte_perm(word, lane8, sel);    // byte * 256 + lane * 8
         const uint2 e = lds64(lut, off);
         lo[j] = e.x;
         hi[j] = e.y;
@@ -309,11 +375,9 @@ __device__ __forceinline__ void trit5_decode_tile(const Problem &pr, int64_t rb,
     w[31] = static_cast<int>(__byte_perm(hi[24], lo[25], 0x6543));
 }
 
-// 2-bit tile: eight words per lane; w[4q + j] keeps pair j of every byte of word q in place
-// (value = code * 4^j), to be multiplied with activation word 4q + j.
-__device__ __forceinline__ void bit2_decode_tile(const Problem &pr, int64_t t, int lane, int (&w)[32]) {
-    const uint4 *src = reinterpret_cast<const uint4 *>(pr.payload) + (t * 2) * kRows + lane;
-    const uint4 v0 = __ldcs(src), v1 = __ldcs(src + kRows);
+// 2-bit: w[4q + j] keeps pair j of every byte of word q in place (value = code * 4^j), to be
+// multiplied with activation word 4q + j.
+__device__ __forceinline__ void bit2_decode_row(const uint4 v0, const uint4 v1, int (&w)[32]) {
     const uint32_t wd[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
     for (int q = 0; q < 8; ++q)
@@ -321,18 +385,17 @@ __device__ __forceinline__ void bit2_decode_tile(const Problem &pr, int64_t t, i
         for (int j = 0; j < 4; ++j) w[4 * q + j] = static_cast<int>(wd[q] & (0x03030303u << (2 * j)));
 }
 
-// int32 accumulator of one row (lane) and group against token activations xg[0..127].
+// int32 accumulator of one row (lane) and group against token activations xg[0..127] (shared memory).
 template <int FMT>
-__device__ __forceinline__ int contract(const int (&w)[32], const int8_t *xg, int lane) {
-    const int4 *xv = reinterpret_cast<const int4 *>(xg);
+__device__ __forceinline__ int contract(const int (&w)[32], const int4 *xg, int lane) {
     if (FMT == kBit2) {
         int a0 = 0, a1 = 0, a2 = 0, a3 = 0;
         // sum of the group's activations, needed because the stored code is weight + 1
-        int sx = __dp4a(0x01010101, __ldg(reinterpret_cast<const int *>(xg) + lane), 0);
+        int sx = __dp4a(0x01010101, reinterpret_cast<const int *>(xg)[lane], 0);
         sx = __reduce_add_sync(0xFFFFFFFFu, sx);
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            const int4 xq = __ldg(xv + q);
+            const int4 xq = xg[q];
             a0 = dp4a_us(static_cast<uint32_t>(w[4 * q + 0]), xq.x, a0);
             a1 = dp4a_us(static_cast<uint32_t>(w[4 * q + 1]), xq.y, a1);
             a2 = dp4a_us(static_cast<uint32_t>(w[4 * q + 2]), xq.z, a2);
@@ -340,94 +403,268 @@ __device__ __forceinline__ int contract(const int (&w)[32], const int8_t *xg, in
         }
         return a0 + (a1 >> 2) + (a2 >> 4) + (a3 >> 6) - sx;
     } else {
-        int a = 0;
+        int a0 = 0, a1 = 0, a2 = 0, a3 = 0;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            const int4 xq = __ldg(xv + q);
-            a = __dp4a(w[4 * q + 0], xq.x, a);
-            a = __dp4a(w[4 * q + 1], xq.y, a);
-            a = __dp4a(w[4 * q + 2], xq.z, a);
-            a = __dp4a(w[4 * q + 3], xq.w, a);
+            const int4 xq = xg[q];
+            a0 = __dp4a(w[4 * q + 0], xq.x, a0);
+            a1 = __dp4a(w[4 * q + 1], xq.y, a1);
+            a2 = __dp4a(w[4 * q + 2], xq.z, a2);
+            a3 = __dp4a(w[4 * q + 3], xq.w, a3);
         }
-        return a;
+        return (a0 + a1) + (a2 + a3);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The persistent, staged kernel body.
+// ---------------------------------------------------------------------------------------------
+
+// Which items a thread block visits, without divisions in the loop: item k of the block is
+// (row-block chunk c0 + k * cstep, column block cs).
+struct Walk {
+    int c0, cstep;   // chunk index of the block's first item, chunk stride between its items
+    int cs;          // column block (0 when CS == 1)
+    int g0;          // first group of the column block
+    int ng;          // groups in the column block
+    int n_items;     // items this block visits
+};
+
+__device__ __forceinline__ Walk make_walk(const Problem &pr, const Plan &pl, int first_item, int item_stride) {
+    Walk w;
+    const int items = static_cast<int>(pl.items);
+    w.n_items = first_item < items ? (items - first_item + item_stride - 1) / item_stride : 0;
+    if (pl.CS == 1) {
+        w.c0 = first_item;
+        w.cstep = item_stride;
+        w.cs = 0;
+    } else {                       // item_stride is a multiple of CS
+        w.c0 = first_item / pl.CS;
+        w.cstep = item_stride / pl.CS;
+        w.cs = first_item - w.c0 * pl.CS;
+    }
+    w.g0 = w.cs * pl.CG;
+    w.ng = pr.G - w.g0 < pl.CG ? pr.G - w.g0 : pl.CG;
+    return w;
+}
+
+struct ItemRange {
+    int rb0;         // first row block
+    int nt;          // tiles (= busy warps)
+    int64_t t0;      // first tile
+};
+
+__device__ __forceinline__ ItemRange item_range(const Problem &pr, const Plan &pl, const Walk &wk, int k) {
+    ItemRange r;
+    r.rb0 = (wk.c0 + k * wk.cstep) * pl.RBC;
+    if (pl.CS == 1) {
+        int nrb = pr.RB - r.rb0;
+        if (nrb > pl.RBC) nrb = pl.RBC;
+        r.nt = nrb * pr.G;
+    } else {
+        r.nt = wk.ng;
+    }
+    r.t0 = static_cast<int64_t>(r.rb0) * pr.G + wk.g0;
+    return r;
+}
+
+// Issues the bulk copies of the block's item k into stage `s` (one thread).  sign_base[s]
+// receives the bit index of the first sign bit held in the stage's sign buffer.
+template <int FMT>
+__device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, const Walk &wk, const SmemLayout &L,
+                                           uint8_t *smem, int k, int s, uint32_t *sign_base) {
+    const ItemRange r = item_range(pr, pl, wk, k);
+    uint8_t *stage = smem + L.stage + static_cast<uint32_t>(s) * L.stage_bytes;
+    const uint32_t bar = smem_addr(smem + L.bar) + 8u * static_cast<uint32_t>(s);
+    const uint32_t d_payload = smem_addr(stage);
+    const uint32_t d_signs = d_payload + L.payload_cap;
+    const uint32_t d_scales = d_signs + L.sign_cap;
+    const uint32_t scale_bytes = static_cast<uint32_t>(r.nt) * 64u;
+    const uint8_t *g_scales = reinterpret_cast<const uint8_t *>(pr.scales) + r.t0 * 64;
+    if (FMT == kBitcos) {
+        const uint32_t o_lo = __ldg(pr.tile_off + r.t0), o_hi = __ldg(pr.tile_off + r.t0 + r.nt);
+        const uint32_t b_lo = (o_lo >> 7) << 4, b_hi = ((o_hi + 127u) >> 7) << 4;
+        const uint32_t sign_bytes = b_hi - b_lo;
+        const uint32_t bm_bytes = static_cast<uint32_t>(r.nt) * 512u;
+        sign_base[s] = b_lo * 8u;
+        mbar_expect_tx(bar, bm_bytes + sign_bytes + scale_bytes);
+        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + r.t0 * 512, bm_bytes, bar);
+        if (sign_bytes) bulk_copy(d_signs, reinterpret_cast<const uint8_t *>(pr.signs) + b_lo, sign_bytes, bar);
+        bulk_copy(d_scales, g_scales, scale_bytes, bar);
+    } else if (FMT == kTrit5) {
+        const int64_t WPR = (26 * static_cast<int64_t>(pr.G) + 3) / 4;
+        const int64_t w_lo = r.rb0 * WPR + ((26 * wk.g0) >> 2);
+        int64_t w_hi;   // exclusive
+        if (pl.CS == 1) w_hi = (r.rb0 + r.nt / pr.G) * WPR;
+        else w_hi = r.rb0 * WPR + ((26 * (wk.g0 + r.nt) - 1) >> 2) + 1;
+        const uint32_t bytes = static_cast<uint32_t>(w_hi - w_lo) * 128u;
+        mbar_expect_tx(bar, bytes + scale_bytes);
+        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + w_lo * 128, bytes, bar);
+        bulk_copy(d_scales, g_scales, scale_bytes, bar);
+    } else {
+        const uint32_t bytes = static_cast<uint32_t>(r.nt) * 1024u;
+        mbar_expect_tx(bar, bytes + scale_bytes);
+        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + r.t0 * 1024, bytes, bar);
+        bulk_copy(d_scales, g_scales, scale_bytes, bar);
     }
 }
 
 template <int FMT, int NB>
-__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem) {
+__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, int first_item,
+                                            int item_stride) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint8_t *lut = smem;
-    float *red = reinterpret_cast<float *>(smem + (FMT == kBit2 ? 0 : kLutBytes));
+    const SmemLayout L = smem_layout(FMT, pl, pr.G, NB);
+    const uint8_t *lut = smem + L.lut;
+    float *red = reinterpret_cast<float *>(smem + L.red);
+    uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 64);
+    const uint32_t bar0 = smem_addr(smem + L.bar);
+    const uint32_t lut_bar = bar0 + 8u * kStages;
     __shared__ int s_last;
 
+    const Walk wk = make_walk(pr, pl, first_item, item_stride);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s <= kStages; ++s) mbar_init(bar0 + 8u * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        for (int k = 0; k < kStages && k < wk.n_items; ++k) issue_item<FMT>(pr, pl, wk, L, smem, k, k, sign_base);
+        if (FMT != kBit2) {
+            mbar_expect_tx(lut_bar, kLutBytes);
+            bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes, lut_bar);
+        }
+    }
+
+    // what this warp works on in every item: CS == 1 -> row block warp / G of the chunk, group
+    // warp % G; else -> the chunk's only row block, group g0 + warp
+    const int my_rbl = (pl.CS == 1) ? warp / pr.G : 0;
+    const int my_g = (pl.CS == 1) ? warp - my_rbl * pr.G : wk.g0 + warp;
+    const bool leader = (pl.CS == 1) ? (my_g == 0) : (warp == 0);
+    const int per_rb = (pl.CS == 1) ? pr.G : wk.ng;              // warps that share a row block
+
+    // activations of this block's groups: all groups when CS == 1, else column block cs
+    const uint32_t xs_stride = static_cast<uint32_t>(pl.CG) * kGroup;     // bytes per token in shared memory
     int xr[NB];
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
         const int bb = b < pr.nb ? b : 0;
         xr[b] = pr.xrow ? __ldg(pr.xrow + bb) : bb;
     }
+    {
+        int4 *xs = reinterpret_cast<int4 *>(smem + L.x);
+        const int per_tok = wk.ng * (kGroup / 16);
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            if (b < pr.nb) {
+                const int4 *src = reinterpret_cast<const int4 *>(pr.x + static_cast<int64_t>(xr[b]) * pr.K + wk.g0 * kGroup);
+                for (int q = threadIdx.x; q < per_tok; q += blockDim.x) xs[b * (xs_stride / 16) + q] = __ldg(src + q);
+            }
+        }
+    }
+    {
+        bool lut_failed = false;
+        if (FMT != kBit2 && threadIdx.x == 0) lut_failed = !mbar_wait(lut_bar, 0);
+        if (__syncthreads_or(lut_failed)) {
+            if (threadIdx.x == 0 && pr.status) *pr.status = 1u;
+            return;
+        }
+    }
 
-    for (int64_t u = blockIdx.x; u < pl.units; u += gridDim.x) {
-        const int64_t rbg = u / pl.CS;
-        const int cs = static_cast<int>(u % pl.CS);
-        const int rbl = warp / pl.SC, run_local = warp % pl.SC;
-        const int64_t rb = rbg * pl.RBC + rbl;
-        const int run = cs * pl.SC + run_local;
-        const bool active = rb < pr.RB;
-        const int64_t m = rb * kRows + lane;
+    for (int k = 0; k < wk.n_items; ++k) {
+        const int s = k % kStages;
+        const uint32_t parity = static_cast<uint32_t>((k / kStages) & 1);
+        const ItemRange r = item_range(pr, pl, wk, k);
+        const bool busy = warp < r.nt;
+        const int rb = r.rb0 + my_rbl;
+        const int g = my_g;
+        const int64_t t = r.t0 + warp;
+        const int64_t m = static_cast<int64_t>(rb) * kRows + lane;
+        uint32_t toff = 0;
+        if (FMT == kBitcos && busy) toff = __ldg(pr.tile_off + t);
 
+        // one thread polls; the barrier below hands the arrival on to everybody (and tells that
+        // every warp is done with the previous item)
+        bool failed = false;
+        if (threadIdx.x == 0) failed = !mbar_wait(bar0 + 8u * s, parity);
+        if (__syncthreads_or(failed)) {
+            if (threadIdx.x == 0 && pr.status) *pr.status = 1u;
+            return;
+        }
+        // refill the stage that the previous item used
+        if (threadIdx.x == 0 && k >= 1 && k - 1 + kStages < wk.n_items) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue_item<FMT>(pr, pl, wk, L, smem, k - 1 + kStages, (k - 1) % kStages, sign_base);
+        }
+
+        const uint8_t *stage = smem + L.stage + static_cast<uint32_t>(s) * L.stage_bytes;
         float ysum[NB];
 #pragma unroll
         for (int b = 0; b < NB; ++b) ysum[b] = 0.f;
 
-        if (active) {
-            for (int g = run * pl.gpw; g < (run + 1) * pl.gpw; ++g) {
-                const int64_t t = rb * pr.G + g;
-                int w[32];
-                if (FMT == kBitcos) bitcos_decode_tile(pr, t, lane, lut, w);
-                else if (FMT == kTrit5) trit5_decode_tile(pr, rb, g, lane, lut, w);
-                else bit2_decode_tile(pr, t, lane, w);
-                const float s = bf16_to_float(__ldg(pr.scales + t * kRows + lane));
+        if (busy) {
+            const uint8_t *xsm = smem + L.x + static_cast<uint32_t>(g - wk.g0) * kGroup;
+            const float sc = bf16_to_float(
+                reinterpret_cast<const uint16_t *>(stage + L.payload_cap + L.sign_cap)[warp * kRows + lane]);
+            int w[32];
+            int acc1 = 0;
+            if (FMT == kBitcos) {
+                const uint4 bm = reinterpret_cast<const uint4 *>(stage)[warp * kRows + lane];
+                const int c = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
+                int incl = c;
 #pragma unroll
-                for (int b = 0; b < NB; ++b) {
-                    if (b < pr.nb) {
-                        const int a = contract<FMT>(w, pr.x + static_cast<int64_t>(xr[b]) * pr.K + g * kGroup, lane);
-                        ysum[b] = fmaf(s, static_cast<float>(a), ysum[b]);
-                        if (pr.acc_debug && m < pr.M)
-                            pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = a;
-                    }
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= d) incl += v;
+                }
+                const uint32_t cursor = toff + static_cast<uint32_t>(incl - c) - sign_base[s];
+                const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + L.payload_cap) + (cursor >> 5);
+                acc1 = bitcos_decode_row<NB == 1>(bm, sp, cursor & 31u, lut, static_cast<uint32_t>(lane) * 4u,
+                                                  reinterpret_cast<const int4 *>(xsm), w);
+            } else if (FMT == kTrit5) {
+                const int WPR = (26 * pr.G + 3) / 4;
+                // words of the stage: row block (rb - rb0) of the chunk, from the chunk's first word
+                const int w_rel = my_rbl * WPR + ((26 * g) >> 2) - ((26 * wk.g0) >> 2);
+                const uint32_t *src = reinterpret_cast<const uint32_t *>(stage) + w_rel * kRows + lane;
+                uint32_t wd[7];
+#pragma unroll
+                for (int i = 0; i < 7; ++i) wd[i] = src[i * kRows];
+                trit5_decode_row(wd, g & 1, lut, static_cast<uint32_t>(lane) * 8u, w);
+            } else {
+                const uint4 *src = reinterpret_cast<const uint4 *>(stage) + (warp * 2) * kRows + lane;
+                bit2_decode_row(src[0], src[kRows], w);
+            }
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                if (b < pr.nb) {
+                    int a;
+                    if (FMT == kBitcos && NB == 1) a = acc1;
+                    else a = contract<FMT>(w, reinterpret_cast<const int4 *>(xsm + b * xs_stride), lane);
+                    ysum[b] = sc * static_cast<float>(a);
+                    if (pr.acc_debug && m < pr.M) pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = a;
                 }
             }
         }
 
-        // ---- reduce the runs of each row block inside the thread block, in run order ----
-        if (pl.SC > 1) {
+        // ---- sum the groups of each row block held by this thread block, in group order ----
 #pragma unroll
-            for (int b = 0; b < NB; ++b) red[(warp * NB + b) * kRows + lane] = ysum[b];
-            __syncthreads();
-            if (run_local == 0) {
+        for (int b = 0; b < NB; ++b) red[(warp * NB + b) * kRows + lane] = ysum[b];
+        __syncthreads();
+        if (busy && leader) {
 #pragma unroll
-                for (int b = 0; b < NB; ++b) {
+            for (int b = 0; b < NB; ++b) {
+                if (b < pr.nb) {
                     float tot = 0.f;
-                    for (int s2 = 0; s2 < pl.SC; ++s2) tot += red[((warp + s2) * NB + b) * kRows + lane];
-                    ysum[b] = tot;
+                    for (int i = 0; i < per_rb; ++i) tot += red[((warp + i) * NB + b) * kRows + lane];
+                    if (pl.CS == 1) {
+                        if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
+                    } else {
+                        pr.partial[((static_cast<int64_t>(rb) * pl.CS + wk.cs) * pr.nb + b) * kRows + lane] = tot;
+                    }
                 }
             }
         }
-        if (pl.CS == 1) {
-            if (run_local == 0 && active && m < pr.M) {
-#pragma unroll
-                for (int b = 0; b < NB; ++b)
-                    if (b < pr.nb) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * ysum[b];
-            }
-        } else {
+        if (pl.CS > 1) {
             // ---- several thread blocks per row block: scratch partials + arrival counter ----
-            if (run_local == 0) {
-#pragma unroll
-                for (int b = 0; b < NB; ++b)
-                    if (b < pr.nb) pr.partial[((rb * pl.CS + cs) * pr.nb + b) * kRows + lane] = ysum[b];
-                __threadfence();
-            }
+            if (warp == 0) __threadfence();
             __syncthreads();
             if (threadIdx.x == 0) {
                 const unsigned int old = atomicAdd(pr.counters + rb, 1u);
@@ -440,32 +677,26 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 for (int b = 0; b < NB; ++b) {
                     if (b < pr.nb) {
                         float tot = 0.f;
-                        for (int c = 0; c < pl.CS; ++c)
-                            tot += __ldcg(pr.partial + ((rb * pl.CS + c) * pr.nb + b) * kRows + lane);
+                        for (int c2 = 0; c2 < pl.CS; ++c2)
+                            tot += __ldcg(pr.partial + ((static_cast<int64_t>(rb) * pl.CS + c2) * pr.nb + b) * kRows + lane);
                         if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
                     }
                 }
                 if (lane == 0) pr.counters[rb] = 0u;   // leave the counter ready for the next call
             }
         }
-        __syncthreads();
     }
 }
 
 template <int FMT, int NB>
-__global__ void __launch_bounds__(kMaxWarps * 32) gemv_kernel(const Problem pr, const Plan pl) {
-    extern __shared__ __align__(16) uint8_t smem[];
-    if (FMT == kBitcos) build_bitcos_lut(smem);
-    if (FMT == kTrit5) build_trit5_lut(smem);
-    if (FMT != kBit2) __syncthreads();
-    run_problem<FMT, NB>(pr, pl, smem);
+__global__ void __launch_bounds__(kMaxWarps * 32, 1) gemv_kernel(const Problem pr, const Plan pl) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    run_problem<FMT, NB>(pr, pl, smem, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
 }
 
 template <int NB>
-__global__ void __launch_bounds__(kMaxWarps * 32) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
-    extern __shared__ __align__(16) uint8_t smem[];
-    build_bitcos_lut(smem);
-    __syncthreads();
+__global__ void __launch_bounds__(kMaxWarps * 32, 1) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
+    extern __shared__ __align__(128) uint8_t smem[];
     const int grp = blockIdx.y;
     const int e = __ldg(ga.group_expert + grp);
     const int begin = __ldg(ga.group_begin + grp), end = __ldg(ga.group_begin + grp + 1);
@@ -478,10 +709,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32) gemv_grouped_kernel(Problem pr
     pr.nb = min(end - begin, NB);
     pr.xrow = pr.xrow + begin;
     pr.out_row0 = begin;
-    uint8_t *ws = reinterpret_cast<uint8_t *>(pr.counters) + static_cast<size_t>(grp) * ga.ws_stride;
-    pr.counters = reinterpret_cast<unsigned int *>(ws);
-    pr.partial = reinterpret_cast<float *>(ws + ((static_cast<size_t>(pr.RB) * 4 + 255) / 256 * 256));
-    run_problem<kBitcos, NB>(pr, pl, smem);
+    uint8_t *ws = reinterpret_cast<uint8_t *>(pr.status) + static_cast<size_t>(grp) * ga.ws_stride;
+    pr.status = reinterpret_cast<unsigned int *>(ws);
+    pr.counters = reinterpret_cast<unsigned int *>(ws + kHeaderBytes);
+    pr.partial = reinterpret_cast<float *>(ws + kHeaderBytes + ((static_cast<size_t>(pr.RB) * 4 + 255) / 256 * 256));
+    run_problem<kBitcos, NB>(pr, pl, smem, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -495,51 +727,50 @@ inline int check_cuda(cudaError_t e) {
     return BITCOS_ERR_CUDA;
 }
 
-size_t smem_bytes(int fmt, int nw, int nb) {
-    return (fmt == kBit2 ? 0 : kLutBytes) + static_cast<size_t>(nw) * nb * kRows * sizeof(float);
-}
-
-// Number of thread blocks to launch: min(units, SMs x resident blocks per SM).  The
-// occupancy query and the opt-in to large dynamic shared memory are done on the first call
-// for a given kernel (one cache per kernel instantiation), block size and device, and remembered (so that first call must not
-// happen during stream capture; later calls only read the cache).
+// Number of multiprocessors of the current device.  The opt-in to large dynamic shared memory is
+// done on the first call for a given kernel instantiation and device and remembered (so that
+// first call must not happen during stream capture; later calls only read the cache).
 template <auto kernel>
-int grid_for(int threads, size_t smem, int64_t units, int *grid) {
+int prepare_kernel(int *sms_out) {
     constexpr int kMaxDev = 32;
-    static int cache[kMaxDev][kMaxWarps + 1][2];      // [device][warps][0: blocks per SM, 1: SMs]; 0 = unknown
+    static int cache[kMaxDev];      // multiprocessor count, 0 = not prepared yet
     int dev = 0;
     int rc = check_cuda(cudaGetDevice(&dev));
     if (rc) return rc;
-    const int nw = threads / 32;
-    int per_sm = 0, sms = 0;
-    if (dev < kMaxDev && cache[dev][nw][0] > 0) {
-        per_sm = cache[dev][nw][0];
-        sms = cache[dev][nw][1];
-    } else {
-        rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        if (rc) return rc;
-        rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutBytes + 32 * 1024));
-        if (rc) return rc;
-        rc = check_cuda(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
-        if (rc) return rc;
-        if (per_sm < 1) per_sm = 1;
-        if (dev < kMaxDev) {
-            cache[dev][nw][1] = sms;
-            cache[dev][nw][0] = per_sm;
-        }
+    if (dev < kMaxDev && cache[dev] > 0) {
+        *sms_out = cache[dev];
+        return BITCOS_OK;
     }
-    const int64_t cap = static_cast<int64_t>(sms) * per_sm;
-    *grid = static_cast<int>(units < cap ? units : cap);
+    int sms = 0, max_smem = 0;
+    rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (rc) return rc;
+    rc = check_cuda(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    if (rc) return rc;
+    rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+    if (rc) return rc;
+    if (dev < kMaxDev) cache[dev] = sms;
+    *sms_out = sms;
     return BITCOS_OK;
+}
+
+// Persistent grid: one block per multiprocessor; a multiple of CS so that a block always works
+// on the same column block and can keep that block's activations in shared memory.
+inline int grid_size(const Plan &pl, int sms) {
+    int64_t g = pl.items < sms ? pl.items : sms;
+    if (pl.CS > 1) {
+        g = g / pl.CS * pl.CS;
+        if (g < pl.CS) g = pl.CS;
+    }
+    return static_cast<int>(g);
 }
 
 template <int FMT, int NB>
 int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
-    const size_t smem = smem_bytes(FMT, pl.NW, NB);
-    int grid = 1;
-    int rc = grid_for<gemv_kernel<FMT, NB>>(pl.NW * 32, smem, pl.units, &grid);
+    int sms = 0;
+    int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms);
     if (rc) return rc;
-    gemv_kernel<FMT, NB><<<grid, pl.NW * 32, smem, stream>>>(pr, pl);
+    const SmemLayout L = smem_layout(FMT, pl, pr.G, NB);
+    gemv_kernel<FMT, NB><<<grid_size(pl, sms), pl.NW * 32, L.total, stream>>>(pr, pl);
     return check_cuda(cudaGetLastError());
 }
 
@@ -554,15 +785,19 @@ int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream) {
 
 template <int NB>
 int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int n_groups, cudaStream_t stream) {
-    const size_t smem = smem_bytes(kBitcos, pl.NW, NB);
-    int grid = 1;
-    int rc = grid_for<gemv_grouped_kernel<NB>>(pl.NW * 32, smem, pl.units, &grid);
+    int sms = 0;
+    int rc = prepare_kernel<gemv_grouped_kernel<NB>>(&sms);
     if (rc) return rc;
-    // the grid's x extent is shared by all groups: spread the machine over them
-    int gx = (grid + n_groups - 1) / n_groups;
+    const SmemLayout L = smem_layout(kBitcos, pl, pr.G, NB);
+    // the machine is shared by all groups: spread its multiprocessors over them
+    int gx = (sms + n_groups - 1) / n_groups;
+    if (gx > pl.items) gx = static_cast<int>(pl.items);
+    if (pl.CS > 1) {
+        gx = gx / pl.CS * pl.CS;
+        if (gx < pl.CS) gx = pl.CS;
+    }
     if (gx < 1) gx = 1;
-    if (gx > pl.units) gx = static_cast<int>(pl.units);
-    gemv_grouped_kernel<NB><<<dim3(gx, n_groups), pl.NW * 32, smem, stream>>>(pr, pl, ga);
+    gemv_grouped_kernel<NB><<<dim3(gx, n_groups), pl.NW * 32, L.total, stream>>>(pr, pl, ga);
     return check_cuda(cudaGetLastError());
 }
 
@@ -572,7 +807,7 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
     if (!payload || !scales || !x || !x_scale || !y || !workspace) return BITCOS_ERR_NULL;
     if (fmt == kBitcos && (!signs || !tile_off)) return BITCOS_ERR_NULL;
     if (M < 1 || K < kGroup || K % kGroup != 0 || batch < 1 || batch > BITCOS_MAX_BATCH) return BITCOS_ERR_SHAPE;
-    if (K / kGroup > 0x7FFFFF || padded_rows(M) / kRows > 0x7FFFFFFF) return BITCOS_ERR_SHAPE;
+    if (K / kGroup > 0x7FFFFF || make_plan(M, K).items > 0x3FFFFFFF) return BITCOS_ERR_SHAPE;
     if (!aligned16(payload) || !aligned16(scales) || !aligned16(x) || !aligned16(y) || !aligned16(workspace) ||
         (signs && !aligned16(signs)) || (tile_off && !aligned16(tile_off)) || (acc_debug && !aligned16(acc_debug)))
         return BITCOS_ERR_ALIGN;
@@ -595,8 +830,10 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
     pr.RB = static_cast<int>(padded_rows(M) / kRows);
     pr.nb = batch;
     pr.out_row0 = 0;
-    pr.counters = static_cast<unsigned int *>(workspace);
-    pr.partial = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + counters_bytes(pr.RB));
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    pr.status = reinterpret_cast<unsigned int *>(ws);
+    pr.counters = reinterpret_cast<unsigned int *>(ws + kHeaderBytes);
+    pr.partial = reinterpret_cast<float *>(ws + kHeaderBytes + counters_bytes(pr.RB));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (fmt == kBitcos) return launch_nb<kBitcos>(pr, pl, stream);
     if (fmt == kTrit5) return launch_nb<kTrit5>(pr, pl, stream);
@@ -617,6 +854,18 @@ size_t bitcos_gemv_workspace_bytes(int64_t M, int64_t K) {
 int bitcos_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream) {
     if (!workspace) return BITCOS_ERR_NULL;
     return check_cuda(cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int bitcos_workspace_status(const void *workspace, void *cuda_stream, int *status) {
+    if (!workspace || !status) return BITCOS_ERR_NULL;
+    unsigned int v = 0;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int rc = check_cuda(cudaMemcpyAsync(&v, workspace, sizeof v, cudaMemcpyDeviceToHost, stream));
+    if (rc) return rc;
+    rc = check_cuda(cudaStreamSynchronize(stream));
+    if (rc) return rc;
+    *status = static_cast<int>(v);
+    return BITCOS_OK;
 }
 
 int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
@@ -699,7 +948,7 @@ int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M,
     pr.K = K;
     pr.G = static_cast<int>(K / kGroup);
     pr.RB = static_cast<int>(padded_rows(M) / kRows);
-    pr.counters = static_cast<unsigned int *>(workspace);
+    pr.status = static_cast<unsigned int *>(workspace);
     GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts};
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (max_group_size <= 1) return launch_grouped<1>(pr, pl, ga, n_groups, stream);
