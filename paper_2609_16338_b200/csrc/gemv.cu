@@ -28,15 +28,17 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstdlib>
 
 namespace {
 
 constexpr int kGroup = BITCOS_GROUP;
 constexpr int kRows = BITCOS_TILE_ROWS;
 constexpr int kMaxWarps = 20;             // warps per thread block = tiles per item
-constexpr int kStages = 3;                // shared-memory ring depth
+constexpr int kMaxStages = 8;             // upper bound on the shared-memory ring depth (Plan::stages)
 constexpr int kLutBytes = 64 * 1024;      // replicated lookup tables (BITCOS, five-trit)
-constexpr uint32_t kSpinLimit = 1u << 22; // bound on mbarrier polls before giving up
+constexpr uint64_t kWaitLimitNs = 500ull * 1000 * 1000;   // an mbarrier wait gives up after half a second
+constexpr int64_t kXResidentBytes = 48 * 1024;   // activations up to this size are kept in shared memory
 
 enum Format { kBitcos = 0, kTrit5 = 1, kBit2 = 2 };
 
@@ -133,6 +135,8 @@ struct Plan {
     int RBC;         // row blocks per item (1 unless CS == 1)
     int NW;          // warps per thread block = CG * RBC
     int64_t items;   // ceil(RB / RBC) * CS
+    int cyclic;      // 1: blocks take whole row-block chunks round robin; 0: contiguous balanced ranges
+    int stages;      // depth of the shared-memory ring (2 .. kMaxStages), set at launch
 };
 
 struct Problem {
@@ -164,16 +168,20 @@ struct GroupedArgs {
 
 inline int64_t padded_rows(int64_t M) { return (M + kRows - 1) / kRows * kRows; }
 
-Plan make_plan(int64_t M, int64_t K) {
+// Decoder warps per thread block: 20, or 10 for more than 8 tokens (their activations and partial
+// sums would not fit in shared memory otherwise).
+inline int decoder_warps(int batch) { return batch > 8 ? kMaxWarps / 2 : kMaxWarps; }
+
+Plan make_plan(int64_t M, int64_t K, int max_warps) {
     const int G = static_cast<int>(K / kGroup);
     const int64_t RB = padded_rows(M) / kRows;
     Plan p{};
-    const int blocks = (G + kMaxWarps - 1) / kMaxWarps;
+    const int blocks = (G + max_warps - 1) / max_warps;
     p.CG = (G + blocks - 1) / blocks;
     p.CS = (G + p.CG - 1) / p.CG;
     p.RBC = 1;
     if (p.CS == 1) {
-        int64_t r = kMaxWarps / p.CG;
+        int64_t r = max_warps / p.CG;
         if (r > RB) r = RB;
         if (r < 1) r = 1;
         p.RBC = static_cast<int>(r);
@@ -188,7 +196,7 @@ constexpr size_t kHeaderBytes = 256;
 size_t counters_bytes(int64_t RB) { return static_cast<size_t>((RB * 4 + 255) / 256 * 256); }
 
 size_t workspace_bytes_for(int64_t M, int64_t K) {
-    const Plan p = make_plan(M, K);
+    const Plan p = make_plan(M, K, kMaxWarps / 2);        // the plan with the most column blocks
     const int64_t RB = padded_rows(M) / kRows;
     size_t b = kHeaderBytes + counters_bytes(RB);
     if (p.CS > 1) b += static_cast<size_t>(RB) * p.CS * BITCOS_MAX_BATCH * kRows * sizeof(float);
@@ -201,15 +209,16 @@ struct SmemLayout {
     uint32_t stage;      // stage 0
     uint32_t stage_bytes;
     uint32_t payload_cap, sign_cap, scale_cap;   // per-stage capacities
-    uint32_t x;          // activations of the block's groups, [nb][CG * 128]
-    uint32_t red;        // [NW][NB][32] floats
-    uint32_t bar;        // kStages mbarriers, then (at +64) per-stage sign base words
+    uint32_t x;          // activations, [nb][K], if x_bytes != 0
+    uint32_t x_bytes;    // 0: the activations do not fit and are read from global memory
+    uint32_t red;        // 2 x [NW][NB][32] floats
+    uint32_t bar;        // mbarriers, then per-stage sign base words
     uint32_t total;
 };
 
 __host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
-__host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G, int nbmax) {
+__host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G, int nbmax, int64_t K) {
     SmemLayout L{};
     uint32_t off = 0;
     L.lut = off;
@@ -231,13 +240,14 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     L.scale_cap = tiles * 64;
     L.stage = off;
     L.stage_bytes = align_up(L.payload_cap + L.sign_cap + L.scale_cap, 128);
-    off += L.stage_bytes * kStages;
+    off += L.stage_bytes * static_cast<uint32_t>(pl.stages);
     L.x = off;
-    off += align_up(static_cast<uint32_t>(nbmax) * static_cast<uint32_t>(pl.CG) * kGroup, 128);
+    L.x_bytes = (static_cast<int64_t>(nbmax) * K <= kXResidentBytes) ? static_cast<uint32_t>(nbmax * K) : 0u;
+    off += align_up(L.x_bytes, 128);
     L.red = off;
-    off += tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
+    off += 2 * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;      // two slots
     L.bar = off;
-    off += 128;
+    off += 256;
     L.total = off;
     return L;
 }
@@ -273,20 +283,31 @@ __device__ __forceinline__ void bulk_copy(uint32_t dst, const void *src, uint32_
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-// Waits for the given phase parity with a bounded number of polls; false if it gave up.
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Waits for the given phase parity, for at most kWaitLimitNs; false if it gave up.  Each poll may
+// suspend the thread for up to about a microsecond.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 0;; ++i) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(1000u)
             : "memory");
         if (done) return true;
+        if ((i & 15u) == 15u) {
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
+        }
     }
-    return false;
 }
 
 // d = (a & c) | (b & ~c): one LOP3
@@ -420,60 +441,89 @@ __device__ __forceinline__ int contract(const int (&w)[32], const int4 *xg, int 
 // The persistent, staged kernel body.
 // ---------------------------------------------------------------------------------------------
 
-// Which items a thread block visits, without divisions in the loop: item k of the block is
-// (row-block chunk c0 + k * cstep, column block cs).
+// Items are numbered row-block chunk major, column block minor: item = c * CS + cs.  A thread
+// block owns a CONTIGUOUS range of items (balanced split of all items over the grid), so it
+// streams a contiguous piece of the packed matrix and usually sees all column blocks of a row
+// block itself; only the row blocks cut by a range boundary need the cross-block protocol.
 struct Walk {
-    int c0, cstep;   // chunk index of the block's first item, chunk stride between its items
-    int cs;          // column block (0 when CS == 1)
-    int g0;          // first group of the column block
-    int ng;          // groups in the column block
-    int n_items;     // items this block visits
+    int first, count;   // this block's first item and number of items
+    int cstride;        // chunk stride after the last column block of a chunk (1 = contiguous range)
+    int q, rem;         // contiguous mode: blocks 0 .. rem-1 own q + 1 items, the others q
 };
 
-__device__ __forceinline__ Walk make_walk(const Problem &pr, const Plan &pl, int first_item, int item_stride) {
+// Two ways to hand items to thread blocks.  Cyclic: block b takes chunks b, b + n, b + 2n, ...
+// with all their column blocks (no row block is ever shared; all blocks read neighbouring
+// addresses at any time).  Contiguous: a balanced split of the item list (perfect balance when
+// there are few chunks per block, at the price of sharing the row blocks cut by a boundary).
+__device__ __forceinline__ Walk make_walk(const Plan &pl, int block, int n_blocks) {
     Walk w;
     const int items = static_cast<int>(pl.items);
-    w.n_items = first_item < items ? (items - first_item + item_stride - 1) / item_stride : 0;
-    if (pl.CS == 1) {
-        w.c0 = first_item;
-        w.cstep = item_stride;
-        w.cs = 0;
-    } else {                       // item_stride is a multiple of CS
-        w.c0 = first_item / pl.CS;
-        w.cstep = item_stride / pl.CS;
-        w.cs = first_item - w.c0 * pl.CS;
+    if (pl.cyclic) {
+        const int chunks = items / pl.CS;
+        w.first = block * pl.CS;
+        w.count = block < chunks ? ((chunks - block + n_blocks - 1) / n_blocks) * pl.CS : 0;
+        w.cstride = n_blocks;
+        w.q = 1;
+        w.rem = 0;
+        return w;
     }
-    w.g0 = w.cs * pl.CG;
-    w.ng = pr.G - w.g0 < pl.CG ? pr.G - w.g0 : pl.CG;
+    w.q = items / n_blocks;
+    w.rem = items - w.q * n_blocks;
+    w.first = block * w.q + (block < w.rem ? block : w.rem);
+    w.count = w.q + (block < w.rem ? 1 : 0);
+    w.cstride = 1;
     return w;
+}
+
+// Which thread block owns an item in contiguous mode (inverse of the split above).
+__device__ __forceinline__ int owner_of(const Walk &w, int item) {
+    const int big = w.rem * (w.q + 1);
+    if (item < big) return item / (w.q + 1);
+    return w.rem + (item - big) / w.q;
 }
 
 struct ItemRange {
     int rb0;         // first row block
+    int cs;          // column block
+    int g0;          // first group
     int nt;          // tiles (= busy warps)
     int64_t t0;      // first tile
 };
 
-__device__ __forceinline__ ItemRange item_range(const Problem &pr, const Plan &pl, const Walk &wk, int k) {
+__device__ __forceinline__ ItemRange item_range(const Problem &pr, const Plan &pl, int c, int cs) {
     ItemRange r;
-    r.rb0 = (wk.c0 + k * wk.cstep) * pl.RBC;
+    r.rb0 = c * pl.RBC;
+    r.cs = cs;
+    r.g0 = cs * pl.CG;
     if (pl.CS == 1) {
         int nrb = pr.RB - r.rb0;
         if (nrb > pl.RBC) nrb = pl.RBC;
         r.nt = nrb * pr.G;
     } else {
-        r.nt = wk.ng;
+        r.nt = pr.G - r.g0 < pl.CG ? pr.G - r.g0 : pl.CG;
     }
-    r.t0 = static_cast<int64_t>(r.rb0) * pr.G + wk.g0;
+    r.t0 = static_cast<int64_t>(r.rb0) * pr.G + r.g0;
     return r;
 }
 
-// Issues the bulk copies of the block's item k into stage `s` (one thread).  sign_base[s]
-// receives the bit index of the first sign bit held in the stage's sign buffer.
+// (chunk, column block) of an item, and the step to the next item, without divisions in loops
+struct ItemIter {
+    int c, cs;
+    __device__ __forceinline__ void init(const Plan &pl, int item) {
+        if (pl.CS == 1) { c = item; cs = 0; }
+        else { c = item / pl.CS; cs = item - c * pl.CS; }
+    }
+    __device__ __forceinline__ void next(const Plan &pl, const Walk &w) {
+        if (++cs == pl.CS) { cs = 0; c += w.cstride; }
+    }
+};
+
+// Issues the bulk copies of one item into stage `s` (one thread).  sign_base[s] receives the bit
+// index of the first sign bit held in the stage's sign buffer.  o_lo / o_hi: sign-vector
+// positions of the item's first tile and of the tile after its last (BITCOS only).
 template <int FMT>
-__device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, const Walk &wk, const SmemLayout &L,
-                                           uint8_t *smem, int k, int s, uint32_t *sign_base) {
-    const ItemRange r = item_range(pr, pl, wk, k);
+__device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, const ItemRange &r, const SmemLayout &L,
+                                           uint8_t *smem, int s, uint32_t *sign_base, uint32_t o_lo, uint32_t o_hi) {
     uint8_t *stage = smem + L.stage + static_cast<uint32_t>(s) * L.stage_bytes;
     const uint32_t bar = smem_addr(smem + L.bar) + 8u * static_cast<uint32_t>(s);
     const uint32_t d_payload = smem_addr(stage);
@@ -482,7 +532,6 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
     const uint32_t scale_bytes = static_cast<uint32_t>(r.nt) * 64u;
     const uint8_t *g_scales = reinterpret_cast<const uint8_t *>(pr.scales) + r.t0 * 64;
     if (FMT == kBitcos) {
-        const uint32_t o_lo = __ldg(pr.tile_off + r.t0), o_hi = __ldg(pr.tile_off + r.t0 + r.nt);
         const uint32_t b_lo = (o_lo >> 7) << 4, b_hi = ((o_hi + 127u) >> 7) << 4;
         const uint32_t sign_bytes = b_hi - b_lo;
         const uint32_t bm_bytes = static_cast<uint32_t>(r.nt) * 512u;
@@ -493,10 +542,10 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
     } else if (FMT == kTrit5) {
         const int64_t WPR = (26 * static_cast<int64_t>(pr.G) + 3) / 4;
-        const int64_t w_lo = r.rb0 * WPR + ((26 * wk.g0) >> 2);
+        const int64_t w_lo = r.rb0 * WPR + ((26 * r.g0) >> 2);
         int64_t w_hi;   // exclusive
         if (pl.CS == 1) w_hi = (r.rb0 + r.nt / pr.G) * WPR;
-        else w_hi = r.rb0 * WPR + ((26 * (wk.g0 + r.nt) - 1) >> 2) + 1;
+        else w_hi = r.rb0 * WPR + ((26 * (r.g0 + r.nt) - 1) >> 2) + 1;
         const uint32_t bytes = static_cast<uint32_t>(w_hi - w_lo) * 128u;
         mbar_expect_tx(bar, bytes + scale_bytes);
         bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + w_lo * 128, bytes, bar);
@@ -509,101 +558,294 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
     }
 }
 
-template <int FMT, int NB>
-__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, int first_item,
-                                            int item_stride) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const SmemLayout L = smem_layout(FMT, pl, pr.G, NB);
-    const uint8_t *lut = smem + L.lut;
-    float *red = reinterpret_cast<float *>(smem + L.red);
-    uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 64);
-    const uint32_t bar0 = smem_addr(smem + L.bar);
-    const uint32_t lut_bar = bar0 + 8u * kStages;
-    __shared__ int s_last;
+// mbarrier slots inside the `bar` region (8 bytes each)
+constexpr int kBarFull = 0;                       // [stages] stage filled by the copy engine
+constexpr int kBarEmpty = kMaxStages;             // [stages] stage released by all decoder warps
+constexpr int kBarRedFull = 2 * kMaxStages;       // [2] partial sums of an item written by all decoder warps
+constexpr int kBarRedEmpty = 2 * kMaxStages + 2;  // [2] partial sums consumed by the epilogue warp
+constexpr int kBarLut = 2 * kMaxStages + 4;       // lookup table arrived
+constexpr int kBarCount = 2 * kMaxStages + 5;
 
-    const Walk wk = make_walk(pr, pl, first_item, item_stride);
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s <= kStages; ++s) mbar_init(bar0 + 8u * s, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        for (int k = 0; k < kStages && k < wk.n_items; ++k) issue_item<FMT>(pr, pl, wk, L, smem, k, k, sign_base);
-        if (FMT != kBit2) {
-            mbar_expect_tx(lut_bar, kLutBytes);
-            bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes, lut_bar);
+// A row block whose column blocks were split over several thread blocks: this block's share.
+struct Share {
+    int rb;             // row block
+    int slot;           // position of this block among the sharers (= order of summation)
+    int sharers;        // number of thread blocks holding a piece of the row block
+    unsigned int old;   // value of the arrival counter before this block's arrival
+};
+
+// If this block's arrival was the last one: add the shares in slot order and write the outputs.
+template <int NB>
+__device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, const int (&xr)[NB], const Share &sh,
+                                             int lane) {
+    const unsigned int old = __shfl_sync(0xFFFFFFFFu, sh.old, 0);
+    if (old != static_cast<unsigned int>(sh.sharers - 1)) return;
+    __threadfence();
+    const int64_t m = static_cast<int64_t>(sh.rb) * kRows + lane;
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        if (b < pr.nb) {
+            float tot = 0.f;
+            for (int j = 0; j < sh.sharers; ++j)
+                tot += __ldcg(pr.partial + ((static_cast<int64_t>(sh.rb) * pl.CS + j) * pr.nb + b) * kRows + lane);
+            if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
         }
     }
+    if (lane == 0) pr.counters[sh.rb] = 0u;    // leave the counter ready for the next call
+}
 
-    // what this warp works on in every item: CS == 1 -> row block warp / G of the chunk, group
-    // warp % G; else -> the chunk's only row block, group g0 + warp
-    const int my_rbl = (pl.CS == 1) ? warp / pr.G : 0;
-    const int my_g = (pl.CS == 1) ? warp - my_rbl * pr.G : wk.g0 + warp;
-    const bool leader = (pl.CS == 1) ? (my_g == 0) : (warp == 0);
-    const int per_rb = (pl.CS == 1) ? pr.G : wk.ng;              // warps that share a row block
+// Warp roles: warps 0 .. NW-1 decode one tile per item each; warp NW feeds the stage ring with
+// bulk copies; warp NW+1 adds the decoders' partial sums in a fixed order and writes the
+// outputs (and runs the cross-block protocol).  The roles meet only through mbarriers, every
+// wait is bounded, and there is no block-wide barrier inside the loop.
+template <int FMT, int NB>
+__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, int block, int n_blocks) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const SmemLayout L = smem_layout(FMT, pl, pr.G, NB, pr.K);
+    const uint8_t *lut = smem + L.lut;
+    float *red = reinterpret_cast<float *>(smem + L.red);
+    uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 8 * kBarCount);
+    const uint32_t bar0 = smem_addr(smem + L.bar);
+    const uint32_t red_slot = static_cast<uint32_t>(pl.NW) * NB * kRows;     // floats per partial-sum slot
+    const Walk wk = make_walk(pl, block, n_blocks);
 
-    // activations of this block's groups: all groups when CS == 1, else column block cs
-    const uint32_t xs_stride = static_cast<uint32_t>(pl.CG) * kGroup;     // bytes per token in shared memory
+    // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as
+    // every block of this one got here; whatever it reads from us it reads after its own
+    // griddepcontrol.wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // ------------------------------------------------------------------ producer warp
+    // It also sets the barriers up, so that the first copies are in flight before anything else
+    // happens in the block.
+    if (warp == pl.NW) {
+        if (lane == 0) {
+            for (int s = 0; s < pl.stages; ++s) {
+                mbar_init(bar0 + 8u * (kBarFull + s), 1);
+                mbar_init(bar0 + 8u * (kBarEmpty + s), pl.NW);
+            }
+            for (int s = 0; s < 2; ++s) {
+                mbar_init(bar0 + 8u * (kBarRedFull + s), pl.NW);
+                mbar_init(bar0 + 8u * (kBarRedEmpty + s), 1);
+            }
+            mbar_init(bar0 + 8u * kBarLut, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        // The first copies go out before the block-wide barrier below, while the other warps are
+        // still fetching the activations.
+        ItemIter it;
+        ItemRange r{};
+        uint32_t o_lo = 0, o_hi = 0;
+        int k0 = 0, ps = 0;
+        uint32_t pphase = 1;       // parity of the phase before the one the decoders complete next
+        bool ok = true;
+        auto issue_loop = [&](int k_end) {
+            for (int k = k0; k < k_end; ++k) {
+                const int s = ps;
+                // offsets of the next item, requested before this item's copies are issued
+                ItemIter nx = it;
+                nx.next(pl, wk);
+                ItemRange rn = r;
+                uint32_t n_lo = 0, n_hi = 0;
+                if (k + 1 < wk.count) {
+                    rn = item_range(pr, pl, nx.c, nx.cs);
+                    if (FMT == kBitcos) {
+                        n_lo = (rn.t0 == r.t0 + r.nt) ? o_hi : __ldg(pr.tile_off + rn.t0);
+                        n_hi = __ldg(pr.tile_off + rn.t0 + rn.nt);
+                    }
+                }
+                if (k >= pl.stages) {
+                    if (!mbar_wait(bar0 + 8u * (kBarEmpty + s), pphase)) {
+                        if (pr.status) *pr.status = 1u;
+                        ok = false;
+                        return;
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                issue_item<FMT>(pr, pl, r, L, smem, s, sign_base, o_lo, o_hi);
+                if (k == 0 && FMT != kBit2) {
+                    mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
+                    bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
+                              bar0 + 8u * kBarLut);
+                }
+                it = nx;
+                r = rn;
+                o_lo = n_lo;
+                o_hi = n_hi;
+                if (++ps == pl.stages) {
+                    ps = 0;
+                    pphase ^= 1u;
+                }
+            }
+            k0 = k_end;
+        };
+        if (lane == 0 && wk.count > 0) {
+            it.init(pl, wk.first);
+            r = item_range(pr, pl, it.c, it.cs);
+            if (FMT == kBitcos) {
+                o_lo = __ldg(pr.tile_off + r.t0);
+                o_hi = __ldg(pr.tile_off + r.t0 + r.nt);
+            }
+            issue_loop(wk.count < pl.stages ? wk.count : pl.stages);
+        }
+        __syncthreads();       // pairs with the barrier the other warps reach after staging the activations
+        if (lane == 0 && ok) issue_loop(wk.count);
+        return;
+    }
+
+    // Everything below may depend on the previous kernel in the stream (activations, outputs,
+    // workspace); the packed weights the producer streams do not.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // activations: kept whole in shared memory ([nb][K]) when they fit, staged by the other
+    // warps while the producer starts the copies; otherwise read from global memory per tile
     int xr[NB];
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
         const int bb = b < pr.nb ? b : 0;
         xr[b] = pr.xrow ? __ldg(pr.xrow + bb) : bb;
     }
-    {
+    const bool x_resident = L.x_bytes != 0;
+    if (x_resident) {
         int4 *xs = reinterpret_cast<int4 *>(smem + L.x);
-        const int per_tok = wk.ng * (kGroup / 16);
+        const int per_tok = static_cast<int>(pr.K / 16);
+        const int nthr = (pl.NW + 2) * 32 - 32;              // all warps but the producer
+        const int tid = warp < pl.NW ? threadIdx.x : threadIdx.x - 32;
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             if (b < pr.nb) {
-                const int4 *src = reinterpret_cast<const int4 *>(pr.x + static_cast<int64_t>(xr[b]) * pr.K + wk.g0 * kGroup);
-                for (int q = threadIdx.x; q < per_tok; q += blockDim.x) xs[b * (xs_stride / 16) + q] = __ldg(src + q);
+                const int4 *src = reinterpret_cast<const int4 *>(pr.x + static_cast<int64_t>(xr[b]) * pr.K);
+                for (int q = tid; q < per_tok; q += nthr) xs[b * per_tok + q] = __ldg(src + q);
             }
         }
     }
-    {
-        bool lut_failed = false;
-        if (FMT != kBit2 && threadIdx.x == 0) lut_failed = !mbar_wait(lut_bar, 0);
-        if (__syncthreads_or(lut_failed)) {
-            if (threadIdx.x == 0 && pr.status) *pr.status = 1u;
+    __syncthreads();          // barriers initialised, activations in place
+    if (wk.count == 0) return;
+
+    // ------------------------------------------------------------------ epilogue warp
+    if (warp == pl.NW + 1) {
+        float run[NB];          // running sum of the current row block over this block's items
+#pragma unroll
+        for (int b = 0; b < NB; ++b) run[b] = 0.f;
+        Share pend[2];
+        int n_pend = 0;
+        ItemIter it;
+        it.init(pl, wk.first);
+        for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
+            const int slot = k & 1;
+            const ItemRange r = item_range(pr, pl, it.c, it.cs);
+            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k >> 1) & 1))) {
+                if (lane == 0 && pr.status) *pr.status = 1u;
+                return;
+            }
+            const float *rs = red + slot * red_slot;
+            if (pl.CS == 1) {
+                // whole row blocks: one output per row, groups added in ascending order
+                const int nrb = r.nt / pr.G;
+                for (int i = 0; i < nrb; ++i) {
+                    const int64_t m = static_cast<int64_t>(r.rb0 + i) * kRows + lane;
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        if (b < pr.nb) {
+                            float tot = 0.f;
+                            for (int j = 0; j < pr.G; ++j) tot += rs[((i * pr.G + j) * NB + b) * kRows + lane];
+                            if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedEmpty + slot));
+                continue;
+            }
+            // one column block of row block rb0: add it to the running sum
+            const bool starts = (r.cs == 0) || (k == 0);
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                if (b < pr.nb) {
+                    float tot = 0.f;
+                    for (int j = 0; j < r.nt; ++j) tot += rs[(j * NB + b) * kRows + lane];
+                    run[b] = starts ? tot : run[b] + tot;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedEmpty + slot));
+            const bool ends = (r.cs == pl.CS - 1) || (k == wk.count - 1);
+            if (!ends) continue;
+            const int first_cs = (k >= r.cs) ? 0 : r.cs - k;       // first column block of rb0 seen by this block
+            const int64_t m = static_cast<int64_t>(r.rb0) * kRows + lane;
+            if (first_cs == 0 && r.cs == pl.CS - 1) {
+                // the whole row block was ours
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    if (b < pr.nb && m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * run[b];
+            } else {
+                // shared row block: publish our share, then count ourselves in
+                Share sh;
+                sh.rb = r.rb0;
+                const int lo = owner_of(wk, r.rb0 * pl.CS), hi = owner_of(wk, r.rb0 * pl.CS + pl.CS - 1);
+                sh.slot = block - lo;
+                sh.sharers = hi - lo + 1;
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    if (b < pr.nb)
+                        pr.partial[((static_cast<int64_t>(sh.rb) * pl.CS + sh.slot) * pr.nb + b) * kRows + lane] = run[b];
+                __syncwarp();
+                sh.old = 0;
+                if (lane == 0) {
+                    __threadfence();
+                    sh.old = atomicAdd(pr.counters + sh.rb, 1u);
+                }
+                pend[n_pend++] = sh;      // at most two per block: its first and its last row block
+            }
+        }
+        for (int i = 0; i < n_pend; ++i) finish_share<NB>(pr, pl, xr, pend[i], lane);
+        return;
+    }
+
+    // ------------------------------------------------------------------ decoder warps
+    // CS == 1: this warp always has row block warp / G of the chunk and group warp % G
+    const int my_rbl = (pl.CS == 1) ? warp / pr.G : 0;
+    const int g_fixed = warp - my_rbl * pr.G;
+    if (FMT != kBit2) {
+        if (!mbar_wait(bar0 + 8u * kBarLut, 0)) {
+            if (lane == 0 && pr.status) *pr.status = 1u;
             return;
         }
     }
-
-    for (int k = 0; k < wk.n_items; ++k) {
-        const int s = k % kStages;
-        const uint32_t parity = static_cast<uint32_t>((k / kStages) & 1);
-        const ItemRange r = item_range(pr, pl, wk, k);
+    ItemIter it;
+    it.init(pl, wk.first);
+    int s = 0;
+    uint32_t phase = 0;
+    for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
+        const int slot = k & 1;
+        const ItemRange r = item_range(pr, pl, it.c, it.cs);
         const bool busy = warp < r.nt;
+        const int g = (pl.CS == 1) ? g_fixed : r.g0 + warp;
         const int rb = r.rb0 + my_rbl;
-        const int g = my_g;
         const int64_t t = r.t0 + warp;
         const int64_t m = static_cast<int64_t>(rb) * kRows + lane;
         uint32_t toff = 0;
         if (FMT == kBitcos && busy) toff = __ldg(pr.tile_off + t);
 
-        // one thread polls; the barrier below hands the arrival on to everybody (and tells that
-        // every warp is done with the previous item)
-        bool failed = false;
-        if (threadIdx.x == 0) failed = !mbar_wait(bar0 + 8u * s, parity);
-        if (__syncthreads_or(failed)) {
-            if (threadIdx.x == 0 && pr.status) *pr.status = 1u;
+        if (!mbar_wait(bar0 + 8u * (kBarFull + s), phase)) {
+            if (lane == 0 && pr.status) *pr.status = 1u;
             return;
         }
-        // refill the stage that the previous item used
-        if (threadIdx.x == 0 && k >= 1 && k - 1 + kStages < wk.n_items) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue_item<FMT>(pr, pl, wk, L, smem, k - 1 + kStages, (k - 1) % kStages, sign_base);
-        }
-
         const uint8_t *stage = smem + L.stage + static_cast<uint32_t>(s) * L.stage_bytes;
         float ysum[NB];
 #pragma unroll
         for (int b = 0; b < NB; ++b) ysum[b] = 0.f;
 
         if (busy) {
-            const uint8_t *xsm = smem + L.x + static_cast<uint32_t>(g - wk.g0) * kGroup;
             const float sc = bf16_to_float(
                 reinterpret_cast<const uint16_t *>(stage + L.payload_cap + L.sign_cap)[warp * kRows + lane]);
+            // activations of group g: in shared memory if resident (xs), else in global memory (xgl)
+            const uint8_t *xs = smem + L.x + static_cast<uint32_t>(g) * kGroup;
+            const uint8_t *xgl = reinterpret_cast<const uint8_t *>(pr.x) + static_cast<int64_t>(g) * kGroup;
             int w[32];
             int acc1 = 0;
             if (FMT == kBitcos) {
@@ -617,12 +859,15 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 }
                 const uint32_t cursor = toff + static_cast<uint32_t>(incl - c) - sign_base[s];
                 const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + L.payload_cap) + (cursor >> 5);
-                acc1 = bitcos_decode_row<NB == 1>(bm, sp, cursor & 31u, lut, static_cast<uint32_t>(lane) * 4u,
-                                                  reinterpret_cast<const int4 *>(xsm), w);
+                if (NB == 1 && x_resident)
+                    acc1 = bitcos_decode_row<true>(bm, sp, cursor & 31u, lut, static_cast<uint32_t>(lane) * 4u,
+                                                   reinterpret_cast<const int4 *>(xs), w);
+                else
+                    bitcos_decode_row<false>(bm, sp, cursor & 31u, lut, static_cast<uint32_t>(lane) * 4u, nullptr, w);
             } else if (FMT == kTrit5) {
                 const int WPR = (26 * pr.G + 3) / 4;
-                // words of the stage: row block (rb - rb0) of the chunk, from the chunk's first word
-                const int w_rel = my_rbl * WPR + ((26 * g) >> 2) - ((26 * wk.g0) >> 2);
+                // words of the stage: row block my_rbl of the chunk, counted from the chunk's first word
+                const int w_rel = my_rbl * WPR + ((26 * g) >> 2) - ((26 * r.g0) >> 2);
                 const uint32_t *src = reinterpret_cast<const uint32_t *>(stage) + w_rel * kRows + lane;
                 uint32_t wd[7];
 #pragma unroll
@@ -636,68 +881,52 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             for (int b = 0; b < NB; ++b) {
                 if (b < pr.nb) {
                     int a;
-                    if (FMT == kBitcos && NB == 1) a = acc1;
-                    else a = contract<FMT>(w, reinterpret_cast<const int4 *>(xsm + b * xs_stride), lane);
+                    if (FMT == kBitcos && NB == 1 && x_resident)
+                        a = acc1;
+                    else if (x_resident)
+                        a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pr.K), lane);
+                    else
+                        a = contract<FMT>(w, reinterpret_cast<const int4 *>(xgl + static_cast<int64_t>(xr[b]) * pr.K), lane);
                     ysum[b] = sc * static_cast<float>(a);
                     if (pr.acc_debug && m < pr.M) pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = a;
                 }
             }
         }
+        // the stage has been read: hand it back to the producer
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar0 + 8u * (kBarEmpty + s));
 
-        // ---- sum the groups of each row block held by this thread block, in group order ----
-#pragma unroll
-        for (int b = 0; b < NB; ++b) red[(warp * NB + b) * kRows + lane] = ysum[b];
-        __syncthreads();
-        if (busy && leader) {
-#pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                if (b < pr.nb) {
-                    float tot = 0.f;
-                    for (int i = 0; i < per_rb; ++i) tot += red[((warp + i) * NB + b) * kRows + lane];
-                    if (pl.CS == 1) {
-                        if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
-                    } else {
-                        pr.partial[((static_cast<int64_t>(rb) * pl.CS + wk.cs) * pr.nb + b) * kRows + lane] = tot;
-                    }
-                }
+        // partial sums for the epilogue warp (two slots, so decoders may run an item ahead of it)
+        if (k >= 2) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>(((k >> 1) - 1) & 1))) {
+                if (lane == 0 && pr.status) *pr.status = 1u;
+                return;
             }
         }
-        if (pl.CS > 1) {
-            // ---- several thread blocks per row block: scratch partials + arrival counter ----
-            if (warp == 0) __threadfence();
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                const unsigned int old = atomicAdd(pr.counters + rb, 1u);
-                s_last = (old == static_cast<unsigned int>(pl.CS - 1));
-            }
-            __syncthreads();
-            if (s_last && warp == 0) {
-                __threadfence();
+        float *rd = red + slot * red_slot;
 #pragma unroll
-                for (int b = 0; b < NB; ++b) {
-                    if (b < pr.nb) {
-                        float tot = 0.f;
-                        for (int c2 = 0; c2 < pl.CS; ++c2)
-                            tot += __ldcg(pr.partial + ((static_cast<int64_t>(rb) * pl.CS + c2) * pr.nb + b) * kRows + lane);
-                        if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
-                    }
-                }
-                if (lane == 0) pr.counters[rb] = 0u;   // leave the counter ready for the next call
-            }
+        for (int b = 0; b < NB; ++b) rd[(warp * NB + b) * kRows + lane] = ysum[b];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedFull + slot));
+        if (++s == pl.stages) {
+            s = 0;
+            phase ^= 1u;
         }
     }
 }
 
 template <int FMT, int NB>
-__global__ void __launch_bounds__(kMaxWarps * 32, 1) gemv_kernel(const Problem pr, const Plan pl) {
+__global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_kernel(const Problem pr, const Plan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
     run_problem<FMT, NB>(pr, pl, smem, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
 }
 
 template <int NB>
-__global__ void __launch_bounds__(kMaxWarps * 32, 1) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
+__global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int grp = blockIdx.y;
+    // the routing lists may come from the previous kernel in the stream
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int e = __ldg(ga.group_expert + grp);
     const int begin = __ldg(ga.group_begin + grp), end = __ldg(ga.group_begin + grp + 1);
     if (e < 0 || e >= ga.n_experts || end <= begin) return;
@@ -731,14 +960,15 @@ inline int check_cuda(cudaError_t e) {
 // done on the first call for a given kernel instantiation and device and remembered (so that
 // first call must not happen during stream capture; later calls only read the cache).
 template <auto kernel>
-int prepare_kernel(int *sms_out) {
+int prepare_kernel(int *sms_out, int *smem_budget_out) {
     constexpr int kMaxDev = 32;
-    static int cache[kMaxDev];      // multiprocessor count, 0 = not prepared yet
+    static int cache[kMaxDev][2];      // [0] multiprocessor count (0 = not prepared yet), [1] dynamic smem budget
     int dev = 0;
     int rc = check_cuda(cudaGetDevice(&dev));
     if (rc) return rc;
-    if (dev < kMaxDev && cache[dev] > 0) {
-        *sms_out = cache[dev];
+    if (dev < kMaxDev && cache[dev][0] > 0) {
+        *sms_out = cache[dev][0];
+        *smem_budget_out = cache[dev][1];
         return BITCOS_OK;
     }
     int sms = 0, max_smem = 0;
@@ -746,32 +976,71 @@ int prepare_kernel(int *sms_out) {
     if (rc) return rc;
     rc = check_cuda(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     if (rc) return rc;
-    rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem - 1024));
+    const int budget = max_smem - 1024;
+    rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, budget));
     if (rc) return rc;
-    if (dev < kMaxDev) cache[dev] = sms;
+    if (dev < kMaxDev) {
+        cache[dev][1] = budget;
+        cache[dev][0] = sms;
+    }
     *sms_out = sms;
+    *smem_budget_out = budget;
     return BITCOS_OK;
 }
 
-// Persistent grid: one block per multiprocessor; a multiple of CS so that a block always works
-// on the same column block and can keep that block's activations in shared memory.
-inline int grid_size(const Plan &pl, int sms) {
-    int64_t g = pl.items < sms ? pl.items : sms;
-    if (pl.CS > 1) {
-        g = g / pl.CS * pl.CS;
-        if (g < pl.CS) g = pl.CS;
+// Ring depth: as many stages as fit next to the tables, activations and partial sums (the loaded
+// DRAM latency of this part needs on the order of 100 KB in flight per multiprocessor).
+inline int choose_stages(int fmt, const Plan &pl, int G, int nb, int64_t K, int smem_budget) {
+    Plan p = pl;
+    for (int st = kMaxStages; st > 2; --st) {
+        p.stages = st;
+        if (static_cast<int>(smem_layout(fmt, p, G, nb, K).total) <= smem_budget) return st;
     }
-    return static_cast<int>(g);
+    return 2;
+}
+
+// Persistent grid: one block per multiprocessor (fewer if there are fewer items).
+inline int grid_size(const Plan &pl, int sms) { return static_cast<int>(pl.items < sms ? pl.items : sms); }
+
+// Round robin over row-block chunks when every block gets many of them (imbalance <= 1/8),
+// else a contiguous balanced split.  BITCOS_WALK=cyclic|contiguous overrides (for A/B runs).
+inline int choose_cyclic(const Plan &pl, int grid) {
+    static const char *force = std::getenv("BITCOS_WALK");
+    if (force && force[0] == 'c' && force[1] == 'y') return 1;
+    if (force && force[0] == 'c' && force[1] == 'o') return 0;
+    return (pl.items / pl.CS) >= 8 * static_cast<int64_t>(grid) ? 1 : 0;
+}
+
+// Launches with programmatic stream serialization, so that this kernel's prologue (barrier
+// set-up, table and first weight copies) may overlap the tail of the previous kernel in the
+// stream.  BITCOS_PDL=0 turns it off (for A/B runs).
+template <typename... KArgs, typename... Args>
+int launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t stream, Args... args) {
+    static const char *env = std::getenv("BITCOS_PDL");
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(static_cast<unsigned>(threads));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (env && env[0] == '0') ? 0 : 1;
+    return check_cuda(cudaLaunchKernelEx(&cfg, kernel, args...));
 }
 
 template <int FMT, int NB>
 int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
-    int sms = 0;
-    int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms);
+    int sms = 0, budget = 0;
+    int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms, &budget);
     if (rc) return rc;
-    const SmemLayout L = smem_layout(FMT, pl, pr.G, NB);
-    gemv_kernel<FMT, NB><<<grid_size(pl, sms), pl.NW * 32, L.total, stream>>>(pr, pl);
-    return check_cuda(cudaGetLastError());
+    const int grid = grid_size(pl, sms);
+    Plan plw = pl;
+    plw.cyclic = choose_cyclic(pl, grid);
+    plw.stages = choose_stages(FMT, pl, pr.G, NB, pr.K, budget);
+    const SmemLayout L = smem_layout(FMT, plw, pr.G, NB, pr.K);
+    return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw);
 }
 
 template <int FMT>
@@ -785,20 +1054,18 @@ int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream) {
 
 template <int NB>
 int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int n_groups, cudaStream_t stream) {
-    int sms = 0;
-    int rc = prepare_kernel<gemv_grouped_kernel<NB>>(&sms);
+    int sms = 0, budget = 0;
+    int rc = prepare_kernel<gemv_grouped_kernel<NB>>(&sms, &budget);
     if (rc) return rc;
-    const SmemLayout L = smem_layout(kBitcos, pl, pr.G, NB);
     // the machine is shared by all groups: spread its multiprocessors over them
     int gx = (sms + n_groups - 1) / n_groups;
     if (gx > pl.items) gx = static_cast<int>(pl.items);
-    if (pl.CS > 1) {
-        gx = gx / pl.CS * pl.CS;
-        if (gx < pl.CS) gx = pl.CS;
-    }
     if (gx < 1) gx = 1;
-    gemv_grouped_kernel<NB><<<dim3(gx, n_groups), pl.NW * 32, L.total, stream>>>(pr, pl, ga);
-    return check_cuda(cudaGetLastError());
+    Plan plw = pl;
+    plw.cyclic = choose_cyclic(pl, gx);
+    plw.stages = choose_stages(kBitcos, pl, pr.G, NB, pr.K, budget);
+    const SmemLayout L = smem_layout(kBitcos, plw, pr.G, NB, pr.K);
+    return launch_pdl(gemv_grouped_kernel<NB>, dim3(gx, n_groups), (pl.NW + 2) * 32, L.total, stream, pr, plw, ga);
 }
 
 int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const uint32_t *tile_off,
@@ -807,13 +1074,13 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
     if (!payload || !scales || !x || !x_scale || !y || !workspace) return BITCOS_ERR_NULL;
     if (fmt == kBitcos && (!signs || !tile_off)) return BITCOS_ERR_NULL;
     if (M < 1 || K < kGroup || K % kGroup != 0 || batch < 1 || batch > BITCOS_MAX_BATCH) return BITCOS_ERR_SHAPE;
-    if (K / kGroup > 0x7FFFFF || make_plan(M, K).items > 0x3FFFFFFF) return BITCOS_ERR_SHAPE;
+    if (K / kGroup > 0x7FFFFF || make_plan(M, K, kMaxWarps / 2).items > 0x3FFFFFFF) return BITCOS_ERR_SHAPE;
     if (!aligned16(payload) || !aligned16(scales) || !aligned16(x) || !aligned16(y) || !aligned16(workspace) ||
         (signs && !aligned16(signs)) || (tile_off && !aligned16(tile_off)) || (acc_debug && !aligned16(acc_debug)))
         return BITCOS_ERR_ALIGN;
     if (workspace_bytes < workspace_bytes_for(M, K)) return BITCOS_ERR_CAPACITY;
 
-    const Plan pl = make_plan(M, K);
+    const Plan pl = make_plan(M, K, decoder_warps(batch));
     Problem pr{};
     pr.payload = payload;
     pr.signs = signs;
@@ -937,7 +1204,7 @@ int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M,
     const size_t stride = workspace_bytes_for(M, K);
     if (workspace_bytes < stride * static_cast<size_t>(n_groups)) return BITCOS_ERR_CAPACITY;
 
-    const Plan pl = make_plan(M, K);
+    const Plan pl = make_plan(M, K, decoder_warps(max_group_size));
     Problem pr{};
     pr.x = x;
     pr.x_scale = x_scale;
