@@ -164,6 +164,31 @@ int bitcos_workspace_status(const void *workspace, void *cuda_stream, int *statu
 int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
                 int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The same product as bitcos_gemv without a caller-provided workspace.  (The paper has no
+ * counterpart: this entry point exists for the library's users, not for the method.)
+ *
+ * Who needs it: code that is not allowed to allocate device memory at the point where it
+ * multiplies -- a serving loop whose memory was sized and handed out at start-up, a plug-in
+ * that runs inside somebody else's memory pool, a latency-critical path where cudaMalloc's
+ * implicit device-wide synchronisation is unacceptable.  The scratch bytes come from a fixed
+ * array of BITCOS_STATIC_WORKSPACE_BYTES inside the library image; every device that loads the
+ * library holds that array until the process exits.  The call allocates nothing and calls no
+ * allocating routine; x, x_scale and y are still the caller's device buffers (as in
+ * bitcos_gemv; acc_debug is not offered).
+ *
+ * Limits and rules
+ *   - ERR_CAPACITY if bitcos_gemv_workspace_bytes(M, K) exceeds BITCOS_STATIC_WORKSPACE_BYTES
+ *     (all shapes of the benchmark configurations fit).
+ *   - The first call on a device looks the array's device address up (cudaGetSymbolAddress,
+ *     with that device current) and keeps it; make that first call outside stream capture.
+ *   - All calls on a device share the one array and it keeps the last call's contents: each
+ *     call first clears the status word and the arrival counters on the given stream.  Two
+ *     calls that may overlap on the GPU (different streams, no ordering between them) race on
+ *     it: order them, or give one of them bitcos_gemv with its own workspace. */
+#define BITCOS_STATIC_WORKSPACE_BYTES (8 * 1024 * 1024)
+int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
+                       void *cuda_stream);
+
 /* Host-buffer form of bitcos_gemv for callers whose activations live in host memory: copies
  * x_host[batch][K] and x_scale_host[batch] into `staging`, runs bitcos_gemv, copies
  * y[batch][M] back to y_host and waits for the stream, so y_host is valid on return.  The

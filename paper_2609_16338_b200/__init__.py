@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     bitcos_gemv_grouped,
     bitcos_gemv_host,
     bitcos_gemv_host_staging_bytes,
+    bitcos_gemv_static,
     group_pairs,
     plain_to_device,
     scales_tile,

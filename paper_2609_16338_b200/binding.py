@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_unpack", "bitcos_scales_tile", "bitcos_scales_untile", "trit5_pack_sizes", "trit5_pack",
     "trit5_unpack", "bit2_pack_sizes", "bit2_pack", "bit2_unpack", "bitcos_gemv_workspace_bytes",
     "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
-    "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host",
+    "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static",
 ]
 
 
@@ -81,6 +81,7 @@ def load_library():
     L.bitcos_gemv_host_staging_bytes.restype = sz
     L.bitcos_gemv_host_staging_bytes.argtypes = [i64, i64, C.c_int]
     L.bitcos_gemv_host.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, sz, vp, sz, vp]
+    L.bitcos_gemv_static.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp]
     _lib = L
     return L
 
@@ -352,6 +353,20 @@ def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, 
                                               acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
                                               workspace.numel(), _stream()), "bitcos_gemv_grouped")
     return y, acc
+
+
+STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024
+
+
+def bitcos_gemv_static(W: DeviceBitcos, x, x_scale, y):
+    """bitcos_gemv for callers that may not allocate: the scratch memory is a fixed array inside
+    the library (at most STATIC_WORKSPACE_BYTES), so nothing is allocated here either -- `y` must be
+    the caller's own [batch, M] float32 CUDA tensor.  Calls on one device share that array: do not
+    let two of them overlap on the GPU.  The first call on a device must not be inside a stream
+    capture."""
+    _check(load_library().bitcos_gemv_static(C.byref(W.desc), x.data_ptr(), x_scale.data_ptr(), x.shape[0],
+                                             y.data_ptr(), _stream()), "bitcos_gemv_static")
+    return y
 
 
 def bitcos_gemv_host_staging_bytes(M: int, K: int, batch: int) -> int:

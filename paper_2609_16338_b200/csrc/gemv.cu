@@ -1142,6 +1142,60 @@ int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, 
                        acc_debug, workspace, workspace_bytes, cuda_stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// bitcos_gemv_static: the same product with the scratch memory taken from a fixed array that is
+// part of the library image, for callers that must not (or cannot) allocate device memory.
+// ---------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+// Scratch of the no-allocation entry point.  Every device that loads the library carries these
+// bytes until the process exits.  In host code the name below is only a handle for
+// cudaGetSymbolAddress; it is not a device address and is never passed to a kernel.
+static __device__ __align__(256) unsigned char g_static_workspace[BITCOS_STATIC_WORKSPACE_BYTES];
+
+// Device address of g_static_workspace on the current device, looked up once per device.
+int static_workspace_ptr(void **out) {
+    constexpr int kMaxDev = 32;
+    static void *cache[kMaxDev];
+    int dev = 0;
+    int rc = check_cuda(cudaGetDevice(&dev));
+    if (rc) return rc;
+    if (dev < kMaxDev && cache[dev]) {
+        *out = cache[dev];
+        return BITCOS_OK;
+    }
+    void *ptr = nullptr;
+    rc = check_cuda(cudaGetSymbolAddress(&ptr, g_static_workspace));
+    if (rc) return rc;
+    if (!ptr) return BITCOS_ERR_CUDA;
+    if (dev < kMaxDev) cache[dev] = ptr;
+    *out = ptr;
+    return BITCOS_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
+                       void *cuda_stream) {
+    if (!W) return BITCOS_ERR_NULL;
+    if (W->M < 1 || W->K < kGroup || W->K % kGroup != 0) return BITCOS_ERR_SHAPE;
+    const size_t need = workspace_bytes_for(W->M, W->K);
+    if (need > static_cast<size_t>(BITCOS_STATIC_WORKSPACE_BYTES)) return BITCOS_ERR_CAPACITY;
+    void *ws = nullptr;
+    int rc = static_workspace_ptr(&ws);
+    if (rc) return rc;
+    // The array keeps whatever the last call left.  The status word and the arrival counters must
+    // start at zero, so they are cleared on the caller's stream ahead of the kernel (the partial
+    // sums behind them are always written before they are read).
+    const size_t head = kHeaderBytes + counters_bytes(padded_rows(W->M) / kRows);
+    rc = check_cuda(cudaMemsetAsync(ws, 0, head, static_cast<cudaStream_t>(cuda_stream)));
+    if (rc) return rc;
+    return gemv_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_scale, batch, y,
+                       nullptr, ws, BITCOS_STATIC_WORKSPACE_BYTES, cuda_stream);
+}
+
 size_t bitcos_gemv_host_staging_bytes(int64_t M, int64_t K, int batch) {
     if (M < 1 || K < kGroup || K % kGroup != 0 || batch < 1 || batch > BITCOS_MAX_BATCH) return 0;
     const size_t xb = (static_cast<size_t>(batch) * K + 255) / 256 * 256;
