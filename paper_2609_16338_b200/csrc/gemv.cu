@@ -137,6 +137,7 @@ struct Plan {
     int64_t items;   // ceil(RB / RBC) * CS
     int cyclic;      // 1: blocks take whole row-block chunks round robin; 0: contiguous balanced ranges
     int stages;      // depth of the shared-memory ring (2 .. kMaxStages), set at launch
+    int probe;       // measurement aid (BITCOS_PROBE=copy): stream the weights but skip the decode
 };
 
 struct Problem {
@@ -218,6 +219,10 @@ struct SmemLayout {
 
 __host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
+// Partial-sum slots between the decoder warps and the epilogue warp (how many items the
+// decoders may run ahead of it).
+__host__ __device__ constexpr int red_slots(int nbmax) { return nbmax <= 2 ? 4 : 2; }
+
 __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G, int nbmax, int64_t K) {
     SmemLayout L{};
     uint32_t off = 0;
@@ -245,7 +250,7 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     L.x_bytes = (static_cast<int64_t>(nbmax) * K <= kXResidentBytes) ? static_cast<uint32_t>(nbmax * K) : 0u;
     off += align_up(L.x_bytes, 128);
     L.red = off;
-    off += 2 * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;      // two slots
+    off += static_cast<uint32_t>(red_slots(nbmax)) * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
     L.bar = off;
     off += 256;
     L.total = off;
@@ -561,10 +566,10 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
 // mbarrier slots inside the `bar` region (8 bytes each)
 constexpr int kBarFull = 0;                       // [stages] stage filled by the copy engine
 constexpr int kBarEmpty = kMaxStages;             // [stages] stage released by all decoder warps
-constexpr int kBarRedFull = 2 * kMaxStages;       // [2] partial sums of an item written by all decoder warps
-constexpr int kBarRedEmpty = 2 * kMaxStages + 2;  // [2] partial sums consumed by the epilogue warp
-constexpr int kBarLut = 2 * kMaxStages + 4;       // lookup table arrived
-constexpr int kBarCount = 2 * kMaxStages + 5;
+constexpr int kBarRedFull = 2 * kMaxStages;       // [slots] partial sums of an item written by all decoder warps
+constexpr int kBarRedEmpty = 2 * kMaxStages + 4;  // [slots] partial sums consumed by the epilogue warp
+constexpr int kBarLut = 2 * kMaxStages + 8;       // lookup table arrived
+constexpr int kBarCount = 2 * kMaxStages + 9;
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -627,7 +632,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 mbar_init(bar0 + 8u * (kBarFull + s), 1);
                 mbar_init(bar0 + 8u * (kBarEmpty + s), pl.NW);
             }
-            for (int s = 0; s < 2; ++s) {
+            for (int s = 0; s < red_slots(NB); ++s) {
                 mbar_init(bar0 + 8u * (kBarRedFull + s), pl.NW);
                 mbar_init(bar0 + 8u * (kBarRedEmpty + s), 1);
             }
@@ -637,26 +642,27 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         }
         // The first copies go out before the block-wide barrier below, while the other warps are
         // still fetching the activations.
-        ItemIter it;
-        ItemRange r{};
-        uint32_t o_lo = 0, o_hi = 0;
+        // Entry offsets are requested two items before they are needed (r0 = item k, r1 = item
+        // k + 1, r2 = item k + 2), so that the load is never waited for.
+        ItemIter it2;
+        ItemRange r0{}, r1{}, r2{};
+        uint32_t lo0 = 0, hi0 = 0, lo1 = 0, hi1 = 0;
         int k0 = 0, ps = 0;
         uint32_t pphase = 1;       // parity of the phase before the one the decoders complete next
         bool ok = true;
+        auto offsets = [&](const ItemRange &prev, uint32_t prev_hi, const ItemRange &r, uint32_t &lo, uint32_t &hi) {
+            if (FMT != kBitcos) return;
+            lo = (r.t0 == prev.t0 + prev.nt) ? prev_hi : __ldg(pr.tile_off + r.t0);
+            hi = __ldg(pr.tile_off + r.t0 + r.nt);
+        };
         auto issue_loop = [&](int k_end) {
             for (int k = k0; k < k_end; ++k) {
                 const int s = ps;
-                // offsets of the next item, requested before this item's copies are issued
-                ItemIter nx = it;
-                nx.next(pl, wk);
-                ItemRange rn = r;
-                uint32_t n_lo = 0, n_hi = 0;
-                if (k + 1 < wk.count) {
-                    rn = item_range(pr, pl, nx.c, nx.cs);
-                    if (FMT == kBitcos) {
-                        n_lo = (rn.t0 == r.t0 + r.nt) ? o_hi : __ldg(pr.tile_off + rn.t0);
-                        n_hi = __ldg(pr.tile_off + rn.t0 + rn.nt);
-                    }
+                uint32_t lo2 = 0, hi2 = 0;
+                if (k + 2 < wk.count) {
+                    it2.next(pl, wk);
+                    r2 = item_range(pr, pl, it2.c, it2.cs);
+                    offsets(r1, hi1, r2, lo2, hi2);
                 }
                 if (k >= pl.stages) {
                     if (!mbar_wait(bar0 + 8u * (kBarEmpty + s), pphase)) {
@@ -666,16 +672,14 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
-                issue_item<FMT>(pr, pl, r, L, smem, s, sign_base, o_lo, o_hi);
+                issue_item<FMT>(pr, pl, r0, L, smem, s, sign_base, lo0, hi0);
                 if (k == 0 && FMT != kBit2) {
                     mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
                     bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
                               bar0 + 8u * kBarLut);
                 }
-                it = nx;
-                r = rn;
-                o_lo = n_lo;
-                o_hi = n_hi;
+                r0 = r1; lo0 = lo1; hi0 = hi1;
+                r1 = r2; lo1 = lo2; hi1 = hi2;
                 if (++ps == pl.stages) {
                     ps = 0;
                     pphase ^= 1u;
@@ -684,11 +688,16 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             k0 = k_end;
         };
         if (lane == 0 && wk.count > 0) {
-            it.init(pl, wk.first);
-            r = item_range(pr, pl, it.c, it.cs);
+            it2.init(pl, wk.first);
+            r0 = item_range(pr, pl, it2.c, it2.cs);
             if (FMT == kBitcos) {
-                o_lo = __ldg(pr.tile_off + r.t0);
-                o_hi = __ldg(pr.tile_off + r.t0 + r.nt);
+                lo0 = __ldg(pr.tile_off + r0.t0);
+                hi0 = __ldg(pr.tile_off + r0.t0 + r0.nt);
+            }
+            if (wk.count > 1) {
+                it2.next(pl, wk);
+                r1 = item_range(pr, pl, it2.c, it2.cs);
+                offsets(r0, hi0, r1, lo1, hi1);
             }
             issue_loop(wk.count < pl.stages ? wk.count : pl.stages);
         }
@@ -731,14 +740,32 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         float run[NB];          // running sum of the current row block over this block's items
 #pragma unroll
         for (int b = 0; b < NB; ++b) run[b] = 0.f;
+        float xsc[NB];          // per-token activation scales
+#pragma unroll
+        for (int b = 0; b < NB; ++b) xsc[b] = __ldg(pr.x_scale + xr[b]);
         Share pend[2];
         int n_pend = 0;
         ItemIter it;
         it.init(pl, wk.first);
+        constexpr int RS = red_slots(NB);
+        // sum of n partial sums of token b, spaced NB * 32 floats apart: four interleaved
+        // accumulators, always combined in the same order
+        auto sum_groups = [&](const float *base, int n) {
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            int j = 0;
+            for (; j + 4 <= n; j += 4) {
+                a0 += base[(j + 0) * NB * kRows];
+                a1 += base[(j + 1) * NB * kRows];
+                a2 += base[(j + 2) * NB * kRows];
+                a3 += base[(j + 3) * NB * kRows];
+            }
+            for (; j < n; ++j) a0 += base[j * NB * kRows];
+            return (a0 + a1) + (a2 + a3);
+        };
         for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
-            const int slot = k & 1;
+            const int slot = k % RS;
             const ItemRange r = item_range(pr, pl, it.c, it.cs);
-            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k >> 1) & 1))) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k / RS) & 1))) {
                 if (lane == 0 && pr.status) *pr.status = 1u;
                 return;
             }
@@ -751,9 +778,8 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 #pragma unroll
                     for (int b = 0; b < NB; ++b) {
                         if (b < pr.nb) {
-                            float tot = 0.f;
-                            for (int j = 0; j < pr.G; ++j) tot += rs[((i * pr.G + j) * NB + b) * kRows + lane];
-                            if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
+                            const float tot = sum_groups(rs + (i * pr.G * NB + b) * kRows + lane, pr.G);
+                            if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = xsc[b] * tot;
                         }
                     }
                 }
@@ -766,8 +792,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 if (b < pr.nb) {
-                    float tot = 0.f;
-                    for (int j = 0; j < r.nt; ++j) tot += rs[(j * NB + b) * kRows + lane];
+                    const float tot = sum_groups(rs + b * kRows + lane, r.nt);
                     run[b] = starts ? tot : run[b] + tot;
                 }
             }
@@ -781,7 +806,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 // the whole row block was ours
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
-                    if (b < pr.nb && m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * run[b];
+                    if (b < pr.nb && m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = xsc[b] * run[b];
             } else {
                 // shared row block: publish our share, then count ourselves in
                 Share sh;
@@ -820,16 +845,24 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     it.init(pl, wk.first);
     int s = 0;
     uint32_t phase = 0;
-    for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
-        const int slot = k & 1;
-        const ItemRange r = item_range(pr, pl, it.c, it.cs);
+    constexpr int RS = red_slots(NB);
+    // the tile's entry offset is requested one item ahead
+    ItemRange r_next = item_range(pr, pl, it.c, it.cs);
+    uint32_t toff_next = 0;
+    if (FMT == kBitcos && warp < r_next.nt) toff_next = __ldg(pr.tile_off + r_next.t0 + warp);
+    for (int k = 0; k < wk.count; ++k) {
+        const int slot = k % RS;
+        const ItemRange r = r_next;
+        const uint32_t toff = toff_next;
         const bool busy = warp < r.nt;
         const int g = (pl.CS == 1) ? g_fixed : r.g0 + warp;
         const int rb = r.rb0 + my_rbl;
-        const int64_t t = r.t0 + warp;
         const int64_t m = static_cast<int64_t>(rb) * kRows + lane;
-        uint32_t toff = 0;
-        if (FMT == kBitcos && busy) toff = __ldg(pr.tile_off + t);
+        if (k + 1 < wk.count) {
+            it.next(pl, wk);
+            r_next = item_range(pr, pl, it.c, it.cs);
+            if (FMT == kBitcos && warp < r_next.nt) toff_next = __ldg(pr.tile_off + r_next.t0 + warp);
+        }
 
         if (!mbar_wait(bar0 + 8u * (kBarFull + s), phase)) {
             if (lane == 0 && pr.status) *pr.status = 1u;
@@ -840,7 +873,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 #pragma unroll
         for (int b = 0; b < NB; ++b) ysum[b] = 0.f;
 
-        if (busy) {
+        if (busy && !pl.probe) {
             const float sc = bf16_to_float(
                 reinterpret_cast<const uint16_t *>(stage + L.payload_cap + L.sign_cap)[warp * kRows + lane]);
             // activations of group g: in shared memory if resident (xs), else in global memory (xgl)
@@ -897,8 +930,8 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         if (lane == 0) mbar_arrive(bar0 + 8u * (kBarEmpty + s));
 
         // partial sums for the epilogue warp (two slots, so decoders may run an item ahead of it)
-        if (k >= 2) {
-            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>(((k >> 1) - 1) & 1))) {
+        if (k >= RS) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>((k / RS - 1) & 1))) {
                 if (lane == 0 && pr.status) *pr.status = 1u;
                 return;
             }
@@ -1039,6 +1072,8 @@ int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
     Plan plw = pl;
     plw.cyclic = choose_cyclic(pl, grid);
     plw.stages = choose_stages(FMT, pl, pr.G, NB, pr.K, budget);
+    static const char *probe = std::getenv("BITCOS_PROBE");
+    plw.probe = (probe && probe[0] == 'c') ? 1 : 0;
     const SmemLayout L = smem_layout(FMT, plw, pr.G, NB, pr.K);
     return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw);
 }
