@@ -221,7 +221,7 @@ __host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v
 
 // Partial-sum slots between the decoder warps and the epilogue warp (how many items the
 // decoders may run ahead of it).
-__host__ __device__ constexpr int red_slots(int nbmax) { return nbmax <= 2 ? 4 : 2; }
+__host__ __device__ constexpr int red_slots(int nbmax) { return nbmax <= 1 ? 8 : nbmax <= 2 ? 4 : 2; }
 
 __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G, int nbmax, int64_t K) {
     SmemLayout L{};
@@ -252,7 +252,7 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     L.red = off;
     off += static_cast<uint32_t>(red_slots(nbmax)) * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
     L.bar = off;
-    off += 256;
+    off += 384;
     L.total = off;
     return L;
 }
@@ -308,6 +308,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
             : "memory");
         if (done) return true;
         if ((i & 15u) == 15u) {
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
+        }
+    }
+}
+
+// The same wait without ever suspending the thread (mbarrier.test_wait in a tight loop): for the
+// one warp whose wake-up latency would otherwise sit on the critical path of every item.
+__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((i & 1023u) == 1023u) {
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > kWaitLimitNs) return false;
@@ -567,9 +589,9 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
 constexpr int kBarFull = 0;                       // [stages] stage filled by the copy engine
 constexpr int kBarEmpty = kMaxStages;             // [stages] stage released by all decoder warps
 constexpr int kBarRedFull = 2 * kMaxStages;       // [slots] partial sums of an item written by all decoder warps
-constexpr int kBarRedEmpty = 2 * kMaxStages + 4;  // [slots] partial sums consumed by the epilogue warp
-constexpr int kBarLut = 2 * kMaxStages + 8;       // lookup table arrived
-constexpr int kBarCount = 2 * kMaxStages + 9;
+constexpr int kBarRedEmpty = 2 * kMaxStages + 8;  // [slots] partial sums consumed by the epilogue warp
+constexpr int kBarLut = 2 * kMaxStages + 16;      // lookup table arrived
+constexpr int kBarCount = 2 * kMaxStages + 17;
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -737,6 +759,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 
     // ------------------------------------------------------------------ epilogue warp
     if (warp == pl.NW + 1) {
+        if (pl.probe == 2) return;
         float run[NB];          // running sum of the current row block over this block's items
 #pragma unroll
         for (int b = 0; b < NB; ++b) run[b] = 0.f;
@@ -765,7 +788,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
             const int slot = k % RS;
             const ItemRange r = item_range(pr, pl, it.c, it.cs);
-            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k / RS) & 1))) {
+            if (!mbar_spin(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k / RS) & 1))) {
                 if (lane == 0 && pr.status) *pr.status = 1u;
                 return;
             }
@@ -929,7 +952,14 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         __syncwarp();
         if (lane == 0) mbar_arrive(bar0 + 8u * (kBarEmpty + s));
 
-        // partial sums for the epilogue warp (two slots, so decoders may run an item ahead of it)
+        if (pl.probe == 2) {
+            if (++s == pl.stages) {
+                s = 0;
+                phase ^= 1u;
+            }
+            continue;
+        }
+        // partial sums for the epilogue warp (several slots, so decoders may run ahead of it)
         if (k >= RS) {
             if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>((k / RS - 1) & 1))) {
                 if (lane == 0 && pr.status) *pr.status = 1u;
@@ -1073,7 +1103,7 @@ int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
     plw.cyclic = choose_cyclic(pl, grid);
     plw.stages = choose_stages(FMT, pl, pr.G, NB, pr.K, budget);
     static const char *probe = std::getenv("BITCOS_PROBE");
-    plw.probe = (probe && probe[0] == 'c') ? 1 : 0;
+    plw.probe = (probe && probe[0] == 'c') ? 1 : (probe && probe[0] == 'd') ? 2 : 0;
     const SmemLayout L = smem_layout(FMT, plw, pr.G, NB, pr.K);
     return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw);
 }
