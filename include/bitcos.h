@@ -36,8 +36,8 @@
  *             32rb + r, bit i <-> k = 128g + 32j + i (LSB first);
  *   signs     uint32[]; bit q of the sign vector is bit (q & 31) of word q >> 5; the q-th
  *             sign bit belongs to the q-th set bit of the bitmap; 1 = negative (Eq. 4);
- *   tile_off  uint32[n_tiles + 1]; tile_off[t] = index of tile t's first sign bit,
- *             tile_off[n_tiles] = number of non-zero weights;
+ *   tile_off  uint32[n_tiles + 1], zero padded to a multiple of 16 bytes; tile_off[t] = index
+ *             of tile t's first sign bit, tile_off[n_tiles] = number of non-zero weights;
  *   scales    uint16[Mp*K/128] bf16 bit patterns, scale of (row 32rb + r, group g) at
  *             t*32 + r (padding rows +0).
  */

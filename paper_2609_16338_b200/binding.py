@@ -113,8 +113,9 @@ class PackedBitcos:
     nnz: int
     bitmap: np.ndarray      # uint32
     signs: np.ndarray       # uint32, zero slack included
-    tile_off: np.ndarray    # uint32 [n_tiles + 1]
+    tile_off: np.ndarray    # uint32 [n_tiles + 1] (a view of tile_off_buf without its padding)
     scales: np.ndarray      # uint16, tile order
+    tile_off_buf: np.ndarray = None     # tile_off zero padded to a multiple of 16 bytes, as uploaded
 
     def payload_bytes(self) -> int:
         """Bytes a GEMV has to read: bitmap, the sign bits (not the slack), offsets, scales."""
@@ -122,8 +123,9 @@ class PackedBitcos:
 
     def to_device(self, device="cuda"):
         import torch
+        off = self.tile_off_buf if self.tile_off_buf is not None else self.tile_off
         t = [torch.from_numpy(a.view(np.int32) if a.dtype == np.uint32 else a.view(np.int16)).to(device)
-             for a in (self.bitmap, self.signs, self.tile_off, self.scales)]
+             for a in (self.bitmap, self.signs, off, self.scales)]
         return DeviceBitcos(self.M, self.K, self.nnz, *t)
 
 
@@ -140,7 +142,8 @@ class DeviceBitcos:
                             self.tile_off.clone(), self.scales.clone())
 
     def payload_bytes(self) -> int:
-        return self.bitmap.numel() * 4 + (self.nnz + 7) // 8 + self.tile_off.numel() * 4 + self.scales.numel() * 2
+        n_tiles = (self.M + TILE_ROWS - 1) // TILE_ROWS * (self.K // GROUP)
+        return self.bitmap.numel() * 4 + (self.nnz + 7) // 8 + (n_tiles + 1) * 4 + self.scales.numel() * 2
 
 
 class DevicePlain:
@@ -167,12 +170,13 @@ def bitcos_pack(trits, scales_bf16) -> PackedBitcos:
     _check(L.bitcos_pack_sizes(M, K, nnz.value, *[C.byref(v) for v in sizes]), "bitcos_pack_sizes")
     bitmap = np.zeros(sizes[0].value // 4, np.uint32)
     signs = np.zeros(sizes[1].value // 4, np.uint32)
-    tile_off = np.zeros(sizes[2].value // 4, np.uint32)
+    tile_off_buf = np.zeros(sizes[2].value // 4, np.uint32)
     scales = np.zeros(sizes[3].value // 2, np.uint16)
     out = C.c_uint64(0)
-    _check(L.bitcos_pack(_ptr(t), _ptr(s), M, K, _ptr(bitmap), _ptr(signs), signs.nbytes, _ptr(tile_off),
+    _check(L.bitcos_pack(_ptr(t), _ptr(s), M, K, _ptr(bitmap), _ptr(signs), signs.nbytes, _ptr(tile_off_buf),
                          _ptr(scales), C.byref(out)), "bitcos_pack")
-    return PackedBitcos(M, K, int(out.value), bitmap, signs, tile_off, scales)
+    n_tiles = (M + TILE_ROWS - 1) // TILE_ROWS * (K // GROUP)
+    return PackedBitcos(M, K, int(out.value), bitmap, signs, tile_off_buf[:n_tiles + 1], scales, tile_off_buf)
 
 
 def bitcos_unpack(p: PackedBitcos) -> np.ndarray:

@@ -209,7 +209,7 @@ struct SmemLayout {
     uint32_t lut;        // lookup tables (0 bytes for 2-bit)
     uint32_t stage;      // stage 0
     uint32_t stage_bytes;
-    uint32_t payload_cap, sign_cap, scale_cap;   // per-stage capacities
+    uint32_t payload_cap, sign_cap, scale_cap, off_cap;   // per-stage capacities
     uint32_t x;          // activations, [nb][K], if x_bytes != 0
     uint32_t x_bytes;    // 0: the activations do not fit and are read from global memory
     uint32_t red;        // 2 x [NW][NB][32] floats
@@ -232,6 +232,7 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     if (fmt == kBitcos) {
         L.payload_cap = tiles * 512;
         L.sign_cap = tiles * 512 + 64;
+        L.off_cap = 128;                 // the item's slice of tile_off (at most 21 + 3 + 3 words)
     } else if (fmt == kTrit5) {
         const uint32_t WPR = (26u * static_cast<uint32_t>(G) + 3) / 4;
         // whole rows when CS == 1, else at most CG groups (+1 shared word) of one row block
@@ -244,7 +245,7 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     }
     L.scale_cap = tiles * 64;
     L.stage = off;
-    L.stage_bytes = align_up(L.payload_cap + L.sign_cap + L.scale_cap, 128);
+    L.stage_bytes = align_up(L.payload_cap + L.sign_cap + L.scale_cap + L.off_cap, 128);
     off += L.stage_bytes * static_cast<uint32_t>(pl.stages);
     L.x = off;
     L.x_bytes = (static_cast<int64_t>(nbmax) * K <= kXResidentBytes) ? static_cast<uint32_t>(nbmax * K) : 0u;
@@ -308,28 +309,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
             : "memory");
         if (done) return true;
         if ((i & 15u) == 15u) {
-            const uint64_t now = global_timer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
-        }
-    }
-}
-
-// The same wait without ever suspending the thread (mbarrier.test_wait in a tight loop): for the
-// one warp whose wake-up latency would otherwise sit on the critical path of every item.
-__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity) {
-    uint64_t t0 = 0;
-    for (uint32_t i = 0;; ++i) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if ((i & 1023u) == 1023u) {
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > kWaitLimitNs) return false;
@@ -563,7 +542,11 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
         const uint32_t sign_bytes = b_hi - b_lo;
         const uint32_t bm_bytes = static_cast<uint32_t>(r.nt) * 512u;
         sign_base[s] = b_lo * 8u;
-        mbar_expect_tx(bar, bm_bytes + sign_bytes + scale_bytes);
+        // the tiles' entry offsets: the 16-byte aligned slice of tile_off that covers t0 .. t0 + nt
+        const uint32_t o_first = static_cast<uint32_t>(r.t0 & 3);
+        const uint32_t off_bytes = ((o_first + static_cast<uint32_t>(r.nt) + 1u + 3u) & ~3u) * 4u;
+        mbar_expect_tx(bar, bm_bytes + sign_bytes + scale_bytes + off_bytes);
+        bulk_copy(d_scales + L.scale_cap, pr.tile_off + (r.t0 - o_first), off_bytes, bar);
         bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + r.t0 * 512, bm_bytes, bar);
         if (sign_bytes) bulk_copy(d_signs, reinterpret_cast<const uint8_t *>(pr.signs) + b_lo, sign_bytes, bar);
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
@@ -788,26 +771,30 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
             const int slot = k % RS;
             const ItemRange r = item_range(pr, pl, it.c, it.cs);
-            if (!mbar_spin(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k / RS) & 1))) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k / RS) & 1))) {
                 if (lane == 0 && pr.status) *pr.status = 1u;
                 return;
             }
             const float *rs = red + slot * red_slot;
             if (pl.CS == 1) {
-                // whole row blocks: one output per row, groups added in ascending order
+                // whole row blocks: one output per row.  The sums are formed first, the slot is
+                // handed back, and only then are the outputs stored, so that the release of the
+                // slot never waits for a global store.
                 const int nrb = r.nt / pr.G;
                 for (int i = 0; i < nrb; ++i) {
                     const int64_t m = static_cast<int64_t>(r.rb0 + i) * kRows + lane;
+                    float t_b[NB];
 #pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        if (b < pr.nb) {
-                            const float tot = sum_groups(rs + (i * pr.G * NB + b) * kRows + lane, pr.G);
-                            if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = xsc[b] * tot;
-                        }
+                    for (int b = 0; b < NB; ++b)
+                        t_b[b] = (b < pr.nb) ? sum_groups(rs + (i * pr.G * NB + b) * kRows + lane, pr.G) : 0.f;
+                    if (i == nrb - 1) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedEmpty + slot));
                     }
+#pragma unroll
+                    for (int b = 0; b < NB; ++b)
+                        if (b < pr.nb && m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = xsc[b] * t_b[b];
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedEmpty + slot));
                 continue;
             }
             // one column block of row block rb0: add it to the running sum
@@ -869,23 +856,13 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     int s = 0;
     uint32_t phase = 0;
     constexpr int RS = red_slots(NB);
-    // the tile's entry offset is requested one item ahead
-    ItemRange r_next = item_range(pr, pl, it.c, it.cs);
-    uint32_t toff_next = 0;
-    if (FMT == kBitcos && warp < r_next.nt) toff_next = __ldg(pr.tile_off + r_next.t0 + warp);
-    for (int k = 0; k < wk.count; ++k) {
+    for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
         const int slot = k % RS;
-        const ItemRange r = r_next;
-        const uint32_t toff = toff_next;
+        const ItemRange r = item_range(pr, pl, it.c, it.cs);
         const bool busy = warp < r.nt;
         const int g = (pl.CS == 1) ? g_fixed : r.g0 + warp;
         const int rb = r.rb0 + my_rbl;
         const int64_t m = static_cast<int64_t>(rb) * kRows + lane;
-        if (k + 1 < wk.count) {
-            it.next(pl, wk);
-            r_next = item_range(pr, pl, it.c, it.cs);
-            if (FMT == kBitcos && warp < r_next.nt) toff_next = __ldg(pr.tile_off + r_next.t0 + warp);
-        }
 
         if (!mbar_wait(bar0 + 8u * (kBarFull + s), phase)) {
             if (lane == 0 && pr.status) *pr.status = 1u;
@@ -913,6 +890,9 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                     const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
                     if (lane >= d) incl += v;
                 }
+                // entry offset of this tile: word (t0 & 3) + warp of the stage's slice of tile_off
+                const uint32_t toff = reinterpret_cast<const uint32_t *>(
+                    stage + L.payload_cap + L.sign_cap + L.scale_cap)[static_cast<uint32_t>(r.t0 & 3) + warp];
                 const uint32_t cursor = toff + static_cast<uint32_t>(incl - c) - sign_base[s];
                 const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + L.payload_cap) + (cursor >> 5);
                 if (NB == 1 && x_resident)

@@ -112,7 +112,7 @@ int bitcos_pack_sizes(int64_t M, int64_t K, uint64_t nnz, size_t *bitmap_bytes, 
     if (nnz > 0xFFFFFFFFull) return BITCOS_ERR_OVERFLOW;
     if (bitmap_bytes) *bitmap_bytes = static_cast<size_t>(Mp * K / 8);
     if (sign_bytes) *sign_bytes = sign_bytes_for(nnz);
-    if (tile_off_bytes) *tile_off_bytes = static_cast<size_t>((Mp / kRows) * G + 1) * 4;
+    if (tile_off_bytes) *tile_off_bytes = (static_cast<size_t>((Mp / kRows) * G + 1) * 4 + 15) / 16 * 16;
     if (scale_bytes) *scale_bytes = static_cast<size_t>(Mp * G) * 2;
     return BITCOS_OK;
 }
@@ -198,6 +198,7 @@ int bitcos_pack(const int8_t *trits, const uint16_t *scales_bf16, int64_t M, int
         if (run > 0xFFFFFFFFull) return BITCOS_ERR_OVERFLOW;
     }
     tile_off[T] = static_cast<uint32_t>(run);
+    for (int64_t t = T + 1; t < (T + 1 + 3) / 4 * 4; ++t) tile_off[t] = 0;     // padding to 16 bytes
     const size_t need = sign_bytes_for(run);
     if (sign_capacity_bytes < need) return BITCOS_ERR_CAPACITY;
     std::memset(signs, 0, need);
