@@ -754,19 +754,17 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         ItemIter it;
         it.init(pl, wk.first);
         constexpr int RS = red_slots(NB);
-        // sum of n partial sums of token b, spaced NB * 32 floats apart: four interleaved
-        // accumulators, always combined in the same order
+        // sum of n <= 20 partial sums of token b, spaced NB * 32 floats apart: all loads are issued
+        // before the first addition, and the additions always follow the same tree
         auto sum_groups = [&](const float *base, int n) {
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-            int j = 0;
-            for (; j + 4 <= n; j += 4) {
-                a0 += base[(j + 0) * NB * kRows];
-                a1 += base[(j + 1) * NB * kRows];
-                a2 += base[(j + 2) * NB * kRows];
-                a3 += base[(j + 3) * NB * kRows];
-            }
-            for (; j < n; ++j) a0 += base[j * NB * kRows];
-            return (a0 + a1) + (a2 + a3);
+            float v[kMaxWarps];
+#pragma unroll
+            for (int j = 0; j < kMaxWarps; ++j) v[j] = (j < n) ? base[j * NB * kRows] : 0.f;
+#pragma unroll
+            for (int w2 = 1; w2 < kMaxWarps; w2 *= 2)
+#pragma unroll
+                for (int j = 0; j + w2 < kMaxWarps; j += 2 * w2) v[j] += v[j + w2];
+            return v[0];
         };
         for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
             const int slot = k % RS;
