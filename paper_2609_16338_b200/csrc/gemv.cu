@@ -253,7 +253,7 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     L.red = off;
     off += static_cast<uint32_t>(red_slots(nbmax)) * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
     L.bar = off;
-    off += 384;
+    off += 512;          // mbarriers, then (16-byte aligned) one 16-byte item descriptor per stage
     L.total = off;
     return L;
 }
@@ -294,26 +294,34 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Waits for the given phase parity, for at most kWaitLimitNs; false if it gave up.  Each poll may
-// suspend the thread for up to about a microsecond.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done;
+}
+// Polls until the phase completes, for at most kWaitLimitNs; false if it gave up.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
     uint64_t t0 = 0;
     for (uint32_t i = 0;; ++i) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity), "r"(1000u)
-            : "memory");
-        if (done) return true;
+        if (mbar_try(bar, parity)) return true;
         if ((i & 15u) == 15u) {
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > kWaitLimitNs) return false;
         }
     }
+}
+// Waits for the given phase parity (bounded); the common case, an already completed phase, costs
+// one instruction.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity);
 }
 
 // d = (a & c) | (b & ~c): one LOP3
@@ -524,8 +532,8 @@ struct ItemIter {
     }
 };
 
-// Issues the bulk copies of one item into stage `s` (one thread).  sign_base[s] receives the bit
-// index of the first sign bit held in the stage's sign buffer.  o_lo / o_hi: sign-vector
+// Issues the bulk copies of one item into stage `s` (one thread) and publishes the item's
+// descriptor (sign_base[4s .. 4s+3]; word 3 = index of the first sign bit held in the stage).  o_lo / o_hi: sign-vector
 // positions of the item's first tile and of the tile after its last (BITCOS only).
 template <int FMT>
 __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, const ItemRange &r, const SmemLayout &L,
@@ -537,11 +545,15 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
     const uint32_t d_scales = d_signs + L.sign_cap;
     const uint32_t scale_bytes = static_cast<uint32_t>(r.nt) * 64u;
     const uint8_t *g_scales = reinterpret_cast<const uint8_t *>(pr.scales) + r.t0 * 64;
+    // what the decoder warps need to know about the item (read by them once the stage is full)
+    sign_base[s * 4 + 0] = static_cast<uint32_t>(r.nt) | (static_cast<uint32_t>(r.t0 & 3) << 8);
+    sign_base[s * 4 + 1] = static_cast<uint32_t>(r.g0);
+    sign_base[s * 4 + 2] = static_cast<uint32_t>(r.rb0);
     if (FMT == kBitcos) {
         const uint32_t b_lo = (o_lo >> 7) << 4, b_hi = ((o_hi + 127u) >> 7) << 4;
         const uint32_t sign_bytes = b_hi - b_lo;
         const uint32_t bm_bytes = static_cast<uint32_t>(r.nt) * 512u;
-        sign_base[s] = b_lo * 8u;
+        sign_base[s * 4 + 3] = b_lo * 8u;
         // the tiles' entry offsets: the 16-byte aligned slice of tile_off that covers t0 .. t0 + nt
         const uint32_t o_first = static_cast<uint32_t>(r.t0 & 3);
         const uint32_t off_bytes = ((o_first + static_cast<uint32_t>(r.nt) + 1u + 3u) & ~3u) * 4u;
@@ -574,7 +586,6 @@ constexpr int kBarEmpty = kMaxStages;             // [stages] stage released by 
 constexpr int kBarRedFull = 2 * kMaxStages;       // [slots] partial sums of an item written by all decoder warps
 constexpr int kBarRedEmpty = 2 * kMaxStages + 8;  // [slots] partial sums consumed by the epilogue warp
 constexpr int kBarLut = 2 * kMaxStages + 16;      // lookup table arrived
-constexpr int kBarCount = 2 * kMaxStages + 17;
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -618,7 +629,8 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     const SmemLayout L = smem_layout(FMT, pl, pr.G, NB, pr.K);
     const uint8_t *lut = smem + L.lut;
     float *red = reinterpret_cast<float *>(smem + L.red);
-    uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 8 * kBarCount);
+    // per stage: {tiles | (first tile & 3) << 8, first group, first row block, first sign bit held}
+    uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 384);
     const uint32_t bar0 = smem_addr(smem + L.bar);
     const uint32_t red_slot = static_cast<uint32_t>(pl.NW) * NB * kRows;     // floats per partial-sum slot
     const Walk wk = make_walk(pl, block, n_blocks);
@@ -849,59 +861,56 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             return;
         }
     }
-    ItemIter it;
-    it.init(pl, wk.first);
-    int s = 0;
-    uint32_t phase = 0;
     constexpr int RS = red_slots(NB);
-    for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
-        const int slot = k % RS;
-        const ItemRange r = item_range(pr, pl, it.c, it.cs);
-        const bool busy = warp < r.nt;
-        const int g = (pl.CS == 1) ? g_fixed : r.g0 + warp;
-        const int rb = r.rb0 + my_rbl;
-        const int64_t m = static_cast<int64_t>(rb) * kRows + lane;
-
-        if (!mbar_wait(bar0 + 8u * (kBarFull + s), phase)) {
+    const uint32_t lane4 = static_cast<uint32_t>(lane) * 4u;
+    const uint32_t tile_lane = static_cast<uint32_t>(warp * kRows + lane);
+    const uint8_t *stage0 = smem + L.stage;
+    const uint8_t *stage = stage0;
+    const uint4 *desc = reinterpret_cast<const uint4 *>(sign_base);
+    uint32_t full_bar = bar0 + 8u * kBarFull, phase = 0;
+    int s = 0;
+    for (int k = 0; k < wk.count; ++k) {
+        if (!mbar_wait(full_bar, phase)) {
             if (lane == 0 && pr.status) *pr.status = 1u;
             return;
         }
-        const uint8_t *stage = smem + L.stage + static_cast<uint32_t>(s) * L.stage_bytes;
+        const uint4 d = desc[s];
+        const int nt = static_cast<int>(d.x & 0xFFu);
+        const bool busy = warp < nt;
+        const int g = (pl.CS == 1) ? g_fixed : static_cast<int>(d.y) + warp;
         float ysum[NB];
 #pragma unroll
         for (int b = 0; b < NB; ++b) ysum[b] = 0.f;
 
         if (busy && !pl.probe) {
-            const float sc = bf16_to_float(
-                reinterpret_cast<const uint16_t *>(stage + L.payload_cap + L.sign_cap)[warp * kRows + lane]);
+            const float sc = bf16_to_float(reinterpret_cast<const uint16_t *>(stage + L.payload_cap + L.sign_cap)[tile_lane]);
             // activations of group g: in shared memory if resident (xs), else in global memory (xgl)
             const uint8_t *xs = smem + L.x + static_cast<uint32_t>(g) * kGroup;
             const uint8_t *xgl = reinterpret_cast<const uint8_t *>(pr.x) + static_cast<int64_t>(g) * kGroup;
             int w[32];
             int acc1 = 0;
             if (FMT == kBitcos) {
-                const uint4 bm = reinterpret_cast<const uint4 *>(stage)[warp * kRows + lane];
+                const uint4 bm = reinterpret_cast<const uint4 *>(stage)[tile_lane];
                 const int c = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
                 int incl = c;
 #pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                    if (lane >= d) incl += v;
+                for (int dd = 1; dd < 32; dd <<= 1) {
+                    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, dd);
+                    if (lane >= dd) incl += v;
                 }
                 // entry offset of this tile: word (t0 & 3) + warp of the stage's slice of tile_off
                 const uint32_t toff = reinterpret_cast<const uint32_t *>(
-                    stage + L.payload_cap + L.sign_cap + L.scale_cap)[static_cast<uint32_t>(r.t0 & 3) + warp];
-                const uint32_t cursor = toff + static_cast<uint32_t>(incl - c) - sign_base[s];
+                    stage + L.payload_cap + L.sign_cap + L.scale_cap)[(d.x >> 8) + static_cast<uint32_t>(warp)];
+                const uint32_t cursor = toff + static_cast<uint32_t>(incl - c) - d.w;
                 const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + L.payload_cap) + (cursor >> 5);
                 if (NB == 1 && x_resident)
-                    acc1 = bitcos_decode_row<true>(bm, sp, cursor & 31u, lut, static_cast<uint32_t>(lane) * 4u,
-                                                   reinterpret_cast<const int4 *>(xs), w);
+                    acc1 = bitcos_decode_row<true>(bm, sp, cursor & 31u, lut, lane4, reinterpret_cast<const int4 *>(xs), w);
                 else
-                    bitcos_decode_row<false>(bm, sp, cursor & 31u, lut, static_cast<uint32_t>(lane) * 4u, nullptr, w);
+                    bitcos_decode_row<false>(bm, sp, cursor & 31u, lut, lane4, nullptr, w);
             } else if (FMT == kTrit5) {
                 const int WPR = (26 * pr.G + 3) / 4;
                 // words of the stage: row block my_rbl of the chunk, counted from the chunk's first word
-                const int w_rel = my_rbl * WPR + ((26 * g) >> 2) - ((26 * r.g0) >> 2);
+                const int w_rel = my_rbl * WPR + ((26 * g) >> 2) - ((26 * static_cast<int>(d.y)) >> 2);
                 const uint32_t *src = reinterpret_cast<const uint32_t *>(stage) + w_rel * kRows + lane;
                 uint32_t wd[7];
 #pragma unroll
@@ -922,22 +931,28 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                     else
                         a = contract<FMT>(w, reinterpret_cast<const int4 *>(xgl + static_cast<int64_t>(xr[b]) * pr.K), lane);
                     ysum[b] = sc * static_cast<float>(a);
-                    if (pr.acc_debug && m < pr.M) pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = a;
+                    if (pr.acc_debug) {
+                        const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + lane;
+                        if (m < pr.M) pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = a;
+                    }
                 }
             }
         }
         // the stage has been read: hand it back to the producer
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar0 + 8u * (kBarEmpty + s));
-
-        if (pl.probe == 2) {
-            if (++s == pl.stages) {
-                s = 0;
-                phase ^= 1u;
-            }
-            continue;
+        if (lane == 0) mbar_arrive(full_bar + 8u * kBarEmpty);
+        stage += L.stage_bytes;
+        full_bar += 8u;
+        if (++s == pl.stages) {
+            s = 0;
+            stage = stage0;
+            full_bar = bar0 + 8u * kBarFull;
+            phase ^= 1u;
         }
+        if (pl.probe == 2) continue;
+
         // partial sums for the epilogue warp (several slots, so decoders may run ahead of it)
+        const int slot = k & (RS - 1);
         if (k >= RS) {
             if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>((k / RS - 1) & 1))) {
                 if (lane == 0 && pr.status) *pr.status = 1u;
@@ -949,10 +964,6 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         for (int b = 0; b < NB; ++b) rd[(warp * NB + b) * kRows + lane] = ysum[b];
         __syncwarp();
         if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedFull + slot));
-        if (++s == pl.stages) {
-            s = 0;
-            phase ^= 1u;
-        }
     }
 }
 
