@@ -1051,16 +1051,23 @@ inline int choose_stages(int fmt, const Plan &pl, int G, int nb, int64_t K, int 
     return 2;
 }
 
-// Persistent grid: one block per multiprocessor (fewer if there are fewer items).
-inline int grid_size(const Plan &pl, int sms) { return static_cast<int>(pl.items < sms ? pl.items : sms); }
-
-// Round robin over row-block chunks when every block gets many of them (imbalance <= 1/8),
-// else a contiguous balanced split.  BITCOS_WALK=cyclic|contiguous overrides (for A/B runs).
-inline int choose_cyclic(const Plan &pl, int grid) {
+// How the items are handed to thread blocks, and how many blocks to launch (persistent: at most
+// one per multiprocessor).  Cost model in units of one item's time: round robin over row-block
+// chunks costs ceil(chunks / blocks) * CS items per block and never shares a row block; a
+// contiguous balanced split costs ceil(items / blocks) items plus, when rows are split into
+// column blocks, the cross-block hand-shake at the end (worth about 2.5 items).
+// BITCOS_WALK=cyclic|contiguous overrides the choice (for A/B runs).
+inline void choose_walk(Plan &pl, int sms, int *grid) {
     static const char *force = std::getenv("BITCOS_WALK");
-    if (force && force[0] == 'c' && force[1] == 'y') return 1;
-    if (force && force[0] == 'c' && force[1] == 'o') return 0;
-    return (pl.items / pl.CS) >= 8 * static_cast<int64_t>(grid) ? 1 : 0;
+    const int64_t chunks = pl.items / pl.CS;
+    const int64_t g_cyc = chunks < sms ? chunks : sms, g_con = pl.items < sms ? pl.items : sms;
+    const double cost_cyc = static_cast<double>((chunks + g_cyc - 1) / g_cyc) * pl.CS;
+    const double cost_con = static_cast<double>((pl.items + g_con - 1) / g_con) + (pl.CS > 1 ? 2.5 : 0.0);
+    int cyclic = cost_cyc <= cost_con ? 1 : 0;
+    if (force && force[0] == 'c' && force[1] == 'y') cyclic = 1;
+    if (force && force[0] == 'c' && force[1] == 'o') cyclic = 0;
+    pl.cyclic = cyclic;
+    *grid = static_cast<int>(cyclic ? g_cyc : g_con);
 }
 
 // Launches with programmatic stream serialization, so that this kernel's prologue (barrier
@@ -1087,9 +1094,9 @@ int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
     int sms = 0, budget = 0;
     int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms, &budget);
     if (rc) return rc;
-    const int grid = grid_size(pl, sms);
+    int grid = 1;
     Plan plw = pl;
-    plw.cyclic = choose_cyclic(pl, grid);
+    choose_walk(plw, sms, &grid);
     plw.stages = choose_stages(FMT, pl, pr.G, NB, pr.K, budget);
     static const char *probe = std::getenv("BITCOS_PROBE");
     plw.probe = (probe && probe[0] == 'c') ? 1 : (probe && probe[0] == 'd') ? 2 : 0;
@@ -1112,11 +1119,11 @@ int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int
     int rc = prepare_kernel<gemv_grouped_kernel<NB>>(&sms, &budget);
     if (rc) return rc;
     // the machine is shared by all groups: spread its multiprocessors over them
-    int gx = (sms + n_groups - 1) / n_groups;
-    if (gx > pl.items) gx = static_cast<int>(pl.items);
-    if (gx < 1) gx = 1;
+    int per_group = (sms + n_groups - 1) / n_groups;
+    if (per_group < 1) per_group = 1;
+    int gx = 1;
     Plan plw = pl;
-    plw.cyclic = choose_cyclic(pl, gx);
+    choose_walk(plw, per_group, &gx);
     plw.stages = choose_stages(kBitcos, pl, pr.G, NB, pr.K, budget);
     const SmemLayout L = smem_layout(kBitcos, plw, pr.G, NB, pr.K);
     return launch_pdl(gemv_grouped_kernel<NB>, dim3(gx, n_groups), (pl.NW + 2) * 32, L.total, stream, pr, plw, ga);
