@@ -150,6 +150,15 @@ int bitcos_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_st
  * *status == 0 means every call that used the workspace so far completed normally. */
 int bitcos_workspace_status(const void *workspace, void *cuda_stream, int *status);
 
+/* Measurement aid for the paper's two-term roofline (Section IV-B.1, Eq. 6: T = max(B/beta, gamma)):
+ * gamma is the cost of the unpack sequence when every operand is already on chip.  Launches
+ * `blocks` thread blocks of `warps_per_block` warps (1..22); each warp decodes one synthetic
+ * 32 x 128 tile held in shared memory `iters` times with the code the GEMV kernels run (format
+ * 0 = BITCOS, 1 = five-trit, 2 = 2-bit) and nothing is read from global memory in the timed loop.
+ * cycles (device, uint64 [blocks]) receives each block's elapsed SM clock cycles; cycles per 32
+ * weights per multiprocessor = cycles / (iters * warps_per_block * 128). */
+int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, uint64_t *cycles, void *cuda_stream);
+
 /* y[b][m] for b < batch, m < M from a BITCOS matrix (steps of Section II-B..II-D on the GPU:
  * entry offset + running population count locate each row's sign window, a 256-entry
  * (presence nibble, sign nibble) table as in Eq. 4 rebuilds four weights at a time as int8,

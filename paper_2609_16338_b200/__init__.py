@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     bitcos_gemv_host,
     bitcos_gemv_host_staging_bytes,
     bitcos_gemv_static,
+    bitcos_decode_probe,
     group_pairs,
     plain_to_device,
     scales_tile,

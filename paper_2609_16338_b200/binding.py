@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_unpack", "bitcos_scales_tile", "bitcos_scales_untile", "trit5_pack_sizes", "trit5_pack",
     "trit5_unpack", "bit2_pack_sizes", "bit2_pack", "bit2_unpack", "bitcos_gemv_workspace_bytes",
     "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
-    "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static",
+    "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe",
 ]
 
 
@@ -82,6 +82,7 @@ def load_library():
     L.bitcos_gemv_host_staging_bytes.argtypes = [i64, i64, C.c_int]
     L.bitcos_gemv_host.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, sz, vp, sz, vp]
     L.bitcos_gemv_static.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp]
+    L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     _lib = L
     return L
 
@@ -357,6 +358,17 @@ def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, 
                                               acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
                                               workspace.numel(), _stream()), "bitcos_gemv_grouped")
     return y, acc
+
+
+def bitcos_decode_probe(fmt: int, warps_per_block: int, iters: int, blocks: int):
+    """Cycles per 32 weights per multiprocessor of the on-chip decode (the roofline's gamma)."""
+    import torch
+    cyc = torch.zeros(blocks, dtype=torch.int64, device="cuda")
+    _check(load_library().bitcos_decode_probe(fmt, warps_per_block, iters, blocks, cyc.data_ptr(), _stream()),
+           "bitcos_decode_probe")
+    torch.cuda.synchronize()
+    c = cyc.cpu().numpy().astype(np.float64)
+    return float(np.median(c)) / (iters * warps_per_block * 128.0)
 
 
 STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024

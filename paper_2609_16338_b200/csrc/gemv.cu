@@ -998,6 +998,87 @@ __global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_grouped_kernel(P
 }
 
 // ---------------------------------------------------------------------------------------------
+// Decode-rate probe: what the paper's roofline calls gamma -- the cost of the unpack sequence when
+// every operand is already on chip (Section IV-B.1, Eq. 6).  Each warp decodes one synthetic tile
+// that sits in shared memory, `iters` times, with the same code the GEMV kernels run (popcounts,
+// prefix sum, sign windows, table lookups, dp4a); nothing is read from global memory inside the
+// timed loop.  cycles[block] receives the block's elapsed clock cycles.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t probe_hash(uint32_t v) {
+    v ^= v >> 16; v *= 0x7FEB352Du; v ^= v >> 15; v *= 0x846CA68Bu; v ^= v >> 16;
+    return v;
+}
+
+template <int FMT>
+__global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) decode_probe_kernel(int iters, unsigned long long *cycles, int *sink) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    uint8_t *lut = smem;
+    uint8_t *tiles = smem + (FMT == kBit2 ? 0 : kLutBytes);          // per warp: 1024 B payload + 640 B signs + 64 B scales
+    uint8_t *xs = tiles + nw * 1792;                                   // 128 activations
+    constexpr uint32_t kTile = 1792;
+    if (FMT != kBit2) {
+        const uint32_t *src = FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v;
+        for (int i = threadIdx.x; i < kLutBytes / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(lut)[i] = src[i];
+    }
+    // synthetic tile: presence bits set with probability 0.5625, random sign bits, valid five-trit bytes
+    uint32_t *mine = reinterpret_cast<uint32_t *>(tiles + warp * kTile);
+    for (int i = lane; i < kTile / 4; i += 32) {
+        const uint32_t h1 = probe_hash(i * 4u + 1), h2 = probe_hash(i * 4u + 2), h3 = probe_hash(i * 4u + 3),
+                       h4 = probe_hash(i * 4u + 4);
+        uint32_t v = h1 | (h2 & h3 & h4);
+        if (FMT == kTrit5) v = ((h1 & 0xFFu) % 243u) | (((h2 & 0xFFu) % 243u) << 8) | (((h3 & 0xFFu) % 243u) << 16) |
+                               (((h4 & 0xFFu) % 243u) << 24);
+        if (FMT == kBit2) v = (h1 | (h2 & h3 & h4)) & 0x55555555u;
+        mine[i] = v;
+    }
+    for (int i = threadIdx.x; i < 32; i += blockDim.x) reinterpret_cast<uint32_t *>(xs)[i] = probe_hash(1000u + i);
+    __syncthreads();
+    const uint8_t *stage = tiles + warp * kTile;
+    const uint32_t lane4 = static_cast<uint32_t>(lane) * 4u;
+    int total = 0;
+    const long long t0 = clock64();
+    for (int it = 0; it < iters; ++it) {
+        int w[32];
+        int a;
+        if (FMT == kBitcos) {
+            const uint4 bm = reinterpret_cast<const uint4 *>(stage)[lane];
+            const int c = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
+            int incl = c;
+#pragma unroll
+            for (int dd = 1; dd < 32; dd <<= 1) {
+                const int v = __shfl_up_sync(0xFFFFFFFFu, incl, dd);
+                if (lane >= dd) incl += v;
+            }
+            const uint32_t cursor = static_cast<uint32_t>(incl - c) + static_cast<uint32_t>(it & 1);
+            const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + 1024) + (cursor >> 5);
+            a = bitcos_decode_row<true>(bm, sp, cursor & 31u, lut, lane4, reinterpret_cast<const int4 *>(xs), w);
+        } else if (FMT == kTrit5) {
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(stage) + lane;
+            uint32_t wd[7];
+#pragma unroll
+            for (int i = 0; i < 7; ++i) wd[i] = src[i * kRows];
+            trit5_decode_row(wd, it & 1, lut, static_cast<uint32_t>(lane) * 8u, w);
+            a = contract<kTrit5>(w, reinterpret_cast<const int4 *>(xs), lane);
+        } else {
+            const uint4 *src = reinterpret_cast<const uint4 *>(stage) + lane + (it & 1);   // keep the loads in the loop
+            bit2_decode_row(src[0], src[kRows], w);
+            a = contract<kBit2>(w, reinterpret_cast<const int4 *>(xs), lane);
+        }
+        const float sc = bf16_to_float(reinterpret_cast<const uint16_t *>(stage + 1024 + 640)[lane]);
+        total += __float_as_int(sc * static_cast<float>(a));
+    }
+    const long long t1 = clock64();
+    __shared__ unsigned long long s_max;
+    if (threadIdx.x == 0) s_max = 0;
+    __syncthreads();
+    if (lane == 0) atomicMax(&s_max, static_cast<unsigned long long>(t1 - t0));
+    __syncthreads();
+    if (threadIdx.x == 0) cycles[blockIdx.x] = s_max;
+    if (total == 0x12345678) *sink = total;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Host side of the device entry points.
 // ---------------------------------------------------------------------------------------------
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -1194,6 +1275,32 @@ int bitcos_workspace_status(const void *workspace, void *cuda_stream, int *statu
     if (rc) return rc;
     *status = static_cast<int>(v);
     return BITCOS_OK;
+}
+
+int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, uint64_t *cycles, void *cuda_stream) {
+    if (!cycles) return BITCOS_ERR_NULL;
+    if (format < 0 || format > 2 || warps_per_block < 1 || warps_per_block > kMaxWarps + 2 || iters < 1 ||
+        iters > (1 << 20) || blocks < 1 || blocks > 4096)
+        return BITCOS_ERR_SHAPE;
+    const size_t smem = (format == kBit2 ? 0 : kLutBytes) + static_cast<size_t>(warps_per_block) * 1792 + 256;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int *sink = reinterpret_cast<int *>(cycles);      // never written in practice
+    unsigned long long *out = reinterpret_cast<unsigned long long *>(cycles);
+    int rc;
+    if (format == kBitcos) {
+        rc = check_cuda(cudaFuncSetAttribute(decode_probe_kernel<kBitcos>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        if (rc) return rc;
+        decode_probe_kernel<kBitcos><<<blocks, warps_per_block * 32, smem, stream>>>(iters, out, sink);
+    } else if (format == kTrit5) {
+        rc = check_cuda(cudaFuncSetAttribute(decode_probe_kernel<kTrit5>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        if (rc) return rc;
+        decode_probe_kernel<kTrit5><<<blocks, warps_per_block * 32, smem, stream>>>(iters, out, sink);
+    } else {
+        rc = check_cuda(cudaFuncSetAttribute(decode_probe_kernel<kBit2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        if (rc) return rc;
+        decode_probe_kernel<kBit2><<<blocks, warps_per_block * 32, smem, stream>>>(iters, out, sink);
+    }
+    return check_cuda(cudaGetLastError());
 }
 
 int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
