@@ -39,6 +39,9 @@ METRIC = "bitcos_gemv_us_per_token"
 UNIT = "us"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per bitcos_gemv launch, averaged over the seven launches
+# of one step, from the ncu capture summarised in profiles/launch_list_and_dram_traffic_bitnet2b_layer_bench.md
+NCU_DRAM_BYTES_PER_LAUNCH = 15627520 / 7.0
 
 
 def layer_config():
@@ -281,15 +284,26 @@ def run_cuda(args):
                     step(first + i)
         return g
 
+    class Eager:
+        """Stand-in for a captured graph: launches the steps directly on the current stream."""
+
+        def __init__(self, n_steps):
+            self.n = n_steps
+
+        def replay(self):
+            for i in range(self.n):
+                step(i)
+
     full, rem = divmod(args.steps, copies)
     with torch.cuda.stream(stream):
         if full:
-            graphs["full"] = capture(copies, 0)
+            graphs["full"] = Eager(copies) if args.no_graph else capture(copies, 0)
         if rem:
-            graphs["rem"] = capture(rem, 0)
-        for _ in range(2):
-            for g in graphs.values():
-                g.replay()
+            graphs["rem"] = Eager(rem) if args.no_graph else capture(rem, 0)
+        if not args.no_graph:
+            for _ in range(2):
+                for g in graphs.values():
+                    g.replay()
         stream.synchronize()
 
     sampler = ClockSampler(local_rank)
@@ -312,7 +326,7 @@ def run_cuda(args):
         dist.barrier()
     ms = e0.elapsed_time(e1)
     # keep the GPU busy a little longer so that the clock sampler sees it under load
-    t_end = time.time() + 0.6
+    t_end = time.time() + (0.0 if args.no_graph else 0.6)
     with torch.cuda.stream(stream):
         while time.time() < t_end:
             (graphs.get("full") or graphs["rem"]).replay()
@@ -336,15 +350,17 @@ def run_cuda(args):
         for j in range(len(layer)):
             bc.bitcos_gemv_host(rep[j], xh_np[j], xsh_np[j], yh_np[j], stagings[j], wss[j])
 
-    e2e_steps = min(args.steps, 200)
-    for i in range(3):
-        e2e_step(i)
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for i in range(e2e_steps):
-        e2e_step(i)
-    torch.cuda.synchronize()
-    e2e_us = (time.perf_counter() - t0) / e2e_steps * 1e6
+    e2e_steps = 0 if args.no_e2e else min(args.steps, 200)
+    e2e_us = float("nan")
+    if e2e_steps:
+        for i in range(3):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        e2e_us = (time.perf_counter() - t0) / e2e_steps * 1e6
     if dist is not None:
         t = torch.tensor([e2e_us], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -362,15 +378,16 @@ def run_cuda(args):
 
     # ---- CPU baseline: the oracle on the host cores, bounded sample ----
     import oracle
-    o_packed = oracle_pack_layer(layer)
-    t0 = time.perf_counter()
-    reps = 0
-    while True:
-        oracle_layer_pass(layer, o_packed)
-        reps += 1
-        if time.perf_counter() - t0 > 10.0 or reps >= 20:
-            break
-    cpu_us = (time.perf_counter() - t0) / reps * 1e6
+    reps, cpu_us = 0, float("nan")
+    if not args.no_cpu_baseline:
+        o_packed = oracle_pack_layer(layer)
+        t0 = time.perf_counter()
+        while True:
+            oracle_layer_pass(layer, o_packed)
+            reps += 1
+            if time.perf_counter() - t0 > 10.0 or reps >= 20:
+                break
+        cpu_us = (time.perf_counter() - t0) / reps * 1e6
 
     peak, which = measured_peaks()
     us_per_step = ms * 1e3 / args.steps
@@ -391,7 +408,7 @@ def run_cuda(args):
         "achieved_gbs": achieved,
         "frac_of_8tbs": achieved / 8000.0,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": f"{which} (STREAM-style copy)",
+                     "traffic": NCU_DRAM_BYTES_PER_LAUNCH, "peak_source": f"{which} (STREAM-style copy)",
                      "kernel": "gemv_kernel<bitcos, 1 token>", "launches": n_launch,
                      "avg_launch_us": ms * 1e3 / n_launch,
                      "algorithmic_bytes_per_launch": layer_bytes / 7.0},
@@ -404,11 +421,28 @@ def run_cuda(args):
         "gpu_launches": n_launch,
         "clocks": clocks,
     }
+    line["two_term_roofline"] = two_term_roofline(bc, cfg["z"], peak, clocks.get("sm_mhz") or 1965.0)
     if detail is not None:
         line["shapes"] = detail
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def two_term_roofline(bc, z, peak_gbs, sm_mhz, sms=148):
+    """The paper's model T = max(B / beta, gamma) per 32 weights (Section IV-B.1), evaluated on this
+    GPU: gamma = measured cycles per 32 weights per multiprocessor with every operand on chip
+    (bitcos_decode_probe, 20 decoder warps), beta = measured HBM bytes per clock per multiprocessor,
+    B = bytes per 32 weights including the 16-bit group scale (and tile offsets for BITCOS)."""
+    beta = peak_gbs * 1e9 / sms / (sm_mhz * 1e6)
+    out = {"beta_bytes_per_clk_per_sm": beta, "sm_mhz": sm_mhz}
+    for fmt, name, B in ((0, "bitcos", 4 + 4 * (1 - z) + 0.5 + 32 / 1024.0), (1, "trit5", 26 / 4.0 + 0.5), (2, "bit2", 8.5)):
+        gamma = bc.bitcos_decode_probe(fmt, 20, 200, sms)
+        mem = B / beta
+        out[name] = {"bytes_per_32_weights": B, "memory_term_cycles": mem, "gamma_cycles": gamma,
+                     "bound_by": "instructions" if gamma > mem else "memory",
+                     "ceiling_gbs": B / max(mem, gamma) * sms * sm_mhz * 1e6 / 1e9}
+    return out
 
 
 def shape_detail(bc, torch, layer, host_packed, stream, launches=64):
@@ -469,6 +503,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-detail", action="store_true", help="skip the per-shape / per-format table")
     ap.add_argument("--serial", action="store_true", help="launch the seven GEMVs of a step strictly in sequence")
+    ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA graphs (for profilers)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps is None:
