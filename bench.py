@@ -39,9 +39,8 @@ METRIC = "bitcos_gemv_us_per_token"
 UNIT = "us"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per bitcos_gemv launch, averaged over the seven launches
-# of one step, from the ncu capture summarised in profiles/launch_list_and_dram_traffic_bitnet2b_layer_bench.md
-NCU_DRAM_BYTES_PER_LAUNCH = 15627520 / 7.0
+# dram__bytes_read.sum + dram__bytes_write.sum of the seven GEMVs of one step, from the ncu capture summarised in profiles/launch_list_and_dram_traffic_bitnet2b_layer_bench.md
+NCU_DRAM_BYTES_PER_STEP = 15627520
 
 
 def layer_config():
@@ -226,6 +225,10 @@ def run_cuda(args):
     wss = [bc.make_workspace(m["M"], m["K"]) for m in layer]
 
     sides = [torch.cuda.Stream(), torch.cuda.Stream()]
+    # fused launches: GEMVs that read the same input and do not depend on one another share a launch
+    groups = [[0, 1, 2], [3], [4, 5], [6]]
+    multi = [[bc.MultiJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in g]) for g in groups]
+             for rep in replicas]
 
     def step(i):
         """One layer pass: q | k | v, then o, then gate | up, then down.  GEMVs that read the same
@@ -239,6 +242,10 @@ def run_cuda(args):
         if args.serial:
             for j in range(len(layer)):
                 run(j)
+            return
+        if not args.branches:
+            for mj in multi[i % copies]:
+                bc.bitcos_gemv_multi(mj)
             return
         cur = torch.cuda.current_stream()
         for sd in sides:
@@ -391,7 +398,8 @@ def run_cuda(args):
 
     peak, which = measured_peaks()
     us_per_step = ms * 1e3 / args.steps
-    n_launch = 7 * args.steps
+    launches_per_step = 7 if (args.serial or args.branches) else len(groups)
+    n_launch = launches_per_step * args.steps
     achieved = layer_bytes * args.steps / (ms * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": us_per_step / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -401,17 +409,22 @@ def run_cuda(args):
                    "packed_bytes_per_step": int(packed_bytes), "algorithmic_bytes_per_step": int(layer_bytes),
                    "l2_policy": f"{copies} rotated copies of the packed layer ({copies * packed_bytes / 2**20:.0f} MiB)"
                                 " so no step finds its weights in L2",
-                   "launch": ("CUDA graphs of the rotation; " + ("7 launches in sequence" if args.serial else
-                              "7 launches per step: q|k|v on parallel branches, o, gate|up on parallel branches, down")
+                   "launch": (("plain stream launches; " if args.no_graph else "CUDA graphs of the rotation; ")
+                              + ("7 launches per step, in sequence" if args.serial else
+                                 "7 launches per step: q|k|v on parallel branches, o, gate|up on parallel branches, down"
+                                 if args.branches else
+                                 "4 launches per step through bitcos_gemv_multi: q+k+v, o, gate+up, down (GEMVs that "
+                                 "read the same input share a launch)")
                               + "; programmatic dependent launch between consecutive kernels of a stream"),
                    "replicas": world},
         "achieved_gbs": achieved,
         "frac_of_8tbs": achieved / 8000.0,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_DRAM_BYTES_PER_LAUNCH, "peak_source": f"{which} (STREAM-style copy)",
-                     "kernel": "gemv_kernel<bitcos, 1 token>", "launches": n_launch,
+                     "traffic": NCU_DRAM_BYTES_PER_STEP / launches_per_step, "peak_source": f"{which} (STREAM-style copy)",
+                     "kernel": "gemv_kernel<bitcos, 1 token>" if launches_per_step == 7 else "gemv_multi_kernel<1 token>",
+                     "launches": n_launch,
                      "avg_launch_us": ms * 1e3 / n_launch,
-                     "algorithmic_bytes_per_launch": layer_bytes / 7.0},
+                     "algorithmic_bytes_per_launch": layer_bytes / launches_per_step},
         "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
                          "sample": f"{reps} full layer passes (7 GEMVs, 69.5 M weights each): BITCOS decode bit by "
                                    "bit, dense int32 dot per group, double scale-and-sum"},
@@ -503,6 +516,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-detail", action="store_true", help="skip the per-shape / per-format table")
     ap.add_argument("--serial", action="store_true", help="launch the seven GEMVs of a step strictly in sequence")
+    ap.add_argument("--branches", action="store_true",
+                    help="seven launches per step with q|k|v and gate|up on parallel graph branches")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA graphs (for profilers)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")

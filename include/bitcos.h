@@ -173,6 +173,23 @@ int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, 
 int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
                 int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Up to four independent BITCOS products in ONE launch (same batch; shapes may differ): e.g. the
+ * q, k and v projections of a decoder layer, which read the same activations and do not depend on
+ * one another, or gate and up.  The multiprocessors are shared between the jobs in proportion to
+ * their sizes, so small matrices run side by side instead of one after the other and the fixed
+ * cost of a launch is paid once.  Every job has its own outputs and its own workspace (sized and
+ * zero filled as for bitcos_gemv; two jobs must not share one).  Results are identical to
+ * n_jobs calls of bitcos_gemv. */
+typedef struct bitcos_gemv_job {
+    const bitcos_weights *W;   /* host struct of device pointers */
+    const int8_t *x;           /* device int8 [batch][K] */
+    const float *x_scale;      /* device float [batch] */
+    float *y;                  /* device float [batch][M] */
+    void *workspace;           /* device scratch, >= bitcos_gemv_workspace_bytes(M, K) */
+    size_t workspace_bytes;
+} bitcos_gemv_job;
+int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
+
 /* The same product as bitcos_gemv without a caller-provided workspace.  (The paper has no
  * counterpart: this entry point exists for the library's users, not for the method.)
  *

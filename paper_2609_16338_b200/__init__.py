@@ -20,6 +20,8 @@ from .binding import (  # noqa: F401
     bitcos_gemv_host,
     bitcos_gemv_host_staging_bytes,
     bitcos_gemv_static,
+    bitcos_gemv_multi,
+    MultiJobs,
     bitcos_decode_probe,
     group_pairs,
     plain_to_device,

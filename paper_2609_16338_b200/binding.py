@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_unpack", "bitcos_scales_tile", "bitcos_scales_untile", "trit5_pack_sizes", "trit5_pack",
     "trit5_unpack", "bit2_pack_sizes", "bit2_pack", "bit2_unpack", "bitcos_gemv_workspace_bytes",
     "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
-    "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe",
+    "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
 ]
 
 
@@ -31,6 +31,11 @@ class BitcosError(RuntimeError):
     def __init__(self, status: int, what: str, detail: str = ""):
         self.status = status
         super().__init__(f"{what}: status {status} ({detail})")
+
+
+class _Job(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("x", C.c_void_p), ("x_scale", C.c_void_p), ("y", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
 class _Weights(C.Structure):
@@ -83,6 +88,7 @@ def load_library():
     L.bitcos_gemv_host.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, sz, vp, sz, vp]
     L.bitcos_gemv_static.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp]
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     _lib = L
     return L
 
@@ -358,6 +364,24 @@ def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, 
                                               acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
                                               workspace.numel(), _stream()), "bitcos_gemv_grouped")
     return y, acc
+
+
+class MultiJobs:
+    """Argument block of bitcos_gemv_multi, built once and reusable: jobs = [(W, x, x_scale, y, workspace)]."""
+
+    def __init__(self, jobs):
+        self.keep = jobs
+        self.batch = jobs[0][1].shape[0]
+        self.arr = (_Job * len(jobs))(*[_Job(C.addressof(W.desc), x.data_ptr(), xs.data_ptr(), y.data_ptr(),
+                                             ws.data_ptr(), ws.numel()) for (W, x, xs, y, ws) in jobs])
+
+
+def bitcos_gemv_multi(jobs):
+    """Up to four independent BITCOS products in one launch; `jobs` is a MultiJobs or a list of
+    (W, x, x_scale, y, workspace) tuples with a common batch size."""
+    mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
+    _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")
+    return [j[3] for j in mj.keep]
 
 
 def bitcos_decode_probe(fmt: int, warps_per_block: int, iters: int, blocks: int):

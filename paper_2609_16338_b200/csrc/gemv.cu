@@ -640,6 +640,13 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     // griddepcontrol.wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+    // A block launched wider than this problem needs (several problems in one launch): the spare
+    // warps only take part in the one block-wide barrier.
+    if (warp >= pl.NW + 2) {
+        __syncthreads();
+        return;
+    }
+
     // ------------------------------------------------------------------ producer warp
     // It also sets the barriers up, so that the first copies are in flight before anything else
     // happens in the block.
@@ -973,6 +980,25 @@ __global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_kernel(const Pro
     run_problem<FMT, NB>(pr, pl, smem, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
 }
 
+// Several independent BITCOS problems in one launch: the grid is cut into one range of thread
+// blocks per problem, and every block runs the ordinary kernel body on its problem.
+constexpr int kMaxJobs = 4;
+struct MultiArgs {
+    Problem pr[kMaxJobs];
+    Plan pl[kMaxJobs];
+    int first_block[kMaxJobs + 1];
+    int n;
+};
+
+template <int NB>
+__global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int b = static_cast<int>(blockIdx.x);
+    int j = 0;
+    while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
+    run_problem<kBitcos, NB>(ma.pr[j], ma.pl[j], smem, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]);
+}
+
 template <int NB>
 __global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -1185,6 +1211,38 @@ int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
     return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw);
 }
 
+template <int NB>
+int launch_multi(MultiArgs &ma, cudaStream_t stream) {
+    int sms = 0, budget = 0;
+    int rc = prepare_kernel<gemv_multi_kernel<NB>>(&sms, &budget);
+    if (rc) return rc;
+    // share the multiprocessors between the problems in proportion to their item counts
+    int64_t total_items = 0;
+    for (int j = 0; j < ma.n; ++j) total_items += ma.pl[j].items;
+    int nw = 0;
+    uint32_t smem = 0;
+    int next = 0;
+    static const char *probe = std::getenv("BITCOS_PROBE");
+    for (int j = 0; j < ma.n; ++j) {
+        int64_t cap = ma.pl[j].items;
+        if (total_items > sms) {
+            cap = ma.pl[j].items * sms / total_items;
+            if (cap < 1) cap = 1;
+        }
+        int grid = 1;
+        choose_walk(ma.pl[j], static_cast<int>(cap), &grid);
+        ma.pl[j].stages = choose_stages(kBitcos, ma.pl[j], ma.pr[j].G, NB, ma.pr[j].K, budget);
+        ma.pl[j].probe = (probe && probe[0] == 'c') ? 1 : (probe && probe[0] == 'd') ? 2 : 0;
+        const SmemLayout L = smem_layout(kBitcos, ma.pl[j], ma.pr[j].G, NB, ma.pr[j].K);
+        if (L.total > smem) smem = L.total;
+        if (ma.pl[j].NW > nw) nw = ma.pl[j].NW;
+        ma.first_block[j] = next;
+        next += grid;
+    }
+    ma.first_block[ma.n] = next;
+    return launch_pdl(gemv_multi_kernel<NB>, dim3(next), (nw + 2) * 32, smem, stream, ma);
+}
+
 template <int FMT>
 int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream) {
     if (pr.nb <= 1) return launch<FMT, 1>(pr, pl, stream);
@@ -1210,9 +1268,10 @@ int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int
     return launch_pdl(gemv_grouped_kernel<NB>, dim3(gx, n_groups), (pl.NW + 2) * 32, L.total, stream, pr, plw, ga);
 }
 
-int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const uint32_t *tile_off,
-                const uint16_t *scales, int64_t M, int64_t K, const int8_t *x, const float *x_scale, int batch,
-                float *y, int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+// Validates the arguments every product shares; fills nothing.
+int check_common(int fmt, const uint32_t *payload, const uint32_t *signs, const uint32_t *tile_off,
+                 const uint16_t *scales, int64_t M, int64_t K, const int8_t *x, const float *x_scale, int batch,
+                 const float *y, const int32_t *acc_debug, const void *workspace, size_t workspace_bytes) {
     if (!payload || !scales || !x || !x_scale || !y || !workspace) return BITCOS_ERR_NULL;
     if (fmt == kBitcos && (!signs || !tile_off)) return BITCOS_ERR_NULL;
     if (M < 1 || K < kGroup || K % kGroup != 0 || batch < 1 || batch > BITCOS_MAX_BATCH) return BITCOS_ERR_SHAPE;
@@ -1221,9 +1280,12 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
         (signs && !aligned16(signs)) || (tile_off && !aligned16(tile_off)) || (acc_debug && !aligned16(acc_debug)))
         return BITCOS_ERR_ALIGN;
     if (workspace_bytes < workspace_bytes_for(M, K)) return BITCOS_ERR_CAPACITY;
+    return BITCOS_OK;
+}
 
-    const Plan pl = make_plan(M, K, decoder_warps(batch));
-    Problem pr{};
+void fill_problem(Problem &pr, const uint32_t *payload, const uint32_t *signs, const uint32_t *tile_off,
+                  const uint16_t *scales, int64_t M, int64_t K, const int8_t *x, const float *x_scale, int batch,
+                  float *y, int32_t *acc_debug, void *workspace) {
     pr.payload = payload;
     pr.signs = signs;
     pr.tile_off = tile_off;
@@ -1243,6 +1305,17 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
     pr.status = reinterpret_cast<unsigned int *>(ws);
     pr.counters = reinterpret_cast<unsigned int *>(ws + kHeaderBytes);
     pr.partial = reinterpret_cast<float *>(ws + kHeaderBytes + counters_bytes(pr.RB));
+}
+
+int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const uint32_t *tile_off,
+                const uint16_t *scales, int64_t M, int64_t K, const int8_t *x, const float *x_scale, int batch,
+                float *y, int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    const int bad = check_common(fmt, payload, signs, tile_off, scales, M, K, x, x_scale, batch, y, acc_debug, workspace,
+                                 workspace_bytes);
+    if (bad) return bad;
+    const Plan pl = make_plan(M, K, decoder_warps(batch));
+    Problem pr{};
+    fill_problem(pr, payload, signs, tile_off, scales, M, K, x, x_scale, batch, y, acc_debug, workspace);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (fmt == kBitcos) return launch_nb<kBitcos>(pr, pl, stream);
     if (fmt == kTrit5) return launch_nb<kTrit5>(pr, pl, stream);
@@ -1362,6 +1435,31 @@ int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_
     if (rc) return rc;
     return gemv_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_scale, batch, y,
                        nullptr, ws, BITCOS_STATIC_WORKSPACE_BYTES, cuda_stream);
+}
+
+int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
+    if (!jobs) return BITCOS_ERR_NULL;
+    if (n_jobs < 1 || n_jobs > kMaxJobs) return BITCOS_ERR_SHAPE;
+    MultiArgs ma{};
+    ma.n = n_jobs;
+    for (int j = 0; j < n_jobs; ++j) {
+        const bitcos_gemv_job &jb = jobs[j];
+        if (!jb.W) return BITCOS_ERR_NULL;
+        const int bad = check_common(kBitcos, jb.W->bitmap, jb.W->signs, jb.W->tile_off, jb.W->scales, jb.W->M, jb.W->K,
+                                     jb.x, jb.x_scale, batch, jb.y, nullptr, jb.workspace, jb.workspace_bytes);
+        if (bad) return bad;
+        for (int i = 0; i < j; ++i)
+            if (jobs[i].workspace == jb.workspace) return BITCOS_ERR_SHAPE;      // jobs run concurrently
+        ma.pl[j] = make_plan(jb.W->M, jb.W->K, decoder_warps(batch));
+        fill_problem(ma.pr[j], jb.W->bitmap, jb.W->signs, jb.W->tile_off, jb.W->scales, jb.W->M, jb.W->K, jb.x,
+                     jb.x_scale, batch, jb.y, nullptr, jb.workspace);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (batch <= 1) return launch_multi<1>(ma, stream);
+    if (batch <= 2) return launch_multi<2>(ma, stream);
+    if (batch <= 4) return launch_multi<4>(ma, stream);
+    if (batch <= 8) return launch_multi<8>(ma, stream);
+    return launch_multi<16>(ma, stream);
 }
 
 size_t bitcos_gemv_host_staging_bytes(int64_t M, int64_t K, int batch) {

@@ -154,6 +154,33 @@ def test_grouped_down_projection_shape(bc):
     check(y, acc, acc_ref, y_ref, mag, "grouped down")
 
 
+@pytest.mark.parametrize("B", [1, 3])
+def test_multi_launch_matches_separate_products(bc, B):
+    """Several independent matrices (different shapes, also different K) in one launch."""
+    shapes = [(2560, 2560), (640, 2560), (96, 6912), (320, 1280)]
+    jobs, refs = [], []
+    for i, (M, K) in enumerate(shapes):
+        W, S = datagen.trits(600 + i, M, K, 0.4219), datagen.scales(600 + i, M, K)
+        x, xs = datagen.activations(600 + i, B, K)
+        refs.append(oracle.gemv_dense(W, S, x, xs))
+        y = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
+        jobs.append((bc.bitcos_pack(W, S).to_device(), dev(x), dev(xs), y, bc.make_workspace(M, K)))
+    for n in (4, 3, 1):
+        for rep in range(2):
+            for j in jobs:
+                j[3].fill_(float("nan"))
+            bc.bitcos_gemv_multi(jobs[:n])
+            for (Wd, _, _, y, _), (acc_ref, y_ref, mag) in zip(jobs[:n], refs[:n]):
+                check(y, None, acc_ref, y_ref, mag, f"multi n={n} rep{rep} {Wd.M}x{Wd.K}")
+    # the same results as the single-matrix entry point, bit for bit
+    bc.bitcos_gemv_multi(jobs)
+    torch.cuda.synchronize()
+    for (Wd, x, xs, y, ws) in jobs:
+        y1, _ = bc.bitcos_gemv(Wd, x, xs, workspace=ws)
+        torch.cuda.synchronize()
+        assert torch.equal(y1, y)
+
+
 def test_host_buffer_entry_point(bc):
     M, K, B = 640, 2560, 4
     W, S = datagen.trits(21, M, K, 0.4219), datagen.scales(21, M, K)
