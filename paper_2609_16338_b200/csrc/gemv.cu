@@ -35,10 +35,14 @@ namespace {
 constexpr int kGroup = BITCOS_GROUP;
 constexpr int kRows = BITCOS_TILE_ROWS;
 constexpr int kMaxWarps = 20;             // warps per thread block = tiles per item
+constexpr int kWarps16 = 16;              // the same for more than 8 tokens (their partial sums need the room)
 constexpr int kMaxStages = 8;             // upper bound on the shared-memory ring depth (Plan::stages)
 constexpr int kLutBytes = 64 * 1024;      // replicated lookup tables (BITCOS, five-trit)
 constexpr uint64_t kWaitLimitNs = 500ull * 1000 * 1000;   // an mbarrier wait gives up after half a second
 constexpr int64_t kXResidentBytes = 48 * 1024;   // activations up to this size are kept in shared memory
+constexpr int kMmaMinBatch = 4;           // from this many tokens on the contraction runs on the tensor cores
+constexpr int kScrRowBytes = 48;          // a quarter of a decoded row (32 int8) + 16 bytes of padding against bank conflicts
+constexpr int kScrBytes = kRows * kScrRowBytes;   // per decoder warp: the transposition buffer in front of ldmatrix
 
 enum Format { kBitcos = 0, kTrit5 = 1, kBit2 = 2 };
 
@@ -169,9 +173,11 @@ struct GroupedArgs {
 
 inline int64_t padded_rows(int64_t M) { return (M + kRows - 1) / kRows * kRows; }
 
-// Decoder warps per thread block: 20, or 10 for more than 8 tokens (their activations and partial
-// sums would not fit in shared memory otherwise).
-inline int decoder_warps(int batch) { return batch > 8 ? kMaxWarps / 2 : kMaxWarps; }
+// Decoder warps per thread block: 20, or 16 for more than 8 tokens (their partial sums would not
+// fit in shared memory otherwise).
+__host__ __device__ constexpr int decoder_warps(int batch) { return batch > 8 ? kWarps16 : kMaxWarps; }
+// Threads of the widest block an instantiation for up to nb tokens is launched with.
+__host__ __device__ constexpr int max_block_threads(int nb) { return (decoder_warps(nb) + 2) * 32; }
 
 Plan make_plan(int64_t M, int64_t K, int max_warps) {
     const int G = static_cast<int>(K / kGroup);
@@ -197,7 +203,7 @@ constexpr size_t kHeaderBytes = 256;
 size_t counters_bytes(int64_t RB) { return static_cast<size_t>((RB * 4 + 255) / 256 * 256); }
 
 size_t workspace_bytes_for(int64_t M, int64_t K) {
-    const Plan p = make_plan(M, K, kMaxWarps / 2);        // the plan with the most column blocks
+    const Plan p = make_plan(M, K, kWarps16);        // the plan with the most column blocks
     const int64_t RB = padded_rows(M) / kRows;
     size_t b = kHeaderBytes + counters_bytes(RB);
     if (p.CS > 1) b += static_cast<size_t>(RB) * p.CS * BITCOS_MAX_BATCH * kRows * sizeof(float);
@@ -213,11 +219,22 @@ struct SmemLayout {
     uint32_t x;          // activations, [nb][K], if x_bytes != 0
     uint32_t x_bytes;    // 0: the activations do not fit and are read from global memory
     uint32_t red;        // 2 x [NW][NB][32] floats
+    uint32_t scr;        // tensor-core path: NW transposition buffers of kScrBytes
     uint32_t bar;        // mbarriers, then per-stage sign base words
     uint32_t total;
 };
 
 __host__ __device__ inline uint32_t align_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+// Partial-sum slots.  Up to two tokens: [warp][token][row] floats.  Tensor-core path:
+// [warp][row][token], tokens fastest, so that a decoder lane stores its accumulator pairs (tokens
+// 2c, 2c + 1) as one 8-byte word and the epilogue warp reads four tokens per load; token t of row r
+// sits at position t ^ red_swizzle(r), which keeps both the stores (lane = row / 4-column pair) and
+// the loads (lane = row) free of bank conflicts without padding.
+template <int NB>
+__host__ __device__ constexpr int red_swizzle(int row) {
+    return NB < 8 ? 0 : ((row >> 2) & 1) * 4 + (NB > 8 ? ((row >> 1) & 1) * 8 : 0);
+}
 
 // Partial-sum slots between the decoder warps and the epilogue warp (how many items the
 // decoders may run ahead of it).
@@ -248,10 +265,14 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     L.stage_bytes = align_up(L.payload_cap + L.sign_cap + L.scale_cap + L.off_cap, 128);
     off += L.stage_bytes * static_cast<uint32_t>(pl.stages);
     L.x = off;
-    L.x_bytes = (static_cast<int64_t>(nbmax) * K <= kXResidentBytes) ? static_cast<uint32_t>(nbmax * K) : 0u;
+    // (the tensor-core path takes its activation fragments straight from global memory)
+    L.x_bytes = (nbmax < kMmaMinBatch && static_cast<int64_t>(nbmax) * K <= kXResidentBytes)
+                    ? static_cast<uint32_t>(nbmax * K) : 0u;
     off += align_up(L.x_bytes, 128);
     L.red = off;
     off += static_cast<uint32_t>(red_slots(nbmax)) * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
+    L.scr = off;
+    off += (nbmax >= kMmaMinBatch) ? tiles * kScrBytes : 0u;
     L.bar = off;
     off += 512;          // mbarriers, then (16-byte aligned) one 16-byte item descriptor per stage
     L.total = off;
@@ -329,6 +350,24 @@ __device__ __forceinline__ uint32_t bit_select(uint32_t a, uint32_t b, uint32_t 
     uint32_t d;
     asm("lop3.b32 %0, %1, %2, %3, 0xE4;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
+}
+
+// Four 8x8 matrices of 16-bit elements from shared memory, one row address per lane: as int8 data
+// this is exactly the A operand (16 rows x 32 bytes) of mma.m16n8k32.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+                 : "r"(addr)
+                 : "memory");
+}
+// c[16 x 8] += a[16 x 32] * b[32 x 8], int8 operands, int32 accumulators.
+__device__ __forceinline__ void mma_s8(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void sts128(uint32_t addr, int a, int b, int c, int d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -418,6 +457,17 @@ __device__ __forceinline__ void bit2_decode_row(const uint4 v0, const uint4 v1, 
     for (int q = 0; q < 8; ++q)
 #pragma unroll
         for (int j = 0; j < 4; ++j) w[4 * q + j] = static_cast<int>(wd[q] & (0x03030303u << (2 * j)));
+}
+
+// 2-bit, as plain int8: w[4q + j] byte b = code - 1 of weight 16 q + 4 j + b.  Per byte,
+// (code + 0x7F) ^ 0x80 maps 0, 1, 2 to -1, 0, +1 without a carry between bytes.
+__device__ __forceinline__ void bit2_decode_row_s8(const uint4 v0, const uint4 v1, int (&w)[32]) {
+    const uint32_t wd[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            w[4 * q + j] = static_cast<int>((((wd[q] >> (2 * j)) & 0x03030303u) + 0x7F7F7F7Fu) ^ 0x80808080u);
 }
 
 // int32 accumulator of one row (lane) and group against token activations xg[0..127] (shared memory).
@@ -785,6 +835,52 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 for (int j = 0; j + w2 < kMaxWarps; j += 2 * w2) v[j] += v[j + w2];
             return v[0];
         };
+        // tensor-core layout: the same for four tokens at a time, n <= 20 float4 spaced one warp's
+        // rows apart, in two batches of ten to bound the registers in flight
+        constexpr int RF = NB;
+        auto sum_groups4 = [&](const float *base, int n) {
+            float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j0 = 0; j0 < kMaxWarps; j0 += 10) {
+                float4 v[10];
+#pragma unroll
+                for (int j = 0; j < 10; ++j)
+                    v[j] = (j0 + j < n) ? *reinterpret_cast<const float4 *>(base + (j0 + j) * kRows * RF)
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w2 = 1; w2 < 10; w2 *= 2)
+#pragma unroll
+                    for (int j = 0; j + w2 < 10; j += 2 * w2) {
+                        v[j].x += v[j + w2].x;
+                        v[j].y += v[j + w2].y;
+                        v[j].z += v[j + w2].z;
+                        v[j].w += v[j + w2].w;
+                    }
+                tot.x += v[0].x;
+                tot.y += v[0].y;
+                tot.z += v[0].z;
+                tot.w += v[0].w;
+            }
+            return tot;
+        };
+        // sums over warps j0 .. j0 + n - 1 of a slot, for this lane's row and every token
+        auto sums = [&](const float *rs, int j0, int n, float (&tot)[NB]) {
+            if (NB >= kMmaMinBatch) {
+#pragma unroll
+                for (int t = 0; t < NB / 4; ++t) {
+                    float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (4 * t < pr.nb) v4 = sum_groups4(rs + (j0 * kRows + lane) * RF + ((4 * t) ^ red_swizzle<NB>(lane)), n);
+                    tot[4 * t + 0] = v4.x;
+                    tot[4 * t + 1] = v4.y;
+                    tot[4 * t + 2] = v4.z;
+                    tot[4 * t + 3] = v4.w;
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    tot[b] = (b < pr.nb) ? sum_groups(rs + (j0 * NB + b) * kRows + lane, n) : 0.f;
+            }
+        };
         for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
             const int slot = k % RS;
             const ItemRange r = item_range(pr, pl, it.c, it.cs);
@@ -801,9 +897,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 for (int i = 0; i < nrb; ++i) {
                     const int64_t m = static_cast<int64_t>(r.rb0 + i) * kRows + lane;
                     float t_b[NB];
-#pragma unroll
-                    for (int b = 0; b < NB; ++b)
-                        t_b[b] = (b < pr.nb) ? sum_groups(rs + (i * pr.G * NB + b) * kRows + lane, pr.G) : 0.f;
+                    sums(rs, i * pr.G, pr.G, t_b);
                     if (i == nrb - 1) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedEmpty + slot));
@@ -816,13 +910,10 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             }
             // one column block of row block rb0: add it to the running sum
             const bool starts = (r.cs == 0) || (k == 0);
+            float t_b[NB];
+            sums(rs, 0, r.nt, t_b);
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                if (b < pr.nb) {
-                    const float tot = sum_groups(rs + b * kRows + lane, r.nt);
-                    run[b] = starts ? tot : run[b] + tot;
-                }
-            }
+            for (int b = 0; b < NB; ++b) run[b] = starts ? t_b[b] : run[b] + t_b[b];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedEmpty + slot));
             const bool ends = (r.cs == pl.CS - 1) || (k == wk.count - 1);
@@ -869,8 +960,45 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         }
     }
     constexpr int RS = red_slots(NB);
+    constexpr bool kMma = NB >= kMmaMinBatch;          // contraction on the tensor cores
+    constexpr int NH = NB > 8 ? 2 : 1;                 // 8-token halves of the batch
+    constexpr int NV = kMma ? NH * 8 : NB;             // partial sums a lane hands to the epilogue warp
     const uint32_t lane4 = static_cast<uint32_t>(lane) * 4u;
     const uint32_t tile_lane = static_cast<uint32_t>(warp * kRows + lane);
+    // Tensor-core path.  The order of the 128 products inside a group is free, so it is chosen to
+    // make the activation loads contiguous: of tokens lane / 4 and lane / 4 + 8 this lane holds
+    // bytes 16 c .. 16 c + 15 and 64 + 16 c .. 64 + 16 c + 15 of the group (c = lane % 4, two 16-byte
+    // loads), and k-block kb of the contraction pairs words 2 kb and 2 kb + 1 of those eight with
+    // the matching weight words.  A operand: each lane stores the row it decoded into the warp's
+    // buffer (32 int8 at a time, in that order), ldmatrix brings it back in fragment order.
+    const int8_t *xfrag[NH];
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+        const int n = 8 * h + (lane >> 2);
+        xfrag[h] = nullptr;
+        if (kMma && n < pr.nb)
+            xfrag[h] = pr.x + static_cast<int64_t>(pr.xrow ? __ldg(pr.xrow + n) : n) * pr.K + 16 * (lane & 3);
+    }
+    uint32_t bf[NH][8];
+    auto load_bf = [&](int g) {
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            int4 u0 = make_int4(0, 0, 0, 0), u1 = make_int4(0, 0, 0, 0);
+            if (xfrag[h]) {
+                const int4 *px = reinterpret_cast<const int4 *>(xfrag[h] + static_cast<int64_t>(g) * kGroup);
+                u0 = __ldg(px);
+                u1 = __ldg(px + 4);
+            }
+            bf[h][0] = u0.x; bf[h][1] = u0.y; bf[h][2] = u0.z; bf[h][3] = u0.w;
+            bf[h][4] = u1.x; bf[h][5] = u1.y; bf[h][6] = u1.z; bf[h][7] = u1.w;
+        }
+    };
+    // whole rows per item: this warp's group never changes, neither do its activation fragments
+    if (kMma && pl.CS == 1) load_bf(g_fixed);
+    const uint32_t scr0 = smem_addr(smem + L.scr) + static_cast<uint32_t>(warp) * kScrBytes;
+    const uint32_t scr_st = scr0 + static_cast<uint32_t>(lane) * kScrRowBytes;
+    const uint32_t scr_ld = scr0 + static_cast<uint32_t>((lane & 7) + ((lane >> 3) & 1) * 8) * kScrRowBytes +
+                            static_cast<uint32_t>(lane >> 4) * 16u;
     const uint8_t *stage0 = smem + L.stage;
     const uint8_t *stage = stage0;
     const uint4 *desc = reinterpret_cast<const uint4 *>(sign_base);
@@ -885,9 +1013,10 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         const int nt = static_cast<int>(d.x & 0xFFu);
         const bool busy = warp < nt;
         const int g = (pl.CS == 1) ? g_fixed : static_cast<int>(d.y) + warp;
-        float ysum[NB];
+        float ysum[NV];
 #pragma unroll
-        for (int b = 0; b < NB; ++b) ysum[b] = 0.f;
+        for (int b = 0; b < NV; ++b) ysum[b] = 0.f;
+        if (kMma && pl.CS != 1 && busy) load_bf(g);        // early, so that the decode hides the latency
 
         if (busy && !pl.probe) {
             const float sc = bf16_to_float(reinterpret_cast<const uint16_t *>(stage + L.payload_cap + L.sign_cap)[tile_lane]);
@@ -925,10 +1054,54 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 trit5_decode_row(wd, g & 1, lut, static_cast<uint32_t>(lane) * 8u, w);
             } else {
                 const uint4 *src = reinterpret_cast<const uint4 *>(stage) + (warp * 2) * kRows + lane;
-                bit2_decode_row(src[0], src[kRows], w);
+                if (kMma) bit2_decode_row_s8(src[0], src[kRows], w);
+                else bit2_decode_row(src[0], src[kRows], w);
+            }
+            if (kMma) {
+                int acc[NH][2][4];
+#pragma unroll
+                for (int h = 0; h < NH; ++h)
+#pragma unroll
+                    for (int mh = 0; mh < 2; ++mh)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) acc[h][mh][r] = 0;
+#pragma unroll
+                for (int kb = 0; kb < 4; ++kb) {
+                    // 32 weights of every row through the buffer: one k-block of the contraction
+                    if (kb) __syncwarp();            // everyone has read the previous block back
+                    const int w0 = (kb < 2) ? 2 * kb : 16 + 2 * (kb - 2);     // first weight word of this block
+                    sts128(scr_st, w[w0], w[w0 + 4], w[w0 + 8], w[w0 + 12]);
+                    sts128(scr_st + 16u, w[w0 + 1], w[w0 + 5], w[w0 + 9], w[w0 + 13]);
+                    __syncwarp();
+#pragma unroll
+                    for (int mh = 0; mh < 2; ++mh) {
+                        uint32_t a[4];
+                        ldmatrix_x4(a, scr_ld + static_cast<uint32_t>(mh * 16 * kScrRowBytes));
+#pragma unroll
+                        for (int h = 0; h < NH; ++h) mma_s8(acc[h][mh], a, bf[h][2 * kb], bf[h][2 * kb + 1]);
+                    }
+                }
+                // accumulator r of (h, mh): row 16 mh + lane / 4 + 8 (r / 2), token 8 h + 2 (lane % 4) + (r & 1)
+                float scq[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) scq[j] = __shfl_sync(0xFFFFFFFFu, sc, (lane >> 2) + 8 * j);
+#pragma unroll
+                for (int h = 0; h < NH; ++h)
+#pragma unroll
+                    for (int mh = 0; mh < 2; ++mh)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            ysum[(h * 2 + mh) * 4 + r] = scq[2 * mh + (r >> 1)] * static_cast<float>(acc[h][mh][r]);
+                            if (pr.acc_debug) {
+                                const int b = 8 * h + 2 * (lane & 3) + (r & 1);
+                                const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + 16 * mh + (lane >> 2) + 8 * (r >> 1);
+                                if (b < pr.nb && m < pr.M) pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = acc[h][mh][r];
+                            }
+                        }
             }
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
+                if (kMma) break;
                 if (b < pr.nb) {
                     int a;
                     if (FMT == kBitcos && NB == 1 && x_resident)
@@ -967,15 +1140,26 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             }
         }
         float *rd = red + slot * red_slot;
+        if (kMma) {
 #pragma unroll
-        for (int b = 0; b < NB; ++b) rd[(warp * NB + b) * kRows + lane] = ysum[b];
+            for (int i = 0; i < NV; i += 2) {
+                const int b = 8 * (i >> 3) + 2 * (lane & 3);                          // and b + 1
+                const int row = 16 * ((i >> 2) & 1) + (lane >> 2) + 8 * ((i >> 1) & 1);
+                if (b < NB)
+                    *reinterpret_cast<float2 *>(rd + (warp * kRows + row) * NB + (b ^ red_swizzle<NB>(row))) =
+                        make_float2(ysum[i], ysum[i + 1]);
+            }
+        } else {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) rd[(warp * NB + b) * kRows + lane] = ysum[b];
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedFull + slot));
     }
 }
 
 template <int FMT, int NB>
-__global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_kernel(const Problem pr, const Plan pl) {
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
     run_problem<FMT, NB>(pr, pl, smem, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
 }
@@ -991,7 +1175,7 @@ struct MultiArgs {
 };
 
 template <int NB>
-__global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma) {
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b = static_cast<int>(blockIdx.x);
     int j = 0;
@@ -1000,7 +1184,7 @@ __global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_multi_kernel(con
 }
 
 template <int NB>
-__global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int grp = blockIdx.y;
     // the routing lists may come from the previous kernel in the stream
@@ -1275,7 +1459,7 @@ int check_common(int fmt, const uint32_t *payload, const uint32_t *signs, const 
     if (!payload || !scales || !x || !x_scale || !y || !workspace) return BITCOS_ERR_NULL;
     if (fmt == kBitcos && (!signs || !tile_off)) return BITCOS_ERR_NULL;
     if (M < 1 || K < kGroup || K % kGroup != 0 || batch < 1 || batch > BITCOS_MAX_BATCH) return BITCOS_ERR_SHAPE;
-    if (K / kGroup > 0x7FFFFF || make_plan(M, K, kMaxWarps / 2).items > 0x3FFFFFFF) return BITCOS_ERR_SHAPE;
+    if (K / kGroup > 0x7FFFFF || make_plan(M, K, kWarps16).items > 0x3FFFFFFF) return BITCOS_ERR_SHAPE;
     if (!aligned16(payload) || !aligned16(scales) || !aligned16(x) || !aligned16(y) || !aligned16(workspace) ||
         (signs && !aligned16(signs)) || (tile_off && !aligned16(tile_off)) || (acc_debug && !aligned16(acc_debug)))
         return BITCOS_ERR_ALIGN;

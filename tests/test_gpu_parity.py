@@ -79,6 +79,9 @@ def test_config0_tiny(bc):
 @pytest.mark.parametrize("M,K,B", [
     (32, 128, 1), (1, 128, 1), (33, 256, 2), (100, 384, 3), (640, 2560, 1), (96, 6912, 1), (64, 2176, 5),
     (256, 512, 16), (50, 1280, 8), (2560, 2560, 1), (160, 25600, 2), (320, 8192, 1),
+    # four tokens and more: the contraction runs on the tensor cores; rows in one piece (K <= 2560,
+    # or 2048 for more than eight tokens) and rows cut into column blocks
+    (96, 6912, 8), (64, 5120, 16), (40, 3072, 4), (2560, 2560, 16), (33, 2560, 9), (700, 2048, 12), (65, 128, 7),
 ])
 def test_shapes_and_batches(bc, M, K, B):
     W, S = datagen.trits(100 + M, M, K, 0.42), datagen.scales(100 + M, M, K)
@@ -200,7 +203,8 @@ def test_host_buffer_entry_point(bc):
 def test_sampled_outputs_at_full_size(bc):
     """The largest layer shapes of the benchmark configurations, in the launch configuration
     the benchmark times; the oracle checks a sample of rows it computes one by one."""
-    for (M, K, z, B) in ((6912, 2560, 0.4219, 1), (2560, 6912, 0.4219, 1), (5120, 25600, 0.4711, 2)):
+    for (M, K, z, B) in ((6912, 2560, 0.4219, 1), (2560, 6912, 0.4219, 1), (5120, 25600, 0.4711, 2),
+                         (8192, 5120, 0.4711, 16), (6912, 2560, 0.4219, 8)):
         W, S = datagen.trits(500 + M, M, K, z), datagen.scales(500 + M, M, K)
         x, xs = datagen.activations(500 + M, B, K)
         rows = np.unique(np.concatenate([np.arange(0, M, max(1, M // 97)), [M - 1, M - 32, 31, 32]]))
