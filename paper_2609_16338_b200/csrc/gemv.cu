@@ -169,6 +169,8 @@ struct GroupedArgs {
     const int32_t *group_begin;
     size_t ws_stride;          // workspace bytes per group
     int n_experts;
+    int n_groups;
+    int flat;                  // 1: one list of all groups' items, split evenly over the thread blocks
 };
 
 inline int64_t padded_rows(int64_t M) { return (M + kRows - 1) / kRows * kRows; }
@@ -637,6 +639,9 @@ constexpr int kBarRedFull = 2 * kMaxStages;       // [slots] partial sums of an 
 constexpr int kBarRedEmpty = 2 * kMaxStages + 8;  // [slots] partial sums consumed by the epilogue warp
 constexpr int kBarLut = 2 * kMaxStages + 16;      // lookup table arrived
 
+__device__ __forceinline__ void mbar_inval(uint32_t bar) {
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -673,8 +678,13 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
 // bulk copies; warp NW+1 adds the decoders' partial sums in a fixed order and writes the
 // outputs (and runs the cross-block protocol).  The roles meet only through mbarriers, every
 // wait is bounded, and there is no block-wide barrier inside the loop.
+// `wk` is this block's share of the problem's items.  `fresh` is false when the block has already
+// run another problem with the same shared-memory layout: the lookup table is still in place and
+// the barriers are invalidated before they are set up again (the caller puts a block-wide barrier
+// between two runs).
 template <int FMT, int NB>
-__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, int block, int n_blocks) {
+__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
+                                            bool fresh = true) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const SmemLayout L = smem_layout(FMT, pl, pr.G, NB, pr.K);
     const uint8_t *lut = smem + L.lut;
@@ -683,7 +693,6 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 384);
     const uint32_t bar0 = smem_addr(smem + L.bar);
     const uint32_t red_slot = static_cast<uint32_t>(pl.NW) * NB * kRows;     // floats per partial-sum slot
-    const Walk wk = make_walk(pl, block, n_blocks);
 
     // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as
     // every block of this one got here; whatever it reads from us it reads after its own
@@ -702,6 +711,17 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     // happens in the block.
     if (warp == pl.NW) {
         if (lane == 0) {
+            if (!fresh) {
+                for (int s = 0; s < pl.stages; ++s) {
+                    mbar_inval(bar0 + 8u * (kBarFull + s));
+                    mbar_inval(bar0 + 8u * (kBarEmpty + s));
+                }
+                for (int s = 0; s < red_slots(NB); ++s) {
+                    mbar_inval(bar0 + 8u * (kBarRedFull + s));
+                    mbar_inval(bar0 + 8u * (kBarRedEmpty + s));
+                }
+                mbar_inval(bar0 + 8u * kBarLut);
+            }
             for (int s = 0; s < pl.stages; ++s) {
                 mbar_init(bar0 + 8u * (kBarFull + s), 1);
                 mbar_init(bar0 + 8u * (kBarEmpty + s), pl.NW);
@@ -747,7 +767,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
                 issue_item<FMT>(pr, pl, r0, L, smem, s, sign_base, lo0, hi0);
-                if (k == 0 && FMT != kBit2) {
+                if (k == 0 && FMT != kBit2 && fresh) {
                     mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
                     bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
                               bar0 + 8u * kBarLut);
@@ -953,7 +973,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     // CS == 1: this warp always has row block warp / G of the chunk and group warp % G
     const int my_rbl = (pl.CS == 1) ? warp / pr.G : 0;
     const int g_fixed = warp - my_rbl * pr.G;
-    if (FMT != kBit2) {
+    if (FMT != kBit2 && fresh) {
         if (!mbar_wait(bar0 + 8u * kBarLut, 0)) {
             if (lane == 0 && pr.status) *pr.status = 1u;
             return;
@@ -1161,7 +1181,8 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 template <int FMT, int NB>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
-    run_problem<FMT, NB>(pr, pl, smem, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
+    run_problem<FMT, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
+                         static_cast<int>(blockIdx.x));
 }
 
 // Several independent BITCOS problems in one launch: the grid is cut into one range of thread
@@ -1180,31 +1201,71 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     const int b = static_cast<int>(blockIdx.x);
     int j = 0;
     while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
-    run_problem<kBitcos, NB>(ma.pr[j], ma.pl[j], smem, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]);
+    run_problem<kBitcos, NB>(ma.pr[j], ma.pl[j], smem,
+                             make_walk(ma.pl[j], b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
+                             b - ma.first_block[j]);
 }
 
+// Fills in what differs between the groups of a grouped product; false if the group is empty or
+// names no expert.
 template <int NB>
-__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(Problem pr, const Plan pl, const GroupedArgs ga) {
-    extern __shared__ __align__(128) uint8_t smem[];
-    const int grp = blockIdx.y;
-    // the routing lists may come from the previous kernel in the stream
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+__device__ __forceinline__ bool grouped_problem(Problem &pr, const Problem &base, const GroupedArgs &ga, int grp) {
     const int e = __ldg(ga.group_expert + grp);
     const int begin = __ldg(ga.group_begin + grp), end = __ldg(ga.group_begin + grp + 1);
-    if (e < 0 || e >= ga.n_experts || end <= begin) return;
+    if (e < 0 || e >= ga.n_experts || end <= begin) return false;
     const bitcos_weights wdesc = ga.experts[e];
+    pr = base;
     pr.payload = wdesc.bitmap;
     pr.signs = wdesc.signs;
     pr.tile_off = wdesc.tile_off;
     pr.scales = wdesc.scales;
     pr.nb = min(end - begin, NB);
-    pr.xrow = pr.xrow + begin;
+    pr.xrow = base.xrow + begin;
     pr.out_row0 = begin;
-    uint8_t *ws = reinterpret_cast<uint8_t *>(pr.status) + static_cast<size_t>(grp) * ga.ws_stride;
+    uint8_t *ws = reinterpret_cast<uint8_t *>(base.status) + static_cast<size_t>(grp) * ga.ws_stride;
     pr.status = reinterpret_cast<unsigned int *>(ws);
     pr.counters = reinterpret_cast<unsigned int *>(ws + kHeaderBytes);
-    pr.partial = reinterpret_cast<float *>(ws + kHeaderBytes + ((static_cast<size_t>(pr.RB) * 4 + 255) / 256 * 256));
-    run_problem<kBitcos, NB>(pr, pl, smem, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x));
+    pr.partial = reinterpret_cast<float *>(ws + kHeaderBytes + ((static_cast<size_t>(base.RB) * 4 + 255) / 256 * 256));
+    return true;
+}
+
+// Grouped product.  Two launch shapes.  Flat (rows in one piece, no cross-block sums): the items
+// of all groups form one list, cut into equal contiguous ranges, one per thread block, so a
+// block runs the tail of one group and the head of the next with the same shared-memory layout.
+// Otherwise: blockIdx.y = group, and the blocks of a row of the grid share that group's items.
+template <int NB>
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(const Problem base, const Plan pl, const GroupedArgs ga) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    // the routing lists may come from the previous kernel in the stream
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    Problem pr;
+    if (!ga.flat) {
+        if (!grouped_problem<NB>(pr, base, ga, static_cast<int>(blockIdx.y))) return;
+        run_problem<kBitcos, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
+                                 static_cast<int>(blockIdx.x));
+        return;
+    }
+    const int64_t ipg = pl.items, total = ipg * ga.n_groups;
+    const int64_t nblk = gridDim.x, b = blockIdx.x;
+    const int64_t q = total / nblk, rem = total - q * nblk;
+    int64_t lo = b * q + (b < rem ? b : rem);
+    const int64_t hi = lo + q + (b < rem ? 1 : 0);
+    bool fresh = true;
+    for (int grp = static_cast<int>(lo / ipg); lo < hi; ++grp) {
+        const int64_t g_lo = static_cast<int64_t>(grp) * ipg;
+        const int64_t seg_hi = hi < g_lo + ipg ? hi : g_lo + ipg;
+        Walk wk;
+        wk.first = static_cast<int>(lo - g_lo);
+        wk.count = static_cast<int>(seg_hi - lo);
+        wk.cstride = 1;
+        wk.q = 1;
+        wk.rem = 0;
+        lo = seg_hi;
+        if (!grouped_problem<NB>(pr, base, ga, grp)) continue;
+        if (!fresh) __syncthreads();          // everybody is done with the previous group's barriers and buffers
+        run_problem<kBitcos, NB>(pr, pl, smem, wk, static_cast<int>(b), fresh);
+        fresh = false;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1441,15 +1502,26 @@ int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int
     int sms = 0, budget = 0;
     int rc = prepare_kernel<gemv_grouped_kernel<NB>>(&sms, &budget);
     if (rc) return rc;
+    Plan plw = pl;
+    plw.stages = choose_stages(kBitcos, pl, pr.G, NB, pr.K, budget);
+    const SmemLayout L = smem_layout(kBitcos, plw, pr.G, NB, pr.K);
+    GroupedArgs gaw = ga;
+    gaw.n_groups = n_groups;
+    if (pl.CS == 1) {
+        // rows in one piece: one balanced list of all groups' items
+        const int64_t total = pl.items * n_groups;
+        gaw.flat = 1;
+        plw.cyclic = 0;
+        return launch_pdl(gemv_grouped_kernel<NB>, dim3(static_cast<unsigned>(total < sms ? total : sms)), (pl.NW + 2) * 32,
+                          L.total, stream, pr, plw, gaw);
+    }
     // the machine is shared by all groups: spread its multiprocessors over them
     int per_group = (sms + n_groups - 1) / n_groups;
     if (per_group < 1) per_group = 1;
     int gx = 1;
-    Plan plw = pl;
     choose_walk(plw, per_group, &gx);
-    plw.stages = choose_stages(kBitcos, pl, pr.G, NB, pr.K, budget);
-    const SmemLayout L = smem_layout(kBitcos, plw, pr.G, NB, pr.K);
-    return launch_pdl(gemv_grouped_kernel<NB>, dim3(gx, n_groups), (pl.NW + 2) * 32, L.total, stream, pr, plw, ga);
+    gaw.flat = 0;
+    return launch_pdl(gemv_grouped_kernel<NB>, dim3(gx, n_groups), (pl.NW + 2) * 32, L.total, stream, pr, plw, gaw);
 }
 
 // Validates the arguments every product shares; fills nothing.
@@ -1720,7 +1792,7 @@ int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M,
     pr.G = static_cast<int>(K / kGroup);
     pr.RB = static_cast<int>(padded_rows(M) / kRows);
     pr.status = static_cast<unsigned int *>(workspace);
-    GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts};
+    GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts, n_groups, 0};
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (max_group_size <= 1) return launch_grouped<1>(pr, pl, ga, n_groups, stream);
     if (max_group_size <= 2) return launch_grouped<2>(pr, pl, ga, n_groups, stream);
