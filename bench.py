@@ -187,6 +187,52 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------
+# Ranks: one process per GPU, independent replicas of the same workload (the path has no exchange
+# step).  The only communication is the barrier around the timed region and the maximum over the
+# ranks' times.
+# ---------------------------------------------------------------------------------------------
+class Ranks:
+    """Process group plumbing of the benchmark: world size and rank from the launcher's environment,
+    a barrier, and the maximum of a per-rank number.  backend "nccl" on GPUs; "gloo" lets the same
+    code run on CPU (the tests do that with two processes)."""
+
+    def __init__(self, backend="nccl", device=None):
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.device = device
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            kw = {"device_id": device} if (backend == "nccl" and device is not None) else {}
+            dist.init_process_group(backend, **kw)
+            self.dist = dist
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+
+    def max(self, value):
+        """Largest `value` over all ranks (every rank gets it)."""
+        if self.dist is None:
+            return float(value)
+        import torch
+        t = torch.tensor([float(value)], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+            self.dist = None
+
+
+def whole_job_value(us_per_step, world):
+    """Time per token of the whole job: every replica finishes one token per step."""
+    return us_per_step / world
+
+
+# ---------------------------------------------------------------------------------------------
 # CUDA arm
 # ---------------------------------------------------------------------------------------------
 def run_cuda(args):
@@ -194,20 +240,15 @@ def run_cuda(args):
     import paper_2609_16338_b200 as bc
     from paper_2609_16338_b200 import build as lib_build
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    ranks = Ranks("nccl", torch.device("cuda", local_rank))
+    world, rank = ranks.world, ranks.rank
     if rank == 0:
         lib_build.build()
-    if dist is not None:
-        dist.barrier()
+    ranks.barrier()
     bc.load_library()
     L = bc.load_library()
 
@@ -316,8 +357,7 @@ def run_cuda(args):
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
-    if dist is not None:
-        dist.barrier()
+    ranks.barrier()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
@@ -329,8 +369,7 @@ def run_cuda(args):
         e1.record(stream)
     stream.synchronize()
     torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
+    ranks.barrier()
     ms = e0.elapsed_time(e1)
     # keep the GPU busy a little longer so that the clock sampler sees it under load
     t_end = time.time() + (0.0 if args.no_graph else 0.6)
@@ -339,10 +378,7 @@ def run_cuda(args):
             (graphs.get("full") or graphs["rem"]).replay()
             stream.synchronize()
     clocks = sampler.stop()
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = ranks.max(ms)
 
     # ---- end to end: host buffers through bitcos_gemv_host, copies inside the timed region ----
     stagings = [torch.empty(bc.bitcos_gemv_host_staging_bytes(m["M"], m["K"], 1), dtype=torch.uint8, device="cuda")
@@ -368,16 +404,12 @@ def run_cuda(args):
             e2e_step(i)
         torch.cuda.synchronize()
         e2e_us = (time.perf_counter() - t0) / e2e_steps * 1e6
-    if dist is not None:
-        t = torch.tensor([e2e_us], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_us = float(t.item())
+    e2e_us = ranks.max(e2e_us)
     h2d = sum(m["K"] + 4 for m in layer)
     d2h = sum(4 * m["M"] for m in layer)
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+        ranks.close()
         return
 
     # ---- per-shape detail: each format on each shape, rotated copies, CUDA graph of 64 launches ----
@@ -402,7 +434,7 @@ def run_cuda(args):
     n_launch = launches_per_step * args.steps
     achieved = layer_bytes * args.steps / (ms * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": us_per_step / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_value(us_per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": us_per_step / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": workload, "batch": 1, "weights": int(sum(m["M"] * m["K"] for m in layer)),
@@ -428,7 +460,7 @@ def run_cuda(args):
         "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
                          "sample": f"{reps} full layer passes (7 GEMVs, 69.5 M weights each): BITCOS decode bit by "
                                    "bit, dense int32 dot per group, double scale-and-sum"},
-        "e2e": {"value": e2e_us / world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        "e2e": {"value": whole_job_value(e2e_us, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "path": "bitcos_gemv_host per GEMV: pinned x -> device, kernel, y -> pinned host, "
                                             "stream wait"},
         "gpu_launches": n_launch,
@@ -437,9 +469,11 @@ def run_cuda(args):
     line["two_term_roofline"] = two_term_roofline(bc, cfg["z"], peak, clocks.get("sm_mhz") or 1965.0)
     if detail is not None:
         line["shapes"] = detail
+        line["batch"] = batch_detail(bc, torch, stream)
+    if args.moe:
+        line["moe"] = moe_detail(bc, torch, stream)
     print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 def two_term_roofline(bc, z, peak_gbs, sm_mhz, sms=148):
@@ -508,6 +542,174 @@ def shape_detail(bc, torch, layer, host_packed, stream, launches=64):
     return out
 
 
+def graph_time_us(torch, stream, launch, n_copies, launches=48, repeats=5):
+    """Median microseconds per launch of `launch(i)` (i = which rotated copy), from CUDA graphs of
+    `launches` launches replayed `repeats` times, events on the launching stream."""
+    launch(0)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(launches):
+                launch(i % n_copies)
+        g.replay()
+        stream.synchronize()
+        times = []
+        for _ in range(repeats):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            stream.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e3 / launches)
+    return float(np.median(times))
+
+
+def graph_time_flushed_us(torch, stream, launch, n_variants, flush, launches=24, repeats=5):
+    """Like graph_time_us for launches whose working set is smaller than L2: every launch is
+    preceded by a write of `flush` (larger than L2); the time of a graph holding only the flushes
+    is subtracted."""
+    launch(0)
+    torch.cuda.synchronize()
+
+    def timed(with_launch):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(launches):
+                    flush.zero_()
+                    if with_launch:
+                        launch(i % n_variants)
+            g.replay()
+            stream.synchronize()
+            times = []
+            for _ in range(repeats):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                g.replay()
+                e1.record(stream)
+                stream.synchronize()
+                times.append(e0.elapsed_time(e1) * 1e3 / launches)
+        return float(np.median(times))
+
+    return timed(True) - timed(False)
+
+
+def batch_detail(bc, torch, stream, M=8192, K=5120, z=0.4711):
+    """Small-batch decode on one Qwen3-32B-shaped matrix (the q projection): the three formats at
+    1, 2, 4, 8, 16 tokens; the weights are read once per call whatever the batch."""
+    import datagen
+    peak, _ = measured_peaks()
+    seed = datagen.config_seed(3, 0)
+    W, S = datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)
+    st = bc.scales_tile(S, M, K)
+    packed = bc.bitcos_pack(W, S)
+    fmts = {"bitcos": (packed.to_device(), bc.bitcos_gemv),
+            "trit5": (bc.plain_to_device(bc.trit5_pack(W), st, M, K), bc.trit5_gemv),
+            "bit2": (bc.plain_to_device(bc.bit2_pack(W), st, M, K), bc.bit2_gemv)}
+    ws = bc.make_workspace(M, K)
+    out = {"M": M, "K": K, "z": z, "rows": []}
+    for B in (1, 2, 4, 8, 16):
+        x, xs = datagen.activations(seed, B, K)
+        xd, xsd = torch.from_numpy(x).cuda(), torch.from_numpy(xs).cuda()
+        y = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        row = {"batch": B, "contraction": "dp4a" if B < 4 else "mma.m16n8k32.s8"}
+        for name, (Wd, f) in fmts.items():
+            n_copies = max(2, int(np.ceil(4.2 * L2_BYTES / Wd.payload_bytes())))
+            reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
+            us = graph_time_us(torch, stream, lambda i: f(reps[i], xd, xsd, y=y, workspace=ws), n_copies)
+            nbytes = algorithmic_bytes(M, K, packed.nnz, B, name)
+            row[name] = {"us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
+                         "us_per_token": us / B}
+            del reps
+        out["rows"].append(row)
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_profile_batch(args):
+    """A few plain stream launches of one format at one batch size on the batch table's matrix
+    (for profilers: no graphs, nothing else on the device).  Prints a small JSON line."""
+    import torch
+    import datagen
+    import paper_2609_16338_b200 as bc
+    from paper_2609_16338_b200 import build as lib_build
+    lib_build.build()
+    bc.load_library()
+    M, K, z, B = 8192, 5120, 0.4711, args.profile_batch
+    seed = datagen.config_seed(3, 0)
+    W, S = datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)
+    packed = bc.bitcos_pack(W, S)
+    Wd = packed.to_device()
+    n_copies = max(2, int(np.ceil(1.5 * L2_BYTES / Wd.payload_bytes())))
+    reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
+    x, xs = datagen.activations(seed, B, K)
+    xd, xsd = torch.from_numpy(x).cuda(), torch.from_numpy(xs).cuda()
+    y = torch.empty((B, M), dtype=torch.float32, device="cuda")
+    ws = bc.make_workspace(M, K)
+    for i in range(3):
+        bc.bitcos_gemv(reps[i % n_copies], xd, xsd, y=y, workspace=ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        bc.bitcos_gemv(reps[i % n_copies], xd, xsd, y=y, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / args.steps
+    print(json.dumps({"profile_batch": B, "M": M, "K": K, "launches": args.steps + 3, "us_per_launch_with_host_gaps": us,
+                      "status": bc.workspace_status(ws)}))
+
+
+def moe_detail(bc, torch, stream, E=128, top_k=8, z=0.3288):
+    """Grouped BITCOS product over the selected experts of a Qwen3-30B-A3B-shaped layer: gate/up
+    (768 x 2048, the token's activations) and down (2048 x 768, one activation row per pair), 1 to 16
+    tokens, expert ids drawn without replacement per token.  The experts of one projection (46 MB
+    packed) would fit in L2, so L2 is flushed before every launch and the routing is redrawn."""
+    import datagen
+    peak, _ = measured_peaks()
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a.view(np.int32) if a.dtype == np.uint32 else a)).cuda()
+
+    out = []
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+    for name, (M, K) in (("gate/up", (768, 2048)), ("down", (2048, 768))):
+        host = [bc.bitcos_pack(datagen.trits(datagen.config_seed(4, e), M, K, z), datagen.scales(datagen.config_seed(4, e), M, K))
+                for e in range(E)]
+        experts = bc.DeviceExperts([h.to_device() for h in host])
+        for tokens in (1, 2, 4, 8, 16):
+            draws = []
+            for d in range(12):
+                ids = datagen.expert_choices(1000 * tokens + d, tokens, E, top_k)
+                pair_expert = ids.reshape(-1)
+                if name == "gate/up":
+                    pair_xrow = np.repeat(np.arange(tokens, dtype=np.int32), top_k)
+                    x, xs = datagen.activations(17, tokens, K)
+                else:
+                    pair_xrow = np.arange(tokens * top_k, dtype=np.int32)
+                    x, xs = datagen.activations(17, tokens * top_k, K)
+                order, ge, gb, xr, mx = bc.group_pairs(pair_expert, pair_xrow)
+                nbytes = sum(algorithmic_bytes(M, K, host[e].nnz, int(gb[i + 1] - gb[i])) for i, e in enumerate(ge))
+                draws.append((dev(ge), dev(gb), dev(xr), mx, len(ge), nbytes))
+            xd, xsd = dev(x), dev(xs)
+            ws = bc.make_workspace(M, K, copies=max(d[4] for d in draws))
+            y = torch.empty((tokens * top_k, M), dtype=torch.float32, device="cuda")
+
+            def launch(i):
+                ge, gb, xr, mx, _, _ = draws[i]
+                bc.bitcos_gemv_grouped(experts, ge, gb, xr, mx, xd, xsd, y=y, workspace=ws)
+
+            us = graph_time_flushed_us(torch, stream, launch, len(draws), flush)
+            nbytes = float(np.mean([d[5] for d in draws]))
+            out.append({"projection": name, "M": M, "K": K, "tokens": tokens,
+                        "distinct_experts": float(np.mean([d[4] for d in draws])), "us": us,
+                        "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak})
+        del experts
+        torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -521,7 +723,15 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA graphs (for profilers)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--profile-batch", type=int, default=0, metavar="B",
+                    help="only launch bitcos_gemv at batch B on the batch table's matrix, --steps times (for profilers)")
+    ap.add_argument("--moe", action="store_true", help="add the grouped mixture-of-experts table (slow to generate)")
     args = ap.parse_args()
+    if args.profile_batch:
+        if args.steps is None:
+            args.steps = 6
+        run_profile_batch(args)
+        return
     if args.impl == "reference":
         if args.steps is None:
             args.steps = 3
