@@ -39,8 +39,11 @@ METRIC = "bitcos_gemv_us_per_token"
 UNIT = "us"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of the seven GEMVs of one step, from the ncu capture summarised in profiles/launch_list_and_dram_traffic_bitnet2b_layer_bench.md
-NCU_DRAM_BYTES_PER_STEP = 15627520
+# dram__bytes_read.sum + dram__bytes_write.sum of all launches of one step, from ncu captures of this
+# command: four launches per step (the default;
+# profiles/launch_list_and_dram_traffic_bitnet2b_layer_bench_default.md) and seven (--serial / --branches,
+# an earlier capture of the same kernels)
+NCU_DRAM_BYTES_PER_STEP = {4: 15312282, 7: 15627520}
 
 
 def layer_config():
@@ -452,7 +455,7 @@ def run_cuda(args):
         "achieved_gbs": achieved,
         "frac_of_8tbs": achieved / 8000.0,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_DRAM_BYTES_PER_STEP / launches_per_step, "peak_source": f"{which} (STREAM-style copy)",
+                     "traffic": NCU_DRAM_BYTES_PER_STEP[launches_per_step] / launches_per_step, "peak_source": f"{which} (STREAM-style copy)",
                      "kernel": "gemv_kernel<bitcos, 1 token>" if launches_per_step == 7 else "gemv_multi_kernel<1 token>",
                      "launches": n_launch,
                      "avg_launch_us": ms * 1e3 / n_launch,
