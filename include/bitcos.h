@@ -163,7 +163,11 @@ int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, 
  * entry offset + running population count locate each row's sign window, a 256-entry
  * (presence nibble, sign nibble) table as in Eq. 4 rebuilds four weights at a time as int8,
  * dp4a accumulates int32 per group, the bf16 group scale and the per-token scale are applied
- * in fp32).
+ * in fp32).  The paper measures one token; for batch >= 3 the same int32 group accumulators come
+ * from int8 tensor-core instructions (mma.m16n8k32) fed with the decoded rows, so that the weights
+ * are decoded once per call whatever the batch.  The accumulators are exact for every batch; y is
+ * deterministic for a given batch size and device (fixed summation order), and the summation
+ * order over groups may differ between batch sizes.
  *   W            host struct holding device pointers
  *   x            device int8 [batch][K], row major
  *   x_scale      device float [batch]
