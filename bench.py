@@ -415,6 +415,13 @@ def run_cuda(args):
         ranks.close()
         return
 
+    # ---- the same seven products as ONE launch per step (what the launch structure costs) ----
+    one_launch_us = None
+    if not args.no_detail:
+        all_jobs = [bc.MultiJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in range(len(layer))])
+                    for rep in replicas]
+        one_launch_us = graph_time_us(torch, stream, lambda i: bc.bitcos_gemv_multi(all_jobs[i]), copies, launches=copies)
+
     # ---- per-shape detail: each format on each shape, rotated copies, CUDA graph of 64 launches ----
     detail = shape_detail(bc, torch, layer, host_packed, stream) if not args.no_detail else None
 
@@ -471,9 +478,17 @@ def run_cuda(args):
     }
     line["two_term_roofline"] = two_term_roofline(bc, cfg["z"], peak, clocks.get("sm_mhz") or 1965.0)
     if detail is not None:
+        line["one_launch_per_step"] = {
+            "us": one_launch_us, "gbs": layer_bytes / one_launch_us / 1e3, "frac": layer_bytes / one_launch_us / 1e3 / peak,
+            "note": "all seven products of the layer in a single bitcos_gemv_multi launch: possible for independent "
+                    "products only (in a decoder layer o follows attention over q, k, v and down follows gate and up), so "
+                    "this is not the headline; it shows how much of the step is launch structure"}
         line["shapes"] = detail
         line["batch"] = batch_detail(bc, torch, stream)
-    if args.moe:
+    if args.all_configs:
+        line["density_sweep"] = sweep_detail(bc, torch, stream)
+        line["qwen32b_layer"] = qwen32b_layer_detail(bc, torch, stream)
+    if args.moe or args.all_configs:
         line["moe"] = moe_detail(bc, torch, stream)
     print(json.dumps(line))
     ranks.close()
@@ -630,6 +645,79 @@ def batch_detail(bc, torch, stream, M=8192, K=5120, z=0.4711):
     return out
 
 
+def sweep_detail(bc, torch, stream):
+    """Zero-density sweep (two matrix shapes, five densities, one token): the three formats on
+    identical weights, realised gain against the byte ratio."""
+    import datagen
+    peak, _ = measured_peaks()
+    out = []
+    for si, (M, K) in enumerate(((4096, 12288), (12288, 4096))):
+        ws = bc.make_workspace(M, K)
+        for zi, z in enumerate((0.30, 0.375, 0.42, 0.47, 0.515)):
+            seed = datagen.config_seed(2, 10 * si + zi)
+            W, S = datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)
+            x, xs = datagen.activations(seed, 1, K)
+            xd, xsd = torch.from_numpy(x).cuda(), torch.from_numpy(xs).cuda()
+            y = torch.empty((1, M), dtype=torch.float32, device="cuda")
+            st = bc.scales_tile(S, M, K)
+            packed = bc.bitcos_pack(W, S)
+            fmts = {"bitcos": (packed.to_device(), bc.bitcos_gemv),
+                    "trit5": (bc.plain_to_device(bc.trit5_pack(W), st, M, K), bc.trit5_gemv),
+                    "bit2": (bc.plain_to_device(bc.bit2_pack(W), st, M, K), bc.bit2_gemv)}
+            row = {"M": M, "K": K, "z": z, "z_realised": 1.0 - packed.nnz / float(M * K)}
+            for name, (Wd, f) in fmts.items():
+                n_copies = max(2, int(np.ceil(4.2 * L2_BYTES / Wd.payload_bytes())))
+                reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
+                us = graph_time_us(torch, stream, lambda i: f(reps[i], xd, xsd, y=y, workspace=ws), n_copies)
+                nbytes = algorithmic_bytes(M, K, packed.nnz, 1, name)
+                row[name] = {"us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak, "bytes": int(nbytes)}
+                del reps
+            row["speedup_vs_trit5"] = row["trit5"]["us"] / row["bitcos"]["us"]
+            row["byte_ratio_trit5"] = row["trit5"]["bytes"] / row["bitcos"]["bytes"]
+            row["speedup_vs_bit2"] = row["bit2"]["us"] / row["bitcos"]["us"]
+            row["byte_ratio_bit2"] = row["bit2"]["bytes"] / row["bitcos"]["bytes"]
+            out.append(row)
+            torch.cuda.empty_cache()
+    return out
+
+
+def qwen32b_layer_detail(bc, torch, stream, z=0.4711):
+    """One decode step through the seven linear maps of a Qwen3-32B-shaped layer at 1 to 16 tokens:
+    four launches per step as in the headline (q+k+v, o, gate+up, down), two rotated copies of the
+    101 MB layer (each launch's weights were last read two steps and more than L2's size ago)."""
+    import datagen
+    peak, _ = measured_peaks()
+    shapes = [("q", 8192, 5120), ("k", 1024, 5120), ("v", 1024, 5120), ("o", 5120, 8192), ("gate", 25600, 5120),
+              ("up", 25600, 5120), ("down", 5120, 25600)]
+    host = []
+    for i, (_, M, K) in enumerate(shapes):
+        seed = datagen.config_seed(3, i)
+        host.append(bc.bitcos_pack(datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)))
+    base = [h.to_device() for h in host]
+    replicas = [base, [w.clone() for w in base]]
+    wss = [bc.make_workspace(M, K) for (_, M, K) in shapes]
+    groups = [[0, 1, 2], [3], [4, 5], [6]]
+    out = []
+    for B in (1, 2, 4, 8, 16):
+        xs_dev = []
+        for i, (_, M, K) in enumerate(shapes):
+            x, xs = datagen.activations(datagen.config_seed(3, i), B, K)
+            xs_dev.append((torch.from_numpy(x).cuda(), torch.from_numpy(xs).cuda()))
+        ys = [torch.empty((B, M), dtype=torch.float32, device="cuda") for (_, M, K) in shapes]
+        multi = [[bc.MultiJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in g]) for g in groups]
+                 for rep in replicas]
+
+        def step(i):
+            for mj in multi[i]:
+                bc.bitcos_gemv_multi(mj)
+
+        us = graph_time_us(torch, stream, step, len(replicas), launches=8)
+        nbytes = sum(algorithmic_bytes(M, K, h.nnz, B) for (_, M, K), h in zip(shapes, host))
+        out.append({"batch": B, "us_per_step": us, "us_per_token": us / B, "gbs": nbytes / us / 1e3,
+                    "frac": nbytes / us / 1e3 / peak, "bytes": int(nbytes)})
+    return out
+
+
 def run_profile_batch(args):
     """A few plain stream launches of one format at one batch size on the batch table's matrix
     (for profilers: no graphs, nothing else on the device).  Prints a small JSON line."""
@@ -728,6 +816,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--profile-batch", type=int, default=0, metavar="B",
                     help="only launch bitcos_gemv at batch B on the batch table's matrix, --steps times (for profilers)")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="add the density sweep and the Qwen3-32B-shaped layer at 1-16 tokens (minutes of host-side packing)")
     ap.add_argument("--moe", action="store_true", help="add the grouped mixture-of-experts table (slow to generate)")
     args = ap.parse_args()
     if args.profile_batch:

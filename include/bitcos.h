@@ -177,7 +177,9 @@ int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, 
 int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
                 int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
-/* Up to four independent BITCOS products in ONE launch (same batch; shapes may differ): e.g. the
+#define BITCOS_MAX_JOBS 8
+
+/* Up to BITCOS_MAX_JOBS independent BITCOS products in ONE launch (same batch; shapes may differ): e.g. the
  * q, k and v projections of a decoder layer, which read the same activations and do not depend on
  * one another, or gate and up.  The multiprocessors are shared between the jobs in proportion to
  * their sizes, so small matrices run side by side instead of one after the other and the fixed

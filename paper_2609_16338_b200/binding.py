@@ -377,7 +377,7 @@ class MultiJobs:
 
 
 def bitcos_gemv_multi(jobs):
-    """Up to four independent BITCOS products in one launch; `jobs` is a MultiJobs or a list of
+    """Up to eight (BITCOS_MAX_JOBS) independent BITCOS products in one launch; `jobs` is a MultiJobs or a list of
     (W, x, x_scale, y, workspace) tuples with a common batch size."""
     mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
     _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")

@@ -1187,7 +1187,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Pr
 
 // Several independent BITCOS problems in one launch: the grid is cut into one range of thread
 // blocks per problem, and every block runs the ordinary kernel body on its problem.
-constexpr int kMaxJobs = 4;
+constexpr int kMaxJobs = BITCOS_MAX_JOBS;
 struct MultiArgs {
     Problem pr[kMaxJobs];
     Plan pl[kMaxJobs];
@@ -1488,10 +1488,19 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream) {
     return launch_pdl(gemv_multi_kernel<NB>, dim3(next), (nw + 2) * 32, smem, stream, ma);
 }
 
+// Which instantiation serves a batch: 1, 2, 4, 8 or 16 tokens.  The one- and two-token paths read
+// the activations from shared memory; when those do not fit there (K beyond 48 K / 24 K), the
+// tensor-core path, which takes its activation fragments from global memory, is the faster one.
+inline int nb_bucket(int batch, int64_t K) {
+    if (batch <= 2 && static_cast<int64_t>(batch) * K > kXResidentBytes) return 4;
+    return batch <= 1 ? 1 : batch <= 2 ? 2 : batch <= 4 ? 4 : batch <= 8 ? 8 : 16;
+}
+
 template <int FMT>
 int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream) {
-    if (pr.nb <= 1) return launch<FMT, 1>(pr, pl, stream);
-    if (pr.nb <= 2) return launch<FMT, 2>(pr, pl, stream);
+    const int nbk = nb_bucket(pr.nb, pr.K);
+    if (nbk == 1) return launch<FMT, 1>(pr, pl, stream);
+    if (nbk == 2) return launch<FMT, 2>(pr, pl, stream);
     if (pr.nb <= 4) return launch<FMT, 4>(pr, pl, stream);
     if (pr.nb <= 8) return launch<FMT, 8>(pr, pl, stream);
     return launch<FMT, 16>(pr, pl, stream);
@@ -1711,8 +1720,11 @@ int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
                      jb.x_scale, batch, jb.y, nullptr, jb.workspace);
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (batch <= 1) return launch_multi<1>(ma, stream);
-    if (batch <= 2) return launch_multi<2>(ma, stream);
+    int64_t kmax = 0;
+    for (int j = 0; j < n_jobs; ++j) kmax = jobs[j].W->K > kmax ? jobs[j].W->K : kmax;
+    const int nbk = nb_bucket(batch, kmax);
+    if (nbk == 1) return launch_multi<1>(ma, stream);
+    if (nbk == 2) return launch_multi<2>(ma, stream);
     if (batch <= 4) return launch_multi<4>(ma, stream);
     if (batch <= 8) return launch_multi<8>(ma, stream);
     return launch_multi<16>(ma, stream);
@@ -1794,8 +1806,9 @@ int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M,
     pr.status = static_cast<unsigned int *>(workspace);
     GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts, n_groups, 0};
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (max_group_size <= 1) return launch_grouped<1>(pr, pl, ga, n_groups, stream);
-    if (max_group_size <= 2) return launch_grouped<2>(pr, pl, ga, n_groups, stream);
+    const int nbk = nb_bucket(max_group_size, K);
+    if (nbk == 1) return launch_grouped<1>(pr, pl, ga, n_groups, stream);
+    if (nbk == 2) return launch_grouped<2>(pr, pl, ga, n_groups, stream);
     if (max_group_size <= 4) return launch_grouped<4>(pr, pl, ga, n_groups, stream);
     if (max_group_size <= 8) return launch_grouped<8>(pr, pl, ga, n_groups, stream);
     return launch_grouped<16>(pr, pl, ga, n_groups, stream);

@@ -160,7 +160,7 @@ def test_grouped_down_projection_shape(bc):
 @pytest.mark.parametrize("B", [1, 3])
 def test_multi_launch_matches_separate_products(bc, B):
     """Several independent matrices (different shapes, also different K) in one launch."""
-    shapes = [(2560, 2560), (640, 2560), (96, 6912), (320, 1280)]
+    shapes = [(2560, 2560), (640, 2560), (96, 6912), (320, 1280), (64, 128), (33, 2560), (1000, 512), (32, 5120)]
     jobs, refs = [], []
     for i, (M, K) in enumerate(shapes):
         W, S = datagen.trits(600 + i, M, K, 0.4219), datagen.scales(600 + i, M, K)
@@ -168,7 +168,7 @@ def test_multi_launch_matches_separate_products(bc, B):
         refs.append(oracle.gemv_dense(W, S, x, xs))
         y = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
         jobs.append((bc.bitcos_pack(W, S).to_device(), dev(x), dev(xs), y, bc.make_workspace(M, K)))
-    for n in (4, 3, 1):
+    for n in (8, 5, 3, 1):
         for rep in range(2):
             for j in jobs:
                 j[3].fill_(float("nan"))
