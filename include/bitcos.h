@@ -132,6 +132,12 @@ typedef struct bitcos_weights {
     const uint16_t *scales;   /* tile order */
     int64_t M;
     int64_t K;
+    /* Optional (NULL if absent): a HOST copy of tile_off, as bitcos_pack wrote it.  With it the
+     * launch hands every thread block the entry offsets of its first tiles by value, which takes one
+     * dependent device-memory round trip out of the start of each call.  The paper has no
+     * counterpart; results do not depend on it.  Ignored by bitcos_gemv_grouped (its descriptors
+     * live in device memory). */
+    const uint32_t *tile_off_host;
 } bitcos_weights;
 
 /* Scratch memory the GEMV entry points need for an M x K matrix (the same value for all

@@ -40,7 +40,7 @@ class _Job(C.Structure):
 
 class _Weights(C.Structure):
     _fields_ = [("bitmap", C.c_void_p), ("signs", C.c_void_p), ("tile_off", C.c_void_p), ("scales", C.c_void_p),
-                ("M", C.c_int64), ("K", C.c_int64)]
+                ("M", C.c_int64), ("K", C.c_int64), ("tile_off_host", C.c_void_p)]
 
 
 _lib = None
@@ -133,20 +133,26 @@ class PackedBitcos:
         off = self.tile_off_buf if self.tile_off_buf is not None else self.tile_off
         t = [torch.from_numpy(a.view(np.int32) if a.dtype == np.uint32 else a.view(np.int16)).to(device)
              for a in (self.bitmap, self.signs, off, self.scales)]
-        return DeviceBitcos(self.M, self.K, self.nnz, *t)
+        return DeviceBitcos(self.M, self.K, self.nnz, *t, tile_off_host=np.ascontiguousarray(self.tile_off))
 
 
 class DeviceBitcos:
     """A BITCOS matrix resident in device memory (tensors only own the bytes)."""
 
-    def __init__(self, M, K, nnz, bitmap, signs, tile_off, scales):
+    def __init__(self, M, K, nnz, bitmap, signs, tile_off, scales, tile_off_host=None):
         self.M, self.K, self.nnz = M, K, nnz
         self.bitmap, self.signs, self.tile_off, self.scales = bitmap, signs, tile_off, scales
-        self.desc = _Weights(bitmap.data_ptr(), signs.data_ptr(), tile_off.data_ptr(), scales.data_ptr(), M, K)
+        self.tile_off_host = tile_off_host           # optional host copy (numpy uint32), kept alive here
+        self.desc = _Weights(bitmap.data_ptr(), signs.data_ptr(), tile_off.data_ptr(), scales.data_ptr(), M, K,
+                             tile_off_host.ctypes.data if tile_off_host is not None else None)
 
     def clone(self):
         return DeviceBitcos(self.M, self.K, self.nnz, self.bitmap.clone(), self.signs.clone(),
-                            self.tile_off.clone(), self.scales.clone())
+                            self.tile_off.clone(), self.scales.clone(), self.tile_off_host)
+
+    def without_host_offsets(self):
+        """The same device buffers, described without the host copy of tile_off."""
+        return DeviceBitcos(self.M, self.K, self.nnz, self.bitmap, self.signs, self.tile_off, self.scales, None)
 
     def payload_bytes(self) -> int:
         n_tiles = (self.M + TILE_ROWS - 1) // TILE_ROWS * (self.K // GROUP)

@@ -163,6 +163,15 @@ struct Problem {
     int64_t out_row0;          // first output row of y / acc_debug for token 0
 };
 
+// Entry offsets of every thread block's first item (sign-vector positions of its first tile and of
+// the tile after its last), passed by value when the caller supplied a host copy of tile_off.
+constexpr int kMaxGrid = 160;
+struct FirstOff {
+    uint32_t lo[kMaxGrid];
+    uint32_t hi[kMaxGrid];
+    int valid;
+};
+
 struct GroupedArgs {
     const bitcos_weights *experts;
     const int32_t *group_expert;
@@ -521,7 +530,7 @@ struct Walk {
 // with all their column blocks (no row block is ever shared; all blocks read neighbouring
 // addresses at any time).  Contiguous: a balanced split of the item list (perfect balance when
 // there are few chunks per block, at the price of sharing the row blocks cut by a boundary).
-__device__ __forceinline__ Walk make_walk(const Plan &pl, int block, int n_blocks) {
+__host__ __device__ __forceinline__ Walk make_walk(const Plan &pl, int block, int n_blocks) {
     Walk w;
     const int items = static_cast<int>(pl.items);
     if (pl.cyclic) {
@@ -556,7 +565,7 @@ struct ItemRange {
     int64_t t0;      // first tile
 };
 
-__device__ __forceinline__ ItemRange item_range(const Problem &pr, const Plan &pl, int c, int cs) {
+__host__ __device__ __forceinline__ ItemRange item_range(const Problem &pr, const Plan &pl, int c, int cs) {
     ItemRange r;
     r.rb0 = c * pl.RBC;
     r.cs = cs;
@@ -575,11 +584,11 @@ __device__ __forceinline__ ItemRange item_range(const Problem &pr, const Plan &p
 // (chunk, column block) of an item, and the step to the next item, without divisions in loops
 struct ItemIter {
     int c, cs;
-    __device__ __forceinline__ void init(const Plan &pl, int item) {
+    __host__ __device__ __forceinline__ void init(const Plan &pl, int item) {
         if (pl.CS == 1) { c = item; cs = 0; }
         else { c = item / pl.CS; cs = item - c * pl.CS; }
     }
-    __device__ __forceinline__ void next(const Plan &pl, const Walk &w) {
+    __host__ __device__ __forceinline__ void next(const Plan &pl, const Walk &w) {
         if (++cs == pl.CS) { cs = 0; c += w.cstride; }
     }
 };
@@ -684,7 +693,7 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
 // between two runs).
 template <int FMT, int NB>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
-                                            bool fresh = true) {
+                                            bool fresh = true, const FirstOff *fo = nullptr, int fo_index = 0) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const SmemLayout L = smem_layout(FMT, pl, pr.G, NB, pr.K);
     const uint8_t *lut = smem + L.lut;
@@ -785,8 +794,13 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             it2.init(pl, wk.first);
             r0 = item_range(pr, pl, it2.c, it2.cs);
             if (FMT == kBitcos) {
-                lo0 = __ldg(pr.tile_off + r0.t0);
-                hi0 = __ldg(pr.tile_off + r0.t0 + r0.nt);
+                if (fo && fo->valid) {
+                    lo0 = fo->lo[fo_index];
+                    hi0 = fo->hi[fo_index];
+                } else {
+                    lo0 = __ldg(pr.tile_off + r0.t0);
+                    hi0 = __ldg(pr.tile_off + r0.t0 + r0.nt);
+                }
             }
             if (wk.count > 1) {
                 it2.next(pl, wk);
@@ -1179,10 +1193,11 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 }
 
 template <int FMT, int NB>
-__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl) {
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl,
+                                                                        const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
     run_problem<FMT, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
-                         static_cast<int>(blockIdx.x));
+                         static_cast<int>(blockIdx.x), true, &fo, static_cast<int>(blockIdx.x));
 }
 
 // Several independent BITCOS problems in one launch: the grid is cut into one range of thread
@@ -1196,14 +1211,15 @@ struct MultiArgs {
 };
 
 template <int NB>
-__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma) {
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma,
+                                                                              const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b = static_cast<int>(blockIdx.x);
     int j = 0;
     while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
     run_problem<kBitcos, NB>(ma.pr[j], ma.pl[j], smem,
                              make_walk(ma.pl[j], b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
-                             b - ma.first_block[j]);
+                             b - ma.first_block[j], true, &fo, b);
 }
 
 // Fills in what differs between the groups of a grouped product; false if the group is empty or
@@ -1441,8 +1457,27 @@ int launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cu
     return check_cuda(cudaLaunchKernelEx(&cfg, kernel, args...));
 }
 
+// Fills fo.lo / fo.hi [base .. base + grid) from a host copy of tile_off: the sign-vector range of
+// the first item of each of the `grid` thread blocks that share the problem.
+void fill_first_off(FirstOff &fo, int base, const uint32_t *off_host, const Problem &pr, const Plan &pl, int grid) {
+    if (!off_host || base + grid > kMaxGrid) {
+        fo.valid = 0;
+        return;
+    }
+    for (int b = 0; b < grid; ++b) {
+        const Walk wk = make_walk(pl, b, grid);
+        fo.lo[base + b] = fo.hi[base + b] = 0;
+        if (wk.count <= 0) continue;
+        ItemIter it;
+        it.init(pl, wk.first);
+        const ItemRange r = item_range(pr, pl, it.c, it.cs);
+        fo.lo[base + b] = off_host[r.t0];
+        fo.hi[base + b] = off_host[r.t0 + r.nt];
+    }
+}
+
 template <int FMT, int NB>
-int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
+int launch(const Problem &pr, const Plan &pl, cudaStream_t stream, const uint32_t *off_host = nullptr) {
     int sms = 0, budget = 0;
     int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms, &budget);
     if (rc) return rc;
@@ -1453,11 +1488,14 @@ int launch(const Problem &pr, const Plan &pl, cudaStream_t stream) {
     static const char *probe = std::getenv("BITCOS_PROBE");
     plw.probe = (probe && probe[0] == 'c') ? 1 : (probe && probe[0] == 'd') ? 2 : 0;
     const SmemLayout L = smem_layout(FMT, plw, pr.G, NB, pr.K);
-    return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw);
+    FirstOff fo;
+    fo.valid = (FMT == kBitcos && off_host) ? 1 : 0;
+    if (fo.valid) fill_first_off(fo, 0, off_host, pr, plw, grid);
+    return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
 template <int NB>
-int launch_multi(MultiArgs &ma, cudaStream_t stream) {
+int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_host) {
     int sms = 0, budget = 0;
     int rc = prepare_kernel<gemv_multi_kernel<NB>>(&sms, &budget);
     if (rc) return rc;
@@ -1468,6 +1506,9 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream) {
     uint32_t smem = 0;
     int next = 0;
     static const char *probe = std::getenv("BITCOS_PROBE");
+    FirstOff fo;
+    fo.valid = 1;
+    for (int j = 0; j < ma.n; ++j) fo.valid = (fo.valid && off_host[j]) ? 1 : 0;
     for (int j = 0; j < ma.n; ++j) {
         int64_t cap = ma.pl[j].items;
         if (total_items > sms) {
@@ -1482,10 +1523,11 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream) {
         if (L.total > smem) smem = L.total;
         if (ma.pl[j].NW > nw) nw = ma.pl[j].NW;
         ma.first_block[j] = next;
+        if (fo.valid) fill_first_off(fo, next, off_host[j], ma.pr[j], ma.pl[j], grid);
         next += grid;
     }
     ma.first_block[ma.n] = next;
-    return launch_pdl(gemv_multi_kernel<NB>, dim3(next), (nw + 2) * 32, smem, stream, ma);
+    return launch_pdl(gemv_multi_kernel<NB>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
 }
 
 // Which instantiation serves a batch: 1, 2, 4, 8 or 16 tokens.  The one- and two-token paths read
@@ -1497,13 +1539,13 @@ inline int nb_bucket(int batch, int64_t K) {
 }
 
 template <int FMT>
-int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream) {
+int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream, const uint32_t *off_host) {
     const int nbk = nb_bucket(pr.nb, pr.K);
-    if (nbk == 1) return launch<FMT, 1>(pr, pl, stream);
-    if (nbk == 2) return launch<FMT, 2>(pr, pl, stream);
-    if (pr.nb <= 4) return launch<FMT, 4>(pr, pl, stream);
-    if (pr.nb <= 8) return launch<FMT, 8>(pr, pl, stream);
-    return launch<FMT, 16>(pr, pl, stream);
+    if (nbk == 1) return launch<FMT, 1>(pr, pl, stream, off_host);
+    if (nbk == 2) return launch<FMT, 2>(pr, pl, stream, off_host);
+    if (pr.nb <= 4) return launch<FMT, 4>(pr, pl, stream, off_host);
+    if (pr.nb <= 8) return launch<FMT, 8>(pr, pl, stream, off_host);
+    return launch<FMT, 16>(pr, pl, stream, off_host);
 }
 
 template <int NB>
@@ -1574,7 +1616,8 @@ void fill_problem(Problem &pr, const uint32_t *payload, const uint32_t *signs, c
 
 int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const uint32_t *tile_off,
                 const uint16_t *scales, int64_t M, int64_t K, const int8_t *x, const float *x_scale, int batch,
-                float *y, int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+                float *y, int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream,
+                const uint32_t *off_host = nullptr) {
     const int bad = check_common(fmt, payload, signs, tile_off, scales, M, K, x, x_scale, batch, y, acc_debug, workspace,
                                  workspace_bytes);
     if (bad) return bad;
@@ -1582,9 +1625,9 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
     Problem pr{};
     fill_problem(pr, payload, signs, tile_off, scales, M, K, x, x_scale, batch, y, acc_debug, workspace);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (fmt == kBitcos) return launch_nb<kBitcos>(pr, pl, stream);
-    if (fmt == kTrit5) return launch_nb<kTrit5>(pr, pl, stream);
-    return launch_nb<kBit2>(pr, pl, stream);
+    if (fmt == kBitcos) return launch_nb<kBitcos>(pr, pl, stream, off_host);
+    if (fmt == kTrit5) return launch_nb<kTrit5>(pr, pl, stream, nullptr);
+    return launch_nb<kBit2>(pr, pl, stream, nullptr);
 }
 
 }  // namespace
@@ -1645,7 +1688,7 @@ int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, 
                 int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     if (!W) return BITCOS_ERR_NULL;
     return gemv_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_scale, batch, y,
-                       acc_debug, workspace, workspace_bytes, cuda_stream);
+                       acc_debug, workspace, workspace_bytes, cuda_stream, W->tile_off_host);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1699,7 +1742,7 @@ int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_
     rc = check_cuda(cudaMemsetAsync(ws, 0, head, static_cast<cudaStream_t>(cuda_stream)));
     if (rc) return rc;
     return gemv_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_scale, batch, y,
-                       nullptr, ws, BITCOS_STATIC_WORKSPACE_BYTES, cuda_stream);
+                       nullptr, ws, BITCOS_STATIC_WORKSPACE_BYTES, cuda_stream, W->tile_off_host);
 }
 
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
@@ -1723,11 +1766,13 @@ int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
     int64_t kmax = 0;
     for (int j = 0; j < n_jobs; ++j) kmax = jobs[j].W->K > kmax ? jobs[j].W->K : kmax;
     const int nbk = nb_bucket(batch, kmax);
-    if (nbk == 1) return launch_multi<1>(ma, stream);
-    if (nbk == 2) return launch_multi<2>(ma, stream);
-    if (batch <= 4) return launch_multi<4>(ma, stream);
-    if (batch <= 8) return launch_multi<8>(ma, stream);
-    return launch_multi<16>(ma, stream);
+    const uint32_t *off_host[kMaxJobs];
+    for (int j = 0; j < n_jobs; ++j) off_host[j] = jobs[j].W->tile_off_host;
+    if (nbk == 1) return launch_multi<1>(ma, stream, off_host);
+    if (nbk == 2) return launch_multi<2>(ma, stream, off_host);
+    if (batch <= 4) return launch_multi<4>(ma, stream, off_host);
+    if (batch <= 8) return launch_multi<8>(ma, stream, off_host);
+    return launch_multi<16>(ma, stream, off_host);
 }
 
 size_t bitcos_gemv_host_staging_bytes(int64_t M, int64_t K, int batch) {

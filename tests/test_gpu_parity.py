@@ -184,6 +184,31 @@ def test_multi_launch_matches_separate_products(bc, B):
         assert torch.equal(y1, y)
 
 
+def test_host_copy_of_entry_offsets_changes_nothing(bc):
+    """With a host copy of tile_off the launch passes each block's first entry offsets by value;
+    without it the kernel loads them.  Same results, bit for bit, and both match the oracle."""
+    for (M, K, B) in ((2560, 2560, 1), (640, 6912, 1), (6912, 2560, 3), (96, 25600, 1)):
+        W, S = datagen.trits(700 + M, M, K, 0.4219), datagen.scales(700 + M, M, K)
+        x, xs = datagen.activations(700 + K, B, K)
+        acc_ref, y_ref, mag = oracle.gemv_dense(W, S, x, xs)
+        Wd = bc.bitcos_pack(W, S).to_device()
+        assert Wd.tile_off_host is not None
+        Wn = Wd.without_host_offsets()
+        xd, xsd = dev(x), dev(xs)
+        ws = bc.make_workspace(M, K)
+        y1, acc1 = bc.bitcos_gemv(Wd, xd, xsd, acc_debug=True, workspace=ws)
+        check(y1, acc1, acc_ref, y_ref, mag, f"host offsets {M}x{K}")
+        y2, acc2 = bc.bitcos_gemv(Wn, xd, xsd, acc_debug=True, workspace=ws)
+        check(y2, acc2, acc_ref, y_ref, mag, f"device offsets {M}x{K}")
+        assert torch.equal(y1, y2)
+        # one job with, one without: the launch falls back to loading them
+        ya = torch.empty_like(y1)
+        yb = torch.empty_like(y1)
+        bc.bitcos_gemv_multi([(Wd, xd, xsd, ya, ws), (Wn, xd, xsd, yb, bc.make_workspace(M, K))])
+        torch.cuda.synchronize()
+        assert torch.equal(ya, y1) and torch.equal(yb, y1)
+
+
 def test_host_buffer_entry_point(bc):
     M, K, B = 640, 2560, 4
     W, S = datagen.trits(21, M, K, 0.4219), datagen.scales(21, M, K)
