@@ -755,7 +755,9 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         bool ok = true;
         auto offsets = [&](const ItemRange &prev, uint32_t prev_hi, const ItemRange &r, uint32_t &lo, uint32_t &hi) {
             if (FMT != kBitcos) return;
-            lo = (r.t0 == prev.t0 + prev.nt) ? prev_hi : __ldg(pr.tile_off + r.t0);
+            // two independent loads (no reuse of the previous item's upper offset: that would make
+            // every request wait for the one before it)
+            lo = __ldg(pr.tile_off + r.t0);
             hi = __ldg(pr.tile_off + r.t0 + r.nt);
         };
         auto issue_loop = [&](int k_end) {
