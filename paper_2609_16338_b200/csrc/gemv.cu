@@ -7,19 +7,23 @@
 // group of one row block (32 x 128 weights); one warp decodes one tile at a time.  An
 // "item" is a run of up to 20 consecutive tiles -- CG groups of one row block, or several
 // whole row blocks when a row has few groups -- and is what one thread block processes per
-// pipeline stage: because tiles are stored in that order, an item's bitmap words, sign bits
-// and scales are three contiguous byte ranges, fetched with three bulk asynchronous copies
-// (cp.async.bulk + mbarrier) into a ring of shared-memory stages while earlier stages are
-// being decoded.  Thread blocks are persistent and walk the item list with a fixed stride.
-// Row sums are formed in a fixed order (groups ascending inside a block through shared
-// memory; column blocks ascending through a scratch buffer and an arrival counter), so
-// results do not depend on scheduling.
+// pipeline stage: because tiles are stored in that order, an item's bitmap words, sign bits,
+// scales and entry offsets are four contiguous byte ranges, fetched with four bulk asynchronous
+// copies (cp.async.bulk + mbarrier) into a ring of shared-memory stages while earlier stages are
+// being decoded.  Thread blocks are persistent and take either a contiguous range of the item
+// list or every n-th row-block chunk.  Row sums are formed in a fixed order (a fixed tree over the
+// groups inside a block through shared memory; column blocks ascending through a scratch buffer
+// and an arrival counter), so results do not depend on scheduling.
+//
+// Contraction.  One or two tokens: dp4a against activations kept in shared memory.  Four tokens
+// and more: the decoded rows pass through a small shared-memory buffer to ldmatrix and
+// mma.m16n8k32 (int8 in, int32 out), so that the decode is paid once per call whatever the batch.
 //
 // BITCOS decode (paper Section II-D, Eq. 4, adapted): the GPU has no bit-deposit
 // instruction, so four weights at a time are rebuilt from a (presence nibble, next four
 // sign bits) key through a 256-entry table held in shared memory, replicated once per lane
 // so that lookups never conflict.  Entries are the four weights as int8 (w = p - 2n, Eq. 2)
-// and feed dp4a directly.  A lane's position in the sign vector is the tile's entry offset
+// ready for dp4a or the tensor cores.  A lane's position in the sign vector is the tile's entry offset
 // plus a warp prefix sum over the rows' population counts; the four 32-bit presence words of
 // a lane's row are decoded as four independent chains, each shifting its own sign window by
 // the number of sign bits a nibble consumed.
@@ -382,15 +386,14 @@ __device__ __forceinline__ void sts128(uint32_t addr, int a, int b, int c, int d
 }
 
 // ---------------------------------------------------------------------------------------------
-// Tile decoders.  For the lane's row they produce either the int32 accumulator against one
-// token (FUSED: decode fused with dp4a) or the 32 int8x4 words of the row.
+// Tile decoders.  For the lane's row they produce the 32 int8x4 words of the row; the contraction
+// follows as a separate step (dp4a per token, or the tensor cores from four tokens on).
 // ---------------------------------------------------------------------------------------------
 
 // BITCOS: bm = the row's four presence words, sp = the stage's sign words at the word holding the
-// row's first sign bit, sh = bit offset inside that word.
-template <bool FUSED>
-__device__ __forceinline__ int bitcos_decode_row(const uint4 bm, const uint32_t *sp, uint32_t sh, const uint8_t *lut,
-                                                 uint32_t lane4, const int4 *xg, int (&w)[32]) {
+// row's first sign bit, sh = bit offset inside that word.  w receives the row's 32 int8x4 words.
+__device__ __forceinline__ void bitcos_decode_row(const uint4 bm, const uint32_t *sp, uint32_t sh, const uint8_t *lut,
+                                                  uint32_t lane4, int (&w)[32]) {
     const int c0 = __popc(bm.x), c1 = __popc(bm.y), c2 = __popc(bm.z);
     const uint32_t s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3], s4 = sp[4];
     uint32_t a0 = __funnelshift_r(s0, s1, sh), a1 = __funnelshift_r(s1, s2, sh);
@@ -406,32 +409,22 @@ __device__ __forceinline__ int bitcos_decode_row(const uint4 bm, const uint32_t 
     S[2] = a0;
     S[3] = __funnelshift_rc(a0, a1, c2);
     const uint32_t P[4] = {bm.x, bm.y, bm.z, bm.w};
-    int acc[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        int4 xq[4];
-        if (FUSED) {
-            // activation words 8j + 2k and 8j + 2k + 1 for the four chains j
-#pragma unroll
-            for (int j = 0; j < 4; ++j) xq[j] = xg[2 * j + (k >> 1)];
-        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             // address bits 0..6 = lane * 4, bits 8..15 = presence byte k of word j (bits 16.. are 0)
             const uint32_t R = __byte_perm(P[j], lane4, 0x6504 | (k << 4));
             uint32_t off = bit_select(S[j] << 12, R, 0xF000u);     // sign nibble over the odd presence nibble
             int e = static_cast<int>(lds32(lut, off));
-            if (FUSED) acc[j] = __dp4a(e, (k & 1) ? xq[j].z : xq[j].x, acc[j]);
-            else w[8 * j + 2 * k] = e;
+            w[8 * j + 2 * k] = e;
             S[j] >>= __dp4a(e, e, 0);                    // non-zeros in the nibble = sign bits consumed
             off = bit_select(S[j] << 8, R, 0x0F00u);               // sign nibble over the even presence nibble
             e = static_cast<int>(lds32(lut + 128, off));
-            if (FUSED) acc[j] = __dp4a(e, (k & 1) ? xq[j].w : xq[j].y, acc[j]);
-            else w[8 * j + 2 * k + 1] = e;
+            w[8 * j + 2 * k + 1] = e;
             S[j] >>= __dp4a(e, e, 0);
         }
     }
-    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
 }
 
 // Five-trit: wd = the seven words that hold the row's 26 bytes, odd = byte offset 2 (odd group).
@@ -1075,7 +1068,6 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             // activations of group g (one or two tokens: always in shared memory)
             const uint8_t *xs = xs_base + static_cast<uint32_t>(g) * kGroup;
             int w[32];
-            int acc1 = 0;
             if (FMT == kBitcos) {
                 const uint4 bm = *reinterpret_cast<const uint4 *>(stage + off_bm);
                 const int c = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
@@ -1089,10 +1081,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 const uint32_t toff = *reinterpret_cast<const uint32_t *>(stage + off_toff + ((d.x >> 8) << 2));
                 const uint32_t cursor = toff + static_cast<uint32_t>(incl - c) - d.w;
                 const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + off_sign + ((cursor >> 5) << 2));
-                if (NB == 1)
-                    acc1 = bitcos_decode_row<true>(bm, sp, cursor & 31u, lut, lane4, reinterpret_cast<const int4 *>(xs), w);
-                else
-                    bitcos_decode_row<false>(bm, sp, cursor & 31u, lut, lane4, nullptr, w);
+                bitcos_decode_row(bm, sp, cursor & 31u, lut, lane4, w);
             } else if (FMT == kTrit5) {
                 const int WPR = (26 * pr.G + 3) / 4;
                 // words of the stage: row block my_rbl of the chunk, counted from the chunk's first word
@@ -1152,16 +1141,12 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             // decode first, contract afterwards: keeps the table lookups of the decode back to back
             // (interleaving them with the contraction's activation loads measured 20 % slower on the
             // five-trit path)
-            if (!kMma && !(FMT == kBitcos && NB == 1)) asm volatile("" ::: "memory");
+            if (!kMma) asm volatile("" ::: "memory");
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 if (kMma) break;
                 if (b < pr.nb) {
-                    int a;
-                    if (FMT == kBitcos && NB == 1)
-                        a = acc1;
-                    else
-                        a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pr.K), lane);
+                    const int a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pr.K), lane);
                     ysum[b] = sc * static_cast<float>(a);
                     if (pr.acc_debug) {
                         const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + lane;
@@ -1357,7 +1342,9 @@ __global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) decode_probe_kernel(i
             }
             const uint32_t cursor = static_cast<uint32_t>(incl - c) + static_cast<uint32_t>(it & 1);
             const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + 1024) + (cursor >> 5);
-            a = bitcos_decode_row<true>(bm, sp, cursor & 31u, lut, lane4, reinterpret_cast<const int4 *>(xs), w);
+            bitcos_decode_row(bm, sp, cursor & 31u, lut, lane4, w);
+            asm volatile("" ::: "memory");
+            a = contract<kBitcos>(w, reinterpret_cast<const int4 *>(xs), lane);
         } else if (FMT == kTrit5) {
             const uint32_t *src = reinterpret_cast<const uint32_t *>(stage) + lane;
             uint32_t wd[7];
