@@ -39,7 +39,7 @@ namespace {
 constexpr int kGroup = BITCOS_GROUP;
 constexpr int kRows = BITCOS_TILE_ROWS;
 constexpr int kMaxWarps = 20;             // warps per thread block = tiles per item
-constexpr int kWarps16 = 16;              // the same for more than 8 tokens (their partial sums need the room)
+constexpr int kWarps16 = 14;              // the same for more than 8 tokens (their partial sums need the room)
 constexpr int kMaxStages = 8;             // upper bound on the shared-memory ring depth (Plan::stages)
 constexpr int kLutBytes = 64 * 1024;      // replicated lookup tables (BITCOS, five-trit)
 constexpr uint64_t kWaitLimitNs = 500ull * 1000 * 1000;   // an mbarrier wait gives up after half a second
@@ -145,7 +145,7 @@ struct Plan {
     int64_t items;   // ceil(RB / RBC) * CS
     int cyclic;      // 1: blocks take whole row-block chunks round robin; 0: contiguous balanced ranges
     int stages;      // depth of the shared-memory ring (2 .. kMaxStages), set at launch
-    int probe;       // measurement aid (BITCOS_PROBE=copy): stream the weights but skip the decode
+    int x_in_stage;  // 1: every stage also receives the item's activation rows (grouped launch, 1-2 tokens)
 };
 
 struct Problem {
@@ -230,7 +230,7 @@ struct SmemLayout {
     uint32_t lut;        // lookup tables (0 bytes for 2-bit)
     uint32_t stage;      // stage 0
     uint32_t stage_bytes;
-    uint32_t payload_cap, sign_cap, scale_cap, off_cap;   // per-stage capacities
+    uint32_t payload_cap, sign_cap, scale_cap, off_cap, x_cap;   // per-stage capacities
     uint32_t x;          // activations, [nb][K], if x_bytes != 0
     uint32_t x_bytes;    // 0: the activations do not fit and are read from global memory
     uint32_t red;        // 2 x [NW][NB][32] floats
@@ -276,12 +276,14 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
         L.sign_cap = 0;
     }
     L.scale_cap = tiles * 64;
+    L.off_cap = align_up(L.off_cap, 16);
+    L.x_cap = pl.x_in_stage ? static_cast<uint32_t>(nbmax * K) : 0u;
     L.stage = off;
-    L.stage_bytes = align_up(L.payload_cap + L.sign_cap + L.scale_cap + L.off_cap, 128);
+    L.stage_bytes = align_up(L.payload_cap + L.sign_cap + L.scale_cap + L.off_cap + L.x_cap, 128);
     off += L.stage_bytes * static_cast<uint32_t>(pl.stages);
     L.x = off;
     // (the tensor-core path takes its activation fragments straight from global memory)
-    L.x_bytes = (nbmax < kMmaMinBatch && static_cast<int64_t>(nbmax) * K <= kXResidentBytes)
+    L.x_bytes = (nbmax < kMmaMinBatch && !pl.x_in_stage && static_cast<int64_t>(nbmax) * K <= kXResidentBytes)
                     ? static_cast<uint32_t>(nbmax * K) : 0u;
     off += align_up(L.x_bytes, 128);
     L.red = off;
@@ -586,19 +588,50 @@ struct ItemIter {
     }
 };
 
+// What differs between the segments of one launch (everything else -- shape, activations,
+// outputs -- is read from the launch's one Problem), behind accessors: the plain kernels read the
+// values from the kernel parameters every time (no registers spent on them), the grouped launch
+// holds the current group's values.
+struct ParamView {
+    __device__ __forceinline__ const uint32_t *payload(const Problem &p) const { return p.payload; }
+    __device__ __forceinline__ const uint32_t *signs(const Problem &p) const { return p.signs; }
+    __device__ __forceinline__ const uint32_t *tile_off(const Problem &p) const { return p.tile_off; }
+    __device__ __forceinline__ const uint16_t *scales(const Problem &p) const { return p.scales; }
+    __device__ __forceinline__ const int32_t *xrow(const Problem &p) const { return p.xrow; }       // NULL: token b reads row b
+    __device__ __forceinline__ unsigned int *status(const Problem &p) const { return p.status; }
+    __device__ __forceinline__ int64_t out_row0(const Problem &p) const { return p.out_row0; }      // first output row of token 0
+    __device__ __forceinline__ int nb(const Problem &p) const { return p.nb; }                      // tokens of the segment
+};
+struct GroupView {
+    const uint32_t *payload_, *signs_, *tile_off_;
+    const uint16_t *scales_;
+    const int32_t *xrow_;
+    unsigned int *status_;
+    int begin_, nb_;
+    __device__ __forceinline__ const uint32_t *payload(const Problem &) const { return payload_; }
+    __device__ __forceinline__ const uint32_t *signs(const Problem &) const { return signs_; }
+    __device__ __forceinline__ const uint32_t *tile_off(const Problem &) const { return tile_off_; }
+    __device__ __forceinline__ const uint16_t *scales(const Problem &) const { return scales_; }
+    __device__ __forceinline__ const int32_t *xrow(const Problem &) const { return xrow_; }
+    __device__ __forceinline__ unsigned int *status(const Problem &) const { return status_; }
+    __device__ __forceinline__ int64_t out_row0(const Problem &) const { return begin_; }
+    __device__ __forceinline__ int nb(const Problem &) const { return nb_; }
+};
+
 // Issues the bulk copies of one item into stage `s` (one thread) and publishes the item's
 // descriptor (sign_base[4s .. 4s+3]; word 3 = index of the first sign bit held in the stage).  o_lo / o_hi: sign-vector
 // positions of the item's first tile and of the tile after its last (BITCOS only).
-template <int FMT>
-__device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, const ItemRange &r, const SmemLayout &L,
-                                           uint8_t *smem, int s, uint32_t *sign_base, uint32_t o_lo, uint32_t o_hi) {
+template <int FMT, typename View>
+__device__ __forceinline__ void issue_item(const Problem &pb, const View &pr, const Plan &pl, const ItemRange &r,
+                                           const SmemLayout &L, uint8_t *smem, int s, uint32_t *sign_base, uint32_t o_lo,
+                                           uint32_t o_hi, const int (&xrows)[2]) {
     uint8_t *stage = smem + L.stage + static_cast<uint32_t>(s) * L.stage_bytes;
     const uint32_t bar = smem_addr(smem + L.bar) + 8u * static_cast<uint32_t>(s);
     const uint32_t d_payload = smem_addr(stage);
     const uint32_t d_signs = d_payload + L.payload_cap;
     const uint32_t d_scales = d_signs + L.sign_cap;
     const uint32_t scale_bytes = static_cast<uint32_t>(r.nt) * 64u;
-    const uint8_t *g_scales = reinterpret_cast<const uint8_t *>(pr.scales) + r.t0 * 64;
+    const uint8_t *g_scales = reinterpret_cast<const uint8_t *>(pr.scales(pb)) + r.t0 * 64;
     // what the decoder warps need to know about the item (read by them once the stage is full)
     sign_base[s * 4 + 0] = static_cast<uint32_t>(r.nt) | (static_cast<uint32_t>(r.t0 & 3) << 8);
     sign_base[s * 4 + 1] = static_cast<uint32_t>(r.g0);
@@ -611,25 +644,33 @@ __device__ __forceinline__ void issue_item(const Problem &pr, const Plan &pl, co
         // the tiles' entry offsets: the 16-byte aligned slice of tile_off that covers t0 .. t0 + nt
         const uint32_t o_first = static_cast<uint32_t>(r.t0 & 3);
         const uint32_t off_bytes = ((o_first + static_cast<uint32_t>(r.nt) + 1u + 3u) & ~3u) * 4u;
-        mbar_expect_tx(bar, bm_bytes + sign_bytes + scale_bytes + off_bytes);
-        bulk_copy(d_scales + L.scale_cap, pr.tile_off + (r.t0 - o_first), off_bytes, bar);
-        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + r.t0 * 512, bm_bytes, bar);
-        if (sign_bytes) bulk_copy(d_signs, reinterpret_cast<const uint8_t *>(pr.signs) + b_lo, sign_bytes, bar);
+        const uint32_t x_bytes = pl.x_in_stage ? static_cast<uint32_t>(pr.nb(pb)) * static_cast<uint32_t>(pb.K) : 0u;
+        mbar_expect_tx(bar, bm_bytes + sign_bytes + scale_bytes + off_bytes + x_bytes);
+        if (pl.x_in_stage) {
+            // the activation rows of this group's tokens (from L2): the decoders of a grouped launch
+            // find them next to the weights and need no block-wide staging step per group
+            for (int b = 0; b < pr.nb(pb) && b < 2; ++b)
+                bulk_copy(d_scales + L.scale_cap + L.off_cap + static_cast<uint32_t>(b) * static_cast<uint32_t>(pb.K),
+                          pb.x + static_cast<int64_t>(xrows[b]) * pb.K, static_cast<uint32_t>(pb.K), bar);
+        }
+        bulk_copy(d_scales + L.scale_cap, pr.tile_off(pb) + (r.t0 - o_first), off_bytes, bar);
+        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload(pb)) + r.t0 * 512, bm_bytes, bar);
+        if (sign_bytes) bulk_copy(d_signs, reinterpret_cast<const uint8_t *>(pr.signs(pb)) + b_lo, sign_bytes, bar);
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
     } else if (FMT == kTrit5) {
-        const int64_t WPR = (26 * static_cast<int64_t>(pr.G) + 3) / 4;
+        const int64_t WPR = (26 * static_cast<int64_t>(pb.G) + 3) / 4;
         const int64_t w_lo = r.rb0 * WPR + ((26 * r.g0) >> 2);
         int64_t w_hi;   // exclusive
-        if (pl.CS == 1) w_hi = (r.rb0 + r.nt / pr.G) * WPR;
+        if (pl.CS == 1) w_hi = (r.rb0 + r.nt / pb.G) * WPR;
         else w_hi = r.rb0 * WPR + ((26 * (r.g0 + r.nt) - 1) >> 2) + 1;
         const uint32_t bytes = static_cast<uint32_t>(w_hi - w_lo) * 128u;
         mbar_expect_tx(bar, bytes + scale_bytes);
-        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + w_lo * 128, bytes, bar);
+        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload(pb)) + w_lo * 128, bytes, bar);
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
     } else {
         const uint32_t bytes = static_cast<uint32_t>(r.nt) * 1024u;
         mbar_expect_tx(bar, bytes + scale_bytes);
-        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload) + r.t0 * 1024, bytes, bar);
+        bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload(pb)) + r.t0 * 1024, bytes, bar);
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
     }
 }
@@ -641,9 +682,6 @@ constexpr int kBarRedFull = 2 * kMaxStages;       // [slots] partial sums of an 
 constexpr int kBarRedEmpty = 2 * kMaxStages + 8;  // [slots] partial sums consumed by the epilogue warp
 constexpr int kBarLut = 2 * kMaxStages + 16;      // lookup table arrived
 
-__device__ __forceinline__ void mbar_inval(uint32_t bar) {
-    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-}
 // Arrival by lane 0 only, as one predicated instruction (no divergent branch around it).
 __device__ __forceinline__ void mbar_arrive_lane0(uint32_t bar, int lane) {
     asm volatile(
@@ -684,19 +722,39 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
     if (lane == 0) pr.counters[sh.rb] = 0u;    // leave the counter ready for the next call
 }
 
+// What a thread block runs back to back: one problem and its share of the items (the plain
+// kernels), or the pieces of several groups (the grouped launch).  Every warp role walks its own
+// copy of the source.
+struct OneSeg {
+    typedef ParamView View;
+    static constexpr bool kSingle = true;      // never more than one segment
+    const Problem *pr;
+    Walk wk;
+    bool used;
+    __device__ __forceinline__ const Problem &shape() const { return *pr; }
+    __device__ __forceinline__ bool next(View &v, Walk &w) {
+        if (used) return false;
+        used = true;
+        (void)v;
+        w = wk;
+        return true;
+    }
+};
+
 // Warp roles: warps 0 .. NW-1 decode one tile per item each; warp NW feeds the stage ring with
 // bulk copies; warp NW+1 adds the decoders' partial sums in a fixed order and writes the
 // outputs (and runs the cross-block protocol).  The roles meet only through mbarriers, every
 // wait is bounded, and there is no block-wide barrier inside the loop.
-// `wk` is this block's share of the problem's items.  `fresh` is false when the block has already
-// run another problem with the same shared-memory layout: the lookup table is still in place and
-// the barriers are invalidated before they are set up again (the caller puts a block-wide barrier
-// between two runs).
-template <int FMT, int NB>
-__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
-                                            bool fresh = true, const FirstOff *fo = nullptr, int fo_index = 0) {
+// `segs` yields the problems this block works on, one after the other, with its share of each
+// one's items; the stage ring, the partial-sum slots and their barriers run on across them.
+template <int FMT, int NB, typename Segs>
+__device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, uint8_t *smem, int block,
+                                             const FirstOff *fo = nullptr, int fo_index = 0) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const SmemLayout L = smem_layout(FMT, pl, pr.G, NB, pr.K);
+    const SmemLayout L = smem_layout(FMT, pl, segs.shape().G, NB, segs.shape().K);
+    const Problem &pb = segs.shape();
+    typename Segs::View pr{};
+    Walk wk{};
     const uint8_t *lut = smem + L.lut;
     float *red = reinterpret_cast<float *>(smem + L.red);
     // per stage: {tiles | (first tile & 3) << 8, first group, first row block, first sign bit held}
@@ -721,17 +779,6 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     // happens in the block.
     if (warp == pl.NW) {
         if (lane == 0) {
-            if (!fresh) {
-                for (int s = 0; s < pl.stages; ++s) {
-                    mbar_inval(bar0 + 8u * (kBarFull + s));
-                    mbar_inval(bar0 + 8u * (kBarEmpty + s));
-                }
-                for (int s = 0; s < red_slots(NB); ++s) {
-                    mbar_inval(bar0 + 8u * (kBarRedFull + s));
-                    mbar_inval(bar0 + 8u * (kBarRedEmpty + s));
-                }
-                mbar_inval(bar0 + 8u * kBarLut);
-            }
             for (int s = 0; s < pl.stages; ++s) {
                 mbar_init(bar0 + 8u * (kBarFull + s), 1);
                 mbar_init(bar0 + 8u * (kBarEmpty + s), pl.NW);
@@ -748,38 +795,41 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         // still fetching the activations.
         // Entry offsets are requested two items before they are needed (r0 = item k, r1 = item
         // k + 1, r2 = item k + 2), so that the load is never waited for.
+        Segs src = segs;
         ItemIter it2;
         ItemRange r0{}, r1{}, r2{};
         uint32_t lo0 = 0, hi0 = 0, lo1 = 0, hi1 = 0;
         int k0 = 0, ps = 0;
+        int kk = 0;                // items issued so far, over all segments
+        int xrows[2] = {0, 0};     // activation rows of the segment's tokens (when they travel with the stage)
         uint32_t pphase = 1;       // parity of the phase before the one the decoders complete next
         bool ok = true;
-        auto offsets = [&](const ItemRange &prev, uint32_t prev_hi, const ItemRange &r, uint32_t &lo, uint32_t &hi) {
+        auto offsets = [&](const ItemRange &r, uint32_t &lo, uint32_t &hi) {
             if (FMT != kBitcos) return;
             // two independent loads (no reuse of the previous item's upper offset: that would make
             // every request wait for the one before it)
-            lo = __ldg(pr.tile_off + r.t0);
-            hi = __ldg(pr.tile_off + r.t0 + r.nt);
+            lo = __ldg(pr.tile_off(pb) + r.t0);
+            hi = __ldg(pr.tile_off(pb) + r.t0 + r.nt);
         };
         auto issue_loop = [&](int k_end) {
-            for (int k = k0; k < k_end; ++k) {
+            for (int k = k0; k < k_end; ++k, ++kk) {
                 const int s = ps;
                 uint32_t lo2 = 0, hi2 = 0;
                 if (k + 2 < wk.count) {
                     it2.next(pl, wk);
-                    r2 = item_range(pr, pl, it2.c, it2.cs);
-                    offsets(r1, hi1, r2, lo2, hi2);
+                    r2 = item_range(pb, pl, it2.c, it2.cs);
+                    offsets(r2, lo2, hi2);
                 }
-                if (k >= pl.stages) {
+                if (kk >= pl.stages) {
                     if (!mbar_wait(bar0 + 8u * (kBarEmpty + s), pphase)) {
-                        if (pr.status) *pr.status = 1u;
+                        if (pr.status(pb)) *pr.status(pb) = 1u;
                         ok = false;
                         return;
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
-                issue_item<FMT>(pr, pl, r0, L, smem, s, sign_base, lo0, hi0);
-                if (k == 0 && FMT != kBit2 && fresh) {
+                issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows);
+                if (kk == 0 && FMT != kBit2) {
                     mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
                     bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
                               bar0 + 8u * kBarLut);
@@ -793,27 +843,44 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             }
             k0 = k_end;
         };
-        if (lane == 0 && wk.count > 0) {
+        // first item(s) of a segment: ranges and entry offsets of items 0 and 1
+        auto prime = [&](bool first_segment) {
+            k0 = 0;
             it2.init(pl, wk.first);
-            r0 = item_range(pr, pl, it2.c, it2.cs);
+            r0 = item_range(pb, pl, it2.c, it2.cs);
             if (FMT == kBitcos) {
-                if (fo && fo->valid) {
+                if (first_segment && fo && fo->valid) {
                     lo0 = fo->lo[fo_index];
                     hi0 = fo->hi[fo_index];
                 } else {
-                    lo0 = __ldg(pr.tile_off + r0.t0);
-                    hi0 = __ldg(pr.tile_off + r0.t0 + r0.nt);
+                    lo0 = __ldg(pr.tile_off(pb) + r0.t0);
+                    hi0 = __ldg(pr.tile_off(pb) + r0.t0 + r0.nt);
                 }
             }
             if (wk.count > 1) {
                 it2.next(pl, wk);
-                r1 = item_range(pr, pl, it2.c, it2.cs);
-                offsets(r0, hi0, r1, lo1, hi1);
+                r1 = item_range(pb, pl, it2.c, it2.cs);
+                offsets(r1, lo1, hi1);
             }
+            if (pl.x_in_stage) {
+                xrows[0] = pr.xrow(pb) ? __ldg(pr.xrow(pb)) : 0;
+                xrows[1] = pr.nb(pb) > 1 ? (pr.xrow(pb) ? __ldg(pr.xrow(pb) + 1) : 1) : 0;
+            }
+        };
+        bool have = src.next(pr, wk);
+        while (have && wk.count <= 0) have = src.next(pr, wk);
+        if (lane == 0 && have) {
+            prime(true);
             issue_loop(wk.count < pl.stages ? wk.count : pl.stages);
         }
         __syncthreads();       // pairs with the barrier the other warps reach after staging the activations
-        if (lane == 0 && ok) issue_loop(wk.count);
+        if (lane != 0 || !have) return;
+        if (ok) issue_loop(wk.count);
+        while (!Segs::kSingle && ok && src.next(pr, wk)) {
+            if (wk.count <= 0) continue;
+            prime(false);
+            issue_loop(wk.count);
+        }
         return;
     }
 
@@ -821,44 +888,58 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     // workspace); the packed weights the producer streams do not.
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // activations: kept whole in shared memory ([nb][K]) when they fit, staged by the other
-    // warps while the producer starts the copies; otherwise read from global memory per tile
+    Segs src = segs;
+    bool have = src.next(pr, wk);
+    while (have && wk.count <= 0) have = src.next(pr, wk);
+    auto next_segment = [&]() {
+        if (Segs::kSingle) return false;
+        bool more = src.next(pr, wk);
+        while (more && wk.count <= 0) more = src.next(pr, wk);
+        return more;
+    };
+
+    // activations of one or two tokens: kept whole in shared memory ([nb][K]), staged by these
+    // warps while the producer starts the copies (plain kernels: one segment), or delivered with
+    // every stage (grouped launch); the tensor-core path reads its fragments from global memory
     int xr[NB];
+    auto token_rows = [&]() {
 #pragma unroll
-    for (int b = 0; b < NB; ++b) {
-        const int bb = b < pr.nb ? b : 0;
-        xr[b] = pr.xrow ? __ldg(pr.xrow + bb) : bb;
-    }
+        for (int b = 0; b < NB; ++b) {
+            const int bb = b < pr.nb(pb) ? b : 0;
+            xr[b] = pr.xrow(pb) ? __ldg(pr.xrow(pb) + bb) : bb;
+        }
+    };
+    if (have) token_rows();
     const bool x_resident = L.x_bytes != 0;
-    if (x_resident) {
+    if (x_resident && have) {
         int4 *xs = reinterpret_cast<int4 *>(smem + L.x);
-        const int per_tok = static_cast<int>(pr.K / 16);
+        const int per_tok = static_cast<int>(pb.K / 16);
         const int nthr = (pl.NW + 2) * 32 - 32;              // all warps but the producer
         const int tid = warp < pl.NW ? threadIdx.x : threadIdx.x - 32;
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
-            if (b < pr.nb) {
-                const int4 *src = reinterpret_cast<const int4 *>(pr.x + static_cast<int64_t>(xr[b]) * pr.K);
+            if (b < pr.nb(pb)) {
+                const int4 *src = reinterpret_cast<const int4 *>(pb.x + static_cast<int64_t>(xr[b]) * pb.K);
                 for (int q = tid; q < per_tok; q += nthr) xs[b * per_tok + q] = __ldg(src + q);
             }
         }
     }
     __syncthreads();          // barriers initialised, activations in place
-    if (wk.count == 0) return;
+    if (!have) return;
 
     // ------------------------------------------------------------------ epilogue warp
     if (warp == pl.NW + 1) {
-        if (pl.probe == 2) return;
         float run[NB];          // running sum of the current row block over this block's items
 #pragma unroll
         for (int b = 0; b < NB; ++b) run[b] = 0.f;
-        float xsc[NB];          // per-token activation scales
-#pragma unroll
-        for (int b = 0; b < NB; ++b) xsc[b] = __ldg(pr.x_scale + xr[b]);
+        // per-token activation scales: kept in registers for up to two tokens, fetched where they
+        // are used (a cached load per output block) for more
+        float xsc[NB < kMmaMinBatch ? NB : 1] = {};
+        auto xscale = [&](int b) { return NB < kMmaMinBatch ? xsc[NB < kMmaMinBatch ? b : 0] : __ldg(pb.x_scale + xr[b]); };
         Share pend[2];
         int n_pend = 0;
         ItemIter it;
-        it.init(pl, wk.first);
+        int kk = 0;             // items consumed so far, over all segments
         constexpr int RS = red_slots(NB);
         // sum of n <= 20 partial sums of token b, spaced NB * 32 floats apart: all loads are issued
         // before the first addition, and the additions always follow the same tree
@@ -906,7 +987,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 #pragma unroll
                 for (int t = 0; t < NB / 4; ++t) {
                     float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (4 * t < pr.nb) v4 = sum_groups4(rs + (j0 * kRows + lane) * RF + ((4 * t) ^ red_swizzle<NB>(lane)), n);
+                    if (4 * t < pr.nb(pb)) v4 = sum_groups4(rs + (j0 * kRows + lane) * RF + ((4 * t) ^ red_swizzle<NB>(lane)), n);
                     tot[4 * t + 0] = v4.x;
                     tot[4 * t + 1] = v4.y;
                     tot[4 * t + 2] = v4.z;
@@ -915,14 +996,21 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             } else {
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
-                    tot[b] = (b < pr.nb) ? sum_groups(rs + (j0 * NB + b) * kRows + lane, n) : 0.f;
+                    tot[b] = (b < pr.nb(pb)) ? sum_groups(rs + (j0 * NB + b) * kRows + lane, n) : 0.f;
             }
         };
-        for (int k = 0; k < wk.count; ++k, it.next(pl, wk)) {
-            const int slot = k % RS;
-            const ItemRange r = item_range(pr, pl, it.c, it.cs);
-            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((k / RS) & 1))) {
-                if (lane == 0 && pr.status) *pr.status = 1u;
+        do {
+        n_pend = 0;
+        it.init(pl, wk.first);
+        if (NB < kMmaMinBatch) {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) xsc[NB < kMmaMinBatch ? b : 0] = __ldg(pb.x_scale + xr[b]);
+        }
+        for (int k = 0; k < wk.count; ++k, ++kk, it.next(pl, wk)) {
+            const int slot = kk % RS;
+            const ItemRange r = item_range(pb, pl, it.c, it.cs);
+            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((kk / RS) & 1))) {
+                if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                 return;
             }
             const float *rs = red + slot * red_slot;
@@ -930,18 +1018,18 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 // whole row blocks: one output per row.  The sums are formed first, the slot is
                 // handed back, and only then are the outputs stored, so that the release of the
                 // slot never waits for a global store.
-                const int nrb = r.nt / pr.G;
+                const int nrb = r.nt / pb.G;
                 for (int i = 0; i < nrb; ++i) {
                     const int64_t m = static_cast<int64_t>(r.rb0 + i) * kRows + lane;
                     float t_b[NB];
-                    sums(rs, i * pr.G, pr.G, t_b);
+                    sums(rs, i * pb.G, pb.G, t_b);
                     if (i == nrb - 1) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar0 + 8u * (kBarRedEmpty + slot));
                     }
 #pragma unroll
                     for (int b = 0; b < NB; ++b)
-                        if (b < pr.nb && m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = xsc[b] * t_b[b];
+                        if (b < pr.nb(pb) && m < pb.M) pb.y[(pr.out_row0(pb) + b) * pb.M + m] = xscale(b) * t_b[b];
                 }
                 continue;
             }
@@ -961,7 +1049,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 // the whole row block was ours
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
-                    if (b < pr.nb && m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = xsc[b] * run[b];
+                    if (b < pr.nb(pb) && m < pb.M) pb.y[(pr.out_row0(pb) + b) * pb.M + m] = xscale(b) * run[b];
             } else {
                 // shared row block: publish our share, then count ourselves in
                 Share sh;
@@ -971,28 +1059,31 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 sh.sharers = hi - lo + 1;
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
-                    if (b < pr.nb)
-                        pr.partial[((static_cast<int64_t>(sh.rb) * pl.CS + sh.slot) * pr.nb + b) * kRows + lane] = run[b];
+                    if (b < pr.nb(pb))
+                        pb.partial[((static_cast<int64_t>(sh.rb) * pl.CS + sh.slot) * pr.nb(pb) + b) * kRows + lane] = run[b];
                 __syncwarp();
                 sh.old = 0;
                 if (lane == 0) {
                     __threadfence();
-                    sh.old = atomicAdd(pr.counters + sh.rb, 1u);
+                    sh.old = atomicAdd(pb.counters + sh.rb, 1u);
                 }
                 pend[n_pend++] = sh;      // at most two per block: its first and its last row block
             }
         }
-        for (int i = 0; i < n_pend; ++i) finish_share<NB>(pr, pl, xr, pend[i], lane);
+        for (int i = 0; i < n_pend; ++i) finish_share<NB>(pb, pl, xr, pend[i], lane);
+        have = next_segment();
+        if (have) token_rows();
+        } while (have);
         return;
     }
 
     // ------------------------------------------------------------------ decoder warps
     // CS == 1: this warp always has row block warp / G of the chunk and group warp % G
-    const int my_rbl = (pl.CS == 1) ? warp / pr.G : 0;
-    const int g_fixed = warp - my_rbl * pr.G;
-    if (FMT != kBit2 && fresh) {
+    const int my_rbl = (pl.CS == 1) ? warp / pb.G : 0;
+    const int g_fixed = warp - my_rbl * pb.G;
+    if (FMT != kBit2) {
         if (!mbar_wait(bar0 + 8u * kBarLut, 0)) {
-            if (lane == 0 && pr.status) *pr.status = 1u;
+            if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
             return;
         }
     }
@@ -1009,13 +1100,15 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     // the matching weight words.  A operand: each lane stores the row it decoded into the warp's
     // buffer (32 int8 at a time, in that order), ldmatrix brings it back in fragment order.
     const int8_t *xfrag[NH];
+    auto token_fragments = [&]() {
 #pragma unroll
-    for (int h = 0; h < NH; ++h) {
-        const int n = 8 * h + (lane >> 2);
-        xfrag[h] = nullptr;
-        if (kMma && n < pr.nb)
-            xfrag[h] = pr.x + static_cast<int64_t>(pr.xrow ? __ldg(pr.xrow + n) : n) * pr.K + 16 * (lane & 3);
-    }
+        for (int h = 0; h < NH; ++h) {
+            const int n = 8 * h + (lane >> 2);
+            xfrag[h] = nullptr;
+            if (kMma && n < pr.nb(pb))
+                xfrag[h] = pb.x + static_cast<int64_t>(pr.xrow(pb) ? __ldg(pr.xrow(pb) + n) : n) * pb.K + 16 * (lane & 3);
+        }
+    };
     uint32_t bf[NH][8];
     auto load_bf = [&](int g) {
 #pragma unroll
@@ -1030,8 +1123,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             bf[h][4] = u1.x; bf[h][5] = u1.y; bf[h][6] = u1.z; bf[h][7] = u1.w;
         }
     };
-    // whole rows per item: this warp's group never changes, neither do its activation fragments
-    if (kMma && pl.CS == 1) load_bf(g_fixed);
+
     const uint32_t scr0 = smem_addr(smem + L.scr) + static_cast<uint32_t>(warp) * kScrBytes;
     const uint32_t scr_st = scr0 + static_cast<uint32_t>(lane) * kScrRowBytes;
     const uint32_t scr_ld = scr0 + static_cast<uint32_t>((lane & 7) + ((lane >> 3) & 1) * 8) * kScrRowBytes +
@@ -1046,27 +1138,36 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
     const uint32_t off_scale = L.payload_cap + L.sign_cap + tile_lane * 2u;           // its row's group scale
     const uint32_t off_toff = L.payload_cap + L.sign_cap + L.scale_cap + static_cast<uint32_t>(warp) * 4u;
     const uint32_t off_sign = L.payload_cap;
+    const uint32_t off_x = L.payload_cap + L.sign_cap + L.scale_cap + L.off_cap;     // activations inside a stage
     const uint8_t *xs_base = smem + L.x;
     // where this lane leaves its partial sums inside a slot (one or two tokens)
     float *rd_lane = red + static_cast<uint32_t>(warp * NB) * kRows + lane;
-    for (int k = 0; k < wk.count; ++k) {
+    int kk = 0;                 // items decoded so far, over all segments
+    do {
+    token_fragments();
+    // whole rows per item: this warp's group never changes, neither do its activation fragments
+    if (kMma && pl.CS == 1) load_bf(g_fixed);
+    for (const int kk_end = kk + wk.count; kk < kk_end; ++kk) {
         if (!mbar_wait(full_bar, phase)) {
-            if (lane == 0 && pr.status) *pr.status = 1u;
+            if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
             return;
         }
         const uint4 d = desc[s];
         const int nt = static_cast<int>(d.x & 0xFFu);
         const bool busy = warp < nt;
-        const int g = (pl.CS == 1) ? g_fixed : static_cast<int>(d.y) + warp;
+        // group of this warp's tile: the item's first group (0 when items are whole rows) + the
+        // warp's place in its row block
+        const int g = static_cast<int>(d.y) + g_fixed;
         float ysum[NV];
 #pragma unroll
         for (int b = 0; b < NV; ++b) ysum[b] = 0.f;
         if (kMma && pl.CS != 1 && busy) load_bf(g);        // early, so that the decode hides the latency
 
-        if (busy && !pl.probe) {
+        if (busy) {
             const float sc = bf16_to_float(*reinterpret_cast<const uint16_t *>(stage + off_scale));
             // activations of group g (one or two tokens: always in shared memory)
-            const uint8_t *xs = xs_base + static_cast<uint32_t>(g) * kGroup;
+            // (only the grouped launch ever delivers activations with the stage)
+            const uint8_t *xs = ((!Segs::kSingle && pl.x_in_stage) ? stage + off_x : xs_base) + static_cast<uint32_t>(g) * kGroup;
             int w[32];
             if (FMT == kBitcos) {
                 const uint4 bm = *reinterpret_cast<const uint4 *>(stage + off_bm);
@@ -1083,7 +1184,7 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
                 const uint32_t *sp = reinterpret_cast<const uint32_t *>(stage + off_sign + ((cursor >> 5) << 2));
                 bitcos_decode_row(bm, sp, cursor & 31u, lut, lane4, w);
             } else if (FMT == kTrit5) {
-                const int WPR = (26 * pr.G + 3) / 4;
+                const int WPR = (26 * pb.G + 3) / 4;
                 // words of the stage: row block my_rbl of the chunk, counted from the chunk's first word
                 const int w_rel = my_rbl * WPR + ((26 * g) >> 2) - ((26 * static_cast<int>(d.y)) >> 2);
                 const uint32_t *src = reinterpret_cast<const uint32_t *>(stage) + w_rel * kRows + lane;
@@ -1131,10 +1232,10 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
                             ysum[(h * 2 + mh) * 4 + r] = scq[2 * mh + (r >> 1)] * static_cast<float>(acc[h][mh][r]);
-                            if (pr.acc_debug) {
+                            if (pb.acc_debug) {
                                 const int b = 8 * h + 2 * (lane & 3) + (r & 1);
                                 const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + 16 * mh + (lane >> 2) + 8 * (r >> 1);
-                                if (b < pr.nb && m < pr.M) pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = acc[h][mh][r];
+                                if (b < pr.nb(pb) && m < pb.M) pb.acc_debug[((pr.out_row0(pb) + b) * pb.M + m) * pb.G + g] = acc[h][mh][r];
                             }
                         }
             }
@@ -1145,12 +1246,12 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 if (kMma) break;
-                if (b < pr.nb) {
-                    const int a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pr.K), lane);
+                if (NB == 1 || b < pr.nb(pb)) {       // a call has at least one token
+                    const int a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pb.K), lane);
                     ysum[b] = sc * static_cast<float>(a);
-                    if (pr.acc_debug) {
+                    if (pb.acc_debug) {
                         const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + lane;
-                        if (m < pr.M) pr.acc_debug[((pr.out_row0 + b) * pr.M + m) * pr.G + g] = a;
+                        if (m < pb.M) pb.acc_debug[((pr.out_row0(pb) + b) * pb.M + m) * pb.G + g] = a;
                     }
                 }
             }
@@ -1166,13 +1267,12 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
             full_bar = bar0 + 8u * kBarFull;
             phase ^= 1u;
         }
-        if (pl.probe == 2) continue;
 
         // partial sums for the epilogue warp (several slots, so decoders may run ahead of it)
-        const int slot = k & (RS - 1);
-        if (k >= RS) {
-            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>((k / RS - 1) & 1))) {
-                if (lane == 0 && pr.status) *pr.status = 1u;
+        const int slot = kk & (RS - 1);
+        if (kk >= RS) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>((kk / RS - 1) & 1))) {
+                if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                 return;
             }
         }
@@ -1193,6 +1293,18 @@ __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, u
         __syncwarp();
         mbar_arrive_lane0(bar0 + 8u * (kBarRedFull + slot), lane);
     }
+    } while (next_segment());
+}
+
+// One problem, this block's share of its items.
+template <int FMT, int NB>
+__device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
+                                            const FirstOff *fo = nullptr, int fo_index = 0) {
+    OneSeg one;
+    one.pr = &pr;
+    one.wk = wk;
+    one.used = false;
+    run_segments<FMT, NB>(one, pl, smem, block, fo, fo_index);
 }
 
 template <int FMT, int NB>
@@ -1200,7 +1312,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Pr
                                                                         const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
     run_problem<FMT, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
-                         static_cast<int>(blockIdx.x), true, &fo, static_cast<int>(blockIdx.x));
+                         static_cast<int>(blockIdx.x), &fo, static_cast<int>(blockIdx.x));
 }
 
 // Several independent BITCOS problems in one launch: the grid is cut into one range of thread
@@ -1222,7 +1334,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
     run_problem<kBitcos, NB>(ma.pr[j], ma.pl[j], smem,
                              make_walk(ma.pl[j], b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
-                             b - ma.first_block[j], true, &fo, b);
+                             b - ma.first_block[j], &fo, b);
 }
 
 // Fills in what differs between the groups of a grouped product; false if the group is empty or
@@ -1248,17 +1360,59 @@ __device__ __forceinline__ bool grouped_problem(Problem &pr, const Problem &base
     return true;
 }
 
-// Grouped product.  Two launch shapes.  Flat (rows in one piece, no cross-block sums): the items
-// of all groups form one list, cut into equal contiguous ranges, one per thread block, so a
-// block runs the tail of one group and the head of the next with the same shared-memory layout.
-// Otherwise: blockIdx.y = group, and the blocks of a row of the grid share that group's items.
+// The pieces of the groups that fall into one thread block's range of the flat item list.
 template <int NB>
-__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(const Problem base, const Plan pl, const GroupedArgs ga) {
+struct GroupedSegs {
+    const Problem *base;
+    const GroupedArgs *ga;
+    int64_t lo, hi, ipg;      // this block's range of the list; items per group
+    int grp;                  // group of item lo
+    typedef GroupView View;
+    static constexpr bool kSingle = false;
+    __device__ __forceinline__ const Problem &shape() const { return *base; }
+    __device__ __forceinline__ bool next(View &v, Walk &w) {
+        while (lo < hi) {
+            const int64_t g_lo = static_cast<int64_t>(grp) * ipg;
+            const int64_t seg_hi = hi < g_lo + ipg ? hi : g_lo + ipg;
+            w.first = static_cast<int>(lo - g_lo);
+            w.count = static_cast<int>(seg_hi - lo);
+            w.cstride = 1;
+            w.q = 1;
+            w.rem = 0;
+            lo = seg_hi;
+            const int g = grp++;
+            const int e = __ldg(ga->group_expert + g);
+            const int begin = __ldg(ga->group_begin + g), end = __ldg(ga->group_begin + g + 1);
+            if (e < 0 || e >= ga->n_experts || end <= begin) continue;
+            const bitcos_weights *wd = ga->experts + e;
+            v.payload_ = wd->bitmap;
+            v.signs_ = wd->signs;
+            v.tile_off_ = wd->tile_off;
+            v.scales_ = wd->scales;
+            v.xrow_ = base->xrow + begin;
+            v.status_ = reinterpret_cast<unsigned int *>(reinterpret_cast<uint8_t *>(base->status) +
+                                                         static_cast<size_t>(g) * ga->ws_stride);
+            v.begin_ = begin;
+            v.nb_ = min(end - begin, NB);
+            return true;
+        }
+        return false;
+    }
+};
+
+// Grouped product.  Two launch shapes.  Flat (rows in one piece, no cross-block sums): the items
+// of all groups form one list, cut into equal contiguous ranges, one per thread block; a block
+// that crosses from one group to the next keeps its pipeline running (the producer is already
+// copying the next group's weights while the last tiles of this one are decoded).  Otherwise:
+// blockIdx.y = group, and the blocks of a row of the grid share that group's items.
+template <int NB>
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(const __grid_constant__ Problem base, const Plan pl,
+                                                                                const __grid_constant__ GroupedArgs ga) {
     extern __shared__ __align__(128) uint8_t smem[];
     // the routing lists may come from the previous kernel in the stream
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    Problem pr;
     if (!ga.flat) {
+        Problem pr;
         if (!grouped_problem<NB>(pr, base, ga, static_cast<int>(blockIdx.y))) return;
         run_problem<kBitcos, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                                  static_cast<int>(blockIdx.x));
@@ -1267,24 +1421,14 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(
     const int64_t ipg = pl.items, total = ipg * ga.n_groups;
     const int64_t nblk = gridDim.x, b = blockIdx.x;
     const int64_t q = total / nblk, rem = total - q * nblk;
-    int64_t lo = b * q + (b < rem ? b : rem);
-    const int64_t hi = lo + q + (b < rem ? 1 : 0);
-    bool fresh = true;
-    for (int grp = static_cast<int>(lo / ipg); lo < hi; ++grp) {
-        const int64_t g_lo = static_cast<int64_t>(grp) * ipg;
-        const int64_t seg_hi = hi < g_lo + ipg ? hi : g_lo + ipg;
-        Walk wk;
-        wk.first = static_cast<int>(lo - g_lo);
-        wk.count = static_cast<int>(seg_hi - lo);
-        wk.cstride = 1;
-        wk.q = 1;
-        wk.rem = 0;
-        lo = seg_hi;
-        if (!grouped_problem<NB>(pr, base, ga, grp)) continue;
-        if (!fresh) __syncthreads();          // everybody is done with the previous group's barriers and buffers
-        run_problem<kBitcos, NB>(pr, pl, smem, wk, static_cast<int>(b), fresh);
-        fresh = false;
-    }
+    GroupedSegs<NB> segs;
+    segs.base = &base;
+    segs.ga = &ga;
+    segs.ipg = ipg;
+    segs.lo = b * q + (b < rem ? b : rem);
+    segs.hi = segs.lo + q + (b < rem ? 1 : 0);
+    segs.grp = static_cast<int>(segs.lo / ipg);
+    run_segments<kBitcos, NB>(segs, pl, smem, static_cast<int>(b));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1492,8 +1636,6 @@ int launch(const Problem &pr, const Plan &pl, cudaStream_t stream, const uint32_
     Plan plw = pl;
     choose_walk(plw, sms, &grid);
     plw.stages = choose_stages(FMT, pl, pr.G, NB, pr.K, budget);
-    static const char *probe = std::getenv("BITCOS_PROBE");
-    plw.probe = (probe && probe[0] == 'c') ? 1 : (probe && probe[0] == 'd') ? 2 : 0;
     const SmemLayout L = smem_layout(FMT, plw, pr.G, NB, pr.K);
     FirstOff fo;
     fo.valid = (FMT == kBitcos && off_host) ? 1 : 0;
@@ -1514,7 +1656,6 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     int nw = 0;
     uint32_t smem = 0;
     int next = 0;
-    static const char *probe = std::getenv("BITCOS_PROBE");
     FirstOff fo;
     fo.valid = 1;
     for (int j = 0; j < ma.n; ++j) fo.valid = (fo.valid && off_host[j]) ? 1 : 0;
@@ -1527,7 +1668,6 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
         int grid = 1;
         choose_walk(ma.pl[j], static_cast<int>(cap), &grid);
         ma.pl[j].stages = choose_stages(kBitcos, ma.pl[j], ma.pr[j].G, NB, ma.pr[j].K, budget);
-        ma.pl[j].probe = (probe && probe[0] == 'c') ? 1 : (probe && probe[0] == 'd') ? 2 : 0;
         const SmemLayout L = smem_layout(kBitcos, ma.pl[j], ma.pr[j].G, NB, ma.pr[j].K);
         if (L.total > smem) smem = L.total;
         if (ma.pl[j].NW > nw) nw = ma.pl[j].NW;
@@ -1569,12 +1709,16 @@ int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int
     GroupedArgs gaw = ga;
     gaw.n_groups = n_groups;
     if (pl.CS == 1) {
-        // rows in one piece: one balanced list of all groups' items
+        // rows in one piece: one balanced list of all groups' items; one or two tokens per group:
+        // their activation rows travel with every stage
         const int64_t total = pl.items * n_groups;
         gaw.flat = 1;
         plw.cyclic = 0;
+        plw.x_in_stage = NB < kMmaMinBatch ? 1 : 0;
+        plw.stages = choose_stages(kBitcos, plw, pr.G, NB, pr.K, budget);
+        const SmemLayout Lf = smem_layout(kBitcos, plw, pr.G, NB, pr.K);
         return launch_pdl(gemv_grouped_kernel<NB>, dim3(static_cast<unsigned>(total < sms ? total : sms)), (pl.NW + 2) * 32,
-                          L.total, stream, pr, plw, gaw);
+                          Lf.total, stream, pr, plw, gaw);
     }
     // the machine is shared by all groups: spread its multiprocessors over them
     int per_group = (sms + n_groups - 1) / n_groups;
