@@ -1332,8 +1332,9 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     const int b = static_cast<int>(blockIdx.x);
     int j = 0;
     while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
-    run_problem<kBitcos, NB>(ma.pr[j], ma.pl[j], smem,
-                             make_walk(ma.pl[j], b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
+    const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
+    const Problem pr = ma.pr[j];
+    run_problem<kBitcos, NB>(pr, pl, smem, make_walk(pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
                              b - ma.first_block[j], &fo, b);
 }
 
