@@ -391,10 +391,17 @@ def run_cuda(args):
     yh = [torch.empty((1, m["M"]), dtype=torch.float32).pin_memory() for m in layer]
     xh_np, xsh_np, yh_np = [t.numpy() for t in xh], [t.numpy() for t in xsh], [t.numpy() for t in yh]
 
+    host_multi = [[bc.MultiHostJobs([(rep[j], xh_np[j], xsh_np[j], yh_np[j], stagings[j], wss[j]) for j in g])
+                   for g in groups] for rep in replicas]
+
     def e2e_step(i):
-        rep = replicas[i % copies]
-        for j in range(len(layer)):
-            bc.bitcos_gemv_host(rep[j], xh_np[j], xsh_np[j], yh_np[j], stagings[j], wss[j])
+        if args.serial or args.branches:
+            rep = replicas[i % copies]
+            for j in range(len(layer)):
+                bc.bitcos_gemv_host(rep[j], xh_np[j], xsh_np[j], yh_np[j], stagings[j], wss[j])
+            return
+        for mj in host_multi[i % copies]:
+            bc.bitcos_gemv_multi_host(mj)
 
     e2e_steps = 0 if args.no_e2e else min(args.steps, 200)
     e2e_us = float("nan")
@@ -471,8 +478,10 @@ def run_cuda(args):
                          "sample": f"{reps} full layer passes (7 GEMVs, 69.5 M weights each): BITCOS decode bit by "
                                    "bit, dense int32 dot per group, double scale-and-sum"},
         "e2e": {"value": whole_job_value(e2e_us, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "path": "bitcos_gemv_host per GEMV: pinned x -> device, kernel, y -> pinned host, "
-                                            "stream wait"},
+                "steps": e2e_steps,
+                "path": ("bitcos_gemv_host per GEMV" if (args.serial or args.branches) else
+                         "bitcos_gemv_multi_host, four calls per step (q+k+v, o, gate+up, down)")
+                        + ": pinned x -> device, kernel, y -> pinned host, stream wait"},
         "gpu_launches": n_launch,
         "clocks": clocks,
     }

@@ -237,6 +237,24 @@ int bitcos_gemv_host(const bitcos_weights *W, const int8_t *x_host, const float 
                      float *y_host, void *staging, size_t staging_bytes, void *workspace,
                      size_t workspace_bytes, void *cuda_stream);
 
+/* Host-buffer form of bitcos_gemv_multi: up to BITCOS_MAX_JOBS independent products whose
+ * activations and results live in host memory, with ONE launch and ONE wait for all of them
+ * (copies every job's x and x_scale into its staging buffer, runs bitcos_gemv_multi, copies every
+ * y back, waits for the stream; all y_host are valid on return).  Per job: staging of
+ * bitcos_gemv_host_staging_bytes(M, K, batch) bytes and a workspace of its own, as for
+ * bitcos_gemv_host.  The paper has no counterpart (it measures resident activations). */
+typedef struct bitcos_gemv_host_job {
+    const bitcos_weights *W;    /* host struct of device pointers */
+    const int8_t *x_host;       /* host int8 [batch][K] (pinned memory keeps the copies asynchronous) */
+    const float *x_scale_host;  /* host float [batch] */
+    float *y_host;              /* host float [batch][M] */
+    void *staging;              /* device scratch */
+    size_t staging_bytes;
+    void *workspace;            /* device scratch, zero filled once */
+    size_t workspace_bytes;
+} bitcos_gemv_host_job;
+int bitcos_gemv_multi_host(const bitcos_gemv_host_job *jobs, int n_jobs, int batch, void *cuda_stream);
+
 /* The same product from the five-trit and 2-bit layouts (device pointers; scales in tile order). */
 int trit5_gemv(const uint32_t *words, const uint16_t *scales_tiled, int64_t M, int64_t K, const int8_t *x,
                const float *x_scale, int batch, float *y, int32_t *acc_debug, void *workspace,

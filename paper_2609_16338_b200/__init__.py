@@ -22,6 +22,8 @@ from .binding import (  # noqa: F401
     bitcos_gemv_static,
     bitcos_gemv_multi,
     MultiJobs,
+    bitcos_gemv_multi_host,
+    MultiHostJobs,
     bitcos_decode_probe,
     group_pairs,
     plain_to_device,

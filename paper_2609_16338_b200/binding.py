@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = [
     "trit5_unpack", "bit2_pack_sizes", "bit2_pack", "bit2_unpack", "bitcos_gemv_workspace_bytes",
     "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
+    "bitcos_gemv_multi_host",
 ]
 
 
@@ -36,6 +37,12 @@ class BitcosError(RuntimeError):
 class _Job(C.Structure):
     _fields_ = [("W", C.c_void_p), ("x", C.c_void_p), ("x_scale", C.c_void_p), ("y", C.c_void_p),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+class _HostJob(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("x_host", C.c_void_p), ("x_scale_host", C.c_void_p), ("y_host", C.c_void_p),
+                ("staging", C.c_void_p), ("staging_bytes", C.c_size_t), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_size_t)]
 
 
 class _Weights(C.Structure):
@@ -89,6 +96,7 @@ def load_library():
     L.bitcos_gemv_static.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp]
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
+    L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
     _lib = L
     return L
 
@@ -413,6 +421,25 @@ def bitcos_gemv_static(W: DeviceBitcos, x, x_scale, y):
     _check(load_library().bitcos_gemv_static(C.byref(W.desc), x.data_ptr(), x_scale.data_ptr(), x.shape[0],
                                              y.data_ptr(), _stream()), "bitcos_gemv_static")
     return y
+
+
+class MultiHostJobs:
+    """Argument block of bitcos_gemv_multi_host, built once and reusable:
+    jobs = [(W, x_host, x_scale_host, y_host, staging, workspace)] with numpy host arrays."""
+
+    def __init__(self, jobs):
+        self.keep = jobs
+        self.batch = jobs[0][1].shape[0]
+        self.arr = (_HostJob * len(jobs))(*[
+            _HostJob(C.addressof(W.desc), xh.ctypes.data, xsh.ctypes.data, yh.ctypes.data, st.data_ptr(), st.numel(),
+                     ws.data_ptr(), ws.numel()) for (W, xh, xsh, yh, st, ws) in jobs])
+
+
+def bitcos_gemv_multi_host(jobs):
+    """Several independent products from host buffers with one launch and one wait."""
+    mj = jobs if isinstance(jobs, MultiHostJobs) else MultiHostJobs(jobs)
+    _check(load_library().bitcos_gemv_multi_host(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi_host")
+    return [j[3] for j in mj.keep]
 
 
 def bitcos_gemv_host_staging_bytes(M: int, K: int, batch: int) -> int:

@@ -1963,6 +1963,49 @@ int bitcos_gemv_host(const bitcos_weights *W, const int8_t *x_host, const float 
     return check_cuda(cudaStreamSynchronize(stream));
 }
 
+int bitcos_gemv_multi_host(const bitcos_gemv_host_job *jobs, int n_jobs, int batch, void *cuda_stream) {
+    if (!jobs) return BITCOS_ERR_NULL;
+    if (n_jobs < 1 || n_jobs > kMaxJobs) return BITCOS_ERR_SHAPE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    bitcos_gemv_job dev_jobs[kMaxJobs];
+    float *y_dev[kMaxJobs];
+    for (int j = 0; j < n_jobs; ++j) {
+        const bitcos_gemv_host_job &jb = jobs[j];
+        if (!jb.W || !jb.x_host || !jb.x_scale_host || !jb.y_host || !jb.staging) return BITCOS_ERR_NULL;
+        const size_t need = bitcos_gemv_host_staging_bytes(jb.W->M, jb.W->K, batch);
+        if (need == 0) return BITCOS_ERR_SHAPE;
+        if (jb.staging_bytes < need) return BITCOS_ERR_CAPACITY;
+        if (!aligned16(jb.staging)) return BITCOS_ERR_ALIGN;
+        uint8_t *base = static_cast<uint8_t *>(jb.staging);
+        const size_t xb = (static_cast<size_t>(batch) * jb.W->K + 255) / 256 * 256;
+        dev_jobs[j].W = jb.W;
+        dev_jobs[j].x = reinterpret_cast<const int8_t *>(base);
+        dev_jobs[j].x_scale = reinterpret_cast<const float *>(base + xb);
+        y_dev[j] = reinterpret_cast<float *>(base + xb + 256);
+        dev_jobs[j].y = y_dev[j];
+        dev_jobs[j].workspace = jb.workspace;
+        dev_jobs[j].workspace_bytes = jb.workspace_bytes;
+    }
+    for (int j = 0; j < n_jobs; ++j) {
+        uint8_t *base = static_cast<uint8_t *>(jobs[j].staging);
+        const size_t xb = (static_cast<size_t>(batch) * jobs[j].W->K + 255) / 256 * 256;
+        int rc = check_cuda(cudaMemcpyAsync(base, jobs[j].x_host, static_cast<size_t>(batch) * jobs[j].W->K,
+                                            cudaMemcpyHostToDevice, stream));
+        if (rc) return rc;
+        rc = check_cuda(cudaMemcpyAsync(base + xb, jobs[j].x_scale_host, static_cast<size_t>(batch) * sizeof(float),
+                                        cudaMemcpyHostToDevice, stream));
+        if (rc) return rc;
+    }
+    int rc = bitcos_gemv_multi(dev_jobs, n_jobs, batch, cuda_stream);
+    if (rc) return rc;
+    for (int j = 0; j < n_jobs; ++j) {
+        rc = check_cuda(cudaMemcpyAsync(jobs[j].y_host, y_dev[j], static_cast<size_t>(batch) * jobs[j].W->M * sizeof(float),
+                                        cudaMemcpyDeviceToHost, stream));
+        if (rc) return rc;
+    }
+    return check_cuda(cudaStreamSynchronize(stream));
+}
+
 int trit5_gemv(const uint32_t *words, const uint16_t *scales_tiled, int64_t M, int64_t K, const int8_t *x,
                const float *x_scale, int batch, float *y, int32_t *acc_debug, void *workspace,
                size_t workspace_bytes, void *cuda_stream) {

@@ -225,6 +225,28 @@ def test_host_buffer_entry_point(bc):
     assert (err <= REL * mag).all()
 
 
+def test_multi_host_buffer_entry_point(bc):
+    """Several products from host buffers in one call: same results as the device entry point."""
+    B = 2
+    jobs, refs = [], []
+    for i, (M, K) in enumerate([(640, 2560), (96, 6912), (2560, 2560)]):
+        W, S = datagen.trits(800 + i, M, K, 0.4219), datagen.scales(800 + i, M, K)
+        x, xs = datagen.activations(800 + i, B, K)
+        refs.append(oracle.gemv_dense(W, S, x, xs))
+        staging = torch.empty(bc.bitcos_gemv_host_staging_bytes(M, K, B), dtype=torch.uint8, device="cuda")
+        xh, xsh = torch.from_numpy(x).pin_memory(), torch.from_numpy(xs).pin_memory()
+        yh = torch.full((B, M), float("nan"), dtype=torch.float32).pin_memory()
+        jobs.append((bc.bitcos_pack(W, S).to_device(), xh.numpy(), xsh.numpy(), yh.numpy(), staging, bc.make_workspace(M, K),
+                     (xh, xsh, yh)))
+    bc.bitcos_gemv_multi_host([j[:6] for j in jobs])
+    for (Wd, xh, xsh, yh, st, ws, _), (acc_ref, y_ref, mag) in zip(jobs, refs):
+        err = np.abs(yh.astype(np.float64) - y_ref)
+        assert (err <= REL * mag).all()
+        y_dev, _ = bc.bitcos_gemv(Wd, dev(xh), dev(xsh), workspace=ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(y_dev.cpu().numpy(), yh)
+
+
 def test_sampled_outputs_at_full_size(bc):
     """The largest layer shapes of the benchmark configurations, in the launch configuration
     the benchmark times; the oracle checks a sample of rows it computes one by one."""
