@@ -142,6 +142,28 @@ def test_grouped_experts(bc):
             check(y, acc, acc_ref, y_ref, mag, f"grouped tokens={tokens} rep{rep}")
 
 
+def test_grouped_many_small_groups(bc):
+    """More items than thread blocks and few items per group: blocks run the tail of one group and
+    the head of the next (and whole small groups) without stopping their pipeline."""
+    E, M, K, top_k = 96, 160, 1280, 6
+    Ws = [datagen.trits(900 + e, M, K, 0.35) for e in range(E)]
+    Ss = [datagen.scales(900 + e, M, K) for e in range(E)]
+    experts = bc.DeviceExperts([bc.bitcos_pack(Ws[e], Ss[e]).to_device() for e in range(E)])
+    for tokens in (16, 12):
+        x, xs = datagen.activations(950 + tokens, tokens, K)
+        ids = datagen.expert_choices(950 + tokens, tokens, E, top_k)
+        pair_expert = ids.reshape(-1)
+        pair_xrow = np.repeat(np.arange(tokens, dtype=np.int32), top_k)
+        order, ge, gb, xr, mx = bc.group_pairs(pair_expert, pair_xrow)
+        assert len(ge) * ((M + 31) // 32 + 1) // 2 > 148 or len(ge) > 50
+        acc_ref, y_ref, mag = oracle.grouped_dense(Ws, Ss, pair_expert[order], pair_xrow[order], x, xs)
+        ws = bc.make_workspace(M, K, copies=len(ge))
+        for rep in range(2):
+            y, acc = bc.bitcos_gemv_grouped(experts, dev(ge), dev(gb), dev(xr), mx, dev(x), dev(xs),
+                                            acc_debug=True, workspace=ws)
+            check(y, acc, acc_ref, y_ref, mag, f"many groups tokens={tokens} rep{rep}")
+
+
 def test_grouped_down_projection_shape(bc):
     # K = 768 (six groups), per-pair activation rows
     E, M, K = 4, 2048, 768
