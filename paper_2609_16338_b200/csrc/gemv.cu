@@ -146,6 +146,7 @@ struct Plan {
     int cyclic;      // 1: blocks take whole row-block chunks round robin; 0: contiguous balanced ranges
     int stages;      // depth of the shared-memory ring (2 .. kMaxStages), set at launch
     int x_in_stage;  // 1: every stage also receives the item's activation rows (grouped launch, 1-2 tokens)
+    int wq, wrem;    // contiguous walk: blocks 0 .. wrem-1 own wq + 1 items, the others wq (set at launch)
 };
 
 struct Problem {
@@ -174,6 +175,10 @@ struct FirstOff {
     uint32_t lo[kMaxGrid];
     uint32_t hi[kMaxGrid];
     int valid;
+    // every block's share of the items, worked out on the host (no divisions at kernel start)
+    int first[kMaxGrid];
+    int count[kMaxGrid];
+    int walks;                 // 1: first / count are filled in
 };
 
 struct GroupedArgs {
@@ -542,6 +547,18 @@ __host__ __device__ __forceinline__ Walk make_walk(const Plan &pl, int block, in
     w.first = block * w.q + (block < w.rem ? block : w.rem);
     w.count = w.q + (block < w.rem ? 1 : 0);
     w.cstride = 1;
+    return w;
+}
+
+// This block's walk: from the launch's table if there is one, else computed here.
+__device__ __forceinline__ Walk block_walk(const FirstOff &fo, int index, const Plan &pl, int block, int n_blocks) {
+    if (!fo.walks) return make_walk(pl, block, n_blocks);
+    Walk w;
+    w.first = fo.first[index];
+    w.count = fo.count[index];
+    w.cstride = pl.cyclic ? n_blocks : 1;
+    w.q = pl.wq;
+    w.rem = pl.wrem;
     return w;
 }
 
@@ -1311,7 +1328,8 @@ template <int FMT, int NB>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl,
                                                                         const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
-    run_problem<FMT, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
+    run_problem<FMT, NB>(pr, pl, smem,
+                         block_walk(fo, static_cast<int>(blockIdx.x), pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                          static_cast<int>(blockIdx.x), &fo, static_cast<int>(blockIdx.x));
 }
 
@@ -1334,7 +1352,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
     const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
     const Problem pr = ma.pr[j];
-    run_problem<kBitcos, NB>(pr, pl, smem, make_walk(pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
+    run_problem<kBitcos, NB>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
                              b - ma.first_block[j], &fo, b);
 }
 
@@ -1586,6 +1604,8 @@ inline void choose_walk(Plan &pl, int sms, int *grid) {
     if (force && force[0] == 'c' && force[1] == 'o') cyclic = 0;
     pl.cyclic = cyclic;
     *grid = static_cast<int>(cyclic ? g_cyc : g_con);
+    pl.wq = cyclic ? 1 : static_cast<int>(pl.items / *grid);
+    pl.wrem = cyclic ? 0 : static_cast<int>(pl.items - static_cast<int64_t>(pl.wq) * *grid);
 }
 
 // Launches with programmatic stream serialization, so that this kernel's prologue (barrier
@@ -1610,10 +1630,18 @@ int launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cu
 // Fills fo.lo / fo.hi [base .. base + grid) from a host copy of tile_off: the sign-vector range of
 // the first item of each of the `grid` thread blocks that share the problem.
 void fill_first_off(FirstOff &fo, int base, const uint32_t *off_host, const Problem &pr, const Plan &pl, int grid) {
-    if (!off_host || base + grid > kMaxGrid) {
+    if (base + grid > kMaxGrid) {
         fo.valid = 0;
+        fo.walks = 0;
         return;
     }
+    for (int b = 0; b < grid; ++b) {
+        const Walk wk = make_walk(pl, b, grid);
+        fo.first[base + b] = wk.first;
+        fo.count[base + b] = wk.count;
+    }
+    if (!off_host) fo.valid = 0;
+    if (!fo.valid) return;
     for (int b = 0; b < grid; ++b) {
         const Walk wk = make_walk(pl, b, grid);
         fo.lo[base + b] = fo.hi[base + b] = 0;
@@ -1640,7 +1668,8 @@ int launch(const Problem &pr, const Plan &pl, cudaStream_t stream, const uint32_
     const SmemLayout L = smem_layout(FMT, plw, pr.G, NB, pr.K);
     FirstOff fo;
     fo.valid = (FMT == kBitcos && off_host) ? 1 : 0;
-    if (fo.valid) fill_first_off(fo, 0, off_host, pr, plw, grid);
+    fo.walks = 1;
+    fill_first_off(fo, 0, off_host, pr, plw, grid);
     return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
@@ -1659,6 +1688,7 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     int next = 0;
     FirstOff fo;
     fo.valid = 1;
+    fo.walks = 1;
     for (int j = 0; j < ma.n; ++j) fo.valid = (fo.valid && off_host[j]) ? 1 : 0;
     for (int j = 0; j < ma.n; ++j) {
         int64_t cap = ma.pl[j].items;
@@ -1673,7 +1703,7 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
         if (L.total > smem) smem = L.total;
         if (ma.pl[j].NW > nw) nw = ma.pl[j].NW;
         ma.first_block[j] = next;
-        if (fo.valid) fill_first_off(fo, next, off_host[j], ma.pr[j], ma.pl[j], grid);
+        fill_first_off(fo, next, fo.valid ? off_host[j] : nullptr, ma.pr[j], ma.pl[j], grid);
         next += grid;
     }
     ma.first_block[ma.n] = next;
