@@ -742,9 +742,11 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
 // What a thread block runs back to back: one problem and its share of the items (the plain
 // kernels), or the pieces of several groups (the grouped launch).  Every warp role walks its own
 // copy of the source.
-struct OneSeg {
+template <bool DEBUG>
+struct OneSegT {
     typedef ParamView View;
     static constexpr bool kSingle = true;      // never more than one segment
+    static constexpr bool kDebug = DEBUG;      // false: acc_debug is known to be NULL (no code for it)
     const Problem *pr;
     Walk wk;
     bool used;
@@ -1249,7 +1251,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
                             ysum[(h * 2 + mh) * 4 + r] = scq[2 * mh + (r >> 1)] * static_cast<float>(acc[h][mh][r]);
-                            if (pb.acc_debug) {
+                            if (Segs::kDebug && pb.acc_debug) {
                                 const int b = 8 * h + 2 * (lane & 3) + (r & 1);
                                 const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + 16 * mh + (lane >> 2) + 8 * (r >> 1);
                                 if (b < pr.nb(pb) && m < pb.M) pb.acc_debug[((pr.out_row0(pb) + b) * pb.M + m) * pb.G + g] = acc[h][mh][r];
@@ -1266,7 +1268,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 if (NB == 1 || b < pr.nb(pb)) {       // a call has at least one token
                     const int a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pb.K), lane);
                     ysum[b] = sc * static_cast<float>(a);
-                    if (pb.acc_debug) {
+                    if (Segs::kDebug && pb.acc_debug) {
                         const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + lane;
                         if (m < pb.M) pb.acc_debug[((pr.out_row0(pb) + b) * pb.M + m) * pb.G + g] = a;
                     }
@@ -1314,10 +1316,10 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 }
 
 // One problem, this block's share of its items.
-template <int FMT, int NB>
+template <int FMT, int NB, bool DEBUG = true>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
                                             const FirstOff *fo = nullptr, int fo_index = 0) {
-    OneSeg one;
+    OneSegT<DEBUG> one;
     one.pr = &pr;
     one.wk = wk;
     one.used = false;
@@ -1352,7 +1354,8 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
     const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
     const Problem pr = ma.pr[j];
-    run_problem<kBitcos, NB>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
+    // (the multi launch has no accumulator dump)
+    run_problem<kBitcos, NB, false>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
                              b - ma.first_block[j], &fo, b);
 }
 
@@ -1388,6 +1391,7 @@ struct GroupedSegs {
     int grp;                  // group of item lo
     typedef GroupView View;
     static constexpr bool kSingle = false;
+    static constexpr bool kDebug = true;
     __device__ __forceinline__ const Problem &shape() const { return *base; }
     __device__ __forceinline__ bool next(View &v, Walk &w) {
         while (lo < hi) {
