@@ -797,19 +797,17 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // It also sets the barriers up, so that the first copies are in flight before anything else
     // happens in the block.
     if (warp == pl.NW) {
-        if (lane == 0) {
-            for (int s = 0; s < pl.stages; ++s) {
-                mbar_init(bar0 + 8u * (kBarFull + s), 1);
-                mbar_init(bar0 + 8u * (kBarEmpty + s), pl.NW);
-            }
-            for (int s = 0; s < red_slots(NB); ++s) {
-                mbar_init(bar0 + 8u * (kBarRedFull + s), pl.NW);
-                mbar_init(bar0 + 8u * (kBarRedEmpty + s), 1);
-            }
-            mbar_init(bar0 + 8u * kBarLut, 1);
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        }
+        // All 33 barrier slots at once, one per lane (slots of unused stages included): slots
+        // kBarEmpty .. kBarRedFull + 7 count the decoder warps, the others one arrival.  Every
+        // barrier is initialised and fenced before the first asynchronous copy is issued.
+        static_assert(kBarFull == 0 && kBarEmpty == 8 && kBarRedFull == 16 && kBarRedEmpty == 24 && kBarLut == 32,
+                      "one barrier slot per lane, plus the table's");
+        mbar_init(bar0 + 8u * static_cast<uint32_t>(lane), (lane >= kBarEmpty && lane < kBarRedEmpty) ? pl.NW : 1);
+        if (lane == 0) mbar_init(bar0 + 8u * kBarLut, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the other lanes' barriers, seen by this lane's copies
         // The first copies go out before the block-wide barrier below, while the other warps are
         // still fetching the activations.
         // Entry offsets are requested two items before they are needed (r0 = item k, r1 = item
