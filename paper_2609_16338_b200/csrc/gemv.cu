@@ -698,6 +698,7 @@ constexpr int kBarEmpty = kMaxStages;             // [stages] stage released by 
 constexpr int kBarRedFull = 2 * kMaxStages;       // [slots] partial sums of an item written by all decoder warps
 constexpr int kBarRedEmpty = 2 * kMaxStages + 8;  // [slots] partial sums consumed by the epilogue warp
 constexpr int kBarLut = 2 * kMaxStages + 16;      // lookup table arrived
+constexpr int kBarX = 2 * kMaxStages + 17;        // activations arrived in shared memory (plain kernels, 1-2 tokens)
 
 // Arrival by lane 0 only, as one predicated instruction (no divergent branch around it).
 __device__ __forceinline__ void mbar_arrive_lane0(uint32_t bar, int lane) {
@@ -804,6 +805,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                       "one barrier slot per lane, plus the table's");
         mbar_init(bar0 + 8u * static_cast<uint32_t>(lane), (lane >= kBarEmpty && lane < kBarRedEmpty) ? pl.NW : 1);
         if (lane == 0) mbar_init(bar0 + 8u * kBarLut, 1);
+        if (lane == 1) mbar_init(bar0 + 8u * kBarX, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
@@ -901,9 +903,13 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         return;
     }
 
-    // Everything below may depend on the previous kernel in the stream (activations, outputs,
-    // workspace); the packed weights the producer streams do not.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // What may depend on the previous kernel in the stream: activations, routing lists, outputs,
+    // workspace.  The packed weights do not, so the producer never waits, and in the plain kernels
+    // with one or two tokens (kEarly) the decoder warps do not either until they have decoded
+    // their first tile: only the contraction needs the activations, which the epilogue warp
+    // fetches into shared memory (one bulk copy per token) as soon as the dependency is resolved.
+    constexpr bool kEarly = Segs::kSingle && NB < kMmaMinBatch;
+    if (!kEarly) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     Segs src = segs;
     bool have = src.next(pr, wk);
@@ -926,9 +932,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             xr[b] = pr.xrow(pb) ? __ldg(pr.xrow(pb) + bb) : bb;
         }
     };
-    if (have) token_rows();
+    if (have && !kEarly) token_rows();
     const bool x_resident = L.x_bytes != 0;
-    if (x_resident && have) {
+    if (x_resident && have && !kEarly) {
         int4 *xs = reinterpret_cast<int4 *>(smem + L.x);
         const int per_tok = static_cast<int>(pb.K / 16);
         const int nthr = (pl.NW + 2) * 32 - 32;              // all warps but the producer
@@ -946,6 +952,18 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 
     // ------------------------------------------------------------------ epilogue warp
     if (warp == pl.NW + 1) {
+        if (kEarly) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            token_rows();
+            if (lane == 0) {
+                mbar_expect_tx(bar0 + 8u * kBarX, static_cast<uint32_t>(pr.nb(pb)) * static_cast<uint32_t>(pb.K));
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    if (b < pr.nb(pb))
+                        bulk_copy(smem_addr(smem + L.x) + static_cast<uint32_t>(b) * static_cast<uint32_t>(pb.K),
+                                  pb.x + static_cast<int64_t>(xr[b]) * pb.K, static_cast<uint32_t>(pb.K), bar0 + 8u * kBarX);
+            }
+        }
         float run[NB];          // running sum of the current row block over this block's items
 #pragma unroll
         for (int b = 0; b < NB; ++b) run[b] = 0.f;
@@ -1160,6 +1178,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // where this lane leaves its partial sums inside a slot (one or two tokens)
     float *rd_lane = red + static_cast<uint32_t>(warp * NB) * kRows + lane;
     int kk = 0;                 // items decoded so far, over all segments
+    bool x_ready = false;
     do {
     token_fragments();
     // whole rows per item: this warp's group never changes, neither do its activation fragments
@@ -1260,6 +1279,16 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             // (interleaving them with the contraction's activation loads measured 20 % slower on the
             // five-trit path)
             if (!kMma) asm volatile("" ::: "memory");
+            if (kEarly && !x_ready) {
+                // first contraction of this warp: the previous kernel must be complete and the
+                // activations in place (the decode above needed neither)
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                if (!mbar_wait(bar0 + 8u * kBarX, 0)) {
+                    if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
+                    return;
+                }
+                x_ready = true;
+            }
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 if (kMma) break;
