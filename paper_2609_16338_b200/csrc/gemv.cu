@@ -908,8 +908,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // with one or two tokens (kEarly) the decoder warps do not either until they have decoded
     // their first tile: only the contraction needs the activations, which the epilogue warp
     // fetches into shared memory (one bulk copy per token) as soon as the dependency is resolved.
-    constexpr bool kEarly = Segs::kSingle && NB < kMmaMinBatch;
-    if (!kEarly) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // With four tokens and more (tensor-core path) the decoders fetch their activation fragments
+    // from global memory right after that first decode instead.
+    constexpr bool kLate = Segs::kSingle;                       // plain kernels: wait as late as possible
+    constexpr bool kEarly = kLate && NB < kMmaMinBatch;         // ... and activations copied by the epilogue warp
+    if (!kLate) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     Segs src = segs;
     bool have = src.next(pr, wk);
@@ -932,7 +935,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             xr[b] = pr.xrow(pb) ? __ldg(pr.xrow(pb) + bb) : bb;
         }
     };
-    if (have && !kEarly) token_rows();
+    if (have && !kLate) token_rows();
     const bool x_resident = L.x_bytes != 0;
     if (x_resident && have && !kEarly) {
         int4 *xs = reinterpret_cast<int4 *>(smem + L.x);
@@ -952,10 +955,10 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 
     // ------------------------------------------------------------------ epilogue warp
     if (warp == pl.NW + 1) {
-        if (kEarly) {
+        if (kLate) {
             asm volatile("griddepcontrol.wait;" ::: "memory");
             token_rows();
-            if (lane == 0) {
+            if (kEarly && lane == 0) {
                 mbar_expect_tx(bar0 + 8u * kBarX, static_cast<uint32_t>(pr.nb(pb)) * static_cast<uint32_t>(pb.K));
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
@@ -1180,9 +1183,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     int kk = 0;                 // items decoded so far, over all segments
     bool x_ready = false;
     do {
-    token_fragments();
-    // whole rows per item: this warp's group never changes, neither do its activation fragments
-    if (kMma && pl.CS == 1) load_bf(g_fixed);
+    if (!(kLate && kMma)) {
+        token_fragments();
+        // whole rows per item: this warp's group never changes, neither do its activation fragments
+        if (kMma && pl.CS == 1) load_bf(g_fixed);
+    }
     for (const int kk_end = kk + wk.count; kk < kk_end; ++kk) {
         if (!mbar_wait(full_bar, phase)) {
             if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
@@ -1197,7 +1202,8 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         float ysum[NV];
 #pragma unroll
         for (int b = 0; b < NV; ++b) ysum[b] = 0.f;
-        if (kMma && pl.CS != 1 && busy) load_bf(g);        // early, so that the decode hides the latency
+        // early, so that the decode hides the latency (not before the dependency is resolved)
+        if (kMma && pl.CS != 1 && busy && (!kLate || x_ready)) load_bf(g);
 
         if (busy) {
             const float sc = bf16_to_float(*reinterpret_cast<const uint16_t *>(stage + off_scale));
@@ -1232,6 +1238,14 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 const uint4 *src = reinterpret_cast<const uint4 *>(stage) + (warp * 2) * kRows + lane;
                 if (kMma) bit2_decode_row_s8(src[0], src[kRows], w);
                 else bit2_decode_row(src[0], src[kRows], w);
+            }
+            if (kLate && kMma && !x_ready) {
+                // first contraction of this warp: the previous kernel must be complete before the
+                // activations are read (the decode above did not need them)
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                token_fragments();
+                load_bf(g);
+                x_ready = true;
             }
             if (kMma) {
                 int acc[NH][2][4];
