@@ -888,9 +888,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         };
         bool have = src.next(pr, wk);
         while (have && wk.count <= 0) have = src.next(pr, wk);
+        // Only the first item goes out before the block-wide barrier: issuing a bulk copy costs this
+        // thread on the order of a hundred nanoseconds, and the other warps wait at that barrier.
         if (lane == 0 && have) {
             prime(true);
-            issue_loop(wk.count < pl.stages ? wk.count : pl.stages);
+            issue_loop(1);
         }
         __syncthreads();       // pairs with the barrier the other warps reach after staging the activations
         if (lane != 0 || !have) return;
