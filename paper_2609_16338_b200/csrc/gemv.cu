@@ -848,11 +848,6 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
                 issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows);
-                if (kk == 0 && FMT != kBit2) {
-                    mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
-                    bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
-                              bar0 + 8u * kBarLut);
-                }
                 r0 = r1; lo0 = lo1; hi0 = hi1;
                 r1 = r2; lo1 = lo2; hi1 = hi2;
                 if (++ps == pl.stages) {
@@ -888,6 +883,13 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         };
         bool have = src.next(pr, wk);
         while (have && wk.count <= 0) have = src.next(pr, wk);
+        // The lookup table first: it is the largest transfer of the start-up (64 KB from L2) and
+        // needs no address arithmetic.
+        if (lane == 0 && have && FMT != kBit2) {
+            mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
+            bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
+                      bar0 + 8u * kBarLut);
+        }
         // Only the first item goes out before the block-wide barrier: issuing a bulk copy costs this
         // thread on the order of a hundred nanoseconds, and the other warps wait at that barrier.
         if (lane == 0 && have) {
