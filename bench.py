@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # command: four launches per step (the default;
 # profiles/launch_list_and_dram_traffic_bitnet2b_layer_bench_default.md) and seven (--serial / --branches,
 # an earlier capture of the same kernels)
-NCU_DRAM_BYTES_PER_STEP = {4: 15297884, 7: 15627520}
+NCU_DRAM_BYTES_PER_STEP = {4: 15288018, 7: 15627520}
 
 
 def layer_config():
