@@ -40,9 +40,8 @@ UNIT = "us"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of all launches of one step, from ncu captures of this
-# command: four launches per step (the default;
-# profiles/launch_list_and_dram_traffic_bitnet2b_layer_bench_default.md) and seven (--serial / --branches,
-# an earlier capture of the same kernels)
+# command (summaries under profiles/): four launches per step (the default) and seven (--serial /
+# --branches, an earlier capture of the same kernels)
 NCU_DRAM_BYTES_PER_STEP = {4: 15288018, 7: 15627520}
 
 
