@@ -140,6 +140,15 @@ typedef struct bitcos_weights {
     const uint32_t *tile_off_host;
 } bitcos_weights;
 
+/* Stream ordering of the device entry points.  They enqueue on the caller's stream and return
+ * without waiting.  Kernels of this library are launched with programmatic stream serialization:
+ * when the previous kernel in the stream is also one of this library's, a call may start reading
+ * its PACKED WEIGHTS (and nothing else) while that kernel is still running; activations, activation
+ * scales, routing lists, outputs, accumulator dumps and workspaces are touched only after every
+ * earlier kernel in the stream has completed, as usual.  Kernels of this library never write packed
+ * weights, so ordinary use needs no extra care; after any other kernel or copy in the stream the
+ * usual order holds in full.  BITCOS_PDL=0 in the environment turns the overlap off. */
+
 /* Scratch memory the GEMV entry points need for an M x K matrix (the same value for all
  * formats and batches): a 256-byte header (word 0 = status), one arrival counter per row
  * block, and the partial row sums of reduction segments that were spread over several
