@@ -39,7 +39,7 @@ namespace {
 constexpr int kGroup = BITCOS_GROUP;
 constexpr int kRows = BITCOS_TILE_ROWS;
 constexpr int kMaxWarps = 20;             // warps per thread block = tiles per item
-constexpr int kWarps16 = 14;              // the same for more than 8 tokens (their partial sums need the room)
+constexpr int kWarps16 = 14;              // the same for more than 8 tokens (16 warps per block: 128 registers per thread)
 constexpr int kMaxStages = 8;             // upper bound on the shared-memory ring depth (Plan::stages)
 constexpr int kLutBytes = 64 * 1024;      // replicated lookup tables (BITCOS, five-trit)
 constexpr uint64_t kWaitLimitNs = 500ull * 1000 * 1000;   // an mbarrier wait gives up after half a second
@@ -193,8 +193,8 @@ struct GroupedArgs {
 
 inline int64_t padded_rows(int64_t M) { return (M + kRows - 1) / kRows * kRows; }
 
-// Decoder warps per thread block: 20, or 16 for more than 8 tokens (their partial sums would not
-// fit in shared memory otherwise).
+// Decoder warps per thread block: 20, or 14 for more than 8 tokens (the tensor-core path then holds
+// 16 accumulators and 16 activation fragments per lane; with 20 warps it spills).
 __host__ __device__ constexpr int decoder_warps(int batch) { return batch > 8 ? kWarps16 : kMaxWarps; }
 // Threads of the widest block an instantiation for up to nb tokens is launched with.
 __host__ __device__ constexpr int max_block_threads(int nb) { return (decoder_warps(nb) + 2) * 32; }
