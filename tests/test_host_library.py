@@ -144,3 +144,28 @@ def test_group_pairs_helper():
     order, ge, gb, xr, mx = bc.group_pairs([5, 2, 5, 7, 2, 5], [0, 0, 1, 1, 2, 2])
     assert list(ge) == [2, 5, 7] and list(gb) == [0, 2, 5, 6] and mx == 3
     assert list(xr) == [0, 2, 0, 1, 2, 1] and list(order) == [1, 4, 0, 2, 5, 3]
+
+
+def test_benchmark_byte_count_is_the_packed_size():
+    """The roofline's numerator (bench.algorithmic_bytes) is exactly what a product has to move:
+    the packed buffers as the packer sizes them (sign bits rounded up to bytes, no slack), the
+    activations with their scales, and the outputs; and it reproduces 2 - z bits per weight plus
+    the scale and entry-offset overheads (Eq. 1, Eq. 5)."""
+    import sys
+    sys.path.insert(0, ROOT)
+    import bench
+    for (M, K, z, B) in ((256, 512, 0.42, 1), (100, 1280, 0.3, 3), (640, 2560, 0.4219, 16)):
+        W, S = datagen.trits(77, M, K, z), datagen.scales(77, M, K)
+        p = bc.bitcos_pack(W, S)
+        Mp = (M + 31) // 32 * 32
+        tiles = Mp // 32 * (K // 128)
+        io = B * (K + 4) + 4 * B * M
+        assert bench.algorithmic_bytes(M, K, p.nnz, B) == p.bitmap.nbytes + (p.nnz + 7) // 8 + p.scales.nbytes + 4 * (tiles + 1) + io
+        assert p.payload_bytes() == bench.algorithmic_bytes(M, K, p.nnz, B) - io
+        # bits per weight of bitmap + signs = 2 - z_realised exactly (padding rows hold no weights)
+        z_real = 1.0 - p.nnz / float(M * K)
+        assert abs((Mp * K + p.nnz) / float(Mp * K) - (2.0 - z_real * M / Mp - (Mp - M) / Mp)) < 1e-12
+        t5 = bc.trit5_pack(W)
+        b2 = bc.bit2_pack(W)
+        assert bench.algorithmic_bytes(M, K, p.nnz, B, "trit5") == t5.nbytes + p.scales.nbytes + io
+        assert bench.algorithmic_bytes(M, K, p.nnz, B, "bit2") == b2.nbytes + p.scales.nbytes + io
