@@ -141,7 +141,8 @@ struct Plan {
     int CG;          // groups per column block
     int CS;          // column blocks per row
     int RBC;         // row blocks per item (1 unless CS == 1)
-    int NW;          // warps per thread block = CG * RBC
+    int NW;          // decoder warps per thread block = ceil(CG * RBC / tpw)
+    int tpw;         // tiles of an item per decoder warp: 1, or 2 on large matrices (one or two tokens)
     int64_t items;   // ceil(RB / RBC) * CS
     int cyclic;      // 1: blocks take whole row-block chunks round robin; 0: contiguous balanced ranges
     int stages;      // depth of the shared-memory ring (2 .. kMaxStages), set at launch
@@ -199,10 +200,12 @@ __host__ __device__ constexpr int decoder_warps(int batch) { return batch > 8 ? 
 // Threads of the widest block an instantiation for up to nb tokens is launched with.
 __host__ __device__ constexpr int max_block_threads(int nb) { return (decoder_warps(nb) + 2) * 32; }
 
-Plan make_plan(int64_t M, int64_t K, int max_warps) {
+Plan make_plan(int64_t M, int64_t K, int max_warps_per_block, int tpw = 1) {
     const int G = static_cast<int>(K / kGroup);
     const int64_t RB = padded_rows(M) / kRows;
     Plan p{};
+    p.tpw = tpw;
+    const int max_warps = max_warps_per_block * tpw;       // tiles an item may hold
     const int blocks = (G + max_warps - 1) / max_warps;
     p.CG = (G + blocks - 1) / blocks;
     p.CS = (G + p.CG - 1) / p.CG;
@@ -213,7 +216,7 @@ Plan make_plan(int64_t M, int64_t K, int max_warps) {
         if (r < 1) r = 1;
         p.RBC = static_cast<int>(r);
     }
-    p.NW = p.CG * p.RBC;
+    p.NW = (p.CG * p.RBC + tpw - 1) / tpw;
     p.items = ((RB + p.RBC - 1) / p.RBC) * p.CS;
     return p;
 }
@@ -265,11 +268,11 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     uint32_t off = 0;
     L.lut = off;
     off += (fmt == kBit2) ? 0 : kLutBytes;
-    const uint32_t tiles = static_cast<uint32_t>(pl.NW);
+    const uint32_t tiles = static_cast<uint32_t>(pl.NW * pl.tpw);
     if (fmt == kBitcos) {
         L.payload_cap = tiles * 512;
         L.sign_cap = tiles * 512 + 64;
-        L.off_cap = 128;                 // the item's slice of tile_off (at most 21 + 3 + 3 words)
+        L.off_cap = 192;                 // the item's slice of tile_off (at most 41 + 3 + 3 words)
     } else if (fmt == kTrit5) {
         const uint32_t WPR = (26u * static_cast<uint32_t>(G) + 3) / 4;
         // whole rows when CS == 1, else at most CG groups (+1 shared word) of one row block
@@ -292,9 +295,9 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
                     ? static_cast<uint32_t>(nbmax * K) : 0u;
     off += align_up(L.x_bytes, 128);
     L.red = off;
-    off += static_cast<uint32_t>(red_slots(nbmax)) * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
+    off += static_cast<uint32_t>(red_slots(nbmax) / pl.tpw) * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
     L.scr = off;
-    off += (nbmax >= kMmaMinBatch) ? tiles * kScrBytes : 0u;
+    off += (nbmax >= kMmaMinBatch) ? static_cast<uint32_t>(pl.NW) * kScrBytes : 0u;
     L.bar = off;
     off += 512;          // mbarriers, then (16-byte aligned) one 16-byte item descriptor per stage
     L.total = off;
@@ -780,7 +783,10 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // per stage: {tiles | (first tile & 3) << 8, first group, first row block, first sign bit held}
     uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 384);
     const uint32_t bar0 = smem_addr(smem + L.bar);
-    const uint32_t red_slot = static_cast<uint32_t>(pl.NW) * NB * kRows;     // floats per partial-sum slot
+    const uint32_t red_slot = static_cast<uint32_t>(pl.NW * pl.tpw) * NB * kRows;     // floats per partial-sum slot
+    // partial-sum slots in use: red_slots(NB), half as many (of twice the size) with two tiles per warp
+    const int rs_log2 = (red_slots(NB) == 8 ? 3 : red_slots(NB) == 4 ? 2 : 1) - (pl.tpw - 1);
+    const int rs_mask = (1 << rs_log2) - 1;
 
     // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as
     // every block of this one got here; whatever it reads from us it reads after its own
@@ -985,7 +991,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         constexpr int RS = red_slots(NB);
         // sum of n <= 20 partial sums of token b, spaced NB * 32 floats apart: all loads are issued
         // before the first addition, and the additions always follow the same tree
-        auto sum_groups = [&](const float *base, int n) {
+        auto sum_groups20 = [&](const float *base, int n) {
             float v[kMaxWarps];
 #pragma unroll
             for (int j = 0; j < kMaxWarps; ++j) v[j] = (j < n) ? base[j * NB * kRows] : 0.f;
@@ -994,6 +1000,12 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 #pragma unroll
                 for (int j = 0; j + w2 < kMaxWarps; j += 2 * w2) v[j] += v[j + w2];
             return v[0];
+        };
+        // (up to 40 partial sums when a warp decodes two tiles per item: two trees of 20)
+        auto sum_groups = [&](const float *base, int n) {
+            float t = sum_groups20(base, n);
+            if (n > kMaxWarps) t += sum_groups20(base + kMaxWarps * NB * kRows, n - kMaxWarps);
+            return t;
         };
         // tensor-core layout: the same for four tokens at a time, n <= 20 float4 spaced one warp's
         // rows apart, in two batches of ten to bound the registers in flight
@@ -1049,9 +1061,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             for (int b = 0; b < NB; ++b) xsc[NB < kMmaMinBatch ? b : 0] = __ldg(pb.x_scale + xr[b]);
         }
         for (int k = 0; k < wk.count; ++k, ++kk, it.next(pl, wk)) {
-            const int slot = kk % RS;
+            const int slot = kk & rs_mask;
             const ItemRange r = item_range(pb, pl, it.c, it.cs);
-            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((kk / RS) & 1))) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedFull + slot), static_cast<uint32_t>((kk >> rs_log2) & 1))) {
                 if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                 return;
             }
@@ -1120,9 +1132,13 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     }
 
     // ------------------------------------------------------------------ decoder warps
-    // CS == 1: this warp always has row block warp / G of the chunk and group warp % G
-    const int my_rbl = (pl.CS == 1) ? warp / pb.G : 0;
-    const int g_fixed = warp - my_rbl * pb.G;
+    // CS == 1: tile t of an item always is row block t / G of the chunk, group t % G; this warp
+    // decodes tile `warp` and, with two tiles per warp, tile `warp + NW`
+    const int tpw = (NB >= kMmaMinBatch) ? 1 : pl.tpw;
+    const int my_rbl0 = (pl.CS == 1) ? warp / pb.G : 0;
+    const int g_fixed0 = warp - my_rbl0 * pb.G;
+    const int my_rbl1 = (pl.CS == 1) ? (warp + pl.NW) / pb.G : 0;
+    const int g_fixed1 = warp + pl.NW - my_rbl1 * pb.G;
     if (FMT != kBit2) {
         if (!mbar_wait(bar0 + 8u * kBarLut, 0)) {
             if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
@@ -1134,7 +1150,6 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     constexpr int NH = NB > 8 ? 2 : 1;                 // 8-token halves of the batch
     constexpr int NV = kMma ? NH * 8 : NB;             // partial sums a lane hands to the epilogue warp
     const uint32_t lane4 = static_cast<uint32_t>(lane) * 4u;
-    const uint32_t tile_lane = static_cast<uint32_t>(warp * kRows + lane);
     // Tensor-core path.  The order of the 128 products inside a group is free, so it is chosen to
     // make the activation loads contiguous: of tokens lane / 4 and lane / 4 + 8 this lane holds
     // bytes 16 c .. 16 c + 15 and 64 + 16 c .. 64 + 16 c + 15 of the group (c = lane % 4, two 16-byte
@@ -1175,22 +1190,25 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     const uint4 *desc = reinterpret_cast<const uint4 *>(sign_base);
     uint32_t full_bar = bar0 + 8u * kBarFull, phase = 0;
     int s = 0;
-    // byte offsets inside a stage that do not change from item to item
-    const uint32_t off_bm = tile_lane * 16u;                                        // this lane's four presence words
-    const uint32_t off_scale = L.payload_cap + L.sign_cap + tile_lane * 2u;           // its row's group scale
-    const uint32_t off_toff = L.payload_cap + L.sign_cap + L.scale_cap + static_cast<uint32_t>(warp) * 4u;
+    // byte offsets inside a stage that do not change from item to item (first tile of this warp;
+    // the second one lies NW tiles further)
+    const uint32_t tile_lane0 = static_cast<uint32_t>(warp * kRows + lane);
+    const uint32_t off_bm0 = tile_lane0 * 16u;                                       // this lane's four presence words
+    const uint32_t off_scale0 = L.payload_cap + L.sign_cap + tile_lane0 * 2u;          // its row's group scale
+    const uint32_t off_toff0 = L.payload_cap + L.sign_cap + L.scale_cap + static_cast<uint32_t>(warp) * 4u;
     const uint32_t off_sign = L.payload_cap;
+    const uint32_t tile_step = static_cast<uint32_t>(pl.NW);
     const uint32_t off_x = L.payload_cap + L.sign_cap + L.scale_cap + L.off_cap;     // activations inside a stage
     const uint8_t *xs_base = smem + L.x;
     // where this lane leaves its partial sums inside a slot (one or two tokens)
-    float *rd_lane = red + static_cast<uint32_t>(warp * NB) * kRows + lane;
+    float *rd_lane0 = red + static_cast<uint32_t>(warp * NB) * kRows + lane;
     int kk = 0;                 // items decoded so far, over all segments
     bool x_ready = false;
     do {
     if (!(kLate && kMma)) {
         token_fragments();
         // whole rows per item: this warp's group never changes, neither do its activation fragments
-        if (kMma && pl.CS == 1) load_bf(g_fixed);
+        if (kMma && pl.CS == 1) load_bf(g_fixed0);
     }
     for (const int kk_end = kk + wk.count; kk < kk_end; ++kk) {
         if (!mbar_wait(full_bar, phase)) {
@@ -1199,11 +1217,29 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         }
         const uint4 d = desc[s];
         const int nt = static_cast<int>(d.x & 0xFFu);
-        const bool busy = warp < nt;
-        // group of this warp's tile: the item's first group (0 when items are whole rows) + the
-        // warp's place in its row block
-        const int g = static_cast<int>(d.y) + g_fixed;
+        const int slot = kk & rs_mask;
+        // Two tiles per warp: the partial sums of a tile are stored as soon as it is done, so the
+        // slot must be free before the first one (with one tile per warp that wait comes after
+        // the decode, further down).
+        if (tpw == 2 && (kk >> rs_log2) > 0) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>(((kk >> rs_log2) - 1) & 1))) {
+                if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
+                return;
+            }
+        }
         float ysum[NV];
+#pragma unroll 1
+        for (int ti = 0; ti < tpw; ++ti) {
+        const int tile = warp + (ti ? pl.NW : 0);
+        const bool busy = tile < nt;
+        const int my_rbl = ti ? my_rbl1 : my_rbl0;
+        // group of this tile: the item's first group (0 when items are whole rows) + the tile's
+        // place in its row block
+        const int g = static_cast<int>(d.y) + (ti ? g_fixed1 : g_fixed0);
+        const uint32_t t_off = ti ? tile_step : 0u;
+        const uint32_t off_bm = off_bm0 + t_off * (kRows * 16u);
+        const uint32_t off_scale = off_scale0 + t_off * (kRows * 2u);
+        const uint32_t off_toff = off_toff0 + t_off * 4u;
 #pragma unroll
         for (int b = 0; b < NV; ++b) ysum[b] = 0.f;
         // early, so that the decode hides the latency (not before the dependency is resolved)
@@ -1239,7 +1275,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 for (int i = 0; i < 7; ++i) wd[i] = src[i * kRows];
                 trit5_decode_row(wd, g & 1, lut, static_cast<uint32_t>(lane) * 8u, w);
             } else {
-                const uint4 *src = reinterpret_cast<const uint4 *>(stage) + (warp * 2) * kRows + lane;
+                const uint4 *src = reinterpret_cast<const uint4 *>(stage) + (tile * 2) * kRows + lane;
                 if (kMma) bit2_decode_row_s8(src[0], src[kRows], w);
                 else bit2_decode_row(src[0], src[kRows], w);
             }
@@ -1320,6 +1356,13 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 }
             }
         }
+        if (tpw == 2) {
+            // (one or two tokens only) this tile's partial sums, zeros if the item has no such tile
+#pragma unroll
+            for (int b = 0; b < NB; ++b)
+                if (!kMma) rd_lane0[slot * red_slot + (t_off * NB + b) * kRows] = ysum[b];
+        }
+        }
         // the stage has been read: hand it back to the producer
         __syncwarp();
         mbar_arrive_lane0(full_bar + 8u * kBarEmpty, lane);
@@ -1333,15 +1376,16 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         }
 
         // partial sums for the epilogue warp (several slots, so decoders may run ahead of it)
-        const int slot = kk & (RS - 1);
-        if (kk >= RS) {
-            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>((kk / RS - 1) & 1))) {
+        if (tpw == 1 && (kk >> rs_log2) > 0) {
+            if (!mbar_wait(bar0 + 8u * (kBarRedEmpty + slot), static_cast<uint32_t>(((kk >> rs_log2) - 1) & 1))) {
                 if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                 return;
             }
         }
         float *rd = red + slot * red_slot;
-        if (kMma) {
+        if (tpw == 2) {
+            // already stored, tile by tile
+        } else if (kMma) {
 #pragma unroll
             for (int i = 0; i < NV; i += 2) {
                 const int b = 8 * (i >> 3) + 2 * (lane & 3);                          // and b + 1
@@ -1352,7 +1396,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             }
         } else {
 #pragma unroll
-            for (int b = 0; b < NB; ++b) rd_lane[slot * red_slot + b * kRows] = ysum[b];
+            for (int b = 0; b < NB; ++b) rd_lane0[slot * red_slot + b * kRows] = ysum[b];
         }
         __syncwarp();
         mbar_arrive_lane0(bar0 + 8u * (kBarRedFull + slot), lane);
@@ -1716,13 +1760,22 @@ void fill_first_off(FirstOff &fo, int base, const uint32_t *off_host, const Prob
     }
 }
 
+// Large matrices, one or two tokens: items of twice the size, two tiles per decoder warp, so that
+// what a decoder warp does per item (barrier waits, descriptor, stage advance, hand-off of the
+// partial sums: about 50 of its 364 instructions per tile) is paid once per two tiles.  Only when
+// every block still gets several items.
+inline bool wants_two_tiles(const Plan &pl, int nb_template, int sms) {
+    return nb_template < kMmaMinBatch && pl.items >= 8 * static_cast<int64_t>(sms);
+}
+
 template <int FMT, int NB>
-int launch(const Problem &pr, const Plan &pl, cudaStream_t stream, const uint32_t *off_host = nullptr) {
+int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint32_t *off_host = nullptr) {
     // the one- and two-token instantiations keep the activations in shared memory (nb_bucket sees to it)
     if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * pr.K > kXResidentBytes) return BITCOS_ERR_SHAPE;
     int sms = 0, budget = 0;
     int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms, &budget);
     if (rc) return rc;
+    const Plan pl = wants_two_tiles(pl_in, NB, sms) ? make_plan(pr.M, pr.K, decoder_warps(pr.nb), 2) : pl_in;
     int grid = 1;
     Plan plw = pl;
     choose_walk(plw, small_launch_cap(pl.items, sms), &grid);

@@ -247,6 +247,32 @@ def test_host_buffer_entry_point(bc):
     assert (err <= REL * mag).all()
 
 
+def test_sampled_outputs_two_tiles_per_warp(bc):
+    """Matrices large enough for the plan with two tiles per decoder warp (eight or more items per
+    multiprocessor): whole rows in one item (K = 2560 and 5120) and rows cut in two column blocks
+    (K = 6912); one and two tokens; all three formats.  The oracle checks a sample of rows."""
+    for (M, K, B) in ((38016, 2560, 1), (38400, 2560, 2), (19200, 5120, 1), (12800, 6912, 2)):
+        z = 0.4219
+        W, S = datagen.trits(900 + K + B, M, K, z), datagen.scales(900 + K + B, M, K)
+        x, xs = datagen.activations(900 + K + B, B, K)
+        rows = np.unique(np.concatenate([np.arange(0, M, max(1, M // 211)), [M - 1, M - 32, M - 33, 31, 32, 63, 64]]))
+        acc_ref, y_ref, mag = oracle.gemv_dense(W[rows], S[rows], x, xs)
+        xd, xsd = dev(x), dev(xs)
+        ws = bc.make_workspace(M, K)
+        st = bc.scales_tile(S, M, K)
+        for fmt, Wd, f in (("bitcos", bc.bitcos_pack(W, S).to_device(), bc.bitcos_gemv),
+                           ("trit5", bc.plain_to_device(bc.trit5_pack(W), st, M, K), bc.trit5_gemv),
+                           ("bit2", bc.plain_to_device(bc.bit2_pack(W), st, M, K), bc.bit2_gemv)):
+            for rep in range(2):
+                y, acc = f(Wd, xd, xsd, acc_debug=True, workspace=ws)
+                torch.cuda.synchronize()
+                assert np.array_equal(acc.cpu().numpy()[:, rows], acc_ref), (fmt, M, K, B)
+                err = np.abs(y.cpu().numpy().astype(np.float64)[:, rows] - y_ref)
+                assert (err <= REL * mag).all(), (fmt, M, K, B)
+            assert bc.workspace_status(ws) == 0
+            del Wd
+
+
 def test_multi_host_buffer_entry_point(bc):
     """Several products from host buffers in one call: same results as the device entry point."""
     B = 2
