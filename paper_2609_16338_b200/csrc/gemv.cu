@@ -272,7 +272,7 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     if (fmt == kBitcos) {
         L.payload_cap = tiles * 512;
         L.sign_cap = tiles * 512 + 64;
-        L.off_cap = 192;                 // the item's slice of tile_off (at most 41 + 3 + 3 words)
+        L.off_cap = pl.tpw == 2 ? 192 : 128;   // the item's slice of tile_off (at most 21 or 41, + 3 + 3 words)
     } else if (fmt == kTrit5) {
         const uint32_t WPR = (26u * static_cast<uint32_t>(G) + 3) / 4;
         // whole rows when CS == 1, else at most CG groups (+1 shared word) of one row block
@@ -770,7 +770,7 @@ struct OneSegT {
 // wait is bounded, and there is no block-wide barrier inside the loop.
 // `segs` yields the problems this block works on, one after the other, with its share of each
 // one's items; the stage ring, the partial-sum slots and their barriers run on across them.
-template <int FMT, int NB, typename Segs>
+template <int FMT, int NB, int TPW, typename Segs>
 __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, uint8_t *smem, int block,
                                              const FirstOff *fo = nullptr, int fo_index = 0) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -783,10 +783,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // per stage: {tiles | (first tile & 3) << 8, first group, first row block, first sign bit held}
     uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 384);
     const uint32_t bar0 = smem_addr(smem + L.bar);
-    const uint32_t red_slot = static_cast<uint32_t>(pl.NW * pl.tpw) * NB * kRows;     // floats per partial-sum slot
+    static_assert(TPW == 1 || (TPW == 2 && NB < kMmaMinBatch), "two tiles per warp: one or two tokens only");
+    const uint32_t red_slot = static_cast<uint32_t>(pl.NW * TPW) * NB * kRows;     // floats per partial-sum slot
     // partial-sum slots in use: red_slots(NB), half as many (of twice the size) with two tiles per warp
-    const int rs_log2 = (red_slots(NB) == 8 ? 3 : red_slots(NB) == 4 ? 2 : 1) - (pl.tpw - 1);
-    const int rs_mask = (1 << rs_log2) - 1;
+    constexpr int rs_log2 = (red_slots(NB) == 8 ? 3 : red_slots(NB) == 4 ? 2 : 1) - (TPW - 1);
+    constexpr int rs_mask = (1 << rs_log2) - 1;
 
     // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as
     // every block of this one got here; whatever it reads from us it reads after its own
@@ -1004,7 +1005,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         // (up to 40 partial sums when a warp decodes two tiles per item: two trees of 20)
         auto sum_groups = [&](const float *base, int n) {
             float t = sum_groups20(base, n);
-            if (n > kMaxWarps) t += sum_groups20(base + kMaxWarps * NB * kRows, n - kMaxWarps);
+            if (TPW == 2 && n > kMaxWarps) t += sum_groups20(base + kMaxWarps * NB * kRows, n - kMaxWarps);
             return t;
         };
         // tensor-core layout: the same for four tokens at a time, n <= 20 float4 spaced one warp's
@@ -1134,7 +1135,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // ------------------------------------------------------------------ decoder warps
     // CS == 1: tile t of an item always is row block t / G of the chunk, group t % G; this warp
     // decodes tile `warp` and, with two tiles per warp, tile `warp + NW`
-    const int tpw = (NB >= kMmaMinBatch) ? 1 : pl.tpw;
+    constexpr int tpw = TPW;
     const int my_rbl0 = (pl.CS == 1) ? warp / pb.G : 0;
     const int g_fixed0 = warp - my_rbl0 * pb.G;
     const int my_rbl1 = (pl.CS == 1) ? (warp + pl.NW) / pb.G : 0;
@@ -1405,21 +1406,21 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 }
 
 // One problem, this block's share of its items.
-template <int FMT, int NB, bool DEBUG = true>
+template <int FMT, int NB, bool DEBUG = true, int TPW = 1>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
                                             const FirstOff *fo = nullptr, int fo_index = 0) {
     OneSegT<DEBUG> one;
     one.pr = &pr;
     one.wk = wk;
     one.used = false;
-    run_segments<FMT, NB>(one, pl, smem, block, fo, fo_index);
+    run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index);
 }
 
-template <int FMT, int NB>
+template <int FMT, int NB, int TPW = 1>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl,
                                                                         const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
-    run_problem<FMT, NB>(pr, pl, smem,
+    run_problem<FMT, NB, true, TPW>(pr, pl, smem,
                          block_walk(fo, static_cast<int>(blockIdx.x), pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                          static_cast<int>(blockIdx.x), &fo, static_cast<int>(blockIdx.x));
 }
@@ -1540,7 +1541,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(
     segs.lo = b * q + (b < rem ? b : rem);
     segs.hi = segs.lo + q + (b < rem ? 1 : 0);
     segs.grp = static_cast<int>(segs.lo / ipg);
-    run_segments<kBitcos, NB>(segs, pl, smem, static_cast<int>(b));
+    run_segments<kBitcos, NB, 1>(segs, pl, smem, static_cast<int>(b));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1763,9 +1764,9 @@ void fill_first_off(FirstOff &fo, int base, const uint32_t *off_host, const Prob
 // Large matrices, one or two tokens: items of twice the size, two tiles per decoder warp, so that
 // what a decoder warp does per item (barrier waits, descriptor, stage advance, hand-off of the
 // partial sums: about 50 of its 364 instructions per tile) is paid once per two tiles.  Only when
-// every block still gets several items.
+// every block still gets several items (three or more of the smaller ones: measured break-even).
 inline bool wants_two_tiles(const Plan &pl, int nb_template, int sms) {
-    return nb_template < kMmaMinBatch && pl.items >= 8 * static_cast<int64_t>(sms);
+    return nb_template < kMmaMinBatch && pl.items >= 3 * static_cast<int64_t>(sms);
 }
 
 template <int FMT, int NB>
@@ -1775,7 +1776,14 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     int sms = 0, budget = 0;
     int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms, &budget);
     if (rc) return rc;
-    const Plan pl = wants_two_tiles(pl_in, NB, sms) ? make_plan(pr.M, pr.K, decoder_warps(pr.nb), 2) : pl_in;
+    const bool two = wants_two_tiles(pl_in, NB, sms);
+    if constexpr (NB < kMmaMinBatch) {
+        if (two) {
+            rc = prepare_kernel<gemv_kernel<FMT, NB, 2>>(&sms, &budget);
+            if (rc) return rc;
+        }
+    }
+    const Plan pl = two ? make_plan(pr.M, pr.K, decoder_warps(pr.nb), 2) : pl_in;
     int grid = 1;
     Plan plw = pl;
     choose_walk(plw, small_launch_cap(pl.items, sms), &grid);
@@ -1785,6 +1793,9 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     fo.valid = (FMT == kBitcos && off_host) ? 1 : 0;
     fo.walks = 1;
     fill_first_off(fo, 0, off_host, pr, plw, grid);
+    if constexpr (NB < kMmaMinBatch) {
+        if (two) return launch_pdl(gemv_kernel<FMT, NB, 2>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
+    }
     return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
