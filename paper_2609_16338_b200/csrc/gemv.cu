@@ -1435,7 +1435,7 @@ struct MultiArgs {
     int n;
 };
 
-template <int NB>
+template <int NB, int TPW = 1>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma,
                                                                               const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -1445,7 +1445,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
     const Problem pr = ma.pr[j];
     // (the multi launch has no accumulator dump)
-    run_problem<kBitcos, NB, false>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
+    run_problem<kBitcos, NB, false, TPW>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
                              b - ma.first_block[j], &fo, b);
 }
 
@@ -1809,6 +1809,21 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     // share the multiprocessors between the problems in proportion to their item counts
     int64_t total_items = 0;
     for (int j = 0; j < ma.n; ++j) total_items += ma.pl[j].items;
+    // enough items altogether: every problem with two tiles per decoder warp
+    Plan all{};
+    all.items = total_items;
+    const bool two = wants_two_tiles(all, NB, sms);
+    if constexpr (NB < kMmaMinBatch) {
+        if (two) {
+            rc = prepare_kernel<gemv_multi_kernel<NB, 2>>(&sms, &budget);
+            if (rc) return rc;
+            total_items = 0;
+            for (int j = 0; j < ma.n; ++j) {
+                ma.pl[j] = make_plan(ma.pr[j].M, ma.pr[j].K, decoder_warps(NB), 2);
+                total_items += ma.pl[j].items;
+            }
+        }
+    }
     sms = small_launch_cap(total_items, sms);
     int nw = 0;
     uint32_t smem = 0;
@@ -1834,6 +1849,9 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
         next += grid;
     }
     ma.first_block[ma.n] = next;
+    if constexpr (NB < kMmaMinBatch) {
+        if (two) return launch_pdl(gemv_multi_kernel<NB, 2>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
+    }
     return launch_pdl(gemv_multi_kernel<NB>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
 }
 

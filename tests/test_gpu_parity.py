@@ -273,6 +273,39 @@ def test_sampled_outputs_two_tiles_per_warp(bc):
             del Wd
 
 
+def test_multi_launch_two_tiles_per_warp(bc):
+    """A multi launch with enough items altogether (three or more per multiprocessor) runs every
+    job with two tiles per decoder warp: jobs of different shapes, among them a small one, one
+    whose rows are cut into column blocks and one with a ragged last row block.  Sampled rows
+    against the oracle; every output written; the same bits from run to run."""
+    shapes = [(12800, 2560), (6400, 5120), (64, 2560), (3200, 6912), (1000, 5120), (4097, 2560)]
+    for B in (1, 2):
+        jobs, refs = [], []
+        for i, (M, K) in enumerate(shapes):
+            W, S = datagen.trits(1300 + i, M, K, 0.4219), datagen.scales(1300 + i, M, K)
+            x, xs = datagen.activations(1300 + i + B, B, K)
+            rows = np.unique(np.concatenate([np.arange(0, M, max(1, M // 97)), [M - 1, 0, 31, 32, 63]]))
+            refs.append((rows,) + tuple(oracle.gemv_dense(W[rows], S[rows], x, xs)))
+            y = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
+            jobs.append((bc.bitcos_pack(W, S).to_device(), dev(x), dev(xs), y, bc.make_workspace(M, K)))
+        for rep in range(2):
+            for j in jobs:
+                j[3].fill_(float("nan"))
+            bc.bitcos_gemv_multi(jobs)
+            torch.cuda.synchronize()
+            for (Wd, _, _, y, ws), (rows, acc_ref, y_ref, mag) in zip(jobs, refs):
+                yh = y.cpu().numpy().astype(np.float64)
+                assert np.isfinite(yh).all(), (Wd.M, Wd.K, B)
+                assert (np.abs(yh[:, rows] - y_ref) <= REL * mag).all(), (Wd.M, Wd.K, B)
+                assert bc.workspace_status(ws) == 0
+        # run to run the same bits (the order of the additions is fixed)
+        first = [j[3].clone() for j in jobs]
+        bc.bitcos_gemv_multi(jobs)
+        torch.cuda.synchronize()
+        for j, y0 in zip(jobs, first):
+            assert torch.equal(j[3], y0)
+
+
 def test_multi_host_buffer_entry_point(bc):
     """Several products from host buffers in one call: same results as the device entry point."""
     B = 2
