@@ -29,6 +29,7 @@ STREAM_SCALES = 1
 STREAM_X = 2
 STREAM_XS = 3
 STREAM_EXPERTS = 4
+STREAM_XF = 5
 
 _GOLD = np.uint64(0x9E3779B97F4A7C15)
 _STREAM_MUL = np.uint64(0xD1B54A32D192ED03)
@@ -99,6 +100,17 @@ def activations(seed: int, B: int, K: int) -> tuple[np.ndarray, np.ndarray]:
     a = 1.0 + 3.0 * uniform(seed, STREAM_XS, 0, B)
     xs = (a / 127.0).astype(np.float32)
     return x, xs
+
+
+def activations_bf16(seed: int, B: int, K: int, outlier_every: int = 97, outlier_gain: float = 24.0) -> np.ndarray:
+    """uint16 [B, K]: bf16 bit patterns of unquantised activations, roughly normal (a sum of
+    four uniforms, variance 1) with every `outlier_every`-th channel scaled up, the shape
+    transformer activations have (a few channels carry most of the range)."""
+    u = uniform(seed, STREAM_XF, 0, 4 * B * K).reshape(B * K, 4)
+    v = (u.sum(axis=1) - 2.0) * np.sqrt(3.0)
+    v = v.reshape(B, K)
+    gain = np.where(np.arange(K) % outlier_every == outlier_every // 2, outlier_gain, 1.0)
+    return f32_to_bf16_bits((v * gain[None, :]).astype(np.float32))
 
 
 def expert_choices(seed: int, tokens: int, n_experts: int, top_k: int) -> np.ndarray:

@@ -342,5 +342,56 @@ def grouped_dense(expert_W, expert_scales, pair_expert, pair_xrow, x, xs):
     return np.stack(accs), np.stack(ys), np.stack(mags)
 
 
+# --- activations quantised per group of 128 (Section III-C: the integer contraction) ---------------
+AMAX_FLOOR = np.float32(2.0 ** -100)
+
+
+def quantize_activations(x, group: int = GROUP):
+    """16- or 32-bit float activations [B, K] -> (int8 codes [B, K], float32 scales).
+
+    Section III-C only says that the integer path quantises the activations to int8 per group
+    of 128 and applies the scales once per group; the rule below is this build's reading of it
+    (symmetric absmax quantisation), taken in float32, the precision the kernel decides in:
+
+        a     = max(max |x| over the group, 2^-100)        (the floor keeps 127 / a finite)
+        scale = a / 127                                     (float32, round to nearest)
+        code  = rint(x * (127 / a))                         (float32 quotient and product, ties to even)
+
+    so that x ~ scale * code with |code| <= 127.  `group` = 128 gives scales [B, K / 128];
+    `group` = 0 takes the whole row as one group (one scale per token, [B]).
+    """
+    x = np.atleast_2d(np.asarray(x, dtype=np.float32))
+    B, K = x.shape
+    gs = K if group == 0 else group
+    if gs < 1 or K % gs:
+        raise ValueError("K must be a multiple of the group size")
+    xg = x.reshape(B, K // gs, gs)
+    a = np.maximum(np.abs(xg).max(axis=2), AMAX_FLOOR).astype(np.float32)
+    scale = (a / np.float32(127.0)).astype(np.float32)
+    inv = (np.float32(127.0) / a).astype(np.float32)
+    prod = (xg * inv[:, :, None]).astype(np.float32)
+    code = np.clip(np.rint(prod), -127, 127).astype(np.int8).reshape(B, K)
+    return code, (scale.reshape(B) if group == 0 else scale)
+
+
+def dense_y_group_scales(acc, scales, xs_g):
+    """y[b, m] = sum over groups g of  s[m, g] * xs_g[b, g] * acc[b, m, g]   in float64
+    (Section III-C: int32 group sums, weight and activation scale applied once per group);
+    also the sum of the absolute values of the terms, for the tolerance."""
+    acc = np.asarray(acc, np.int64)
+    B, M, G = acc.shape
+    s = (np.asarray(scales, np.uint16).reshape(M, G).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    xs_g = np.asarray(xs_g, np.float32).reshape(B, G).astype(np.float64)
+    terms = acc.astype(np.float64) * s[None, :, :] * xs_g[:, None, :]
+    return terms.sum(axis=2), np.abs(terms).sum(axis=2)
+
+
+def gemv_dense_group_scales(W, scales, x, xs_g):
+    """Dense definition with one activation scale per token and group: (acc, y, mag)."""
+    acc = dense_acc(W, x)
+    y, mag = dense_y_group_scales(acc, scales, xs_g)
+    return acc, y, mag
+
+
 def threads() -> int:
     return int(lib().o_threads())

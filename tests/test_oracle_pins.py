@@ -433,3 +433,159 @@ def test_generator_is_counter_based_and_has_the_stated_distribution():
     assert x.min() >= -127 and x.max() <= 127 and (xs > 0).all()
     ids = datagen.expert_choices(2, 16, 128, 8)
     assert all(len(set(r)) == 8 for r in ids) and ids.min() >= 0 and ids.max() < 128
+
+
+# --- Section III-C: activations quantised per group of 128, scales applied once per group ---------
+def _bf16(vals):
+    return datagen.bf16_bits_to_f32(datagen.f32_to_bf16_bits(np.asarray(vals, np.float32)))
+
+
+def test_quantiser_worked_examples():
+    """Two groups worked out by hand.  Largest magnitude 1: the factor is 127, and 0.5 lands on
+    the tie 63.5, which goes to the even 64.  Largest magnitude 127: the factor is 1, the scale
+    exactly 1, and the ties 0.5, 2.5, 126.5 go to the even 0, 2, 126, while 1.5 goes to 2."""
+    x = np.zeros((2, 128), np.float32)
+    x[0, :7] = [1.0, -0.5, 0.25, 0.0, 1.0 / 256, -1.0, 0.75]
+    x[1, 5:13] = [127.0, 0.5, 1.5, 2.5, -2.5, 126.5, -0.5, -1.5]
+    assert np.array_equal(_bf16(x), x)                    # all of them are bf16 values
+    q, s = oracle.quantize_activations(x)
+    assert q.dtype == np.int8 and s.dtype == np.float32 and s.shape == (2, 1)
+    assert q[0, :7].tolist() == [127, -64, 32, 0, 0, -127, 95] and not q[0, 7:].any()
+    assert q[1, 5:13].tolist() == [127, 0, 2, 2, -2, 126, 0, -2] and not q[1, :5].any() and not q[1, 13:].any()
+    assert s[1, 0] == np.float32(1.0)
+    assert s[0, 0] == np.float32(1.0) / np.float32(127.0) and abs(float(s[0, 0]) * 127 - 1) < 2.0 ** -23
+
+
+def _round_to_f32(fr):
+    """Nearest float32 (ties to even) of a rational of normal magnitude, in exact arithmetic."""
+    from fractions import Fraction
+    if fr == 0:
+        return Fraction(0)
+    e = 0
+    a = abs(fr)
+    while a >= 2:
+        a /= 2
+        e += 1
+    while a < 1:
+        a *= 2
+        e -= 1
+    quantum = Fraction(2) ** (e - 23)
+    return round(fr / quantum) * quantum               # round() of a Fraction: ties to even
+
+
+def test_quantiser_against_exact_rational_arithmetic():
+    """The stated rule carried out in exact rationals with explicit roundings, element by
+    element, on a few groups (with outliers, a tiny group and an all-zero group)."""
+    from fractions import Fraction
+    x = datagen.bf16_bits_to_f32(datagen.activations_bf16(31, 3, 256))
+    x[1, 128:] *= np.float32(2.0 ** -60)
+    x[2, :128] = 0
+    q, s = oracle.quantize_activations(x)
+    for b in range(3):
+        for g in range(2):
+            grp = [Fraction(float(v)) for v in x[b, 128 * g:128 * g + 128]]
+            a = max(max(abs(v) for v in grp), Fraction(2) ** -100)
+            scale = _round_to_f32(a / 127)
+            inv = _round_to_f32(Fraction(127) / a)
+            assert Fraction(float(s[b, g])) == scale
+            for k, v in enumerate(grp):
+                code = round(_round_to_f32(v * inv))
+                assert -127 <= code <= 127
+                assert int(q[b, 128 * g + k]) == code, (b, g, k)
+    assert not q[2, :128].any() and Fraction(float(s[2, 0])) == _round_to_f32(Fraction(2) ** -100 / 127)
+
+
+def test_quantiser_invariants():
+    B, K = 4, 1024
+    x = datagen.bf16_bits_to_f32(datagen.activations_bf16(32, B, K))
+    for group in (128, 0):
+        q, s = oracle.quantize_activations(x, group)
+        sg = s.reshape(B, -1)
+        gs = K // sg.shape[1]
+        xg, qg = x.reshape(B, -1, gs), q.reshape(B, -1, gs).astype(np.float64)
+        # reconstruction error at most half a step (plus the rounding of the float32 factor)
+        err = np.abs(xg.astype(np.float64) - qg * sg[:, :, None].astype(np.float64))
+        assert (err <= 0.5 * sg[:, :, None] * (1 + 2.0 ** -14)).all()
+        # the largest magnitude of every group gets code +-127, with its sign
+        am = np.abs(xg).argmax(axis=2)
+        top = np.take_along_axis(qg, am[:, :, None], 2)[:, :, 0]
+        assert np.array_equal(top, 127 * np.sign(np.take_along_axis(xg, am[:, :, None], 2)[:, :, 0]))
+        assert np.abs(q.astype(np.int32)).max() == 127
+        # odd symmetry, and scaling by a power of two moves only the scale
+        q2, s2 = oracle.quantize_activations(-x, group)
+        assert np.array_equal(q2, -q) and np.array_equal(s2, s)
+        q3, s3 = oracle.quantize_activations(x * np.float32(2.0 ** -9), group)
+        assert np.array_equal(q3, q) and np.array_equal(s3, s * np.float32(2.0 ** -9))
+    # groups do not see each other: swapping two groups swaps their codes and scales
+    q, s = oracle.quantize_activations(x)
+    xs = x.copy()
+    xs[:, 0:128], xs[:, 256:384] = x[:, 256:384], x[:, 0:128]
+    q4, s4 = oracle.quantize_activations(xs)
+    assert np.array_equal(q4[:, 0:128], q[:, 256:384]) and np.array_equal(s4[:, 0], s[:, 2])
+    assert np.array_equal(q4[:, 128:256], q[:, 128:256])
+    # one scale per token = one group as long as the row
+    q5, s5 = oracle.quantize_activations(x[:, :128], 0)
+    assert np.array_equal(q5, q[:, :128]) and np.array_equal(s5, s[:, 0])
+    with pytest.raises(ValueError):
+        oracle.quantize_activations(x[:, :100])
+
+
+def test_group_scale_product_bruteforce_and_special_cases():
+    rng = np.random.default_rng(33)
+    M, K, B = 5, 384, 2
+    G = K // 128
+    W = rng.integers(-1, 2, (M, K)).astype(np.int8)
+    S = datagen.scales(33, M, K)
+    Sf = datagen.bf16_bits_to_f32(S).astype(np.float64)
+    x = rng.integers(-127, 128, (B, K)).astype(np.int8)
+    xg = rng.uniform(0.001, 0.05, (B, G)).astype(np.float32)
+    acc, y, mag = oracle.gemv_dense_group_scales(W, S, x, xg)
+    for b in range(B):
+        for m in range(M):
+            tot, tot_abs = 0.0, 0.0
+            for g in range(G):
+                a = sum(int(W[m, k]) * int(x[b, k]) for k in range(128 * g, 128 * g + 128))
+                assert acc[b, m, g] == a
+                tot += Sf[m, g] * float(xg[b, g]) * a
+                tot_abs += abs(Sf[m, g] * float(xg[b, g]) * a)
+            assert y[b, m] == pytest.approx(tot, rel=1e-13, abs=1e-300)
+            assert mag[b, m] == pytest.approx(tot_abs, rel=1e-13)
+    # as a dense float64 matrix product of the two de-quantised operands
+    Wd = W.astype(np.float64) * np.repeat(Sf, 128, axis=1)
+    xd = x.astype(np.float64) * np.repeat(xg.astype(np.float64), 128, axis=1)
+    assert np.allclose(y, xd @ Wd.T, rtol=0, atol=1e-12 * mag.max())
+    # the same scale in every group: the per-token product
+    xs = np.array([0.02, 0.007], np.float32)
+    _, y1, m1 = oracle.gemv_dense(W, S, x, xs)
+    _, y2, m2 = oracle.gemv_dense_group_scales(W, S, x, np.repeat(xs[:, None], G, axis=1))
+    assert np.allclose(y1, y2, rtol=0, atol=1e-13 * m1.max()) and np.allclose(m1, m2, rtol=1e-13)
+    # a scale of zero removes its group; scaling one group's scale scales that group's term
+    xz = xg.copy()
+    xz[:, 1] = 0
+    _, y3, _ = oracle.gemv_dense_group_scales(W, S, x, xz)
+    x0 = x.copy()
+    x0[:, 128:256] = 0
+    _, y4, _ = oracle.gemv_dense_group_scales(W, S, x0, xg)
+    assert np.allclose(y3, y4, rtol=0, atol=1e-13 * mag.max())
+
+
+def test_quantised_product_stays_within_the_quantisation_bound():
+    """Quantise, multiply, compare with the product of the unquantised activations: every
+    weight of a group contributes an error of at most half a quantisation step."""
+    M, K, B = 64, 1024, 3
+    W = datagen.trits(34, M, K, 0.42)
+    S = datagen.scales(34, M, K)
+    Sf = datagen.bf16_bits_to_f32(S).astype(np.float64)
+    x = datagen.bf16_bits_to_f32(datagen.activations_bf16(34, B, K))
+    exact = x.astype(np.float64) @ (W.astype(np.float64) * np.repeat(Sf, 128, axis=1)).T
+    nnz = np.abs(W).reshape(M, K // 128, 128).sum(axis=2).astype(np.float64)
+    errs = {}
+    for group in (128, 0):
+        q, s = oracle.quantize_activations(x, group)
+        sg = s.reshape(B, -1) if group else np.repeat(s[:, None], K // 128, axis=1)
+        _, y, _ = oracle.gemv_dense_group_scales(W, S, q, sg)
+        bound = 0.5 * (1 + 2.0 ** -14) * np.einsum("mg,bg->bm", Sf * nnz, sg.astype(np.float64))
+        assert (np.abs(y - exact) <= bound + 1e-12).all()
+        errs[group] = np.sqrt(np.mean((y - exact) ** 2))
+    # with outlier channels, scales per group lose less than one scale per token
+    assert errs[128] < errs[0]
