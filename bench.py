@@ -428,6 +428,28 @@ def run_cuda(args):
                     for rep in replicas]
         one_launch_us = graph_time_us(torch, stream, lambda i: bc.bitcos_gemv_multi(all_jobs[i]), copies, launches=copies)
 
+    # ---- the layer pass with an activation quantiser in front of each of its four launches ----
+    # (bf16 activations -> int8 and one scale per token, then the fused launch that reads them)
+    with_quant_us = None
+    if not args.no_detail and not (args.serial or args.branches):
+        import datagen
+        xb, qx, qs = [], [], []
+        for gi, g in enumerate(groups):
+            K = layer[g[0]]["K"]
+            bits = datagen.activations_bf16(datagen.config_seed(1, 60 + gi), 1, K)
+            xb.append(torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16))
+            qx.append(torch.empty((1, K), dtype=torch.int8, device="cuda"))
+            qs.append(torch.empty((1,), dtype=torch.float32, device="cuda"))
+        multi_q = [[bc.MultiJobs([(rep[j], qx[gi], qs[gi], ys[j], wss[j]) for j in g]) for gi, g in enumerate(groups)]
+                   for rep in replicas]
+
+        def step_q(i):
+            for gi, mj in enumerate(multi_q[i]):
+                bc.bitcos_quantize_activations(xb[gi], 0, xq=qx[gi], x_scale=qs[gi])
+                bc.bitcos_gemv_multi(mj)
+
+        with_quant_us = graph_time_us(torch, stream, step_q, copies, launches=copies)
+
     # ---- per-shape detail: each format on each shape, rotated copies, CUDA graph of 64 launches ----
     detail = shape_detail(bc, torch, layer, host_packed, stream) if not args.no_detail else None
 
@@ -491,8 +513,15 @@ def run_cuda(args):
             "note": "all seven products of the layer in a single bitcos_gemv_multi launch: possible for independent "
                     "products only (in a decoder layer o follows attention over q, k, v and down follows gate and up), so "
                     "this is not the headline; it shows how much of the step is launch structure"}
+        if with_quant_us is not None:
+            line["layer_with_quantisers"] = {
+                "us": with_quant_us,
+                "note": "the timed step with bitcos_quantize_activations (bf16 -> int8, one scale per token) in front "
+                        "of each of its four launches: eight kernels per step, each overlapping its start-up with the "
+                        "kernel before it"}
         line["shapes"] = detail
         line["batch"] = batch_detail(bc, torch, stream)
+        line["activation_quant"] = quant_detail(bc, torch, stream)
     if args.all_configs:
         line["density_sweep"] = sweep_detail(bc, torch, stream)
         line["qwen32b_layer"] = qwen32b_layer_detail(bc, torch, stream)
@@ -649,6 +678,56 @@ def batch_detail(bc, torch, stream, M=8192, K=5120, z=0.4711):
                          "us_per_token": us / B}
             del reps
         out["rows"].append(row)
+        torch.cuda.empty_cache()
+    return out
+
+
+def quant_detail(bc, torch, stream):
+    """The quantised-activation front end: bf16 activations -> int8 quantiser (one scale per group
+    of 128, or per token) -> product, on two matrices at 1, 4 and 16 tokens.  `chain` is one
+    quantiser launch plus one product launch back to back on the stream (the product's start-up
+    overlaps the quantiser); `gemv` is the product alone on ready int8 activations."""
+    import datagen
+    out = []
+    for (M, K, z, ci) in ((2560, 6912, 0.4219, 1), (8192, 5120, 0.4711, 3)):
+        seed = datagen.config_seed(ci, 40)
+        W, S = datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)
+        packed = bc.bitcos_pack(W, S)
+        Wd = packed.to_device()
+        n_copies = max(2, int(np.ceil(4.2 * L2_BYTES / Wd.payload_bytes())))
+        reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
+        ws = bc.make_workspace(M, K)
+        G = K // 128
+        for B in (1, 4, 16):
+            xb = torch.from_numpy(datagen.activations_bf16(seed + B, B, K).view(np.int16)).cuda().view(torch.bfloat16)
+            q = torch.empty((B, K), dtype=torch.int8, device="cuda")
+            sg = torch.empty((B, G), dtype=torch.float32, device="cuda")
+            st = torch.empty((B,), dtype=torch.float32, device="cuda")
+            y = torch.empty((B, M), dtype=torch.float32, device="cuda")
+            bc.bitcos_quantize_activations(xb, 128, xq=q, x_scale=sg)
+            bc.bitcos_quantize_activations(xb, 0, xq=q, x_scale=st)
+            row = {"M": M, "K": K, "batch": B}
+            row["gemv_us"] = graph_time_us(torch, stream, lambda i: bc.bitcos_gemv(reps[i], q, st, y=y, workspace=ws), n_copies)
+            row["gemv_group_scales_us"] = graph_time_us(
+                torch, stream, lambda i: bc.bitcos_gemv_group_scales(reps[i], q, sg, y=y, workspace=ws), n_copies)
+            row["quantise_groups_us"] = graph_time_us(
+                torch, stream, lambda i: bc.bitcos_quantize_activations(xb, 128, xq=q, x_scale=sg), 1)
+            row["quantise_tokens_us"] = graph_time_us(
+                torch, stream, lambda i: bc.bitcos_quantize_activations(xb, 0, xq=q, x_scale=st), 1)
+
+            def chain_groups(i):
+                bc.bitcos_quantize_activations(xb, 128, xq=q, x_scale=sg)
+                bc.bitcos_gemv_group_scales(reps[i], q, sg, y=y, workspace=ws)
+
+            def chain_tokens(i):
+                bc.bitcos_quantize_activations(xb, 0, xq=q, x_scale=st)
+                bc.bitcos_gemv(reps[i], q, st, y=y, workspace=ws)
+
+            row["chain_groups_us"] = graph_time_us(torch, stream, chain_groups, n_copies)
+            row["chain_tokens_us"] = graph_time_us(torch, stream, chain_tokens, n_copies)
+            row["quantiser_bytes"] = int(B * K * 3 + 4 * B * G)
+            out.append(row)
+        del reps
         torch.cuda.empty_cache()
     return out
 

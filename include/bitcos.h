@@ -192,6 +192,29 @@ int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, 
 int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
                 int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Activation quantiser in front of the product.  Section III-C has the integer contraction
+ * quantise the activations to int8 per group of 128 and apply the scales once per group; the
+ * paper does not spell the rule out, and this library uses symmetric absmax quantisation, decided
+ * in float32:
+ *     a = max(max |x| over the group, 2^-100)     scale = a / 127     code = rint(x * (127 / a))
+ * (IEEE quotient and product, ties to even; |code| <= 127; an all-zero group gets codes 0).
+ *   x_bf16   device bf16 [batch][K] (bit patterns; finite values), 16-byte aligned
+ *   group    128: one scale per token and group of 128, x_scale = device float [batch][K/128]
+ *            0:   one scale per token (the whole row is one group), x_scale = device float [batch]
+ *   xq       device int8 [batch][K], 16-byte aligned, overwritten
+ * ERR_SHAPE for any other group, K not a multiple of 128, batch outside 1..BITCOS_MAX_BATCH.
+ * Stream ordered like the products: it waits for the kernel before it before reading x_bf16,
+ * and the product launched after it overlaps its own start-up with this kernel. */
+int bitcos_quantize_activations(const uint16_t *x_bf16, int batch, int64_t K, int group, int8_t *xq, float *x_scale,
+                                void *cuda_stream);
+
+/* bitcos_gemv with one activation scale per token and group of 128 (Section III-C):
+ *     y[b][m] = sum over groups g of  s[m][g] * x_group_scale[b][g] * (int32 sum over the group)
+ *   x_group_scale   device float [batch][K/128], e.g. from bitcos_quantize_activations(group = 128)
+ * Everything else as for bitcos_gemv (same accumulators, same workspace rules). */
+int bitcos_gemv_group_scales(const bitcos_weights *W, const int8_t *x, const float *x_group_scale, int batch, float *y,
+                             int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 #define BITCOS_MAX_JOBS 8
 
 /* Up to BITCOS_MAX_JOBS independent BITCOS products in ONE launch (same batch; shapes may differ): e.g. the

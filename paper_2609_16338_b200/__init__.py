@@ -23,6 +23,8 @@ from .binding import (  # noqa: F401
     bitcos_gemv_multi,
     MultiJobs,
     bitcos_gemv_multi_host,
+    bitcos_quantize_activations,
+    bitcos_gemv_group_scales,
     MultiHostJobs,
     bitcos_decode_probe,
     group_pairs,

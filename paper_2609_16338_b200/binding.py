@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "trit5_unpack", "bit2_pack_sizes", "bit2_pack", "bit2_unpack", "bitcos_gemv_workspace_bytes",
     "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
-    "bitcos_gemv_multi_host",
+    "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
 ]
 
 
@@ -97,6 +97,8 @@ def load_library():
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
+    L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
+    L.bitcos_gemv_group_scales.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, vp, sz, vp]
     _lib = L
     return L
 
@@ -314,6 +316,38 @@ def bitcos_gemv(W: DeviceBitcos, x, x_scale, y=None, acc_debug=None, workspace=N
                                       acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
                                       workspace.numel(), _stream()), "bitcos_gemv")
     return y, acc
+
+
+def bitcos_gemv_group_scales(W: DeviceBitcos, x, x_group_scale, y=None, acc_debug=None, workspace=None):
+    """bitcos_gemv with one activation scale per token and group of 128: x_group_scale float32 [batch, K / 128]."""
+    batch = x.shape[0]
+    if tuple(x_group_scale.shape) != (batch, W.K // 128):
+        raise ValueError("x_group_scale must be [batch, K / 128]")
+    if workspace is None:
+        workspace = make_workspace(W.M, W.K, x.device)
+    y, acc = _outputs(W.M, W.K, batch, y, acc_debug, x.device)
+    _check(load_library().bitcos_gemv_group_scales(C.byref(W.desc), x.data_ptr(), x_group_scale.data_ptr(), batch,
+                                                   y.data_ptr(), acc.data_ptr() if acc is not None else None,
+                                                   workspace.data_ptr(), workspace.numel(), _stream()),
+           "bitcos_gemv_group_scales")
+    return y, acc
+
+
+def bitcos_quantize_activations(x_bf16, group: int = 128, xq=None, x_scale=None):
+    """bf16 activations [batch, K] on the device -> (int8 codes [batch, K], float32 scales
+    [batch, K / 128] for group = 128, [batch] for group = 0)."""
+    import torch
+    if x_bf16.dtype != torch.bfloat16 or x_bf16.dim() != 2 or not x_bf16.is_contiguous():
+        raise ValueError("x_bf16 must be a contiguous bfloat16 [batch, K] tensor")
+    batch, K = x_bf16.shape
+    if xq is None:
+        xq = torch.empty((batch, K), dtype=torch.int8, device=x_bf16.device)
+    if x_scale is None:
+        shape = (batch,) if group == 0 else (batch, K // 128)
+        x_scale = torch.empty(shape, dtype=torch.float32, device=x_bf16.device)
+    _check(load_library().bitcos_quantize_activations(x_bf16.data_ptr(), batch, K, group, xq.data_ptr(),
+                                                      x_scale.data_ptr(), _stream()), "bitcos_quantize_activations")
+    return xq, x_scale
 
 
 def _plain_gemv(name, W: DevicePlain, x, x_scale, y, acc_debug, workspace):

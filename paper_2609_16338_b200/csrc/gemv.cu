@@ -724,7 +724,7 @@ struct Share {
 };
 
 // If this block's arrival was the last one: add the shares in slot order and write the outputs.
-template <int NB>
+template <int NB, bool XG>
 __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, const int (&xr)[NB], const Share &sh,
                                              int lane) {
     const unsigned int old = __shfl_sync(0xFFFFFFFFu, sh.old, 0);
@@ -737,7 +737,7 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
             float tot = 0.f;
             for (int j = 0; j < sh.sharers; ++j)
                 tot += __ldcg(pr.partial + ((static_cast<int64_t>(sh.rb) * pl.CS + j) * pr.nb + b) * kRows + lane);
-            if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = __ldg(pr.x_scale + xr[b]) * tot;
+            if (m < pr.M) pr.y[(pr.out_row0 + b) * pr.M + m] = XG ? tot : __ldg(pr.x_scale + xr[b]) * tot;
         }
     }
     if (lane == 0) pr.counters[sh.rb] = 0u;    // leave the counter ready for the next call
@@ -746,11 +746,12 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
 // What a thread block runs back to back: one problem and its share of the items (the plain
 // kernels), or the pieces of several groups (the grouped launch).  Every warp role walks its own
 // copy of the source.
-template <bool DEBUG>
+template <bool DEBUG, bool XG = false>
 struct OneSegT {
     typedef ParamView View;
     static constexpr bool kSingle = true;      // never more than one segment
     static constexpr bool kDebug = DEBUG;      // false: acc_debug is known to be NULL (no code for it)
+    static constexpr bool kGroupScales = XG;   // x_scale holds one scale per token AND group: [nb][G]
     const Problem *pr;
     Walk wk;
     bool used;
@@ -784,6 +785,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     uint32_t *sign_base = reinterpret_cast<uint32_t *>(smem + L.bar + 384);
     const uint32_t bar0 = smem_addr(smem + L.bar);
     static_assert(TPW == 1 || (TPW == 2 && NB < kMmaMinBatch), "two tiles per warp: one or two tokens only");
+    // one activation scale per token and group (applied by the decoder warps, tile by tile)
+    // instead of one per token (applied by the epilogue warp to the finished sums)
+    constexpr bool kXG = Segs::kGroupScales;
     const uint32_t red_slot = static_cast<uint32_t>(pl.NW * TPW) * NB * kRows;     // floats per partial-sum slot
     // partial-sum slots in use: red_slots(NB), half as many (of twice the size) with two tiles per warp
     constexpr int rs_log2 = (red_slots(NB) == 8 ? 3 : red_slots(NB) == 4 ? 2 : 1) - (TPW - 1);
@@ -984,7 +988,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         // per-token activation scales: kept in registers for up to two tokens, fetched where they
         // are used (a cached load per output block) for more
         float xsc[NB < kMmaMinBatch ? NB : 1] = {};
-        auto xscale = [&](int b) { return NB < kMmaMinBatch ? xsc[NB < kMmaMinBatch ? b : 0] : __ldg(pb.x_scale + xr[b]); };
+        auto xscale = [&](int b) {
+            return kXG ? 1.f : NB < kMmaMinBatch ? xsc[NB < kMmaMinBatch ? b : 0] : __ldg(pb.x_scale + xr[b]);
+        };
         Share pend[2];
         int n_pend = 0;
         ItemIter it;
@@ -1057,7 +1063,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         do {
         n_pend = 0;
         it.init(pl, wk.first);
-        if (NB < kMmaMinBatch) {
+        if (NB < kMmaMinBatch && !kXG) {
 #pragma unroll
             for (int b = 0; b < NB; ++b) xsc[NB < kMmaMinBatch ? b : 0] = __ldg(pb.x_scale + xr[b]);
         }
@@ -1125,7 +1131,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 pend[n_pend++] = sh;      // at most two per block: its first and its last row block
             }
         }
-        for (int i = 0; i < n_pend; ++i) finish_share<NB>(pb, pl, xr, pend[i], lane);
+        for (int i = 0; i < n_pend; ++i) finish_share<NB, kXG>(pb, pl, xr, pend[i], lane);
         have = next_segment();
         if (have) token_rows();
         } while (have);
@@ -1168,9 +1174,17 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         }
     };
     uint32_t bf[NH][8];
+    float xgq[NH][2];           // group scales of the two tokens whose accumulators this lane holds
     auto load_bf = [&](int g) {
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
+            if (kXG) {
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int b = 8 * h + 2 * (lane & 3) + r;
+                    xgq[h][r] = (b < pr.nb(pb)) ? __ldg(pb.x_scale + static_cast<int64_t>(b) * pb.G + g) : 0.f;
+                }
+            }
             int4 u0 = make_int4(0, 0, 0, 0), u1 = make_int4(0, 0, 0, 0);
             if (xfrag[h]) {
                 const int4 *px = reinterpret_cast<const int4 *>(xfrag[h] + static_cast<int64_t>(g) * kGroup);
@@ -1323,6 +1337,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
                             ysum[(h * 2 + mh) * 4 + r] = scq[2 * mh + (r >> 1)] * static_cast<float>(acc[h][mh][r]);
+                            if (kXG) ysum[(h * 2 + mh) * 4 + r] *= xgq[h][r & 1];
                             if (Segs::kDebug && pb.acc_debug) {
                                 const int b = 8 * h + 2 * (lane & 3) + (r & 1);
                                 const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + 16 * mh + (lane >> 2) + 8 * (r >> 1);
@@ -1344,12 +1359,21 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 }
                 x_ready = true;
             }
+            float xgs[NB < kMmaMinBatch ? NB : 1];
+            if (kXG && !kMma) {
+                // (after the dependency wait: the scales come from the kernel before this one)
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    if (NB == 1 || b < pr.nb(pb))
+                        xgs[NB < kMmaMinBatch ? b : 0] = __ldg(pb.x_scale + static_cast<int64_t>(b) * pb.G + g);
+            }
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 if (kMma) break;
                 if (NB == 1 || b < pr.nb(pb)) {       // a call has at least one token
                     const int a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pb.K), lane);
                     ysum[b] = sc * static_cast<float>(a);
+                    if (kXG) ysum[b] *= xgs[NB < kMmaMinBatch ? b : 0];
                     if (Segs::kDebug && pb.acc_debug) {
                         const int64_t m = (static_cast<int64_t>(d.z) + my_rbl) * kRows + lane;
                         if (m < pb.M) pb.acc_debug[((pr.out_row0(pb) + b) * pb.M + m) * pb.G + g] = a;
@@ -1406,21 +1430,21 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 }
 
 // One problem, this block's share of its items.
-template <int FMT, int NB, bool DEBUG = true, int TPW = 1>
+template <int FMT, int NB, bool DEBUG = true, int TPW = 1, bool XG = false>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
                                             const FirstOff *fo = nullptr, int fo_index = 0) {
-    OneSegT<DEBUG> one;
+    OneSegT<DEBUG, XG> one;
     one.pr = &pr;
     one.wk = wk;
     one.used = false;
     run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index);
 }
 
-template <int FMT, int NB, int TPW = 1>
+template <int FMT, int NB, int TPW = 1, bool XG = false>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl,
                                                                         const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
-    run_problem<FMT, NB, true, TPW>(pr, pl, smem,
+    run_problem<FMT, NB, true, TPW, XG>(pr, pl, smem,
                          block_walk(fo, static_cast<int>(blockIdx.x), pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                          static_cast<int>(blockIdx.x), &fo, static_cast<int>(blockIdx.x));
 }
@@ -1482,6 +1506,7 @@ struct GroupedSegs {
     typedef GroupView View;
     static constexpr bool kSingle = false;
     static constexpr bool kDebug = true;
+    static constexpr bool kGroupScales = false;
     __device__ __forceinline__ const Problem &shape() const { return *base; }
     __device__ __forceinline__ bool next(View &v, Walk &w) {
         while (lo < hi) {
@@ -1769,17 +1794,17 @@ inline bool wants_two_tiles(const Plan &pl, int nb_template, int sms) {
     return nb_template < kMmaMinBatch && pl.items >= 3 * static_cast<int64_t>(sms);
 }
 
-template <int FMT, int NB>
+template <int FMT, int NB, bool XG = false>
 int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint32_t *off_host = nullptr) {
     // the one- and two-token instantiations keep the activations in shared memory (nb_bucket sees to it)
     if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * pr.K > kXResidentBytes) return BITCOS_ERR_SHAPE;
     int sms = 0, budget = 0;
-    int rc = prepare_kernel<gemv_kernel<FMT, NB>>(&sms, &budget);
+    int rc = prepare_kernel<gemv_kernel<FMT, NB, 1, XG>>(&sms, &budget);
     if (rc) return rc;
     const bool two = wants_two_tiles(pl_in, NB, sms);
     if constexpr (NB < kMmaMinBatch) {
         if (two) {
-            rc = prepare_kernel<gemv_kernel<FMT, NB, 2>>(&sms, &budget);
+            rc = prepare_kernel<gemv_kernel<FMT, NB, 2, XG>>(&sms, &budget);
             if (rc) return rc;
         }
     }
@@ -1794,9 +1819,9 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     fo.walks = 1;
     fill_first_off(fo, 0, off_host, pr, plw, grid);
     if constexpr (NB < kMmaMinBatch) {
-        if (two) return launch_pdl(gemv_kernel<FMT, NB, 2>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
+        if (two) return launch_pdl(gemv_kernel<FMT, NB, 2, XG>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
     }
-    return launch_pdl(gemv_kernel<FMT, NB>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
+    return launch_pdl(gemv_kernel<FMT, NB, 1, XG>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
 template <int NB>
@@ -1863,14 +1888,14 @@ inline int nb_bucket(int batch, int64_t K) {
     return batch <= 1 ? 1 : batch <= 2 ? 2 : batch <= 4 ? 4 : batch <= 8 ? 8 : 16;
 }
 
-template <int FMT>
+template <int FMT, bool XG = false>
 int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream, const uint32_t *off_host) {
     const int nbk = nb_bucket(pr.nb, pr.K);
-    if (nbk == 1) return launch<FMT, 1>(pr, pl, stream, off_host);
-    if (nbk == 2) return launch<FMT, 2>(pr, pl, stream, off_host);
-    if (pr.nb <= 4) return launch<FMT, 4>(pr, pl, stream, off_host);
-    if (pr.nb <= 8) return launch<FMT, 8>(pr, pl, stream, off_host);
-    return launch<FMT, 16>(pr, pl, stream, off_host);
+    if (nbk == 1) return launch<FMT, 1, XG>(pr, pl, stream, off_host);
+    if (nbk == 2) return launch<FMT, 2, XG>(pr, pl, stream, off_host);
+    if (pr.nb <= 4) return launch<FMT, 4, XG>(pr, pl, stream, off_host);
+    if (pr.nb <= 8) return launch<FMT, 8, XG>(pr, pl, stream, off_host);
+    return launch<FMT, 16, XG>(pr, pl, stream, off_host);
 }
 
 template <int NB>
@@ -1947,7 +1972,7 @@ void fill_problem(Problem &pr, const uint32_t *payload, const uint32_t *signs, c
 int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const uint32_t *tile_off,
                 const uint16_t *scales, int64_t M, int64_t K, const int8_t *x, const float *x_scale, int batch,
                 float *y, int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream,
-                const uint32_t *off_host = nullptr) {
+                const uint32_t *off_host = nullptr, bool group_scales = false) {
     const int bad = check_common(fmt, payload, signs, tile_off, scales, M, K, x, x_scale, batch, y, acc_debug, workspace,
                                  workspace_bytes);
     if (bad) return bad;
@@ -1955,9 +1980,85 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
     Problem pr{};
     fill_problem(pr, payload, signs, tile_off, scales, M, K, x, x_scale, batch, y, acc_debug, workspace);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (group_scales) return fmt == kBitcos ? launch_nb<kBitcos, true>(pr, pl, stream, off_host) : BITCOS_ERR_SHAPE;
     if (fmt == kBitcos) return launch_nb<kBitcos>(pr, pl, stream, off_host);
     if (fmt == kTrit5) return launch_nb<kTrit5>(pr, pl, stream, nullptr);
     return launch_nb<kBit2>(pr, pl, stream, nullptr);
+}
+
+
+// ------------------------------------------------------------------ activation quantiser
+// bf16 activations -> int8 codes and float scales, one scale per group of 128 or per token:
+//   a = max(max |x| over the group, 2^-100),  scale = a / 127,  code = rint(x * (127 / a))
+// with IEEE float32 quotient and product and ties to even (the explicit intrinsics keep the
+// compiler from contracting or approximating them, so the codes do not depend on build flags).
+constexpr float kAmaxFloor = 7.888609052210118e-31f;      // 2^-100
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t quant_code(float x, float inv) {
+    int c = __float2int_rn(__fmul_rn(x, inv));
+    c = c > 127 ? 127 : (c < -127 ? -127 : c);
+    return static_cast<uint32_t>(c) & 0xFFu;
+}
+// the two values of a 32-bit word -> two codes in the low 16 bits
+__device__ __forceinline__ uint32_t quant_pair(uint32_t u, float inv) {
+    return quant_code(bf16_lo(u), inv) | (quant_code(bf16_hi(u), inv) << 8);
+}
+
+// One warp per group of 128: a lane holds four consecutive values.
+__global__ void __launch_bounds__(256) quantize_groups_kernel(const uint16_t *__restrict__ x, int8_t *__restrict__ q,
+                                                              float *__restrict__ scale, int64_t n_groups) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = static_cast<int64_t>(gridDim.x) * (blockDim.x >> 5);
+    for (int64_t grp = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); grp < n_groups; grp += warps) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(x + grp * kGroup) + lane);
+        float a = fmaxf(fmaxf(fabsf(bf16_lo(v.x)), fabsf(bf16_hi(v.x))), fmaxf(fabsf(bf16_lo(v.y)), fabsf(bf16_hi(v.y))));
+#pragma unroll
+        for (int d = 16; d; d >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, d));
+        a = fmaxf(a, kAmaxFloor);
+        const float inv = __fdiv_rn(127.0f, a);
+        reinterpret_cast<uint32_t *>(q + grp * kGroup)[lane] = quant_pair(v.x, inv) | (quant_pair(v.y, inv) << 16);
+        if (lane == 0) scale[grp] = __fdiv_rn(a, 127.0f);
+    }
+}
+
+// One thread block per token: largest magnitude of the row, then the codes (the row is read
+// twice, the second time from cache).
+constexpr int kQuantThreads = 512;
+__global__ void __launch_bounds__(kQuantThreads) quantize_tokens_kernel(const uint16_t *__restrict__ x, int8_t *__restrict__ q,
+                                                                        float *__restrict__ scale, int64_t K) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    __shared__ float warp_max[kQuantThreads / 32];
+    const int64_t row = blockIdx.x;
+    const uint4 *src = reinterpret_cast<const uint4 *>(x + row * K);      // eight values per load
+    const int64_t n = K / 8;
+    float a = 0.f;
+    for (int64_t i = threadIdx.x; i < n; i += kQuantThreads) {
+        const uint4 v = __ldg(src + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) a = fmaxf(a, fmaxf(fabsf(bf16_lo(w[j])), fabsf(bf16_hi(w[j]))));
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, d));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = a;
+    __syncthreads();
+    a = warp_max[0];
+#pragma unroll
+    for (int j = 1; j < kQuantThreads / 32; ++j) a = fmaxf(a, warp_max[j]);
+    a = fmaxf(a, kAmaxFloor);
+    const float inv = __fdiv_rn(127.0f, a);
+    uint2 *dst = reinterpret_cast<uint2 *>(q + row * K);
+    for (int64_t i = threadIdx.x; i < n; i += kQuantThreads) {
+        const uint4 v = __ldg(src + i);
+        dst[i] = make_uint2(quant_pair(v.x, inv) | (quant_pair(v.y, inv) << 16),
+                            quant_pair(v.z, inv) | (quant_pair(v.w, inv) << 16));
+    }
+    if (threadIdx.x == 0) scale[row] = __fdiv_rn(a, 127.0f);
 }
 
 }  // namespace
@@ -2073,6 +2174,29 @@ int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_
     if (rc) return rc;
     return gemv_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_scale, batch, y,
                        nullptr, ws, BITCOS_STATIC_WORKSPACE_BYTES, cuda_stream, W->tile_off_host);
+}
+
+int bitcos_quantize_activations(const uint16_t *x_bf16, int batch, int64_t K, int group, int8_t *xq, float *x_scale,
+                                void *cuda_stream) {
+    if (!x_bf16 || !xq || !x_scale) return BITCOS_ERR_NULL;
+    if (batch < 1 || batch > BITCOS_MAX_BATCH || K < kGroup || K % kGroup != 0) return BITCOS_ERR_SHAPE;
+    if (group != 0 && group != kGroup) return BITCOS_ERR_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(xq)) return BITCOS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (group == 0)
+        return launch_pdl(quantize_tokens_kernel, dim3(static_cast<unsigned>(batch)), kQuantThreads, 0, stream, x_bf16, xq,
+                          x_scale, K);
+    const int64_t n_groups = static_cast<int64_t>(batch) * (K / kGroup);
+    const int64_t blocks = (n_groups + 7) / 8;
+    return launch_pdl(quantize_groups_kernel, dim3(static_cast<unsigned>(blocks)), 256, 0, stream, x_bf16, xq, x_scale,
+                      n_groups);
+}
+
+int bitcos_gemv_group_scales(const bitcos_weights *W, const int8_t *x, const float *x_group_scale, int batch, float *y,
+                             int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!W) return BITCOS_ERR_NULL;
+    return gemv_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_group_scale, batch, y,
+                       acc_debug, workspace, workspace_bytes, cuda_stream, W->tile_off_host, true);
 }
 
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
