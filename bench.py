@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of all launches of one step, from ncu captures of this
 # command (summaries under profiles/): four launches per step (the default) and seven (--serial /
 # --branches, an earlier capture of the same kernels)
-NCU_DRAM_BYTES_PER_STEP = {4: 15288018, 7: 15627520}
+NCU_DRAM_BYTES_PER_STEP = {4: 15289129, 7: 15627520}
 
 
 def layer_config():
