@@ -120,6 +120,36 @@ int bit2_pack_sizes(int64_t M, int64_t K, size_t *bytes);
 int bit2_pack(const int8_t *trits, int64_t M, int64_t K, uint32_t *words);
 int bit2_unpack(const uint32_t *words, int64_t M, int64_t K, int8_t *trits_out);
 
+/* Which of the two compact formats stores an M x K matrix with nnz non-zero weights in fewer
+ * bytes (Section II-A: BITCOS spends 2 - z bits per weight and the five-trit format 26 bytes
+ * per 128 weights, so BITCOS wins above a zero density of 0.375; a tensor takes whichever rate
+ * it meets first).  All bytes a product reads are counted, entry offsets included.
+ * *format = 0 (BITCOS) or 1 (five-trit); the two byte counts are optional outputs. */
+int bitcos_choose_format(int64_t M, int64_t K, uint64_t nnz, int *format, size_t *bitcos_bytes, size_t *trit5_bytes);
+
+/* ---------------------------------------------------------------------------------------
+ * Device side: packing.  The same four BITCOS buffers as bitcos_pack writes, byte for byte, from
+ * trits and scales that are already in device memory (a checkpoint converted on the GPU).  A
+ * set-up path: both calls enqueue on the given stream and WAIT for it before they return (they
+ * report counts and errors to the host), so a product launched afterwards finds the packed
+ * weights complete.  scratch: BITCOS_PACK_SCRATCH_BYTES of device memory, 16-byte aligned.
+ * ------------------------------------------------------------------------------------- */
+#define BITCOS_PACK_SCRATCH_BYTES 256
+
+/* Number of non-zero weights of trits[M][K] (device, row major, int8); ERR_TRIT on a value
+ * outside {-1, 0, +1}.  Size the sign vector with bitcos_pack_sizes from it. */
+int bitcos_count_nnz_device(const int8_t *trits, int64_t M, int64_t K, uint64_t *nnz, void *scratch, void *cuda_stream);
+
+/* Packs trits[M][K] (device int8, row major) and scales_bf16[M][K/128] (device, row major) into
+ * the device buffers bitmap, signs (sign_capacity_bytes, zero filled here), tile_off and
+ * scales_tiled, all sized by bitcos_pack_sizes.  tile_off_host (optional): host buffer of the
+ * tile_off size receiving a copy (for bitcos_weights.tile_off_host).  nnz_out (optional, host).
+ * ERR_TRIT / ERR_SCALE / ERR_OVERFLOW as for bitcos_pack; ERR_CAPACITY if the sign vector does
+ * not fit (outputs are then incomplete). */
+int bitcos_pack_device(const int8_t *trits, const uint16_t *scales_bf16, int64_t M, int64_t K, uint32_t *bitmap,
+                       uint32_t *signs, size_t sign_capacity_bytes, uint32_t *tile_off, uint16_t *scales_tiled,
+                       uint32_t *tile_off_host, uint64_t *nnz_out, void *scratch, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------------------
  * Device side: the products.
  * ------------------------------------------------------------------------------------- */

@@ -25,6 +25,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
+    "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device",
 ]
 
 
@@ -98,6 +99,9 @@ def load_library():
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
     L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
+    L.bitcos_choose_format.argtypes = [i64, i64, u64, C.POINTER(C.c_int), psz, psz]
+    L.bitcos_count_nnz_device.argtypes = [vp, i64, i64, C.POINTER(u64), vp, vp]
+    L.bitcos_pack_device.argtypes = [vp, vp, i64, i64, vp, vp, sz, vp, vp, vp, C.POINTER(u64), vp, vp]
     L.bitcos_gemv_group_scales.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, vp, sz, vp]
     _lib = L
     return L
@@ -200,6 +204,54 @@ def bitcos_pack(trits, scales_bf16) -> PackedBitcos:
                          _ptr(scales), C.byref(out)), "bitcos_pack")
     n_tiles = (M + TILE_ROWS - 1) // TILE_ROWS * (K // GROUP)
     return PackedBitcos(M, K, int(out.value), bitmap, signs, tile_off_buf[:n_tiles + 1], scales, tile_off_buf)
+
+
+def bitcos_choose_format(M: int, K: int, nnz: int):
+    """('bitcos' or 'trit5', BITCOS bytes, five-trit bytes): the format that stores the matrix in fewer bytes."""
+    fmt, a, b = C.c_int(0), C.c_size_t(0), C.c_size_t(0)
+    _check(load_library().bitcos_choose_format(M, K, nnz, C.byref(fmt), C.byref(a), C.byref(b)), "bitcos_choose_format")
+    return ("bitcos", "trit5")[fmt.value], int(a.value), int(b.value)
+
+
+PACK_SCRATCH_BYTES = 256
+
+
+def bitcos_count_nnz_device(trits) -> int:
+    """Non-zero weights of an int8 [M, K] tensor in device memory (waits for the stream)."""
+    import torch
+    M, K = trits.shape
+    scratch = torch.empty(PACK_SCRATCH_BYTES, dtype=torch.uint8, device=trits.device)
+    nnz = C.c_uint64(0)
+    _check(load_library().bitcos_count_nnz_device(trits.data_ptr(), M, K, C.byref(nnz), scratch.data_ptr(), _stream()),
+           "bitcos_count_nnz_device")
+    return int(nnz.value)
+
+
+def bitcos_pack_device(trits, scales_bf16) -> "DeviceBitcos":
+    """Packs an int8 [M, K] tensor of trits and an int16/bfloat16 [M, K / 128] tensor of bf16 scales,
+    both in device memory, into a DeviceBitcos (with the host copy of tile_off) on the same device."""
+    import torch
+    L = load_library()
+    if trits.dtype != torch.int8 or trits.dim() != 2 or not trits.is_contiguous() or not scales_bf16.is_contiguous():
+        raise ValueError("trits must be a contiguous int8 [M, K] tensor, scales contiguous")
+    M, K = trits.shape
+    nnz = bitcos_count_nnz_device(trits)
+    sizes = [C.c_size_t(0) for _ in range(4)]
+    _check(L.bitcos_pack_sizes(M, K, nnz, *[C.byref(v) for v in sizes]), "bitcos_pack_sizes")
+    dev = trits.device
+    bitmap = torch.empty(sizes[0].value // 4, dtype=torch.int32, device=dev)
+    signs = torch.empty(sizes[1].value // 4, dtype=torch.int32, device=dev)
+    tile_off = torch.empty(sizes[2].value // 4, dtype=torch.int32, device=dev)
+    scales = torch.empty(sizes[3].value // 2, dtype=torch.int16, device=dev)
+    off_host = np.zeros(sizes[2].value // 4, np.uint32)
+    scratch = torch.empty(PACK_SCRATCH_BYTES, dtype=torch.uint8, device=dev)
+    out = C.c_uint64(0)
+    _check(L.bitcos_pack_device(trits.data_ptr(), scales_bf16.data_ptr(), M, K, bitmap.data_ptr(), signs.data_ptr(),
+                                sizes[1].value, tile_off.data_ptr(), scales.data_ptr(), _ptr(off_host), C.byref(out),
+                                scratch.data_ptr(), _stream()), "bitcos_pack_device")
+    n_tiles = (M + TILE_ROWS - 1) // TILE_ROWS * (K // GROUP)
+    return DeviceBitcos(M, K, int(out.value), bitmap, signs, tile_off, scales,
+                        tile_off_host=np.ascontiguousarray(off_host[:n_tiles + 1]))
 
 
 def bitcos_unpack(p: PackedBitcos) -> np.ndarray:

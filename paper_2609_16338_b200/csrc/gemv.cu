@@ -2063,6 +2063,11 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_tokens_kernel(const ui
 
 }  // namespace
 
+namespace bitcos_detail {
+// for the library's other translation units: the error bitcos_last_cuda_error reports
+void record_cuda_error(int e) { g_last_cuda_error = e; }
+}  // namespace bitcos_detail
+
 extern "C" {
 
 int bitcos_last_cuda_error(void) { return g_last_cuda_error; }

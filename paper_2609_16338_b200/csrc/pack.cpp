@@ -117,6 +117,25 @@ int bitcos_pack_sizes(int64_t M, int64_t K, uint64_t nnz, size_t *bitmap_bytes, 
     return BITCOS_OK;
 }
 
+int bitcos_choose_format(int64_t M, int64_t K, uint64_t nnz, int *format, size_t *bitcos_bytes, size_t *trit5_bytes) {
+    if (!format) return BITCOS_ERR_NULL;
+    size_t bm = 0, sg = 0, off = 0, t5 = 0;
+    int rc = bitcos_pack_sizes(M, K, nnz, &bm, &sg, &off, nullptr);
+    if (rc) return rc;
+    rc = trit5_pack_sizes(M, K, &t5);
+    if (rc) return rc;
+    // what a product reads: the sign bits themselves (not the vector's alignment slack) and the
+    // entry offsets without their padding; the scales are the same in both formats
+    const size_t n_tiles = static_cast<size_t>(padded_rows(M) / kRows) * static_cast<size_t>(K / kGroup);
+    const size_t bc = bm + static_cast<size_t>((nnz + 7) / 8) + (n_tiles + 1) * 4;
+    (void)sg;
+    (void)off;
+    *format = bc <= t5 ? 0 : 1;
+    if (bitcos_bytes) *bitcos_bytes = bc;
+    if (trit5_bytes) *trit5_bytes = t5;
+    return BITCOS_OK;
+}
+
 int bitcos_count_nnz(const int8_t *trits, int64_t M, int64_t K, uint64_t *nnz) {
     if (!trits || !nnz) return BITCOS_ERR_NULL;
     if (!shape_ok(M, K)) return BITCOS_ERR_SHAPE;

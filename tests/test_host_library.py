@@ -169,3 +169,26 @@ def test_benchmark_byte_count_is_the_packed_size():
         b2 = bc.bit2_pack(W)
         assert bench.algorithmic_bytes(M, K, p.nnz, B, "trit5") == t5.nbytes + p.scales.nbytes + io
         assert bench.algorithmic_bytes(M, K, p.nnz, B, "bit2") == b2.nbytes + p.scales.nbytes + io
+
+
+def test_choose_format_breaks_even_near_three_eighths():
+    """Section II-A: 2 - z bits per weight against 26 bytes per 128 weights (1.625 bits) break even
+    at z = 0.375; with the entry offsets counted (32 bits per 4096 weights) a little above it.
+    The byte counts are those of the oracle's packed buffers."""
+    M, K = 256, 1024
+    for z in (0.30, 0.36, 0.40, 0.47):
+        W = datagen.trits(77, M, K, z)
+        pk = oracle.bitcos_pack(W)
+        fmt, b_bytes, t_bytes = bc.bitcos_choose_format(M, K, pk.nnz)
+        assert b_bytes == pk.bitmap.nbytes + (pk.nnz + 7) // 8 + pk.tile_off.nbytes
+        assert t_bytes == oracle.trit5_pack(W).nbytes
+        assert fmt == ("bitcos" if b_bytes <= t_bytes else "trit5")
+        assert fmt == ("bitcos" if z >= 0.40 else "trit5")
+    # the exact crossing: bits per weight 2 - z + 32/4096 (+ the last offset) against 1.625
+    n = M * K
+    nnz_even = n - int(round(0.375 * n))
+    assert bc.bitcos_choose_format(M, K, nnz_even)[0] == "trit5"                  # offsets tip it
+    nnz_cross = n - int(np.ceil((0.375 + 32.0 / 4096) * n + 32))
+    assert bc.bitcos_choose_format(M, K, nnz_cross)[0] == "bitcos"
+    with pytest.raises(bc.BitcosError):
+        bc.bitcos_choose_format(M, 100, 5)
