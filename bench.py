@@ -525,6 +525,7 @@ def run_cuda(args):
     if args.all_configs:
         line["density_sweep"] = sweep_detail(bc, torch, stream)
         line["qwen32b_layer"] = qwen32b_layer_detail(bc, torch, stream)
+        line["device_pack"] = pack_detail(bc, torch)
     if args.moe or args.all_configs:
         line["moe"] = moe_detail(bc, torch, stream)
     print(json.dumps(line))
@@ -728,6 +729,34 @@ def quant_detail(bc, torch, stream):
             row["quantiser_bytes"] = int(B * K * 3 + 4 * B * G)
             out.append(row)
         del reps
+        torch.cuda.empty_cache()
+    return out
+
+
+def pack_detail(bc, torch):
+    """Device-side packing (set-up path): int8 trits + bf16 scales in device memory -> the BITCOS
+    buffers.  Wall time of the whole call (count pass, three kernels, two stream waits), against
+    the bytes it has to move once: the trits in, the packed buffers out."""
+    import time
+    import datagen
+    peak, _ = measured_peaks()
+    out = []
+    for (M, K, z, ci) in ((8192, 5120, 0.4711, 3), (25600, 5120, 0.4711, 3)):
+        seed = datagen.config_seed(ci, 50)
+        W, S = datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)
+        Wt, St = torch.from_numpy(W).cuda(), torch.from_numpy(S.view(np.int16)).cuda()
+        Wd = bc.bitcos_pack_device(Wt, St)
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(5):
+            t0 = time.perf_counter()
+            Wd = bc.bitcos_pack_device(Wt, St)
+            times.append((time.perf_counter() - t0) * 1e6)
+        us = float(np.median(times))
+        nbytes = M * K + S.nbytes + Wd.payload_bytes()
+        out.append({"M": M, "K": K, "us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
+                    "bytes_once": int(nbytes), "note": "the trits are read three times (count, bitmap, signs)"})
+        del Wt, St, Wd
         torch.cuda.empty_cache()
     return out
 

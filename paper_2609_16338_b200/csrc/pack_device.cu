@@ -37,14 +37,15 @@ inline int64_t padded_rows(int64_t M) { return (M + kRows - 1) / kRows * kRows; 
 
 // Presence and negative masks of the four bytes of a word (bit i <-> byte i), and whether all
 // four are in {-1, 0, +1}.
+__device__ __forceinline__ uint32_t byte_tops(uint32_t m) {
+    // bits 7, 15, 23, 31 -> bits 0..3 (the four partial products land on distinct bits: no carries)
+    return ((m & 0x80808080u) * 0x00204081u) >> 28;
+}
 __device__ __forceinline__ void masks4(uint32_t w, uint32_t &pres, uint32_t &neg, bool &ok) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t b = (w >> (8 * i)) & 0xFFu;
-        pres |= static_cast<uint32_t>(b != 0u) << i;
-        neg |= static_cast<uint32_t>(b == 0xFFu) << i;
-        ok = ok && (b == 0u || b == 1u || b == 0xFFu);
-    }
+    const uint32_t zero = __vcmpeq4(w, 0u), one = __vcmpeq4(w, 0x01010101u), minus = __vcmpeq4(w, 0xFFFFFFFFu);
+    pres |= byte_tops(~zero);
+    neg |= byte_tops(minus);
+    ok = ok && ((zero | one | minus) == 0xFFFFFFFFu);
 }
 
 // The 128 weights of (row m, group g) as four presence words and four negative words (bit i of
@@ -149,15 +150,24 @@ __global__ void __launch_bounds__(kScanThreads) scan_counts_kernel(uint32_t *__r
 // The bits of `src` at the set positions of `mask`, packed towards bit 0 (the inverse of the
 // deposit of Fig. 4).
 __device__ __forceinline__ uint32_t extract_bits(uint32_t src, uint32_t mask) {
-    uint32_t out = 0u;
-    int k = 0;
-    while (mask) {
-        const uint32_t low = mask & (0u - mask);
-        out |= static_cast<uint32_t>((src & low) != 0u) << k;
-        ++k;
-        mask &= mask - 1u;
+    // parallel-suffix compress: in round i every selected bit moves right by 2^i if the number of
+    // unselected positions below it has bit i set (five rounds for 32 bits)
+    uint32_t x = src & mask, m = mask;
+    uint32_t mk = ~m << 1;                       // the unselected positions, moved up by one: what lies below each bit
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        uint32_t mp = mk ^ (mk << 1);            // prefix parity of mk
+        mp ^= mp << 2;
+        mp ^= mp << 4;
+        mp ^= mp << 8;
+        mp ^= mp << 16;
+        const uint32_t mv = mp & m;              // bits to move in this round
+        m = (m ^ mv) | (mv >> (1 << i));
+        const uint32_t t = x & mv;
+        x = (x ^ t) | (t >> (1 << i));
+        mk &= ~mp;
     }
-    return out;
+    return x;
 }
 
 // Kernel 3: the sign vector.  Row r of tile t owns the bits [tile_off[t] + (non-zeros of rows
