@@ -843,7 +843,8 @@ def run_profile_batch(args):
     from paper_2609_16338_b200 import build as lib_build
     lib_build.build()
     bc.load_library()
-    M, K, z, B = 8192, 5120, 0.4711, args.profile_batch
+    M, K = (int(v) for v in args.profile_shape.split("x"))
+    z, B = 0.4711, args.profile_batch
     seed = datagen.config_seed(3, 0)
     W, S = datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)
     packed = bc.bitcos_pack(W, S)
@@ -930,6 +931,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA graphs (for profilers)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--profile-shape", default="8192x5120", metavar="MxK",
+                    help="matrix of --profile-batch (default: the batch table's q projection)")
     ap.add_argument("--profile-batch", type=int, default=0, metavar="B",
                     help="only launch bitcos_gemv at batch B on the batch table's matrix, --steps times (for profilers)")
     ap.add_argument("--all-configs", action="store_true",

@@ -1789,9 +1789,11 @@ void fill_first_off(FirstOff &fo, int base, const uint32_t *off_host, const Prob
 // Large matrices, one or two tokens: items of twice the size, two tiles per decoder warp, so that
 // what a decoder warp does per item (barrier waits, descriptor, stage advance, hand-off of the
 // partial sums: about 50 of its 364 instructions per tile) is paid once per two tiles.  Only when
-// every block still gets several items (three or more of the smaller ones: measured break-even).
+// every block still gets several items: from eight of the one-tile items per multiprocessor on.  (Between
+// three and eight the gain depends on the shape and the format: 8192x5120 -3 % at one token but +6 % at
+// two, 4096x12288 +3 %, 2-bit +3 %; so those keep one tile per warp.)
 inline bool wants_two_tiles(const Plan &pl, int nb_template, int sms) {
-    return nb_template < kMmaMinBatch && pl.items >= 3 * static_cast<int64_t>(sms);
+    return nb_template < kMmaMinBatch && pl.items >= 8 * static_cast<int64_t>(sms);
 }
 
 template <int FMT, int NB, bool XG = false>

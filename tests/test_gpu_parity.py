@@ -248,7 +248,7 @@ def test_host_buffer_entry_point(bc):
 
 
 def test_sampled_outputs_two_tiles_per_warp(bc):
-    """Matrices large enough for the plan with two tiles per decoder warp (three or more items per
+    """Matrices large enough for the plan with two tiles per decoder warp (eight or more items per
     multiprocessor): whole rows in one item (K = 2560 and 5120) and rows cut in two column blocks
     (K = 6912); one and two tokens; all three formats.  The oracle checks a sample of rows."""
     for (M, K, B) in ((38016, 2560, 1), (38400, 2560, 2), (19200, 5120, 1), (12800, 6912, 2)):
@@ -274,7 +274,7 @@ def test_sampled_outputs_two_tiles_per_warp(bc):
 
 
 def test_multi_launch_two_tiles_per_warp(bc):
-    """A multi launch with enough items altogether (three or more per multiprocessor) runs every
+    """A multi launch with enough items altogether (eight or more per multiprocessor) runs every
     job with two tiles per decoder warp: jobs of different shapes, among them a small one, one
     whose rows are cut into column blocks and one with a ragged last row block.  Sampled rows
     against the oracle; every output written; the same bits from run to run."""
