@@ -430,7 +430,7 @@ def run_cuda(args):
 
     # ---- the layer pass with an activation quantiser in front of each of its four launches ----
     # (bf16 activations -> int8 and one scale per token, then the fused launch that reads them)
-    with_quant_us = None
+    with_quant_us = fused_quant_us = None
     if not args.no_detail and not (args.serial or args.branches):
         import datagen
         xb, qx, qs = [], [], []
@@ -449,6 +449,15 @@ def run_cuda(args):
                 bc.bitcos_gemv_multi(mj)
 
         with_quant_us = graph_time_us(torch, stream, step_q, copies, launches=copies)
+        # the same with the quantiser inside the products (scales per group of 128): four launches
+        multi_b = [[bc.MultiJobs([(rep[j], xb[gi], None, ys[j], wss[j]) for j in g]) for gi, g in enumerate(groups)]
+                   for rep in replicas]
+
+        def step_b(i):
+            for mj in multi_b[i]:
+                bc.bitcos_gemv_multi_bf16(mj)
+
+        fused_quant_us = graph_time_us(torch, stream, step_b, copies, launches=copies)
 
     # ---- per-shape detail: each format on each shape, rotated copies, CUDA graph of 64 launches ----
     detail = shape_detail(bc, torch, layer, host_packed, stream) if not args.no_detail else None
@@ -518,7 +527,10 @@ def run_cuda(args):
                 "us": with_quant_us,
                 "note": "the timed step with bitcos_quantize_activations (bf16 -> int8, one scale per token) in front "
                         "of each of its four launches: eight kernels per step, each overlapping its start-up with the "
-                        "kernel before it"}
+                        "kernel before it",
+                "fused_us": fused_quant_us,
+                "fused_note": "bitcos_gemv_multi_bf16: the same four launches as the timed step, reading bf16 activations "
+                              "and quantising them per group of 128 inside the decoder warps"}
         line["shapes"] = detail
         line["batch"] = batch_detail(bc, torch, stream)
         line["activation_quant"] = quant_detail(bc, torch, stream)
@@ -699,7 +711,7 @@ def quant_detail(bc, torch, stream):
         reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
         ws = bc.make_workspace(M, K)
         G = K // 128
-        for B in (1, 4, 16):
+        for B in (1, 2, 4, 16):
             xb = torch.from_numpy(datagen.activations_bf16(seed + B, B, K).view(np.int16)).cuda().view(torch.bfloat16)
             q = torch.empty((B, K), dtype=torch.int8, device="cuda")
             sg = torch.empty((B, G), dtype=torch.float32, device="cuda")
@@ -724,6 +736,10 @@ def quant_detail(bc, torch, stream):
                 bc.bitcos_quantize_activations(xb, 0, xq=q, x_scale=st)
                 bc.bitcos_gemv(reps[i], q, st, y=y, workspace=ws)
 
+            if B <= 2:
+                # the quantiser inside the product's thread blocks (one and two tokens)
+                row["gemv_bf16_us"] = graph_time_us(
+                    torch, stream, lambda i: bc.bitcos_gemv_bf16(reps[i], xb, y=y, workspace=ws), n_copies)
             row["chain_groups_us"] = graph_time_us(torch, stream, chain_groups, n_copies)
             row["chain_tokens_us"] = graph_time_us(torch, stream, chain_tokens, n_copies)
             row["quantiser_bytes"] = int(B * K * 3 + 4 * B * G)

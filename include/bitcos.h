@@ -245,6 +245,16 @@ int bitcos_quantize_activations(const uint16_t *x_bf16, int batch, int64_t K, in
 int bitcos_gemv_group_scales(const bitcos_weights *W, const int8_t *x, const float *x_group_scale, int batch, float *y,
                              int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The quantiser fused into the product, for one or two tokens: x_bf16 = device bf16 [batch][K]
+ * (bit patterns, 16-byte aligned); every decoder warp quantises the group of 128 its tile
+ * multiplies (the rule of bitcos_quantize_activations, group = 128) and applies the group's
+ * scale, so the result is exactly that of bitcos_quantize_activations followed by
+ * bitcos_gemv_group_scales, without the separate launch and without the int8 copy in memory.
+ * ERR_SHAPE for batch > 2 (use the two calls) and for rows too long for the one- and two-token
+ * kernels (batch * K > 49152).  Everything else as for bitcos_gemv. */
+int bitcos_gemv_bf16(const bitcos_weights *W, const uint16_t *x_bf16, int batch, float *y, int32_t *acc_debug,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 #define BITCOS_MAX_JOBS 8
 
 /* Up to BITCOS_MAX_JOBS independent BITCOS products in ONE launch (same batch; shapes may differ): e.g. the
@@ -263,6 +273,9 @@ typedef struct bitcos_gemv_job {
     size_t workspace_bytes;
 } bitcos_gemv_job;
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
+/* The same with 16-bit activations quantised inside the launch (see bitcos_gemv_bf16): every
+ * job's x points to device bf16 [batch][K], x_scale is ignored (may be NULL); batch 1 or 2. */
+int bitcos_gemv_multi_bf16(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
 
 /* The same product as bitcos_gemv without a caller-provided workspace.  (The paper has no
  * counterpart: this entry point exists for the library's users, not for the method.)

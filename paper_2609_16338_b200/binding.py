@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_workspace_init", "bitcos_workspace_status", "bitcos_gemv", "trit5_gemv", "bit2_gemv", "bitcos_gemv_grouped",
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
-    "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device",
+    "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
 ]
 
 
@@ -99,6 +99,8 @@ def load_library():
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
     L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
+    L.bitcos_gemv_bf16.argtypes = [C.POINTER(_Weights), vp, C.c_int, vp, vp, vp, sz, vp]
+    L.bitcos_gemv_multi_bf16.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_choose_format.argtypes = [i64, i64, u64, C.POINTER(C.c_int), psz, psz]
     L.bitcos_count_nnz_device.argtypes = [vp, i64, i64, C.POINTER(u64), vp, vp]
     L.bitcos_pack_device.argtypes = [vp, vp, i64, i64, vp, vp, sz, vp, vp, vp, C.POINTER(u64), vp, vp]
@@ -385,6 +387,21 @@ def bitcos_gemv_group_scales(W: DeviceBitcos, x, x_group_scale, y=None, acc_debu
     return y, acc
 
 
+def bitcos_gemv_bf16(W: DeviceBitcos, x_bf16, y=None, acc_debug=None, workspace=None):
+    """The product from bfloat16 activations [batch, K] (batch 1 or 2), quantised per group of 128 inside the launch."""
+    import torch
+    if x_bf16.dtype != torch.bfloat16 or x_bf16.dim() != 2 or not x_bf16.is_contiguous():
+        raise ValueError("x_bf16 must be a contiguous bfloat16 [batch, K] tensor")
+    batch = x_bf16.shape[0]
+    if workspace is None:
+        workspace = make_workspace(W.M, W.K, x_bf16.device)
+    y, acc = _outputs(W.M, W.K, batch, y, acc_debug, x_bf16.device)
+    _check(load_library().bitcos_gemv_bf16(C.byref(W.desc), x_bf16.data_ptr(), batch, y.data_ptr(),
+                                           acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
+                                           workspace.numel(), _stream()), "bitcos_gemv_bf16")
+    return y, acc
+
+
 def bitcos_quantize_activations(x_bf16, group: int = 128, xq=None, x_scale=None):
     """bf16 activations [batch, K] on the device -> (int8 codes [batch, K], float32 scales
     [batch, K / 128] for group = 128, [batch] for group = 0)."""
@@ -472,8 +489,8 @@ class MultiJobs:
     def __init__(self, jobs):
         self.keep = jobs
         self.batch = jobs[0][1].shape[0]
-        self.arr = (_Job * len(jobs))(*[_Job(C.addressof(W.desc), x.data_ptr(), xs.data_ptr(), y.data_ptr(),
-                                             ws.data_ptr(), ws.numel()) for (W, x, xs, y, ws) in jobs])
+        self.arr = (_Job * len(jobs))(*[_Job(C.addressof(W.desc), x.data_ptr(), xs.data_ptr() if xs is not None else None,
+                                             y.data_ptr(), ws.data_ptr(), ws.numel()) for (W, x, xs, y, ws) in jobs])
 
 
 def bitcos_gemv_multi(jobs):
@@ -481,6 +498,14 @@ def bitcos_gemv_multi(jobs):
     (W, x, x_scale, y, workspace) tuples with a common batch size."""
     mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
     _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")
+    return [j[3] for j in mj.keep]
+
+
+def bitcos_gemv_multi_bf16(jobs):
+    """bitcos_gemv_multi with bfloat16 activations quantised inside the launch: jobs = MultiJobs or a list of
+    (W, x_bf16, None, y, workspace) tuples, batch 1 or 2."""
+    mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
+    _check(load_library().bitcos_gemv_multi_bf16(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi_bf16")
     return [j[3] for j in mj.keep]
 
 

@@ -293,7 +293,11 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
     // (the tensor-core path takes its activation fragments straight from global memory)
     L.x_bytes = (nbmax < kMmaMinBatch && !pl.x_in_stage && static_cast<int64_t>(nbmax) * K <= kXResidentBytes)
                     ? static_cast<uint32_t>(nbmax * K) : 0u;
-    off += align_up(L.x_bytes, 128);
+    // (at least 128 bytes per decoder warp and token: the products that take 16-bit activations
+    // quantise each warp's group into its own slice of this area)
+    uint32_t x_area = L.x_bytes;
+    if (L.x_bytes && x_area < static_cast<uint32_t>(pl.NW * nbmax * kGroup)) x_area = static_cast<uint32_t>(pl.NW * nbmax * kGroup);
+    off += align_up(x_area, 128);
     L.red = off;
     off += static_cast<uint32_t>(red_slots(nbmax) / pl.tpw) * tiles * static_cast<uint32_t>(nbmax) * kRows * 4;
     L.scr = off;
@@ -513,6 +517,23 @@ __device__ __forceinline__ int contract(const int (&w)[32], const int4 *xg, int 
         }
         return (a0 + a1) + (a2 + a3);
     }
+}
+
+// Activation quantiser arithmetic (used by the quantiser kernels and by the products that take
+// 16-bit activations): a = max(max |x| over the group, 2^-100), scale = a / 127,
+// code = rint(x * (127 / a)), IEEE float32 quotient and product, ties to even.
+constexpr float kAmaxFloor = 7.888609052210118e-31f;      // 2^-100
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t quant_code(float x, float inv) {
+    int c = __float2int_rn(__fmul_rn(x, inv));
+    c = c > 127 ? 127 : (c < -127 ? -127 : c);
+    return static_cast<uint32_t>(c) & 0xFFu;
+}
+// the two values of a 32-bit word -> two codes in the low 16 bits
+__device__ __forceinline__ uint32_t quant_pair(uint32_t u, float inv) {
+    return quant_code(bf16_lo(u), inv) | (quant_code(bf16_hi(u), inv) << 8);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -746,12 +767,13 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
 // What a thread block runs back to back: one problem and its share of the items (the plain
 // kernels), or the pieces of several groups (the grouped launch).  Every warp role walks its own
 // copy of the source.
-template <bool DEBUG, bool XG = false>
+template <bool DEBUG, bool XG = false, bool XQ = false>
 struct OneSegT {
     typedef ParamView View;
     static constexpr bool kSingle = true;      // never more than one segment
     static constexpr bool kDebug = DEBUG;      // false: acc_debug is known to be NULL (no code for it)
     static constexpr bool kGroupScales = XG;   // x_scale holds one scale per token AND group: [nb][G]
+    static constexpr bool kQuantize = XQ;      // x holds bf16 activations: quantised per group of 128 by the decoder warps
     const Problem *pr;
     Walk wk;
     bool used;
@@ -787,7 +809,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     static_assert(TPW == 1 || (TPW == 2 && NB < kMmaMinBatch), "two tiles per warp: one or two tokens only");
     // one activation scale per token and group (applied by the decoder warps, tile by tile)
     // instead of one per token (applied by the epilogue warp to the finished sums)
-    constexpr bool kXG = Segs::kGroupScales;
+    constexpr bool kXQ = Segs::kQuantize;                      // (one or two tokens only)
+    constexpr bool kXG = Segs::kGroupScales || kXQ;
+    static_assert(!kXQ || NB < kMmaMinBatch, "16-bit activations: one or two tokens only");
     const uint32_t red_slot = static_cast<uint32_t>(pl.NW * TPW) * NB * kRows;     // floats per partial-sum slot
     // partial-sum slots in use: red_slots(NB), half as many (of twice the size) with two tiles per warp
     constexpr int rs_log2 = (red_slots(NB) == 8 ? 3 : red_slots(NB) == 4 ? 2 : 1) - (TPW - 1);
@@ -973,7 +997,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         if (kLate) {
             asm volatile("griddepcontrol.wait;" ::: "memory");
             token_rows();
-            if (kEarly && lane == 0) {
+            if (kEarly && !kXQ && lane == 0) {
                 mbar_expect_tx(bar0 + 8u * kBarX, static_cast<uint32_t>(pr.nb(pb)) * static_cast<uint32_t>(pb.K));
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
@@ -1178,7 +1202,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     auto load_bf = [&](int g) {
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
-            if (kXG) {
+            if (kXG && !kXQ) {
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
                     const int b = 8 * h + 2 * (lane & 3) + r;
@@ -1219,6 +1243,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     float *rd_lane0 = red + static_cast<uint32_t>(warp * NB) * kRows + lane;
     int kk = 0;                 // items decoded so far, over all segments
     bool x_ready = false;
+    // 16-bit activations: the group this warp has quantised last, its scales, and its buffer
+    // ([token][128] int8 inside the activation area)
+    int q_g = -1;
+    float q_scale[NB < kMmaMinBatch ? NB : 1] = {};
+    uint32_t *q_scr = reinterpret_cast<uint32_t *>(smem + L.x) + static_cast<uint32_t>(warp) * (NB * kRows);
     do {
     if (!(kLate && kMma)) {
         token_fragments();
@@ -1259,12 +1288,26 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         for (int b = 0; b < NV; ++b) ysum[b] = 0.f;
         // early, so that the decode hides the latency (not before the dependency is resolved)
         if (kMma && pl.CS != 1 && busy && (!kLate || x_ready)) load_bf(g);
+        // 16-bit activations of a group this warp has not quantised yet: fetched ahead of the decode too
+        uint2 qv[NB < kMmaMinBatch ? NB : 1];
+        bool q_have = false;
+        auto fetch_group = [&]() {
+#pragma unroll
+            for (int b = 0; b < NB; ++b)
+                if (NB == 1 || b < pr.nb(pb))
+                    qv[NB < kMmaMinBatch ? b : 0] =
+                        __ldg(reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(pb.x) + static_cast<int64_t>(b) * pb.K +
+                                                              static_cast<int64_t>(g) * kGroup) + lane);
+            q_have = true;
+        };
+        if (kXQ && busy && x_ready && g != q_g) fetch_group();
 
         if (busy) {
             const float sc = bf16_to_float(*reinterpret_cast<const uint16_t *>(stage + off_scale));
             // activations of group g (one or two tokens: always in shared memory)
             // (only the grouped launch ever delivers activations with the stage)
-            const uint8_t *xs = ((!Segs::kSingle && pl.x_in_stage) ? stage + off_x : xs_base) + static_cast<uint32_t>(g) * kGroup;
+            const uint8_t *xs = kXQ ? reinterpret_cast<const uint8_t *>(q_scr)
+                                    : ((!Segs::kSingle && pl.x_in_stage) ? stage + off_x : xs_base) + static_cast<uint32_t>(g) * kGroup;
             int w[32];
             if (FMT == kBitcos) {
                 const uint4 bm = *reinterpret_cast<const uint4 *>(stage + off_bm);
@@ -1353,14 +1396,39 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 // first contraction of this warp: the previous kernel must be complete and the
                 // activations in place (the decode above needed neither)
                 asm volatile("griddepcontrol.wait;" ::: "memory");
-                if (!mbar_wait(bar0 + 8u * kBarX, 0)) {
+                if (!kXQ && !mbar_wait(bar0 + 8u * kBarX, 0)) {
                     if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                     return;
                 }
                 x_ready = true;
             }
+            if (kXQ && g != q_g) {
+                // 16-bit activations: this warp quantises the group its tile multiplies (four values
+                // per lane, largest magnitude by shuffles) into its own 128 bytes per token
+                if (!q_have) fetch_group();        // (first tile: the dependency has only just been resolved)
+                __syncwarp();                     // the previous tile's contraction has read the buffer
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    if (NB == 1 || b < pr.nb(pb)) {
+                        const uint2 v = qv[NB < kMmaMinBatch ? b : 0];
+                        float a = fmaxf(fmaxf(fabsf(bf16_lo(v.x)), fabsf(bf16_hi(v.x))),
+                                        fmaxf(fabsf(bf16_lo(v.y)), fabsf(bf16_hi(v.y))));
+#pragma unroll
+                        for (int dd = 16; dd; dd >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, dd));
+                        a = fmaxf(a, kAmaxFloor);
+                        const float inv = __fdiv_rn(127.0f, a);
+                        q_scale[NB < kMmaMinBatch ? b : 0] = __fdiv_rn(a, 127.0f);
+                        q_scr[b * kRows + lane] = quant_pair(v.x, inv) | (quant_pair(v.y, inv) << 16);
+                    }
+                }
+                __syncwarp();
+                q_g = g;
+            }
             float xgs[NB < kMmaMinBatch ? NB : 1];
-            if (kXG && !kMma) {
+            if (kXQ) {
+#pragma unroll
+                for (int b = 0; b < NB; ++b) xgs[NB < kMmaMinBatch ? b : 0] = q_scale[NB < kMmaMinBatch ? b : 0];
+            } else if (kXG && !kMma) {
                 // (after the dependency wait: the scales come from the kernel before this one)
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
@@ -1371,7 +1439,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             for (int b = 0; b < NB; ++b) {
                 if (kMma) break;
                 if (NB == 1 || b < pr.nb(pb)) {       // a call has at least one token
-                    const int a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * pb.K), lane);
+                    const int a = contract<FMT>(w, reinterpret_cast<const int4 *>(xs + static_cast<uint32_t>(b) * (kXQ ? static_cast<uint32_t>(kGroup) : static_cast<uint32_t>(pb.K))), lane);
                     ysum[b] = sc * static_cast<float>(a);
                     if (kXG) ysum[b] *= xgs[NB < kMmaMinBatch ? b : 0];
                     if (Segs::kDebug && pb.acc_debug) {
@@ -1430,21 +1498,21 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 }
 
 // One problem, this block's share of its items.
-template <int FMT, int NB, bool DEBUG = true, int TPW = 1, bool XG = false>
+template <int FMT, int NB, bool DEBUG = true, int TPW = 1, bool XG = false, bool XQ = false>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
                                             const FirstOff *fo = nullptr, int fo_index = 0) {
-    OneSegT<DEBUG, XG> one;
+    OneSegT<DEBUG, XG, XQ> one;
     one.pr = &pr;
     one.wk = wk;
     one.used = false;
     run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index);
 }
 
-template <int FMT, int NB, int TPW = 1, bool XG = false>
+template <int FMT, int NB, int TPW = 1, bool XG = false, bool XQ = false>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl,
                                                                         const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
-    run_problem<FMT, NB, true, TPW, XG>(pr, pl, smem,
+    run_problem<FMT, NB, true, TPW, XG, XQ>(pr, pl, smem,
                          block_walk(fo, static_cast<int>(blockIdx.x), pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                          static_cast<int>(blockIdx.x), &fo, static_cast<int>(blockIdx.x));
 }
@@ -1459,7 +1527,7 @@ struct MultiArgs {
     int n;
 };
 
-template <int NB, int TPW = 1>
+template <int NB, int TPW = 1, bool XQ = false>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma,
                                                                               const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -1469,7 +1537,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
     const Problem pr = ma.pr[j];
     // (the multi launch has no accumulator dump)
-    run_problem<kBitcos, NB, false, TPW>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
+    run_problem<kBitcos, NB, false, TPW, false, XQ>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
                              b - ma.first_block[j], &fo, b);
 }
 
@@ -1507,6 +1575,7 @@ struct GroupedSegs {
     static constexpr bool kSingle = false;
     static constexpr bool kDebug = true;
     static constexpr bool kGroupScales = false;
+    static constexpr bool kQuantize = false;
     __device__ __forceinline__ const Problem &shape() const { return *base; }
     __device__ __forceinline__ bool next(View &v, Walk &w) {
         while (lo < hi) {
@@ -1796,17 +1865,17 @@ inline bool wants_two_tiles(const Plan &pl, int nb_template, int sms) {
     return nb_template < kMmaMinBatch && pl.items >= 8 * static_cast<int64_t>(sms);
 }
 
-template <int FMT, int NB, bool XG = false>
+template <int FMT, int NB, bool XG = false, bool XQ = false>
 int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint32_t *off_host = nullptr) {
     // the one- and two-token instantiations keep the activations in shared memory (nb_bucket sees to it)
     if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * pr.K > kXResidentBytes) return BITCOS_ERR_SHAPE;
     int sms = 0, budget = 0;
-    int rc = prepare_kernel<gemv_kernel<FMT, NB, 1, XG>>(&sms, &budget);
+    int rc = prepare_kernel<gemv_kernel<FMT, NB, 1, XG, XQ>>(&sms, &budget);
     if (rc) return rc;
     const bool two = wants_two_tiles(pl_in, NB, sms);
     if constexpr (NB < kMmaMinBatch) {
         if (two) {
-            rc = prepare_kernel<gemv_kernel<FMT, NB, 2, XG>>(&sms, &budget);
+            rc = prepare_kernel<gemv_kernel<FMT, NB, 2, XG, XQ>>(&sms, &budget);
             if (rc) return rc;
         }
     }
@@ -1821,17 +1890,17 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     fo.walks = 1;
     fill_first_off(fo, 0, off_host, pr, plw, grid);
     if constexpr (NB < kMmaMinBatch) {
-        if (two) return launch_pdl(gemv_kernel<FMT, NB, 2, XG>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
+        if (two) return launch_pdl(gemv_kernel<FMT, NB, 2, XG, XQ>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
     }
-    return launch_pdl(gemv_kernel<FMT, NB, 1, XG>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
+    return launch_pdl(gemv_kernel<FMT, NB, 1, XG, XQ>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
-template <int NB>
+template <int NB, bool XQ = false>
 int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_host) {
     for (int j = 0; j < ma.n; ++j)
         if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * ma.pr[j].K > kXResidentBytes) return BITCOS_ERR_SHAPE;
     int sms = 0, budget = 0;
-    int rc = prepare_kernel<gemv_multi_kernel<NB>>(&sms, &budget);
+    int rc = prepare_kernel<gemv_multi_kernel<NB, 1, XQ>>(&sms, &budget);
     if (rc) return rc;
     // share the multiprocessors between the problems in proportion to their item counts
     int64_t total_items = 0;
@@ -1842,7 +1911,7 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     const bool two = wants_two_tiles(all, NB, sms);
     if constexpr (NB < kMmaMinBatch) {
         if (two) {
-            rc = prepare_kernel<gemv_multi_kernel<NB, 2>>(&sms, &budget);
+            rc = prepare_kernel<gemv_multi_kernel<NB, 2, XQ>>(&sms, &budget);
             if (rc) return rc;
             total_items = 0;
             for (int j = 0; j < ma.n; ++j) {
@@ -1877,9 +1946,9 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     }
     ma.first_block[ma.n] = next;
     if constexpr (NB < kMmaMinBatch) {
-        if (two) return launch_pdl(gemv_multi_kernel<NB, 2>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
+        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
     }
-    return launch_pdl(gemv_multi_kernel<NB>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
+    return launch_pdl(gemv_multi_kernel<NB, 1, XQ>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
 }
 
 // Which instantiation serves a batch: 1, 2, 4, 8 or 16 tokens.  The one- and two-token paths read
@@ -1994,20 +2063,6 @@ int gemv_common(int fmt, const uint32_t *payload, const uint32_t *signs, const u
 //   a = max(max |x| over the group, 2^-100),  scale = a / 127,  code = rint(x * (127 / a))
 // with IEEE float32 quotient and product and ties to even (the explicit intrinsics keep the
 // compiler from contracting or approximating them, so the codes do not depend on build flags).
-constexpr float kAmaxFloor = 7.888609052210118e-31f;      // 2^-100
-
-__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
-__device__ __forceinline__ uint32_t quant_code(float x, float inv) {
-    int c = __float2int_rn(__fmul_rn(x, inv));
-    c = c > 127 ? 127 : (c < -127 ? -127 : c);
-    return static_cast<uint32_t>(c) & 0xFFu;
-}
-// the two values of a 32-bit word -> two codes in the low 16 bits
-__device__ __forceinline__ uint32_t quant_pair(uint32_t u, float inv) {
-    return quant_code(bf16_lo(u), inv) | (quant_code(bf16_hi(u), inv) << 8);
-}
-
 // One warp per group of 128: a lane holds four consecutive values.
 __global__ void __launch_bounds__(256) quantize_groups_kernel(const uint16_t *__restrict__ x, int8_t *__restrict__ q,
                                                               float *__restrict__ scale, int64_t n_groups) {
@@ -2206,14 +2261,21 @@ int bitcos_gemv_group_scales(const bitcos_weights *W, const int8_t *x, const flo
                        acc_debug, workspace, workspace_bytes, cuda_stream, W->tile_off_host, true);
 }
 
-int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
+}  // extern "C"
+
+namespace {
+// bf16 = true: every job's x holds 16-bit activations (x_scale is not used) and the decoder warps
+// quantise them per group of 128; one or two tokens.
+int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream, bool bf16) {
     if (!jobs) return BITCOS_ERR_NULL;
     if (n_jobs < 1 || n_jobs > kMaxJobs) return BITCOS_ERR_SHAPE;
+    if (bf16 && batch > 2) return BITCOS_ERR_SHAPE;
     MultiArgs ma{};
     ma.n = n_jobs;
     for (int j = 0; j < n_jobs; ++j) {
-        const bitcos_gemv_job &jb = jobs[j];
+        bitcos_gemv_job jb = jobs[j];
         if (!jb.W) return BITCOS_ERR_NULL;
+        if (bf16) jb.x_scale = reinterpret_cast<const float *>(jb.x);        // never read; passes the NULL check
         const int bad = check_common(kBitcos, jb.W->bitmap, jb.W->signs, jb.W->tile_off, jb.W->scales, jb.W->M, jb.W->K,
                                      jb.x, jb.x_scale, batch, jb.y, nullptr, jb.workspace, jb.workspace_bytes);
         if (bad) return bad;
@@ -2229,11 +2291,45 @@ int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
     const int nbk = nb_bucket(batch, kmax);
     const uint32_t *off_host[kMaxJobs];
     for (int j = 0; j < n_jobs; ++j) off_host[j] = jobs[j].W->tile_off_host;
+    if (bf16) {
+        if (nbk == 1) return launch_multi<1, true>(ma, stream, off_host);
+        if (nbk == 2) return launch_multi<2, true>(ma, stream, off_host);
+        return BITCOS_ERR_SHAPE;          // rows too long for the one- and two-token kernels
+    }
     if (nbk == 1) return launch_multi<1>(ma, stream, off_host);
     if (nbk == 2) return launch_multi<2>(ma, stream, off_host);
     if (batch <= 4) return launch_multi<4>(ma, stream, off_host);
     if (batch <= 8) return launch_multi<8>(ma, stream, off_host);
     return launch_multi<16>(ma, stream, off_host);
+}
+}  // namespace
+
+extern "C" {
+
+int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
+    return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, false);
+}
+
+int bitcos_gemv_multi_bf16(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
+    return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, true);
+}
+
+int bitcos_gemv_bf16(const bitcos_weights *W, const uint16_t *x_bf16, int batch, float *y, int32_t *acc_debug,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!W) return BITCOS_ERR_NULL;
+    if (batch > 2) return BITCOS_ERR_SHAPE;
+    const int8_t *x = reinterpret_cast<const int8_t *>(x_bf16);
+    const int bad = check_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x,
+                                 reinterpret_cast<const float *>(x), batch, y, acc_debug, workspace, workspace_bytes);
+    if (bad) return bad;
+    const Plan pl = make_plan(W->M, W->K, decoder_warps(batch));
+    Problem pr{};
+    fill_problem(pr, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, nullptr, batch, y, acc_debug, workspace);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int nbk = nb_bucket(batch, W->K);
+    if (nbk == 1) return launch<kBitcos, 1, false, true>(pr, pl, stream, W->tile_off_host);
+    if (nbk == 2) return launch<kBitcos, 2, false, true>(pr, pl, stream, W->tile_off_host);
+    return BITCOS_ERR_SHAPE;              // rows too long for the one- and two-token kernels
 }
 
 size_t bitcos_gemv_host_staging_bytes(int64_t M, int64_t K, int batch) {

@@ -178,3 +178,78 @@ def test_quantise_then_multiply_on_one_stream(bc, B):
         assert np.array_equal(q.cpu().numpy(), q_ref)
         assert (np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= REL * mag).all(), (B, rep, "tokens")
     assert bc.workspace_status(ws) == 0
+
+
+@pytest.mark.parametrize("M,K,B", [(64, 128, 1), (2560, 2560, 1), (2560, 2560, 2), (2560, 6912, 1), (2560, 6912, 2),
+                                   (6912, 2560, 1), (333, 1280, 2), (640, 640, 1), (96, 25600, 1), (1000, 5120, 2)])
+def test_product_from_bf16_activations(bc, M, K, B):
+    """The quantiser fused into the product: the same codes (seen through the bit-exact int32
+    accumulators), scales and outputs as the oracle's quantise-then-multiply chain."""
+    W, S = datagen.trits(2400 + M, M, K, 0.4219), datagen.scales(2400 + M, M, K)
+    bits = special_rows(datagen.activations_bf16(2400 + K + B, B, K))
+    xf = datagen.bf16_bits_to_f32(bits)
+    q_ref, s_ref = oracle.quantize_activations(xf, 128)
+    acc_ref, y_ref, mag = oracle.gemv_dense_group_scales(W, S, q_ref, s_ref)
+    Wd = bc.bitcos_pack(W, S).to_device()
+    ws = bc.make_workspace(M, K)
+    xd = dev_bf16(bits)
+    for rep in range(2):
+        y, acc = bc.bitcos_gemv_bf16(Wd, xd, acc_debug=(rep == 0) or None, workspace=ws)
+        torch.cuda.synchronize()
+        if acc is not None:
+            assert np.array_equal(acc.cpu().numpy(), acc_ref), (M, K, B)
+        yv = y.cpu().numpy().astype(np.float64)
+        assert (np.abs(yv - y_ref) <= REL * mag).all(), (M, K, B, rep)
+        assert (yv[mag == 0] == 0).all()
+    assert bc.workspace_status(ws) == 0
+
+
+def test_product_from_bf16_activations_large_and_multi(bc):
+    """Two tiles per warp (a large matrix), and a layer's worth of jobs in fused launches."""
+    M, K, B = 19200, 5120, 1
+    W, S = datagen.trits(2500, M, K, 0.4219), datagen.scales(2500, M, K)
+    bits = datagen.activations_bf16(2500, B, K)
+    q_ref, s_ref = oracle.quantize_activations(datagen.bf16_bits_to_f32(bits), 128)
+    rows = np.unique(np.concatenate([np.arange(0, M, M // 211), [M - 1, M - 32, M - 33, 31, 32, 63, 64]]))
+    acc_ref, y_ref, mag = oracle.gemv_dense_group_scales(W[rows], S[rows], q_ref, s_ref)
+    Wd = bc.bitcos_pack(W, S).to_device()
+    y, acc = bc.bitcos_gemv_bf16(Wd, dev_bf16(bits), acc_debug=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(acc.cpu().numpy()[:, rows], acc_ref)
+    assert (np.abs(y.cpu().numpy().astype(np.float64)[:, rows] - y_ref) <= REL * mag).all()
+    del Wd
+    for B in (1, 2):
+        shapes = [(2560, 2560), (640, 2560), (640, 2560), (96, 6912), (33, 1280)]
+        jobs, refs = [], []
+        for i, (M, K) in enumerate(shapes):
+            W, S = datagen.trits(2600 + i, M, K, 0.4219), datagen.scales(2600 + i, M, K)
+            bits = datagen.activations_bf16(2600 + i + B, B, K)
+            q_ref, s_ref = oracle.quantize_activations(datagen.bf16_bits_to_f32(bits), 128)
+            refs.append(oracle.gemv_dense_group_scales(W, S, q_ref, s_ref))
+            yj = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
+            jobs.append((bc.bitcos_pack(W, S).to_device(), dev_bf16(bits), None, yj, bc.make_workspace(M, K)))
+        for n in (5, 3, 1):
+            for j in jobs:
+                j[3].fill_(float("nan"))
+            bc.bitcos_gemv_multi_bf16(jobs[:n])
+            torch.cuda.synchronize()
+            for (Wd, _, _, yj, ws), (_, y_ref, mag) in zip(jobs[:n], refs[:n]):
+                assert (np.abs(yj.cpu().numpy().astype(np.float64) - y_ref) <= REL * mag).all(), (Wd.M, Wd.K, B, n)
+                assert bc.workspace_status(ws) == 0
+
+
+def test_product_from_bf16_activations_rejects_what_it_cannot_do(bc):
+    W, S = datagen.trits(2700, 64, 256, 0.4), datagen.scales(2700, 64, 256)
+    Wd = bc.bitcos_pack(W, S).to_device()
+    with pytest.raises(bc.BitcosError) as e:
+        bc.bitcos_gemv_bf16(Wd, torch.zeros((3, 256), dtype=torch.bfloat16, device="cuda"))
+    assert e.value.status == 2
+    W, S = datagen.trits(2701, 32, 25600, 0.4), datagen.scales(2701, 32, 25600)
+    Wl = bc.bitcos_pack(W, S).to_device()
+    with pytest.raises(bc.BitcosError) as e:
+        bc.bitcos_gemv_bf16(Wl, torch.zeros((2, 25600), dtype=torch.bfloat16, device="cuda"))
+    assert e.value.status == 2
+    with pytest.raises(bc.BitcosError) as e:
+        bc.bitcos_gemv_multi_bf16([(Wd, torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda"), None,
+                                    torch.zeros((4, 64), dtype=torch.float32, device="cuda"), bc.make_workspace(64, 256))])
+    assert e.value.status == 2
