@@ -322,6 +322,19 @@ def run_cuda(args):
         step(i)
     torch.cuda.synchronize()
 
+    if args.profile_quant:
+        # for profilers: plain stream launches of the layer pass from bf16 activations, nothing else
+        step_q, step_b = quantised_layer_steps(bc, torch, layer, groups, replicas, ys, wss)
+        run = step_q if args.profile_quant == "chain" else step_b
+        for i in range(args.steps):
+            run(i)
+        torch.cuda.synchronize()
+        status = max(bc.workspace_status(w) for w in wss)
+        if rank == 0:
+            print(json.dumps({"profile_quant": args.profile_quant, "steps": args.steps, "status": status}))
+        ranks.close()
+        return
+
     # Capture the rotation as CUDA graphs so that the host's launch cost is not what is timed.
     stream = torch.cuda.Stream()
     graphs = {}
@@ -432,31 +445,8 @@ def run_cuda(args):
     # (bf16 activations -> int8 and one scale per token, then the fused launch that reads them)
     with_quant_us = fused_quant_us = None
     if not args.no_detail and not (args.serial or args.branches):
-        import datagen
-        xb, qx, qs = [], [], []
-        for gi, g in enumerate(groups):
-            K = layer[g[0]]["K"]
-            bits = datagen.activations_bf16(datagen.config_seed(1, 60 + gi), 1, K)
-            xb.append(torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16))
-            qx.append(torch.empty((1, K), dtype=torch.int8, device="cuda"))
-            qs.append(torch.empty((1,), dtype=torch.float32, device="cuda"))
-        multi_q = [[bc.MultiJobs([(rep[j], qx[gi], qs[gi], ys[j], wss[j]) for j in g]) for gi, g in enumerate(groups)]
-                   for rep in replicas]
-
-        def step_q(i):
-            for gi, mj in enumerate(multi_q[i]):
-                bc.bitcos_quantize_activations(xb[gi], 0, xq=qx[gi], x_scale=qs[gi])
-                bc.bitcos_gemv_multi(mj)
-
+        step_q, step_b = quantised_layer_steps(bc, torch, layer, groups, replicas, ys, wss)
         with_quant_us = graph_time_us(torch, stream, step_q, copies, launches=copies)
-        # the same with the quantiser inside the products (scales per group of 128): four launches
-        multi_b = [[bc.MultiJobs([(rep[j], xb[gi], None, ys[j], wss[j]) for j in g]) for gi, g in enumerate(groups)]
-                   for rep in replicas]
-
-        def step_b(i):
-            for mj in multi_b[i]:
-                bc.bitcos_gemv_multi_bf16(mj)
-
         fused_quant_us = graph_time_us(torch, stream, step_b, copies, launches=copies)
 
     # ---- per-shape detail: each format on each shape, rotated copies, CUDA graph of 64 launches ----
@@ -542,6 +532,35 @@ def run_cuda(args):
         line["moe"] = moe_detail(bc, torch, stream)
     print(json.dumps(line))
     ranks.close()
+
+
+def quantised_layer_steps(bc, torch, layer, groups, replicas, ys, wss):
+    """The layer pass from bf16 activations, two ways.  step_q: bitcos_quantize_activations (one scale
+    per token) in front of each fused launch, eight kernels per step.  step_b: the quantiser inside
+    the products (bitcos_gemv_multi_bf16, scales per group of 128), four launches per step."""
+    import datagen
+    xb, qx, qs = [], [], []
+    for gi, g in enumerate(groups):
+        K = layer[g[0]]["K"]
+        bits = datagen.activations_bf16(datagen.config_seed(1, 60 + gi), 1, K)
+        xb.append(torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16))
+        qx.append(torch.empty((1, K), dtype=torch.int8, device="cuda"))
+        qs.append(torch.empty((1,), dtype=torch.float32, device="cuda"))
+    multi_q = [[bc.MultiJobs([(rep[j], qx[gi], qs[gi], ys[j], wss[j]) for j in g]) for gi, g in enumerate(groups)]
+               for rep in replicas]
+    multi_b = [[bc.MultiJobs([(rep[j], xb[gi], None, ys[j], wss[j]) for j in g]) for gi, g in enumerate(groups)]
+               for rep in replicas]
+
+    def step_q(i):
+        for gi, mj in enumerate(multi_q[i % len(multi_q)]):
+            bc.bitcos_quantize_activations(xb[gi], 0, xq=qx[gi], x_scale=qs[gi])
+            bc.bitcos_gemv_multi(mj)
+
+    def step_b(i):
+        for mj in multi_b[i % len(multi_b)]:
+            bc.bitcos_gemv_multi_bf16(mj)
+
+    return step_q, step_b
 
 
 def two_term_roofline(bc, z, peak_gbs, sm_mhz, sms=148):
@@ -947,6 +966,9 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA graphs (for profilers)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--profile-quant", default="", choices=["", "chain", "fused"],
+                    help="only launch --steps layer passes from bf16 activations (quantiser kernels in front of the "
+                         "products, or inside them), without graphs (for profilers)")
     ap.add_argument("--profile-shape", default="8192x5120", metavar="MxK",
                     help="matrix of --profile-batch (default: the batch table's q projection)")
     ap.add_argument("--profile-batch", type=int, default=0, metavar="B",
@@ -966,7 +988,7 @@ def main():
         run_reference(args)
     else:
         if args.steps is None:
-            args.steps = 2000
+            args.steps = 20 if args.profile_quant else 2000
         run_cuda(args)
 
 
