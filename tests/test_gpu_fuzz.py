@@ -76,3 +76,46 @@ def test_seeded_sweep(bc, seed):
         assert (np.abs(yv - y_ref) <= REL * mag).all(), what
         assert (yv[mag == 0] == 0).all(), what
         assert bc.workspace_status(ws) == 0, what
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_seeded_sweep_quantised_front_end(bc, seed):
+    """The same sweep for the quantised-activation entry points: quantiser (both granularities),
+    product with group scales (every batch size), product from bf16 activations (one and two
+    tokens, single and multi launch), and the device packer in front of them."""
+    rng = np.random.default_rng(seed)
+    for it in range(14):
+        M = int(rng.choice(ROWS))
+        K = 128 * int(rng.choice(GROUPS))
+        B = int(rng.integers(1, 17))
+        z = float(rng.choice(DENSITIES))
+        what = f"seed {seed} case {it}: {M}x{K} batch {B} z {z}"
+        s = 7000 + 100 * seed + it
+        W, S = datagen.trits(s, M, K, z), datagen.scales(s, M, K)
+        bits = datagen.activations_bf16(s, B, K)
+        xf = datagen.bf16_bits_to_f32(bits)
+        xb = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+        Wd = bc.bitcos_pack_device(torch.from_numpy(W).cuda(), torch.from_numpy(S.view(np.int16)).cuda())
+        ws = bc.make_workspace(M, K)
+        q_ref, s_ref = oracle.quantize_activations(xf, 128)
+        acc_ref, y_ref, mag = oracle.gemv_dense_group_scales(W, S, q_ref, s_ref)
+        q, sg = bc.bitcos_quantize_activations(xb, 128)
+        y, acc = bc.bitcos_gemv_group_scales(Wd, q, sg, acc_debug=True, workspace=ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(sg.cpu().numpy(), s_ref), what
+        assert np.array_equal(acc.cpu().numpy(), acc_ref), what
+        assert (np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= REL * mag).all(), what
+        qt_ref, st_ref = oracle.quantize_activations(xf, 0)
+        qt, st = bc.bitcos_quantize_activations(xb, 0)
+        torch.cuda.synchronize()
+        assert np.array_equal(qt.cpu().numpy(), qt_ref) and np.array_equal(st.cpu().numpy(), st_ref), what
+        nb = 1 + it % 2
+        if nb * K <= 49152:
+            y2, acc2 = bc.bitcos_gemv_bf16(Wd, xb[:nb].contiguous(), acc_debug=True, workspace=ws)
+            y3 = torch.empty((nb, M), dtype=torch.float32, device="cuda")
+            bc.bitcos_gemv_multi_bf16([(Wd, xb[:nb].contiguous(), None, y3, bc.make_workspace(M, K))])
+            torch.cuda.synchronize()
+            assert np.array_equal(acc2.cpu().numpy(), acc_ref[:nb]), what
+            assert (np.abs(y2.cpu().numpy().astype(np.float64) - y_ref[:nb]) <= REL * mag[:nb]).all(), what
+            assert (np.abs(y3.cpu().numpy().astype(np.float64) - y_ref[:nb]) <= REL * mag[:nb]).all(), what
+        assert bc.workspace_status(ws) == 0, what
