@@ -273,6 +273,9 @@ typedef struct bitcos_gemv_job {
     size_t workspace_bytes;
 } bitcos_gemv_job;
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
+/* The same with one activation scale per token and group of 128 (see bitcos_gemv_group_scales):
+ * every job's x_scale points to device float [batch][K/128]. */
+int bitcos_gemv_multi_group_scales(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
 /* The same with 16-bit activations quantised inside the launch (see bitcos_gemv_bf16): every
  * job's x points to device bf16 [batch][K], x_scale is ignored (may be NULL); batch 1 or 2. */
 int bitcos_gemv_multi_bf16(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);

@@ -26,6 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
+    "bitcos_gemv_multi_group_scales",
 ]
 
 
@@ -101,6 +102,7 @@ def load_library():
     L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
     L.bitcos_gemv_bf16.argtypes = [C.POINTER(_Weights), vp, C.c_int, vp, vp, vp, sz, vp]
     L.bitcos_gemv_multi_bf16.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
+    L.bitcos_gemv_multi_group_scales.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_choose_format.argtypes = [i64, i64, u64, C.POINTER(C.c_int), psz, psz]
     L.bitcos_count_nnz_device.argtypes = [vp, i64, i64, C.POINTER(u64), vp, vp]
     L.bitcos_pack_device.argtypes = [vp, vp, i64, i64, vp, vp, sz, vp, vp, vp, C.POINTER(u64), vp, vp]
@@ -498,6 +500,15 @@ def bitcos_gemv_multi(jobs):
     (W, x, x_scale, y, workspace) tuples with a common batch size."""
     mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
     _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")
+    return [j[3] for j in mj.keep]
+
+
+def bitcos_gemv_multi_group_scales(jobs):
+    """bitcos_gemv_multi with one activation scale per token and group: jobs = MultiJobs or a list of
+    (W, x, x_group_scale [batch, K / 128], y, workspace) tuples."""
+    mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
+    _check(load_library().bitcos_gemv_multi_group_scales(mj.arr, len(mj.arr), mj.batch, _stream()),
+           "bitcos_gemv_multi_group_scales")
     return [j[3] for j in mj.keep]
 
 

@@ -1527,7 +1527,7 @@ struct MultiArgs {
     int n;
 };
 
-template <int NB, int TPW = 1, bool XQ = false>
+template <int NB, int TPW = 1, bool XQ = false, bool XG = false>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma,
                                                                               const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -1537,7 +1537,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
     const Problem pr = ma.pr[j];
     // (the multi launch has no accumulator dump)
-    run_problem<kBitcos, NB, false, TPW, false, XQ>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
+    run_problem<kBitcos, NB, false, TPW, XG, XQ>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
                              b - ma.first_block[j], &fo, b);
 }
 
@@ -1895,12 +1895,12 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     return launch_pdl(gemv_kernel<FMT, NB, 1, XG, XQ>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
-template <int NB, bool XQ = false>
+template <int NB, bool XQ = false, bool XG = false>
 int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_host) {
     for (int j = 0; j < ma.n; ++j)
         if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * ma.pr[j].K > kXResidentBytes) return BITCOS_ERR_SHAPE;
     int sms = 0, budget = 0;
-    int rc = prepare_kernel<gemv_multi_kernel<NB, 1, XQ>>(&sms, &budget);
+    int rc = prepare_kernel<gemv_multi_kernel<NB, 1, XQ, XG>>(&sms, &budget);
     if (rc) return rc;
     // share the multiprocessors between the problems in proportion to their item counts
     int64_t total_items = 0;
@@ -1911,7 +1911,7 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     const bool two = wants_two_tiles(all, NB, sms);
     if constexpr (NB < kMmaMinBatch) {
         if (two) {
-            rc = prepare_kernel<gemv_multi_kernel<NB, 2, XQ>>(&sms, &budget);
+            rc = prepare_kernel<gemv_multi_kernel<NB, 2, XQ, XG>>(&sms, &budget);
             if (rc) return rc;
             total_items = 0;
             for (int j = 0; j < ma.n; ++j) {
@@ -1946,9 +1946,9 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     }
     ma.first_block[ma.n] = next;
     if constexpr (NB < kMmaMinBatch) {
-        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
+        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ, XG>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
     }
-    return launch_pdl(gemv_multi_kernel<NB, 1, XQ>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
+    return launch_pdl(gemv_multi_kernel<NB, 1, XQ, XG>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
 }
 
 // Which instantiation serves a batch: 1, 2, 4, 8 or 16 tokens.  The one- and two-token paths read
@@ -2266,7 +2266,8 @@ int bitcos_gemv_group_scales(const bitcos_weights *W, const int8_t *x, const flo
 namespace {
 // bf16 = true: every job's x holds 16-bit activations (x_scale is not used) and the decoder warps
 // quantise them per group of 128; one or two tokens.
-int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream, bool bf16) {
+int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream, bool bf16,
+                      bool group_scales = false) {
     if (!jobs) return BITCOS_ERR_NULL;
     if (n_jobs < 1 || n_jobs > kMaxJobs) return BITCOS_ERR_SHAPE;
     if (bf16 && batch > 2) return BITCOS_ERR_SHAPE;
@@ -2296,6 +2297,13 @@ int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
         if (nbk == 2) return launch_multi<2, true>(ma, stream, off_host);
         return BITCOS_ERR_SHAPE;          // rows too long for the one- and two-token kernels
     }
+    if (group_scales) {
+        if (nbk == 1) return launch_multi<1, false, true>(ma, stream, off_host);
+        if (nbk == 2) return launch_multi<2, false, true>(ma, stream, off_host);
+        if (batch <= 4) return launch_multi<4, false, true>(ma, stream, off_host);
+        if (batch <= 8) return launch_multi<8, false, true>(ma, stream, off_host);
+        return launch_multi<16, false, true>(ma, stream, off_host);
+    }
     if (nbk == 1) return launch_multi<1>(ma, stream, off_host);
     if (nbk == 2) return launch_multi<2>(ma, stream, off_host);
     if (batch <= 4) return launch_multi<4>(ma, stream, off_host);
@@ -2308,6 +2316,10 @@ extern "C" {
 
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
     return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, false);
+}
+
+int bitcos_gemv_multi_group_scales(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
+    return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, false, true);
 }
 
 int bitcos_gemv_multi_bf16(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {

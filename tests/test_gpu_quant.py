@@ -253,3 +253,28 @@ def test_product_from_bf16_activations_rejects_what_it_cannot_do(bc):
         bc.bitcos_gemv_multi_bf16([(Wd, torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda"), None,
                                     torch.zeros((4, 64), dtype=torch.float32, device="cuda"), bc.make_workspace(64, 256))])
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("B", [1, 2, 5, 16])
+def test_multi_launch_with_group_scales(bc, B):
+    shapes = [(2560, 2560), (640, 2560), (96, 6912), (320, 1280), (33, 2560)]
+    jobs, refs = [], []
+    for i, (M, K) in enumerate(shapes):
+        W, S = datagen.trits(2800 + i, M, K, 0.4219), datagen.scales(2800 + i, M, K)
+        x, _ = datagen.activations(2800 + i + B, B, K)
+        G = K // 128
+        xg = (0.001 * (1.0 + 19.0 * datagen.uniform(2800 + i, datagen.STREAM_XS, 0, B * G))).astype(np.float32).reshape(B, G)
+        refs.append(oracle.gemv_dense_group_scales(W, S, x, xg))
+        y = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
+        jobs.append((bc.bitcos_pack(W, S).to_device(), dev(x), dev(xg), y, bc.make_workspace(M, K)))
+    for n in (5, 2):
+        for j in jobs:
+            j[3].fill_(float("nan"))
+        bc.bitcos_gemv_multi_group_scales(jobs[:n])
+        torch.cuda.synchronize()
+        for (Wd, x, xg, y, ws), (_, y_ref, mag) in zip(jobs[:n], refs[:n]):
+            assert (np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= REL * mag).all(), (Wd.M, Wd.K, B, n)
+            y1, _ = bc.bitcos_gemv_group_scales(Wd, x, xg, workspace=ws)
+            torch.cuda.synchronize()
+            assert torch.equal(y1, y)
+            assert bc.workspace_status(ws) == 0
