@@ -175,8 +175,9 @@ typedef struct bitcos_weights {
  * when the previous kernel in the stream is also one of this library's, a call may start reading
  * its PACKED WEIGHTS (and nothing else) while that kernel is still running; activations, activation
  * scales, routing lists, outputs, accumulator dumps and workspaces are touched only after every
- * earlier kernel in the stream has completed, as usual.  Kernels of this library never write packed
- * weights, so ordinary use needs no extra care; after any other kernel or copy in the stream the
+ * earlier kernel in the stream has completed, as usual.  The products and the quantiser never write
+ * packed weights, and bitcos_pack_device waits for the stream before it returns, so ordinary use needs
+ * no extra care; after any other kernel or copy in the stream the
  * usual order holds in full.  BITCOS_PDL=0 in the environment turns the overlap off. */
 
 /* Scratch memory the GEMV entry points need for an M x K matrix (the same value for all
