@@ -393,5 +393,26 @@ def gemv_dense_group_scales(W, scales, x, xs_g):
     return acc, y, mag
 
 
+# --- unquantised 16-bit activations against weights +-s (Sections II-B and II-D: the scale blended
+# --- into the reconstructed weight, multiply-add against 16-bit activations) -----------------------
+def gemv_dense_blend(W, scales, x):
+    """y[b, m] = sum over k of (W[m, k] * s[m, k // 128]) * x[b, k] in float64, x = float values of
+    16-bit activations [B, K] (no quantisation anywhere); also the sum of |terms| for the tolerance."""
+    W = np.asarray(W, np.int8)
+    M, K = W.shape
+    G = K // GROUP
+    s = (np.asarray(scales, np.uint16).reshape(M, G).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    x = np.atleast_2d(np.asarray(x, np.float64))
+    B = x.shape[0]
+    y = np.zeros((B, M), np.float64)
+    mag = np.zeros((B, M), np.float64)
+    for m in range(M):
+        ws = W[m].astype(np.float64) * np.repeat(s[m], GROUP)          # the row's weights +-s (or 0)
+        terms = x * ws[None, :]
+        y[:, m] = terms.sum(axis=1)
+        mag[:, m] = np.abs(terms).sum(axis=1)
+    return y, mag
+
+
 def threads() -> int:
     return int(lib().o_threads())

@@ -589,3 +589,39 @@ def test_quantised_product_stays_within_the_quantisation_bound():
         errs[group] = np.sqrt(np.mean((y - exact) ** 2))
     # with outlier channels, scales per group lose less than one scale per token
     assert errs[128] < errs[0]
+
+
+# --- Sections II-B / II-D: weights rebuilt as +-s, multiplied with unquantised 16-bit activations ---
+def test_blend_product_bruteforce_and_cross_checks():
+    rng = np.random.default_rng(35)
+    M, K, B = 4, 256, 2
+    W = rng.integers(-1, 2, (M, K)).astype(np.int8)
+    S = datagen.scales(35, M, K)
+    Sf = datagen.bf16_bits_to_f32(S).astype(np.float64)
+    x = datagen.bf16_bits_to_f32(datagen.activations_bf16(35, B, K)).astype(np.float64)
+    y, mag = oracle.gemv_dense_blend(W, S, x)
+    for b in range(B):
+        for m in range(M):
+            tot = sum(int(W[m, k]) * Sf[m, k // 128] * x[b, k] for k in range(K))
+            tot_abs = sum(abs(int(W[m, k]) * Sf[m, k // 128] * x[b, k]) for k in range(K))
+            assert y[b, m] == pytest.approx(tot, rel=1e-12, abs=1e-300)
+            assert mag[b, m] == pytest.approx(tot_abs, rel=1e-12)
+    # as a library matrix product
+    assert np.allclose(y, x @ (W.astype(np.float64) * np.repeat(Sf, 128, axis=1)).T, rtol=0, atol=1e-12 * mag.max())
+    # activations that are small integers times a power of two are 16-bit values and int8 codes at
+    # once: then this product is the integer path's (pinned on its own), with that power as the scale
+    q, _ = datagen.activations(36, B, K)
+    xq = q.astype(np.float64) * 2.0 ** -7
+    assert np.array_equal(datagen.bf16_bits_to_f32(datagen.f32_to_bf16_bits(xq.astype(np.float32))).astype(np.float64), xq)
+    y2, m2 = oracle.gemv_dense_blend(W, S, xq)
+    _, y_int, m_int = oracle.gemv_dense(W, S, q, np.full(B, 2.0 ** -7, np.float32))
+    assert np.allclose(y2, y_int, rtol=0, atol=1e-12 * m2.max())
+    assert (m2 >= m_int * (1 - 1e-12)).all()          # |sum over a group| <= sum of |terms|
+    # closed forms: all +1 with unit scales sums the activations; a single -1 picks one of them
+    ones = np.full((M, K // 128), 0x3F80, np.uint16)
+    y3, _ = oracle.gemv_dense_blend(np.ones((M, K), np.int8), ones, x)
+    assert np.allclose(y3, np.repeat(x.sum(axis=1)[:, None], M, axis=1), rtol=1e-13)
+    Wz = np.zeros((M, K), np.int8)
+    Wz[1, 200] = -1
+    y4, m4 = oracle.gemv_dense_blend(Wz, S, x)
+    assert np.array_equal(y4[:, 1], -Sf[1, 1] * x[:, 200]) and not y4[:, [0, 2, 3]].any() and np.array_equal(m4, np.abs(y4))
