@@ -730,7 +730,7 @@ def quant_detail(bc, torch, stream):
         reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
         ws = bc.make_workspace(M, K)
         G = K // 128
-        for B in (1, 2, 4, 16):
+        for B in (1, 2, 4, 8, 16):
             xb = torch.from_numpy(datagen.activations_bf16(seed + B, B, K).view(np.int16)).cuda().view(torch.bfloat16)
             q = torch.empty((B, K), dtype=torch.int8, device="cuda")
             sg = torch.empty((B, G), dtype=torch.float32, device="cuda")
@@ -759,6 +759,10 @@ def quant_detail(bc, torch, stream):
                 # the quantiser inside the product's thread blocks (one and two tokens)
                 row["gemv_bf16_us"] = graph_time_us(
                     torch, stream, lambda i: bc.bitcos_gemv_bf16(reps[i], xb, y=y, workspace=ws), n_copies)
+            if B <= 8:
+                # the 16-bit variant: weights rebuilt as +-s against the unquantised activations (tensor cores)
+                row["gemv_blend_bf16_us"] = graph_time_us(
+                    torch, stream, lambda i: bc.bitcos_gemv_blend_bf16(reps[i], xb, y=y, workspace=ws), n_copies)
             row["chain_groups_us"] = graph_time_us(torch, stream, chain_groups, n_copies)
             row["chain_tokens_us"] = graph_time_us(torch, stream, chain_tokens, n_copies)
             row["quantiser_bytes"] = int(B * K * 3 + 4 * B * G)

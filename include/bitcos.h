@@ -256,6 +256,19 @@ int bitcos_gemv_group_scales(const bitcos_weights *W, const int8_t *x, const flo
 int bitcos_gemv_bf16(const bitcos_weights *W, const uint16_t *x_bf16, int batch, float *y, int32_t *acc_debug,
                      void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The 16-bit variant of Sections II-B / II-D: no activation quantisation; the weights are rebuilt
+ * as +s / 0 / -s (the bf16 group scale blended into the weight, exact) and multiplied with the
+ * bf16 activations as they are,
+ *     y[b][m] = sum over k of (W[m][k] * s[m][k / 128]) * x[b][k],
+ * on the tensor cores (mma.m16n8k16, bf16 operands, fp32 accumulation over each group of 128; the
+ * groups are then added in fp32 in the fixed order of the other products).  Every product is exact
+ * in fp32; the sums are within 4e-5 of the sum of |terms|.  batch 1..8 (ERR_SHAPE above);
+ * x_bf16 = device bf16 [batch][K], 16-byte aligned; no accumulator dump.  About twice the cost of
+ * the integer product at one token (the decoded weights are expanded to 16 bits on the way to the
+ * tensor cores), the same at eight. */
+int bitcos_gemv_blend_bf16(const bitcos_weights *W, const uint16_t *x_bf16, int batch, float *y, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream);
+
 #define BITCOS_MAX_JOBS 8
 
 /* Up to BITCOS_MAX_JOBS independent BITCOS products in ONE launch (same batch; shapes may differ): e.g. the

@@ -27,6 +27,7 @@ from .binding import (  # noqa: F401
     bitcos_gemv_group_scales,
     bitcos_gemv_bf16,
     bitcos_gemv_multi_bf16,
+    bitcos_gemv_blend_bf16,
     bitcos_gemv_multi_group_scales,
     bitcos_choose_format,
     bitcos_count_nnz_device,

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16",
 ]
 
 
@@ -102,6 +102,7 @@ def load_library():
     L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
     L.bitcos_gemv_bf16.argtypes = [C.POINTER(_Weights), vp, C.c_int, vp, vp, vp, sz, vp]
     L.bitcos_gemv_multi_bf16.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
+    L.bitcos_gemv_blend_bf16.argtypes = [C.POINTER(_Weights), vp, C.c_int, vp, vp, sz, vp]
     L.bitcos_gemv_multi_group_scales.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_choose_format.argtypes = [i64, i64, u64, C.POINTER(C.c_int), psz, psz]
     L.bitcos_count_nnz_device.argtypes = [vp, i64, i64, C.POINTER(u64), vp, vp]
@@ -402,6 +403,21 @@ def bitcos_gemv_bf16(W: DeviceBitcos, x_bf16, y=None, acc_debug=None, workspace=
                                            acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
                                            workspace.numel(), _stream()), "bitcos_gemv_bf16")
     return y, acc
+
+
+def bitcos_gemv_blend_bf16(W: DeviceBitcos, x_bf16, y=None, workspace=None):
+    """The 16-bit variant: weights rebuilt as +-s times unquantised bfloat16 activations [batch, K], batch 1..8."""
+    import torch
+    if x_bf16.dtype != torch.bfloat16 or x_bf16.dim() != 2 or not x_bf16.is_contiguous():
+        raise ValueError("x_bf16 must be a contiguous bfloat16 [batch, K] tensor")
+    batch = x_bf16.shape[0]
+    if workspace is None:
+        workspace = make_workspace(W.M, W.K, x_bf16.device)
+    y, _ = _outputs(W.M, W.K, batch, y, None, x_bf16.device)
+    _check(load_library().bitcos_gemv_blend_bf16(C.byref(W.desc), x_bf16.data_ptr(), batch, y.data_ptr(),
+                                                 workspace.data_ptr(), workspace.numel(), _stream()),
+           "bitcos_gemv_blend_bf16")
+    return y
 
 
 def bitcos_quantize_activations(x_bf16, group: int = 128, xq=None, x_scale=None):

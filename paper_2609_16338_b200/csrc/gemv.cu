@@ -395,6 +395,31 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], const uint32_t (&a)[4], uint
                  : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// c[16 x 8] += a[16 x 16] * b[16 x 8], bf16 operands, fp32 accumulators.
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+// Four decoded weights (bytes 0x00, 0x01, 0xFF) -> four bf16 values 0, +s, -s (the scale blended
+// into the weight, Section II-B): the low three bits of a weight byte (0, 1, 7) pick the high and
+// the low byte of its bf16 value out of two small byte tables built from the scale.
+//   hi_a / hi_b: bytes {0, s_hi, -, -} / {-, -, -, s_hi | 0x80};  lo_a / lo_b: {0, s_lo, -, -} / {-, -, -, s_lo}
+// p01 = (w0, w1), p23 = (w2, w3) as bf16x2.
+__device__ __forceinline__ void blend4(uint32_t t, uint32_t hi_a, uint32_t hi_b, uint32_t lo_a, uint32_t lo_b, uint32_t &p01,
+                                       uint32_t &p23) {
+    uint32_t u = t & 0x07070707u;
+    u |= u >> 4;                                   // byte 0: n0 | n1 << 4, byte 2: n2 | n3 << 4
+    const uint32_t sel = prmt(u, 0u, 0x4420u);     // n0 | n1 << 4 | n2 << 8 | n3 << 12
+    const uint32_t hi = prmt(hi_a, hi_b, sel), lo = prmt(lo_a, lo_b, sel);
+    p01 = prmt(lo, hi, 0x5140u);
+    p23 = prmt(lo, hi, 0x7362u);
+}
 __device__ __forceinline__ void sts128(uint32_t addr, int a, int b, int c, int d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -767,13 +792,14 @@ __device__ __forceinline__ void finish_share(const Problem &pr, const Plan &pl, 
 // What a thread block runs back to back: one problem and its share of the items (the plain
 // kernels), or the pieces of several groups (the grouped launch).  Every warp role walks its own
 // copy of the source.
-template <bool DEBUG, bool XG = false, bool XQ = false>
+template <bool DEBUG, bool XG = false, bool XQ = false, bool BL = false>
 struct OneSegT {
     typedef ParamView View;
     static constexpr bool kSingle = true;      // never more than one segment
     static constexpr bool kDebug = DEBUG;      // false: acc_debug is known to be NULL (no code for it)
     static constexpr bool kGroupScales = XG;   // x_scale holds one scale per token AND group: [nb][G]
     static constexpr bool kQuantize = XQ;      // x holds bf16 activations: quantised per group of 128 by the decoder warps
+    static constexpr bool kBlend = BL;         // x holds bf16 activations, used as they are against weights +-s (tensor cores)
     const Problem *pr;
     Walk wk;
     bool used;
@@ -810,7 +836,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // one activation scale per token and group (applied by the decoder warps, tile by tile)
     // instead of one per token (applied by the epilogue warp to the finished sums)
     constexpr bool kXQ = Segs::kQuantize;                      // (one or two tokens only)
-    constexpr bool kXG = Segs::kGroupScales || kXQ;
+    constexpr bool kBlend = Segs::kBlend;                      // (tensor-core path, up to eight tokens)
+    static_assert(!kBlend || (NB == 8 && FMT == kBitcos && TPW == 1), "blended weights: the eight-token BITCOS kernel");
+    constexpr bool kXG = Segs::kGroupScales || kXQ || kBlend;   // no token scale in the epilogue
     static_assert(!kXQ || NB < kMmaMinBatch, "16-bit activations: one or two tokens only");
     const uint32_t red_slot = static_cast<uint32_t>(pl.NW * TPW) * NB * kRows;     // floats per partial-sum slot
     // partial-sum slots in use: red_slots(NB), half as many (of twice the size) with two tiles per warp
@@ -1194,14 +1222,27 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             const int n = 8 * h + (lane >> 2);
             xfrag[h] = nullptr;
             if (kMma && n < pr.nb(pb))
-                xfrag[h] = pb.x + static_cast<int64_t>(pr.xrow(pb) ? __ldg(pr.xrow(pb) + n) : n) * pb.K + 16 * (lane & 3);
+                xfrag[h] = kBlend ? pb.x + static_cast<int64_t>(n) * pb.K * 2 + 64 * (lane & 3)
+                                  : pb.x + static_cast<int64_t>(pr.xrow(pb) ? __ldg(pr.xrow(pb) + n) : n) * pb.K + 16 * (lane & 3);
         }
     };
-    uint32_t bf[NH][8];
+    // (blended weights: of token lane / 4 this lane holds bytes 64 c .. 64 c + 63 of the group's 256,
+    // four 16-byte loads; k-step j of the contraction uses words 2 j and 2 j + 1 of those sixteen)
+    uint32_t bf[NH][kBlend ? 16 : 8];
     float xgq[NH][2];           // group scales of the two tokens whose accumulators this lane holds
     auto load_bf = [&](int g) {
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
+            if (kBlend) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    int4 u = make_int4(0, 0, 0, 0);
+                    if (xfrag[h]) u = __ldg(reinterpret_cast<const int4 *>(xfrag[h] + static_cast<int64_t>(g) * (2 * kGroup)) + q);
+                    bf[h][(kBlend ? 4 : 0) * q + 0] = u.x; bf[h][(kBlend ? 4 : 0) * q + 1] = u.y;
+                    bf[h][(kBlend ? 4 : 0) * q + 2] = u.z; bf[h][(kBlend ? 4 : 0) * q + 3] = u.w;
+                }
+                continue;
+            }
             if (kXG && !kXQ) {
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
@@ -1345,7 +1386,44 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 load_bf(g);
                 x_ready = true;
             }
-            if (kMma) {
+            if (kBlend) {
+                // Weights +-s as bf16 against the unquantised activations: eight k-steps of sixteen
+                // products.  K-step j takes weight word j of each of the row's four 32-weight runs
+                // (k = 32 c + 4 j .. + 3), which is the order the activation words above are held in.
+                float accf[NH][2][4];
+#pragma unroll
+                for (int h = 0; h < NH; ++h)
+#pragma unroll
+                    for (int mh = 0; mh < 2; ++mh)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) accf[h][mh][r] = 0.f;
+                const uint32_t sbits = *reinterpret_cast<const uint16_t *>(stage + off_scale);
+                const uint32_t s_hi = sbits >> 8, s_lo = sbits & 0xFFu;
+                const uint32_t hi_a = s_hi << 8, hi_b = (s_hi | 0x80u) << 24, lo_a = s_lo << 8, lo_b = s_lo << 24;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (j) __syncwarp();             // everyone has read the previous block back
+                    uint32_t p01[4], p23[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) blend4(static_cast<uint32_t>(w[8 * c + j]), hi_a, hi_b, lo_a, lo_b, p01[c], p23[c]);
+                    sts128(scr_st, p01[0], p01[1], p01[2], p01[3]);
+                    sts128(scr_st + 16u, p23[0], p23[1], p23[2], p23[3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int mh = 0; mh < 2; ++mh) {
+                        uint32_t a[4];
+                        ldmatrix_x4(a, scr_ld + static_cast<uint32_t>(mh * 16 * kScrRowBytes));
+#pragma unroll
+                        for (int h = 0; h < NH; ++h) mma_bf16(accf[h][mh], a, bf[h][(kBlend ? 2 : 0) * j], bf[h][(kBlend ? 2 : 0) * j + (kBlend ? 1 : 0)]);
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < NH; ++h)
+#pragma unroll
+                    for (int mh = 0; mh < 2; ++mh)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) ysum[(h * 2 + mh) * 4 + r] = accf[h][mh][r];
+            } else if (kMma) {
                 int acc[NH][2][4];
 #pragma unroll
                 for (int h = 0; h < NH; ++h)
@@ -1498,21 +1576,21 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 }
 
 // One problem, this block's share of its items.
-template <int FMT, int NB, bool DEBUG = true, int TPW = 1, bool XG = false, bool XQ = false>
+template <int FMT, int NB, bool DEBUG = true, int TPW = 1, bool XG = false, bool XQ = false, bool BL = false>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
                                             const FirstOff *fo = nullptr, int fo_index = 0) {
-    OneSegT<DEBUG, XG, XQ> one;
+    OneSegT<DEBUG, XG, XQ, BL> one;
     one.pr = &pr;
     one.wk = wk;
     one.used = false;
     run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index);
 }
 
-template <int FMT, int NB, int TPW = 1, bool XG = false, bool XQ = false>
+template <int FMT, int NB, int TPW = 1, bool XG = false, bool XQ = false, bool BL = false>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_kernel(const Problem pr, const Plan pl,
                                                                         const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
-    run_problem<FMT, NB, true, TPW, XG, XQ>(pr, pl, smem,
+    run_problem<FMT, NB, !BL, TPW, XG, XQ, BL>(pr, pl, smem,
                          block_walk(fo, static_cast<int>(blockIdx.x), pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                          static_cast<int>(blockIdx.x), &fo, static_cast<int>(blockIdx.x));
 }
@@ -1576,6 +1654,7 @@ struct GroupedSegs {
     static constexpr bool kDebug = true;
     static constexpr bool kGroupScales = false;
     static constexpr bool kQuantize = false;
+    static constexpr bool kBlend = false;
     __device__ __forceinline__ const Problem &shape() const { return *base; }
     __device__ __forceinline__ bool next(View &v, Walk &w) {
         while (lo < hi) {
@@ -1865,12 +1944,12 @@ inline bool wants_two_tiles(const Plan &pl, int nb_template, int sms) {
     return nb_template < kMmaMinBatch && pl.items >= 8 * static_cast<int64_t>(sms);
 }
 
-template <int FMT, int NB, bool XG = false, bool XQ = false>
+template <int FMT, int NB, bool XG = false, bool XQ = false, bool BL = false>
 int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint32_t *off_host = nullptr) {
     // the one- and two-token instantiations keep the activations in shared memory (nb_bucket sees to it)
     if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * pr.K > kXResidentBytes) return BITCOS_ERR_SHAPE;
     int sms = 0, budget = 0;
-    int rc = prepare_kernel<gemv_kernel<FMT, NB, 1, XG, XQ>>(&sms, &budget);
+    int rc = prepare_kernel<gemv_kernel<FMT, NB, 1, XG, XQ, BL>>(&sms, &budget);
     if (rc) return rc;
     const bool two = wants_two_tiles(pl_in, NB, sms);
     if constexpr (NB < kMmaMinBatch) {
@@ -1892,7 +1971,7 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     if constexpr (NB < kMmaMinBatch) {
         if (two) return launch_pdl(gemv_kernel<FMT, NB, 2, XG, XQ>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
     }
-    return launch_pdl(gemv_kernel<FMT, NB, 1, XG, XQ>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
+    return launch_pdl(gemv_kernel<FMT, NB, 1, XG, XQ, BL>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
 template <int NB, bool XQ = false, bool XG = false>
@@ -2324,6 +2403,20 @@ int bitcos_gemv_multi_group_scales(const bitcos_gemv_job *jobs, int n_jobs, int 
 
 int bitcos_gemv_multi_bf16(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
     return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, true);
+}
+
+int bitcos_gemv_blend_bf16(const bitcos_weights *W, const uint16_t *x_bf16, int batch, float *y, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream) {
+    if (!W) return BITCOS_ERR_NULL;
+    if (batch > 8) return BITCOS_ERR_SHAPE;
+    const int8_t *x = reinterpret_cast<const int8_t *>(x_bf16);
+    const int bad = check_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x,
+                                 reinterpret_cast<const float *>(x), batch, y, nullptr, workspace, workspace_bytes);
+    if (bad) return bad;
+    const Plan pl = make_plan(W->M, W->K, decoder_warps(8));
+    Problem pr{};
+    fill_problem(pr, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, nullptr, batch, y, nullptr, workspace);
+    return launch<kBitcos, 8, false, false, true>(pr, pl, static_cast<cudaStream_t>(cuda_stream), W->tile_off_host);
 }
 
 int bitcos_gemv_bf16(const bitcos_weights *W, const uint16_t *x_bf16, int batch, float *y, int32_t *acc_debug,
