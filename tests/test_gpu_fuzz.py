@@ -118,4 +118,9 @@ def test_seeded_sweep_quantised_front_end(bc, seed):
             assert np.array_equal(acc2.cpu().numpy(), acc_ref[:nb]), what
             assert (np.abs(y2.cpu().numpy().astype(np.float64) - y_ref[:nb]) <= REL * mag[:nb]).all(), what
             assert (np.abs(y3.cpu().numpy().astype(np.float64) - y_ref[:nb]) <= REL * mag[:nb]).all(), what
+        nbl = min(B, 1 + it % 8)
+        yb = bc.bitcos_gemv_blend_bf16(Wd, xb[:nbl].contiguous(), workspace=ws)
+        torch.cuda.synchronize()
+        yb_ref, magb = oracle.gemv_dense_blend(W, S, xf[:nbl])
+        assert (np.abs(yb.cpu().numpy().astype(np.float64) - yb_ref) <= 4e-5 * magb).all(), what
         assert bc.workspace_status(ws) == 0, what
