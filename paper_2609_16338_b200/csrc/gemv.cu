@@ -1233,13 +1233,13 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     auto load_bf = [&](int g) {
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
-            if (kBlend) {
+            if constexpr (kBlend) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     int4 u = make_int4(0, 0, 0, 0);
                     if (xfrag[h]) u = __ldg(reinterpret_cast<const int4 *>(xfrag[h] + static_cast<int64_t>(g) * (2 * kGroup)) + q);
-                    bf[h][(kBlend ? 4 : 0) * q + 0] = u.x; bf[h][(kBlend ? 4 : 0) * q + 1] = u.y;
-                    bf[h][(kBlend ? 4 : 0) * q + 2] = u.z; bf[h][(kBlend ? 4 : 0) * q + 3] = u.w;
+                    bf[h][4 * q + 0] = u.x; bf[h][4 * q + 1] = u.y;
+                    bf[h][4 * q + 2] = u.z; bf[h][4 * q + 3] = u.w;
                 }
                 continue;
             }
@@ -1386,7 +1386,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 load_bf(g);
                 x_ready = true;
             }
-            if (kBlend) {
+            if constexpr (kBlend) {
                 // Weights +-s as bf16 against the unquantised activations: eight k-steps of sixteen
                 // products.  K-step j takes weight word j of each of the row's four 32-weight runs
                 // (k = 32 c + 4 j .. + 3), which is the order the activation words above are held in.
@@ -1414,7 +1414,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                         uint32_t a[4];
                         ldmatrix_x4(a, scr_ld + static_cast<uint32_t>(mh * 16 * kScrRowBytes));
 #pragma unroll
-                        for (int h = 0; h < NH; ++h) mma_bf16(accf[h][mh], a, bf[h][(kBlend ? 2 : 0) * j], bf[h][(kBlend ? 2 : 0) * j + (kBlend ? 1 : 0)]);
+                        for (int h = 0; h < NH; ++h) mma_bf16(accf[h][mh], a, bf[h][2 * j], bf[h][2 * j + 1]);
                     }
                 }
 #pragma unroll
