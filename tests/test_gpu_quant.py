@@ -278,3 +278,41 @@ def test_multi_launch_with_group_scales(bc, B):
             torch.cuda.synchronize()
             assert torch.equal(y1, y)
             assert bc.workspace_status(ws) == 0
+
+
+def test_entry_points_inside_a_cuda_graph(bc):
+    """Quantiser, products with group scales, from bf16 activations and the 16-bit variant captured
+    into one CUDA graph (after a first eager call each, which does the one-time set-up) and
+    replayed: the same bits as the eager calls."""
+    M, K, B = 2560, 2560, 2
+    W, S = datagen.trits(2900, M, K, 0.4219), datagen.scales(2900, M, K)
+    Wd = bc.bitcos_pack(W, S).to_device()
+    ws = bc.make_workspace(M, K)
+    xb = dev_bf16(datagen.activations_bf16(2900, B, K))
+    q = torch.empty((B, K), dtype=torch.int8, device="cuda")
+    sg = torch.empty((B, K // 128), dtype=torch.float32, device="cuda")
+    y1, y2, y3 = (torch.empty((B, M), dtype=torch.float32, device="cuda") for _ in range(3))
+
+    def run():
+        bc.bitcos_quantize_activations(xb, 128, xq=q, x_scale=sg)
+        bc.bitcos_gemv_group_scales(Wd, q, sg, y=y1, workspace=ws)
+        bc.bitcos_gemv_bf16(Wd, xb, y=y2, workspace=ws)
+        bc.bitcos_gemv_blend_bf16(Wd, xb, y=y3, workspace=ws)
+
+    run()
+    torch.cuda.synchronize()
+    eager = [t.clone() for t in (q, sg, y1, y2, y3)]
+    assert torch.equal(y1, y2)                       # the fused product is the two-step chain, bit for bit
+    stream = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            run()
+        for rep in range(2):
+            for t in (q, sg, y1, y2, y3):
+                t.zero_()
+            g.replay()
+            stream.synchronize()
+            for t, e in zip((q, sg, y1, y2, y3), eager):
+                assert torch.equal(t, e), rep
+    assert bc.workspace_status(ws) == 0
