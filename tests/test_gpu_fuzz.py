@@ -109,7 +109,7 @@ def test_seeded_sweep_quantised_front_end(bc, seed):
         qt, st = bc.bitcos_quantize_activations(xb, 0)
         torch.cuda.synchronize()
         assert np.array_equal(qt.cpu().numpy(), qt_ref) and np.array_equal(st.cpu().numpy(), st_ref), what
-        nb = 1 + it % 2
+        nb = min(B, 1 + it % 2)
         if nb * K <= 49152:
             y2, acc2 = bc.bitcos_gemv_bf16(Wd, xb[:nb].contiguous(), acc_debug=True, workspace=ws)
             y3 = torch.empty((nb, M), dtype=torch.float32, device="cuda")
