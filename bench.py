@@ -894,17 +894,26 @@ def run_profile_batch(args):
     xd, xsd = torch.from_numpy(x).cuda(), torch.from_numpy(xs).cuda()
     y = torch.empty((B, M), dtype=torch.float32, device="cuda")
     ws = bc.make_workspace(M, K)
+    if args.profile_entry == "blend":
+        # the 16-bit variant: weights +-s against unquantised bf16 activations
+        xb = torch.from_numpy(datagen.activations_bf16(seed, B, K).view(np.int16)).cuda().view(torch.bfloat16)
+
+        def call(i):
+            bc.bitcos_gemv_blend_bf16(reps[i % n_copies], xb, y=y, workspace=ws)
+    else:
+        def call(i):
+            bc.bitcos_gemv(reps[i % n_copies], xd, xsd, y=y, workspace=ws)
     for i in range(3):
-        bc.bitcos_gemv(reps[i % n_copies], xd, xsd, y=y, workspace=ws)
+        call(i)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
-        bc.bitcos_gemv(reps[i % n_copies], xd, xsd, y=y, workspace=ws)
+        call(i)
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / args.steps
-    print(json.dumps({"profile_batch": B, "M": M, "K": K, "launches": args.steps + 3, "us_per_launch_with_host_gaps": us,
+    print(json.dumps({"profile_batch": B, "entry": args.profile_entry, "M": M, "K": K, "launches": args.steps + 3, "us_per_launch_with_host_gaps": us,
                       "status": bc.workspace_status(ws)}))
 
 
@@ -973,6 +982,8 @@ def main():
     ap.add_argument("--profile-quant", default="", choices=["", "chain", "fused"],
                     help="only launch --steps layer passes from bf16 activations (quantiser kernels in front of the "
                          "products, or inside them), without graphs (for profilers)")
+    ap.add_argument("--profile-entry", default="gemv", choices=["gemv", "blend"],
+                    help="entry point --profile-batch launches: bitcos_gemv or bitcos_gemv_blend_bf16")
     ap.add_argument("--profile-shape", default="8192x5120", metavar="MxK",
                     help="matrix of --profile-batch (default: the batch table's q projection)")
     ap.add_argument("--profile-batch", type=int, default=0, metavar="B",
