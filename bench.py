@@ -774,7 +774,7 @@ def quant_detail(bc, torch, stream):
 
 def pack_detail(bc, torch):
     """Device-side packing (set-up path): int8 trits + bf16 scales in device memory -> the BITCOS
-    buffers.  Wall time of the whole call (count pass, three kernels, two stream waits), against
+    buffers.  Wall time of the whole call (three kernels, two stream waits, the sign vector cut to size), against
     the bytes it has to move once: the trits in, the packed buffers out."""
     import time
     import datagen
@@ -794,7 +794,7 @@ def pack_detail(bc, torch):
         us = float(np.median(times))
         nbytes = M * K + S.nbytes + Wd.payload_bytes()
         out.append({"M": M, "K": K, "us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
-                    "bytes_once": int(nbytes), "note": "the trits are read three times (count, bitmap, signs)"})
+                    "bytes_once": int(nbytes), "note": "the trits are read twice (bitmap and counts, signs)"})
         del Wt, St, Wd
         torch.cuda.empty_cache()
     return out

@@ -240,20 +240,26 @@ def bitcos_pack_device(trits, scales_bf16) -> "DeviceBitcos":
     if trits.dtype != torch.int8 or trits.dim() != 2 or not trits.is_contiguous() or not scales_bf16.is_contiguous():
         raise ValueError("trits must be a contiguous int8 [M, K] tensor, scales contiguous")
     M, K = trits.shape
-    nnz = bitcos_count_nnz_device(trits)
+    # the sign vector is sized for the worst case (every weight non-zero) and cut to size afterwards:
+    # one pass over the trits less than counting first
+    Mp = (M + TILE_ROWS - 1) // TILE_ROWS * TILE_ROWS
     sizes = [C.c_size_t(0) for _ in range(4)]
-    _check(L.bitcos_pack_sizes(M, K, nnz, *[C.byref(v) for v in sizes]), "bitcos_pack_sizes")
+    _check(L.bitcos_pack_sizes(M, K, min(Mp * K, 0xFFFFFFFF), *[C.byref(v) for v in sizes]), "bitcos_pack_sizes")
     dev = trits.device
     bitmap = torch.empty(sizes[0].value // 4, dtype=torch.int32, device=dev)
-    signs = torch.empty(sizes[1].value // 4, dtype=torch.int32, device=dev)
+    signs_max = torch.empty(sizes[1].value // 4, dtype=torch.int32, device=dev)
     tile_off = torch.empty(sizes[2].value // 4, dtype=torch.int32, device=dev)
     scales = torch.empty(sizes[3].value // 2, dtype=torch.int16, device=dev)
     off_host = np.zeros(sizes[2].value // 4, np.uint32)
     scratch = torch.empty(PACK_SCRATCH_BYTES, dtype=torch.uint8, device=dev)
     out = C.c_uint64(0)
-    _check(L.bitcos_pack_device(trits.data_ptr(), scales_bf16.data_ptr(), M, K, bitmap.data_ptr(), signs.data_ptr(),
+    _check(L.bitcos_pack_device(trits.data_ptr(), scales_bf16.data_ptr(), M, K, bitmap.data_ptr(), signs_max.data_ptr(),
                                 sizes[1].value, tile_off.data_ptr(), scales.data_ptr(), _ptr(off_host), C.byref(out),
                                 scratch.data_ptr(), _stream()), "bitcos_pack_device")
+    need = C.c_size_t(0)
+    _check(L.bitcos_pack_sizes(M, K, out.value, None, C.byref(need), None, None), "bitcos_pack_sizes")
+    signs = signs_max[:need.value // 4].clone()
+    del signs_max
     n_tiles = (M + TILE_ROWS - 1) // TILE_ROWS * (K // GROUP)
     return DeviceBitcos(M, K, int(out.value), bitmap, signs, tile_off, scales,
                         tile_off_host=np.ascontiguousarray(off_host[:n_tiles + 1]))
