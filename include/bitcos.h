@@ -205,6 +205,30 @@ int bitcos_workspace_status(const void *workspace, void *cuda_stream, int *statu
  * weights per multiprocessor = cycles / (iters * warps_per_block * 128). */
 int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, uint64_t *cycles, void *cuda_stream);
 
+/* The same measurement for each of the library's BITCOS decoders, on real packed tiles, with the
+ * accumulators handed back so that every decoder can be checked (Section II-D notes that the unpack
+ * sequence, not the format, decides whether the saved bytes turn into time; Eq. 6's gamma is what
+ * this measures).  bitmap / signs / tile_off describe one item of n_tiles consecutive tiles of a
+ * packed matrix (device pointers: bitmap = the first tile's, tile_off = its entry, signs = the
+ * matrix's whole sign vector of sign_bytes bytes); x = device int8 [n_tiles][128], the activations of
+ * tile t's group.  A block of n_tiles warps (1..32) copies the item into shared memory once; warp t then
+ * computes, `iters` times, the 32 int32 group accumulators of tile t (row r in lane r) from shared
+ * memory only.  cycles (device uint64 [blocks]) as for bitcos_decode_probe; acc_out = NULL or device
+ * int32 [n_tiles][32], written by block 0.
+ *   variant 0  shifted window: (presence nibble, sign nibble) table of Eq. 4, the window of a word
+ *              shifted by each nibble's population count; decode into registers, then contract
+ *   variant 1  running position: the same table, windows never shifted, a running bit position per
+ *              word updated by the dp4a that counts; contraction fused (what the products run)
+ *   variant 2  byte table: eight weights per step from a 3^8-entry table behind a 256-entry index
+ *   variant 3  no table: the deposit of Fig. 4 with shifts and masks, contraction on bit planes
+ *   variant 4  lane = bit: one presence word per warp step, sign slot = population count of the
+ *              lower bits, products added across the warp
+ * ERR_CAPACITY if the item does not fit into shared memory with the variant's tables. */
+#define BITCOS_PROBE_VARIANTS 5
+int bitcos_decode_probe_variant(int variant, const uint32_t *bitmap, const uint32_t *signs, size_t sign_bytes,
+                                const uint32_t *tile_off, int n_tiles, const int8_t *x, int iters, int blocks,
+                                uint64_t *cycles, int32_t *acc_out, void *cuda_stream);
+
 /* y[b][m] for b < batch, m < M from a BITCOS matrix (steps of Section II-B..II-D on the GPU:
  * entry offset + running population count locate each row's sign window, a 256-entry
  * (presence nibble, sign nibble) table as in Eq. 4 rebuilds four weights at a time as int8,

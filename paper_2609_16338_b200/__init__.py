@@ -34,6 +34,8 @@ from .binding import (  # noqa: F401
     bitcos_pack_device,
     MultiHostJobs,
     bitcos_decode_probe,
+    bitcos_decode_probe_variant,
+    PROBE_VARIANTS,
     group_pairs,
     plain_to_device,
     scales_tile,

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant",
 ]
 
 
@@ -97,6 +97,7 @@ def load_library():
     L.bitcos_gemv_host.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, sz, vp, sz, vp]
     L.bitcos_gemv_static.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp]
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.bitcos_decode_probe_variant.argtypes = [C.c_int, vp, vp, sz, vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp]
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
     L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
@@ -551,6 +552,27 @@ def bitcos_decode_probe(fmt: int, warps_per_block: int, iters: int, blocks: int)
     torch.cuda.synchronize()
     c = cyc.cpu().numpy().astype(np.float64)
     return float(np.median(c)) / (iters * warps_per_block * 128.0)
+
+
+PROBE_VARIANTS = ("shifted window", "running position", "byte table", "no table", "lane = bit")
+
+
+def bitcos_decode_probe_variant(variant: int, W: DeviceBitcos, first_tile: int, n_tiles: int, x, iters: int, blocks: int,
+                                want_acc: bool = False):
+    """On-chip cost of one BITCOS decoder on tiles first_tile .. first_tile + n_tiles - 1 of W (x = int8
+    [n_tiles, 128], the activations of each tile's group): cycles per 32 weights per multiprocessor, and the
+    int32 accumulators [n_tiles, 32] of the last pass if asked for."""
+    import torch
+    cyc = torch.zeros(blocks, dtype=torch.int64, device="cuda")
+    acc = torch.zeros((n_tiles, TILE_ROWS), dtype=torch.int32, device="cuda") if want_acc else None
+    _check(load_library().bitcos_decode_probe_variant(
+        variant, W.bitmap.data_ptr() + first_tile * 512, W.signs.data_ptr(), W.signs.numel() * 4,
+        W.tile_off.data_ptr() + first_tile * 4, n_tiles, x.data_ptr(), iters, blocks, cyc.data_ptr(),
+        acc.data_ptr() if acc is not None else None, _stream()), "bitcos_decode_probe_variant")
+    torch.cuda.synchronize()
+    c = cyc.cpu().numpy().astype(np.float64)
+    gamma = float(np.median(c)) / (iters * n_tiles * 128.0)
+    return (gamma, acc) if want_acc else gamma
 
 
 STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024

@@ -8,8 +8,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbitcos.so")
-SOURCES = [os.path.join(CSRC, "gemv.cu"), os.path.join(CSRC, "pack_device.cu"), os.path.join(CSRC, "pack.cpp")]
-HEADERS = [os.path.join(ROOT, "include", "bitcos.h")]
+SOURCES = [os.path.join(CSRC, "gemv.cu"), os.path.join(CSRC, "probe.cu"), os.path.join(CSRC, "pack_device.cu"),
+           os.path.join(CSRC, "pack.cpp")]
+HEADERS = [os.path.join(ROOT, "include", "bitcos.h"), os.path.join(CSRC, "decode.cuh")]
 
 
 def nvcc_command(extra=()):

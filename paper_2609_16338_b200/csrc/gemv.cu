@@ -28,6 +28,7 @@
 // a lane's row are decoded as four independent chains, each shifting its own sign window by
 // the number of sign bits a nibble consumed.
 #include "bitcos.h"
+#include "decode.cuh"
 
 #include <cuda_runtime.h>
 
@@ -36,12 +37,13 @@
 
 namespace {
 
+using namespace bitcos_dev;
+
 constexpr int kGroup = BITCOS_GROUP;
 constexpr int kRows = BITCOS_TILE_ROWS;
 constexpr int kMaxWarps = 20;             // warps per thread block = tiles per item
 constexpr int kWarps16 = 14;              // the same for more than 8 tokens (16 warps per block: 128 registers per thread)
 constexpr int kMaxStages = 8;             // upper bound on the shared-memory ring depth (Plan::stages)
-constexpr int kLutBytes = 64 * 1024;      // replicated lookup tables (BITCOS, five-trit)
 constexpr uint64_t kWaitLimitNs = 500ull * 1000 * 1000;   // an mbarrier wait gives up after half a second
 constexpr int64_t kXResidentBytes = 48 * 1024;   // activations up to this size are kept in shared memory
 constexpr int kMmaMinBatch = 4;           // from this many tokens on the contraction runs on the tensor cores
@@ -52,85 +54,8 @@ enum Format { kBitcos = 0, kTrit5 = 1, kBit2 = 2 };
 
 thread_local int g_last_cuda_error = 0;
 
-// ---------------------------------------------------------------------------------------------
-// Lookup tables, generated at compile time.
-// ---------------------------------------------------------------------------------------------
-struct Lut256 {
-    uint32_t v[256];
-};
-struct Lut256x2 {
-    uint32_t lo[256];
-    uint32_t hi[256];
-};
-
-// Entry (m, s) of Eq. 4 as four int8: byte i = 0 if bit i of m is clear, else +1 / -1 by the
-// sign bit whose index is the rank of i among the set bits of m.  Index = (s << 4) | m.
-constexpr Lut256 make_nibble_lut() {
-    Lut256 t{};
-    for (int key = 0; key < 256; ++key) {
-        const int m = key & 15, s = key >> 4;
-        uint32_t e = 0;
-        int r = 0;
-        for (int i = 0; i < 4; ++i) {
-            if ((m >> i) & 1) {
-                e |= (((s >> r) & 1) ? 0xFFu : 0x01u) << (8 * i);
-                ++r;
-            }
-        }
-        t.v[key] = e;
-    }
-    return t;
-}
-
-// Five-trit byte -> digits t0..t4 (value - 1 each) as int8: lo = (t0,t1,t2,t3), hi = (t1,t2,t3,t4).
-constexpr Lut256x2 make_trit5_lut() {
-    Lut256x2 t{};
-    for (int b = 0; b < 256; ++b) {
-        int v = b;
-        uint32_t d[5] = {0, 0, 0, 0, 0};
-        for (int i = 0; i < 5; ++i) {
-            d[i] = static_cast<uint32_t>((v % 3) - 1) & 0xFFu;
-            v /= 3;
-        }
-        t.lo[b] = d[0] | (d[1] << 8) | (d[2] << 16) | (d[3] << 24);
-        t.hi[b] = d[1] | (d[2] << 8) | (d[3] << 16) | (d[4] << 24);
-    }
-    return t;
-}
-
-// The tables as they sit in shared memory, replicated once per lane (32 copies) so that a warp's
-// 32 lookups always fall into 32 different banks.  They live in global memory in that final
-// form and each thread block fetches its copy with one bulk asynchronous copy.
-struct LutBig {
-    uint32_t v[kLutBytes / 4];
-};
-
-// BITCOS: byte address = key * 256 + sub * 128 + lane * 4;
-//   sub 0 ("even" nibbles): key = (s << 4) | m;  sub 1 ("odd" nibbles): key = (m << 4) | s,
-// so that a presence BYTE placed in address bits 8..15 needs only its other nibble replaced
-// by the four sign bits.
-constexpr LutBig make_bitcos_lut() {
-    const Lut256 base = make_nibble_lut();
-    LutBig t{};
-    for (int idx = 0; idx < kLutBytes / 4; ++idx) {
-        const int key = idx >> 6, sub = (idx >> 5) & 1;
-        const int src = sub ? (((key & 15) << 4) | (key >> 4)) : key;
-        t.v[idx] = base.v[src];
-    }
-    return t;
-}
-
-// Five-trit: byte address = byte value * 256 + lane * 8 (lo word, hi word).
-constexpr LutBig make_trit5_big() {
-    const Lut256x2 base = make_trit5_lut();
-    LutBig t{};
-    for (int idx = 0; idx < kLutBytes / 4; ++idx) {
-        const int key = idx >> 6;
-        t.v[idx] = (idx & 1) ? base.hi[key] : base.lo[key];
-    }
-    return t;
-}
-
+// The replicated lookup tables in their shared-memory form (decode.cuh); each thread block fetches
+// its copy from global memory with one bulk asynchronous copy.
 __device__ __align__(128) const LutBig g_bitcos_lut = make_bitcos_lut();
 __device__ __align__(128) const LutBig g_trit5_lut = make_trit5_big();
 
@@ -311,18 +236,6 @@ __host__ __device__ inline SmemLayout smem_layout(int fmt, const Plan &pl, int G
 // ---------------------------------------------------------------------------------------------
 // Device helpers.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t lds32(const uint8_t *base, uint32_t off) {
-    return *reinterpret_cast<const uint32_t *>(base + off);
-}
-__device__ __forceinline__ uint2 lds64(const uint8_t *base, uint32_t off) {
-    return *reinterpret_cast<const uint2 *>(base + off);
-}
-// dot product of four unsigned bytes of a with four signed bytes of b, plus c
-__device__ __forceinline__ int dp4a_us(uint32_t a, int b, int c) {
-    int d;
-    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
 __device__ __forceinline__ float bf16_to_float(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -374,13 +287,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return mbar_wait_slow(bar, parity);
 }
 
-// d = (a & c) | (b & ~c): one LOP3
-__device__ __forceinline__ uint32_t bit_select(uint32_t a, uint32_t b, uint32_t c) {
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xE4;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-
 // Four 8x8 matrices of 16-bit elements from shared memory, one row address per lane: as int8 data
 // this is exactly the A operand (16 rows x 32 bytes) of mma.m16n8k32.
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr) {
@@ -400,11 +306,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t r;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-    return r;
 }
 // Four decoded weights (bytes 0x00, 0x01, 0xFF) -> four bf16 values 0, +s, -s (the scale blended
 // into the weight, Section II-B): the low three bits of a weight byte (0, 1, 7) pick the high and
@@ -428,90 +329,6 @@ __device__ __forceinline__ void sts128(uint32_t addr, int a, int b, int c, int d
 // Tile decoders.  For the lane's row they produce the 32 int8x4 words of the row; the contraction
 // follows as a separate step (dp4a per token, or the tensor cores from four tokens on).
 // ---------------------------------------------------------------------------------------------
-
-// BITCOS: bm = the row's four presence words, sp = the stage's sign words at the word holding the
-// row's first sign bit, sh = bit offset inside that word.  w receives the row's 32 int8x4 words.
-__device__ __forceinline__ void bitcos_decode_row(const uint4 bm, const uint32_t *sp, uint32_t sh, const uint8_t *lut,
-                                                  uint32_t lane4, int (&w)[32]) {
-    const int c0 = __popc(bm.x), c1 = __popc(bm.y), c2 = __popc(bm.z);
-    const uint32_t s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3], s4 = sp[4];
-    uint32_t a0 = __funnelshift_r(s0, s1, sh), a1 = __funnelshift_r(s1, s2, sh);
-    uint32_t a2 = __funnelshift_r(s2, s3, sh), a3 = __funnelshift_r(s3, s4, sh);
-    uint32_t S[4];
-    S[0] = a0;
-    a0 = __funnelshift_rc(a0, a1, c0);
-    a1 = __funnelshift_rc(a1, a2, c0);
-    a2 = __funnelshift_rc(a2, a3, c0);
-    S[1] = a0;
-    a0 = __funnelshift_rc(a0, a1, c1);
-    a1 = __funnelshift_rc(a1, a2, c1);
-    S[2] = a0;
-    S[3] = __funnelshift_rc(a0, a1, c2);
-    const uint32_t P[4] = {bm.x, bm.y, bm.z, bm.w};
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            // address bits 0..6 = lane * 4, bits 8..15 = presence byte k of word j (bits 16.. are 0)
-            const uint32_t R = __byte_perm(P[j], lane4, 0x6504 | (k << 4));
-            uint32_t off = bit_select(S[j] << 12, R, 0xF000u);     // sign nibble over the odd presence nibble
-            int e = static_cast<int>(lds32(lut, off));
-            w[8 * j + 2 * k] = e;
-            S[j] >>= __dp4a(e, e, 0);                    // non-zeros in the nibble = sign bits consumed
-            off = bit_select(S[j] << 8, R, 0x0F00u);               // sign nibble over the even presence nibble
-            e = static_cast<int>(lds32(lut + 128, off));
-            w[8 * j + 2 * k + 1] = e;
-            S[j] >>= __dp4a(e, e, 0);
-        }
-    }
-}
-
-// Five-trit: wd = the seven words that hold the row's 26 bytes, odd = byte offset 2 (odd group).
-__device__ __forceinline__ void trit5_decode_row(const uint32_t (&wd)[7], int odd, const uint8_t *lut, uint32_t lane8,
-                                                 int (&w)[32]) {
-    uint32_t lo[26], hi[26];
-#pragma unroll
-    for (int j = 0; j < 26; ++j) {
-        const int be = j, bo = j + 2;
-        const uint32_t word = odd ? wd[bo >> 2] : wd[be >> 2];
-        const uint32_t sel = odd ? (0x6504u | ((bo & 3) << 4)) : (0x6504u | ((be & 3) << 4));
-        const uint32_t off = __byte_perm(word, lane8, sel);    // byte * 256 + lane * 8
-        const uint2 e = lds64(lut, off);
-        lo[j] = e.x;
-        hi[j] = e.y;
-    }
-#pragma unroll
-    for (int q = 0; q < 6; ++q) {
-        w[5 * q + 0] = static_cast<int>(lo[4 * q]);
-        w[5 * q + 1] = static_cast<int>(__byte_perm(hi[4 * q], lo[4 * q + 1], 0x6543));
-        w[5 * q + 2] = static_cast<int>(__byte_perm(hi[4 * q + 1], lo[4 * q + 2], 0x5432));
-        w[5 * q + 3] = static_cast<int>(__byte_perm(hi[4 * q + 2], lo[4 * q + 3], 0x4321));
-        w[5 * q + 4] = static_cast<int>(hi[4 * q + 3]);
-    }
-    w[30] = static_cast<int>(lo[24]);
-    w[31] = static_cast<int>(__byte_perm(hi[24], lo[25], 0x6543));
-}
-
-// 2-bit: w[4q + j] keeps pair j of every byte of word q in place (value = code * 4^j), to be
-// multiplied with activation word 4q + j.
-__device__ __forceinline__ void bit2_decode_row(const uint4 v0, const uint4 v1, int (&w)[32]) {
-    const uint32_t wd[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-    for (int q = 0; q < 8; ++q)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) w[4 * q + j] = static_cast<int>(wd[q] & (0x03030303u << (2 * j)));
-}
-
-// 2-bit, as plain int8: w[4q + j] byte b = code - 1 of weight 16 q + 4 j + b.  Per byte,
-// (code + 0x7F) ^ 0x80 maps 0, 1, 2 to -1, 0, +1 without a carry between bytes.
-__device__ __forceinline__ void bit2_decode_row_s8(const uint4 v0, const uint4 v1, int (&w)[32]) {
-    const uint32_t wd[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-    for (int q = 0; q < 8; ++q)
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            w[4 * q + j] = static_cast<int>((((wd[q] >> (2 * j)) & 0x03030303u) + 0x7F7F7F7Fu) ^ 0x80808080u);
-}
 
 // int32 accumulator of one row (lane) and group against token activations xg[0..127] (shared memory).
 template <int FMT>
