@@ -20,6 +20,10 @@ group of 128 reduction elements drawn from U[0.01, 0.05], int8 activations unifo
 """
 from __future__ import annotations
 
+import ctypes as C
+import os
+import subprocess
+
 import numpy as np
 
 GROUP = 128
@@ -64,9 +68,41 @@ def _chunks(total: int, step: int = 1 << 24):
         pos += n
 
 
-def trits(seed: int, M: int, K: int, z: float) -> np.ndarray:
-    """int8 [M, K] with values in {-1, 0, +1}: 0 with probability z, else +-1 evenly."""
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_FILL_SRC = os.path.join(_HERE, "datagen_fill.c")
+_FILL_LIB = os.path.join(_HERE, "libdatagen_fill.so")
+_fill = None
+
+
+def build_native(force: bool = False) -> str:
+    """Compiles the native filler for large tensors (gcc); returns the library's path."""
+    if force or not os.path.exists(_FILL_LIB) or os.path.getmtime(_FILL_LIB) < os.path.getmtime(_FILL_SRC):
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-o", _FILL_LIB, _FILL_SRC])
+    return _FILL_LIB
+
+
+def _native_fill():
+    """The native filler, or None if it cannot be built here (the numpy formulation then serves)."""
+    global _fill
+    if _fill is None:
+        try:
+            L = C.CDLL(build_native())
+            L.datagen_fill_trits.restype = None
+            L.datagen_fill_trits.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64, C.c_double, C.c_void_p]
+            _fill = L
+        except (OSError, subprocess.CalledProcessError):
+            _fill = False
+    return _fill or None
+
+
+def trits(seed: int, M: int, K: int, z: float, native: bool = True) -> np.ndarray:
+    """int8 [M, K] with values in {-1, 0, +1}: 0 with probability z, else +-1 evenly.  Large
+    tensors are filled by the native helper (the same values, bit for bit)."""
     out = np.empty(M * K, dtype=np.int8)
+    L = _native_fill() if (native and M * K >= (1 << 16)) else None
+    if L is not None:
+        L.datagen_fill_trits(seed & 0xFFFFFFFFFFFFFFFF, STREAM_TRITS, 0, M * K, float(z), out.ctypes.data)
+        return out.reshape(M, K)
     half = z + (1.0 - z) / 2.0
     for pos, n in _chunks(M * K):
         u = uniform(seed, STREAM_TRITS, pos, n)

@@ -223,8 +223,10 @@ int bitcos_decode_probe(int format, int warps_per_block, int iters, int blocks, 
  *   variant 3  no table: the deposit of Fig. 4 with shifts and masks, contraction on bit planes
  *   variant 4  lane = bit: one presence word per warp step, sign slot = population count of the
  *              lower bits, products added across the warp
+ *   variant 5, 6, 7  split row: the first 1, 2, 3 presence words of a row as variant 1, the others as
+ *              variant 3 (loads the shared-memory pipe and the integer ALU at the same time)
  * ERR_CAPACITY if the item does not fit into shared memory with the variant's tables. */
-#define BITCOS_PROBE_VARIANTS 5
+#define BITCOS_PROBE_VARIANTS 8
 int bitcos_decode_probe_variant(int variant, const uint32_t *bitmap, const uint32_t *signs, size_t sign_bytes,
                                 const uint32_t *tile_off, int n_tiles, const int8_t *x, int iters, int blocks,
                                 uint64_t *cycles, int32_t *acc_out, void *cuda_stream);

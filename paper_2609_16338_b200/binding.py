@@ -554,7 +554,8 @@ def bitcos_decode_probe(fmt: int, warps_per_block: int, iters: int, blocks: int)
     return float(np.median(c)) / (iters * warps_per_block * 128.0)
 
 
-PROBE_VARIANTS = ("shifted window", "running position", "byte table", "no table", "lane = bit")
+PROBE_VARIANTS = ("shifted window", "running position", "byte table", "no table", "lane = bit", "split row 1+3",
+                  "split row 2+2", "split row 3+1")
 
 
 def bitcos_decode_probe_variant(variant: int, W: DeviceBitcos, first_tile: int, n_tiles: int, x, iters: int, blocks: int,

@@ -395,6 +395,74 @@ __device__ __forceinline__ int bitcos_row_dot_planes(const uint4 bm, const uint3
 }
 
 // ---------------------------------------------------------------------------------------------
+// Decoder F ("split row"): the first NL presence words of a row through the table with running
+// positions (decoder B), the others through the table-free deposit and bit planes (decoder D).
+// The table path is bound by shared-memory wavefronts, the table-free path by the integer ALU;
+// splitting a row between them loads both pipes.
+//   xs   the group's activations in natural order, xp the same in bit-plane order (decoder D)
+// ---------------------------------------------------------------------------------------------
+template <int NL>
+__device__ __forceinline__ int bitcos_row_dot_split(const uint4 bm, const uint32_t *sp, uint32_t sh, const uint8_t *lut,
+                                                    uint32_t lane4, const uint8_t *xs, const uint8_t *xp) {
+    uint32_t S[4];
+    sign_windows(bm, sp, sh, S);
+    const uint32_t P[4] = {bm.x, bm.y, bm.z, bm.w};
+    int acc = 0;
+    // table part
+    uint32_t A[NL > 0 ? NL : 1], B[NL > 0 ? NL : 1];
+    int pos[NL > 0 ? NL : 1], a[NL > 0 ? NL : 1];
+#pragma unroll
+    for (int j = 0; j < NL; ++j) {
+        A[j] = __funnelshift_l(S[j], S[j], 12);
+        B[j] = __funnelshift_l(S[j], S[j], 8);
+        pos[j] = 0;
+        a[j] = 0;
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+        for (int j = 0; j < NL; ++j) {
+            const int4 xq = reinterpret_cast<const int4 *>(xs)[2 * j + h];
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+                const int k = 2 * h + kk;
+                const uint32_t R = __byte_perm(P[j], lane4, 0x6504 | (k << 4));
+                uint32_t t = __funnelshift_r(A[j], A[j], pos[j]);
+                int e = static_cast<int>(lds32(lut, bit_select(t, R, 0xF000u)));
+                pos[j] = __dp4a(e, e, pos[j]);
+                a[j] = __dp4a(e, kk ? xq.z : xq.x, a[j]);
+                t = __funnelshift_r(B[j], B[j], pos[j]);
+                e = static_cast<int>(lds32(lut + 128, bit_select(t, R, 0x0F00u)));
+                pos[j] = __dp4a(e, e, pos[j]);
+                a[j] = __dp4a(e, kk ? xq.w : xq.y, a[j]);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < NL; ++j) acc += a[j];
+    // table-free part
+    if (NL < 4) {
+        int ap[8], an[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ap[i] = an[i] = 0;
+#pragma unroll
+        for (int j = NL; j < 4; ++j) {
+            const uint32_t N = deposit32(S[j], P[j]);
+            const int4 x0 = reinterpret_cast<const int4 *>(xp)[2 * j], x1 = reinterpret_cast<const int4 *>(xp)[2 * j + 1];
+            const int xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                ap[i] = dp4a_us(P[j] & (0x01010101u << i), xw[i], ap[i]);
+                an[i] = dp4a_us(N & (0x01010101u << i), xw[i], an[i]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc += (ap[i] - 2 * an[i]) >> i;
+    }
+    return acc;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Decoder E ("lane = bit"): the whole warp works on one presence word at a time, lane i on bit i:
 // a weight's sign slot is the population count of the word's lower bits, its sign is that bit of
 // the window at the warp's running cursor, and the 32 products are added across the warp.  Rows

@@ -35,7 +35,7 @@ __host__ __device__ inline ProbeLayout probe_layout(int variant, int n_tiles) {
     ProbeLayout L{};
     uint32_t off = 0;
     L.lut = off;
-    off += (variant <= 2) ? kLutBytes : 0;
+    off += (variant <= 2 || variant >= 5) ? kLutBytes : 0;
     L.second = off;
     off += (variant == 2) ? ((kByteTableBytes + 127) / 128 * 128) : 0;
     L.bitmap = off;
@@ -67,7 +67,7 @@ probe_variant_kernel(const uint32_t *__restrict__ bitmap, const uint32_t *__rest
     uint8_t *s_x = smem + L.x, *s_xp = smem + L.xp;
 
     // ---- set-up (untimed): tables, the item's packed bytes, activations in both orders
-    if (VAR <= 1) {
+    if (VAR <= 1 || VAR >= 5) {
         // byte address = key * 256 + sub * 128 + lane * 4 (see make_bitcos_lut)
         for (int idx = threadIdx.x; idx < kLutBytes / 4; idx += blockDim.x) {
             const int key = idx >> 6, sub = (idx >> 5) & 1;
@@ -123,8 +123,10 @@ probe_variant_kernel(const uint32_t *__restrict__ bitmap, const uint32_t *__rest
                 a = acc[0];
             } else if (VAR == 2) {
                 a = bitcos_row_dot_bytes(bm, sp, cursor & 31u, lut, smem + L.second, lane4, xg);
-            } else {
+            } else if (VAR == 3) {
                 a = bitcos_row_dot_planes(bm, sp, cursor & 31u, xpg);
+            } else {
+                a = bitcos_row_dot_split<VAR - 4>(bm, sp, cursor & 31u, lut, lane4, xg, xpg);     // variants 5, 6, 7: 1, 2, 3 words through the table
             }
         }
         last = a;
@@ -183,6 +185,9 @@ extern "C" int bitcos_decode_probe_variant(int variant, const uint32_t *bitmap, 
         case 1: return launch_probe<1>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
         case 2: return launch_probe<2>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
         case 3: return launch_probe<3>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
-        default: return launch_probe<4>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
+        case 4: return launch_probe<4>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
+        case 5: return launch_probe<5>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
+        case 6: return launch_probe<6>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
+        default: return launch_probe<7>(bitmap, signs, tile_off, sw, x, n_tiles, iters, blocks, out, acc_out, stream);
     }
 }

@@ -55,7 +55,7 @@ def special_matrix(seed, M, K):
     return W
 
 
-@pytest.mark.parametrize("variant", range(5))
+@pytest.mark.parametrize("variant", range(8))
 def test_every_decoder_matches_the_oracle(bc, variant):
     for case, (M, K) in enumerate(((320, 384), (64, 1024))):
         W = special_matrix(100 + case, M, K) if case == 0 else datagen.trits(77, M, K, 0.42)
