@@ -273,6 +273,10 @@ def run_cuda(args):
     multi = [[bc.MultiJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in g]) for g in groups]
              for rep in replicas]
 
+    phases = [p for p, g in enumerate(groups) for _ in g]
+    order = [j for g in groups for j in g]
+    phased = [bc.PhasedJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in order], phases) for rep in replicas]
+
     def step(i):
         """One layer pass: q | k | v, then o, then gate | up, then down.  GEMVs that read the same
         input have no dependency on one another and are launched on forked streams (parallel
@@ -285,6 +289,9 @@ def run_cuda(args):
         if args.serial:
             for j in range(len(layer)):
                 run(j)
+            return
+        if args.launch == "phased":
+            bc.bitcos_gemv_phased(phased[i % copies])
             return
         if not args.branches:
             for mj in multi[i % copies]:
@@ -357,43 +364,37 @@ def run_cuda(args):
             for i in range(self.n):
                 step(i)
 
-    full, rem = divmod(args.steps, copies)
-    with torch.cuda.stream(stream):
-        if full:
-            graphs["full"] = Eager(copies) if args.no_graph else capture(copies, 0)
-        if rem:
-            graphs["rem"] = Eager(rem) if args.no_graph else capture(rem, 0)
-        if not args.no_graph:
-            for _ in range(2):
-                for g in graphs.values():
-                    g.replay()
-        stream.synchronize()
-
+    # One graph holds exactly --steps layer passes (rotating over the weight copies).  It is replayed
+    # back to back at least 30 times (and for at least a second, so that the clock sampler sees the
+    # load); every replay is bracketed by CUDA events on the launching stream, and the reported time
+    # is the median replay.  The clock sampler runs from before the untimed replays to the end.
     sampler = ClockSampler(local_rank)
     sampler.start()
-    time.sleep(0.3)
+    with torch.cuda.stream(stream):
+        timed_graph = Eager(args.steps) if args.no_graph else capture(args.steps, 0)
+        for _ in range(3):
+            timed_graph.replay()
+        stream.synchronize()
     ranks.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    replay_ms = []
+    t_begin = time.time()
     with torch.cuda.stream(stream):
-        e0.record(stream)
-        for _ in range(full):
-            graphs["full"].replay()
-        if rem:
-            graphs["rem"].replay()
-        e1.record(stream)
-    stream.synchronize()
-    torch.cuda.synchronize()
-    ranks.barrier()
-    ms = e0.elapsed_time(e1)
-    # keep the GPU busy a little longer so that the clock sampler sees it under load
-    t_end = time.time() + (0.0 if args.no_graph else 0.6)
-    with torch.cuda.stream(stream):
-        while time.time() < t_end:
-            (graphs.get("full") or graphs["rem"]).replay()
+        while len(replay_ms) < 30 or (time.time() - t_begin < 1.0 and len(replay_ms) < 2000):
+            evs = []
+            for _ in range(10):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                timed_graph.replay()
+                e1.record(stream)
+                evs.append((e0, e1))
             stream.synchronize()
+            replay_ms += [a.elapsed_time(b) for a, b in evs]
+    torch.cuda.synchronize()
+    ranks.barrier()
     clocks = sampler.stop()
-    ms = ranks.max(ms)
+    ms = ranks.max(float(np.median(replay_ms)))
+    ms_min, ms_max = ranks.max(float(np.min(replay_ms))), ranks.max(float(np.max(replay_ms)))
 
     # ---- end to end: host buffers through bitcos_gemv_host, copies inside the timed region ----
     stagings = [torch.empty(bc.bitcos_gemv_host_staging_bytes(m["M"], m["K"], 1), dtype=torch.uint8, device="cuda")
@@ -406,14 +407,24 @@ def run_cuda(args):
     host_multi = [[bc.MultiHostJobs([(rep[j], xh_np[j], xsh_np[j], yh_np[j], stagings[j], wss[j]) for j in g])
                    for g in groups] for rep in replicas]
 
+    # one call per step: one pinned block in, the four launches, one pinned block out, one wait
+    host_phases = [bc.HostPhases([(rep[j], wss[j]) for j in order], phases) for rep in replicas]
+    for hp in host_phases:
+        for n, j in enumerate(order):
+            hp.x[n][:] = layer[j]["x"]
+            hp.x_scale[n][:] = layer[j]["xs"]
+
     def e2e_step(i):
         if args.serial or args.branches:
             rep = replicas[i % copies]
             for j in range(len(layer)):
                 bc.bitcos_gemv_host(rep[j], xh_np[j], xsh_np[j], yh_np[j], stagings[j], wss[j])
             return
-        for mj in host_multi[i % copies]:
-            bc.bitcos_gemv_multi_host(mj)
+        if args.e2e_per_phase:
+            for mj in host_multi[i % copies]:
+                bc.bitcos_gemv_multi_host(mj)
+            return
+        host_phases[i % copies].run()
 
     e2e_steps = 0 if args.no_e2e else min(args.steps, 200)
     e2e_us = float("nan")
@@ -427,8 +438,11 @@ def run_cuda(args):
         torch.cuda.synchronize()
         e2e_us = (time.perf_counter() - t0) / e2e_steps * 1e6
     e2e_us = ranks.max(e2e_us)
-    h2d = sum(m["K"] + 4 for m in layer)
-    d2h = sum(4 * m["M"] for m in layer)
+    if args.serial or args.branches or args.e2e_per_phase:
+        h2d = sum(m["K"] + 4 for m in layer)
+        d2h = sum(4 * m["M"] for m in layer)
+    else:
+        h2d, d2h = host_phases[0].in_bytes, host_phases[0].out_bytes      # the two blocks as copied (16-byte padding included)
 
     if rank != 0:
         ranks.close()
@@ -499,10 +513,15 @@ def run_cuda(args):
                                    "bit, dense int32 dot per group, double scale-and-sum"},
         "e2e": {"value": whole_job_value(e2e_us, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps,
-                "path": ("bitcos_gemv_host per GEMV" if (args.serial or args.branches) else
-                         "bitcos_gemv_multi_host, four calls per step (q+k+v, o, gate+up, down)")
-                        + ": pinned x -> device, kernel, y -> pinned host, stream wait"},
+                "path": ("bitcos_gemv_host per GEMV: pinned x -> device, kernel, y -> pinned host, stream wait"
+                         if (args.serial or args.branches) else
+                         "bitcos_gemv_multi_host, four calls per step, each: pinned x -> device, launch, y -> pinned host, stream wait"
+                         if args.e2e_per_phase else
+                         "bitcos_gemv_phases_host, one call per step: one pinned block with all activations -> device, "
+                         "four launches (q+k+v, o, gate+up, down), all outputs -> one pinned block, one stream wait")},
         "gpu_launches": n_launch,
+        "timing": {"replays": len(replay_ms), "steps_per_replay": args.steps, "statistic": "median replay",
+                   "us_per_step_min": ms_min * 1e3 / args.steps, "us_per_step_max": ms_max * 1e3 / args.steps},
         "clocks": clocks,
     }
     line["two_term_roofline"] = two_term_roofline(bc, cfg["z"], peak, clocks.get("sm_mhz") or 1965.0)
@@ -976,7 +995,12 @@ def main():
     ap.add_argument("--serial", action="store_true", help="launch the seven GEMVs of a step strictly in sequence")
     ap.add_argument("--branches", action="store_true",
                     help="seven launches per step with q|k|v and gate|up on parallel graph branches")
+    ap.add_argument("--launch", default="multi", choices=["multi", "phased"],
+                    help="multi: four bitcos_gemv_multi launches per step; phased: the whole layer pass as one "
+                         "bitcos_gemv_phased launch (phases q|k|v, o, gate|up, down)")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA graphs (for profilers)")
+    ap.add_argument("--e2e-per-phase", action="store_true",
+                    help="end-to-end leg through four bitcos_gemv_multi_host calls per step instead of one bitcos_gemv_phases_host call")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--profile-quant", default="", choices=["", "chain", "fused"],
@@ -1003,7 +1027,7 @@ def main():
         run_reference(args)
     else:
         if args.steps is None:
-            args.steps = 20 if args.profile_quant else 2000
+            args.steps = 20 if args.profile_quant else 200
         run_cuda(args)
 
 

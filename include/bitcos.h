@@ -320,6 +320,30 @@ int bitcos_gemv_multi_group_scales(const bitcos_gemv_job *jobs, int n_jobs, int 
  * job's x points to device bf16 [batch][K], x_scale is ignored (may be NULL); batch 1 or 2. */
 int bitcos_gemv_multi_bf16(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
 
+/* Jobs in dependency order inside ONE launch.  job_phase[j] (0 .. BITCOS_MAX_PHASES - 1, non-decreasing
+ * in j, starting at 0, no phase skipped) puts every job into a phase; the jobs of a phase are
+ * independent of one another (as in bitcos_gemv_multi), and a job's activations x, x_scale are read
+ * only after EVERY job of the phase before it has written all of its outputs -- so a job may consume
+ * what the phase before produced.  The seven products of a decoder layer make four phases:
+ * q | k | v, then o, then gate | up, then down (the paper's end-to-end runs execute exactly this
+ * sequence per layer, one launch per product; Section III-B.5).  What does not depend on the phase
+ * before runs ahead of the dependency: the next phase's packed weights are streamed and its first
+ * tiles decoded while the current phase is still being finished, which is what a sequence of
+ * launches cannot do.  Inside one launch nothing else can run between two phases: a layer whose
+ * attention, normalisation or activation kernels sit between the products uses bitcos_gemv_multi
+ * per phase instead.
+ *   jobs, n_jobs   as for bitcos_gemv_multi (1 .. BITCOS_MAX_JOBS; own outputs and own workspace each)
+ *   batch          1 or 2 (ERR_SHAPE above, and for rows too long for the one- and two-token kernels)
+ *   sync           device scratch of BITCOS_PHASED_SYNC_BYTES, 16-byte aligned, zero filled ONCE; the
+ *                  launch leaves it zero.  Two phased launches that may overlap must not share it.
+ * Results are identical, bit for bit, to one bitcos_gemv_multi call per phase.  Every thread block
+ * waits for the phase before with a bounded wait (status word of the job's workspace on expiry);
+ * the launch uses at most one thread block per multiprocessor, so all blocks are resident together. */
+#define BITCOS_MAX_PHASES 4
+#define BITCOS_PHASED_SYNC_BYTES 64
+int bitcos_gemv_phased(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, void *sync,
+                       void *cuda_stream);
+
 /* The same product as bitcos_gemv without a caller-provided workspace.  (The paper has no
  * counterpart: this entry point exists for the library's users, not for the method.)
  *
@@ -372,6 +396,21 @@ typedef struct bitcos_gemv_host_job {
     size_t workspace_bytes;
 } bitcos_gemv_host_job;
 int bitcos_gemv_multi_host(const bitcos_gemv_host_job *jobs, int n_jobs, int batch, void *cuda_stream);
+
+/* A whole sequence of phases from host buffers with ONE copy in, ONE copy out and ONE wait: the
+ * host-buffer form for callers that run several dependent products per step (a decoder layer's
+ * q | k | v, o, gate | up, down) and keep activations and results on the host.  The caller lays every
+ * job's x and x_scale out inside one device block `in_device` (and the same bytes, at the same
+ * offsets, inside the host block `in_host`), and every job's y inside one device block
+ * `out_device`; jobs[] holds the DEVICE addresses, as for bitcos_gemv_multi.  The call copies
+ * in_host -> in_device (in_bytes), runs one bitcos_gemv_multi launch per phase (job_phase as for
+ * bitcos_gemv_phased), copies out_device -> out_host (out_bytes) and waits for the stream, so
+ * out_host is valid on return.  Pinned host blocks keep the two copies asynchronous until the wait.
+ * ERR_CAPACITY if a job's x, x_scale or y lies outside its block.  The paper has no counterpart (it
+ * measures resident activations). */
+int bitcos_gemv_phases_host(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, const void *in_host,
+                            void *in_device, size_t in_bytes, void *out_host, const void *out_device, size_t out_bytes,
+                            void *cuda_stream);
 
 /* The same product from the five-trit and 2-bit layouts (device pointers; scales in tile order). */
 int trit5_gemv(const uint32_t *words, const uint16_t *scales_tiled, int64_t M, int64_t K, const int8_t *x,

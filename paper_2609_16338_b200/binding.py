@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host",
 ]
 
 
@@ -99,6 +99,8 @@ def load_library():
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.bitcos_decode_probe_variant.argtypes = [C.c_int, vp, vp, sz, vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp]
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
+    L.bitcos_gemv_phased.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp]
+    L.bitcos_gemv_phases_host.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp, sz, vp, vp, sz, vp]
     L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
     L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
     L.bitcos_gemv_bf16.argtypes = [C.POINTER(_Weights), vp, C.c_int, vp, vp, vp, sz, vp]
@@ -524,6 +526,77 @@ def bitcos_gemv_multi(jobs):
     mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
     _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")
     return [j[3] for j in mj.keep]
+
+
+PHASED_SYNC_BYTES = 64
+
+
+def make_phased_sync(device="cuda"):
+    """Zero-filled device scratch for bitcos_gemv_phased (the launch leaves it zero)."""
+    import torch
+    return torch.zeros(PHASED_SYNC_BYTES, dtype=torch.uint8, device=device)
+
+
+class PhasedJobs(MultiJobs):
+    """Argument block of bitcos_gemv_phased: jobs as for MultiJobs plus one phase per job."""
+
+    def __init__(self, jobs, phases, sync=None):
+        super().__init__(jobs)
+        self.phases = (C.c_int * len(jobs))(*[int(p) for p in phases])
+        self.sync = sync if sync is not None else make_phased_sync()
+
+
+def bitcos_gemv_phased(jobs, phases=None, sync=None):
+    """Jobs in dependency order in one launch: `jobs` is a PhasedJobs, or a list of (W, x, x_scale, y, workspace)
+    tuples with `phases` (one int per job, non-decreasing from 0) and a sync buffer from make_phased_sync."""
+    pj = jobs if isinstance(jobs, PhasedJobs) else PhasedJobs(jobs, phases, sync)
+    _check(load_library().bitcos_gemv_phased(pj.arr, pj.phases, len(pj.arr), pj.batch, pj.sync.data_ptr(), _stream()),
+           "bitcos_gemv_phased")
+    return [j[3] for j in pj.keep]
+
+
+class HostPhases:
+    """Everything bitcos_gemv_phases_host needs for a fixed set of matrices, built once: one pinned host block and
+    one device block for all jobs' activations and scales, one of each for all outputs, and the job list.
+    weights = [(DeviceBitcos, workspace)], phases = one int per job; fill x[j] / x_scale[j] (numpy views
+    of the pinned block), call run(), read y[j]."""
+
+    def __init__(self, weights, phases, batch: int = 1):
+        import torch
+        self.batch = batch
+        off, self.x_off, self.xs_off = 0, [], []
+        for W, _ in weights:
+            self.x_off.append(off)
+            off += (batch * W.K + 15) // 16 * 16
+            self.xs_off.append(off)
+            off += (batch * 4 + 15) // 16 * 16
+        self.in_bytes = off
+        off, self.y_off = 0, []
+        for W, _ in weights:
+            self.y_off.append(off)
+            off += (batch * W.M * 4 + 15) // 16 * 16
+        self.out_bytes = off
+        self.in_host = torch.zeros(self.in_bytes, dtype=torch.uint8).pin_memory()
+        self.out_host = torch.zeros(self.out_bytes, dtype=torch.uint8).pin_memory()
+        self.in_dev = torch.zeros(self.in_bytes, dtype=torch.uint8, device="cuda")
+        self.out_dev = torch.zeros(self.out_bytes, dtype=torch.uint8, device="cuda")
+        hin, hout = self.in_host.numpy(), self.out_host.numpy()
+        self.x = [hin[o:o + batch * W.K].view(np.int8).reshape(batch, W.K) for o, (W, _) in zip(self.x_off, weights)]
+        self.x_scale = [hin[o:o + batch * 4].view(np.float32) for o in self.xs_off]
+        self.y = [hout[o:o + batch * W.M * 4].view(np.float32).reshape(batch, W.M) for o, (W, _) in zip(self.y_off, weights)]
+        base_in, base_out = self.in_dev.data_ptr(), self.out_dev.data_ptr()
+        self.keep = weights
+        self.arr = (_Job * len(weights))(*[_Job(C.addressof(W.desc), base_in + xo, base_in + so, base_out + yo,
+                                                ws.data_ptr(), ws.numel())
+                                           for (W, ws), xo, so, yo in zip(weights, self.x_off, self.xs_off, self.y_off)])
+        self.phases = (C.c_int * len(weights))(*[int(p) for p in phases])
+
+    def run(self):
+        _check(load_library().bitcos_gemv_phases_host(self.arr, self.phases, len(self.arr), self.batch,
+                                                      self.in_host.data_ptr(), self.in_dev.data_ptr(), self.in_bytes,
+                                                      self.out_host.data_ptr(), self.out_dev.data_ptr(), self.out_bytes,
+                                                      _stream()), "bitcos_gemv_phases_host")
+        return self.y
 
 
 def bitcos_gemv_multi_group_scales(jobs):

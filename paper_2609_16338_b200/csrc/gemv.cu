@@ -34,6 +34,7 @@
 
 #include <cstdint>
 #include <cstdlib>
+#include <mutex>
 
 namespace {
 
@@ -613,6 +614,7 @@ template <bool DEBUG, bool XG = false, bool XQ = false, bool BL = false>
 struct OneSegT {
     typedef ParamView View;
     static constexpr bool kSingle = true;      // never more than one segment
+    static constexpr bool kHetero = false;     // all segments share one problem shape and one plan
     static constexpr bool kDebug = DEBUG;      // false: acc_debug is known to be NULL (no code for it)
     static constexpr bool kGroupScales = XG;   // x_scale holds one scale per token AND group: [nb][G]
     static constexpr bool kQuantize = XQ;      // x holds bf16 activations: quantised per group of 128 by the decoder warps
@@ -621,6 +623,7 @@ struct OneSegT {
     Walk wk;
     bool used;
     __device__ __forceinline__ const Problem &shape() const { return *pr; }
+    __device__ __forceinline__ int block_in_job(int block) const { return block; }
     __device__ __forceinline__ bool next(View &v, Walk &w) {
         if (used) return false;
         used = true;
@@ -637,11 +640,19 @@ struct OneSegT {
 // `segs` yields the problems this block works on, one after the other, with its share of each
 // one's items; the stage ring, the partial-sum slots and their barriers run on across them.
 template <int FMT, int NB, int TPW, typename Segs>
-__device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, uint8_t *smem, int block,
+__device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in, uint8_t *smem, int block,
                                              const FirstOff *fo = nullptr, int fo_index = 0) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // The problem and the plan of the segment a warp role is working on.  The plain and the grouped
+    // launches have one shape and one plan for all their segments.  A phased launch (kHetero) moves
+    // from job to job: only what the shared-memory layout and the barrier counts need -- the widest
+    // plan, the longest row -- is common (pl_in, segs.shape()), and every role re-binds pb / pl to its
+    // own copy of the current job's problem and plan.
+    const Problem *pbp = &segs.shape();
+    const Plan *plp = &pl_in;
+#define pb (*pbp)
+#define pl (*plp)
     const SmemLayout L = smem_layout(FMT, pl, segs.shape().G, NB, segs.shape().K);
-    const Problem &pb = segs.shape();
     typename Segs::View pr{};
     Walk wk{};
     const uint8_t *lut = smem + L.lut;
@@ -695,6 +706,10 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         // Entry offsets are requested two items before they are needed (r0 = item k, r1 = item
         // k + 1, r2 = item k + 2), so that the load is never waited for.
         Segs src = segs;
+        if constexpr (Segs::kHetero) {
+            pbp = src.problem_ptr();
+            plp = src.plan_ptr();
+        }
         ItemIter it2;
         ItemRange r0{}, r1{}, r2{};
         uint32_t lo0 = 0, hi0 = 0, lo1 = 0, hi1 = 0;
@@ -794,11 +809,15 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // fetches into shared memory (one bulk copy per token) as soon as the dependency is resolved.
     // With four tokens and more (tensor-core path) the decoders fetch their activation fragments
     // from global memory right after that first decode instead.
-    constexpr bool kLate = Segs::kSingle;                       // plain kernels: wait as late as possible
+    constexpr bool kLate = Segs::kSingle || Segs::kHetero;      // plain and phased kernels: wait as late as possible
     constexpr bool kEarly = kLate && NB < kMmaMinBatch;         // ... and activations copied by the epilogue warp
     if (!kLate) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     Segs src = segs;
+    if constexpr (Segs::kHetero) {
+        pbp = src.problem_ptr();
+        plp = src.plan_ptr();
+    }
     bool have = src.next(pr, wk);
     while (have && wk.count <= 0) have = src.next(pr, wk);
     auto next_segment = [&]() {
@@ -839,8 +858,8 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
 
     // ------------------------------------------------------------------ epilogue warp
     if (warp == pl.NW + 1) {
-        if (kLate) {
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+        // the segment's activations into shared memory: one bulk copy per token (one or two tokens)
+        auto fetch_x = [&]() {
             token_rows();
             if (kEarly && !kXQ && lane == 0) {
                 mbar_expect_tx(bar0 + 8u * kBarX, static_cast<uint32_t>(pr.nb(pb)) * static_cast<uint32_t>(pb.K));
@@ -850,6 +869,10 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                         bulk_copy(smem_addr(smem + L.x) + static_cast<uint32_t>(b) * static_cast<uint32_t>(pb.K),
                                   pb.x + static_cast<int64_t>(xr[b]) * pb.K, static_cast<uint32_t>(pb.K), bar0 + 8u * kBarX);
             }
+        };
+        if (kLate) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            if (!Segs::kHetero) fetch_x();
         }
         float run[NB];          // running sum of the current row block over this block's items
 #pragma unroll
@@ -930,6 +953,18 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             }
         };
         do {
+        if constexpr (Segs::kHetero) {
+            // A phased launch: this segment's activations (and whatever else its job reads) may be
+            // written by the jobs of the phase before it, so they are fetched only once every thread
+            // block has finished that phase.  All decoder warps have left the previous segment's
+            // contractions by now (its last partial sums were consumed above), so the one activation
+            // buffer is free.
+            if (!src.wait_dependency(lane)) {
+                if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
+                return;
+            }
+            fetch_x();
+        }
         n_pend = 0;
         it.init(pl, wk.first);
         if (NB < kMmaMinBatch && !kXG) {
@@ -985,7 +1020,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 Share sh;
                 sh.rb = r.rb0;
                 const int lo = owner_of(wk, r.rb0 * pl.CS), hi = owner_of(wk, r.rb0 * pl.CS + pl.CS - 1);
-                sh.slot = block - lo;
+                sh.slot = src.block_in_job(block) - lo;
                 sh.sharers = hi - lo + 1;
 #pragma unroll
                 for (int b = 0; b < NB; ++b)
@@ -1001,8 +1036,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
             }
         }
         for (int i = 0; i < n_pend; ++i) finish_share<NB, kXG>(pb, pl, xr, pend[i], lane);
+        if constexpr (Segs::kHetero) src.signal_done(lane);      // this block's outputs of the phase are written
         have = next_segment();
-        if (have) token_rows();
+        if (have && !Segs::kHetero) token_rows();
         } while (have);
         return;
     }
@@ -1011,10 +1047,12 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     // CS == 1: tile t of an item always is row block t / G of the chunk, group t % G; this warp
     // decodes tile `warp` and, with two tiles per warp, tile `warp + NW`
     constexpr int tpw = TPW;
-    const int my_rbl0 = (pl.CS == 1) ? warp / pb.G : 0;
-    const int g_fixed0 = warp - my_rbl0 * pb.G;
-    const int my_rbl1 = (pl.CS == 1) ? (warp + pl.NW) / pb.G : 0;
-    const int g_fixed1 = warp + pl.NW - my_rbl1 * pb.G;
+    // (a phased launch works these out again for every job)
+    int my_rbl0 = (pl.CS == 1) ? warp / pb.G : 0;
+    int g_fixed0 = warp - my_rbl0 * pb.G;
+    int my_rbl1 = (pl.CS == 1) ? (warp + pl.NW) / pb.G : 0;
+    int g_fixed1 = warp + pl.NW - my_rbl1 * pb.G;
+    uint32_t x_parity = 0;      // phase parity of the activations' barrier: one phase per segment of a phased launch
     if (FMT != kBit2) {
         if (!mbar_wait(bar0 + 8u * kBarLut, 0)) {
             if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
@@ -1106,6 +1144,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
     int q_g = -1;
     float q_scale[NB < kMmaMinBatch ? NB : 1] = {};
     uint32_t *q_scr = reinterpret_cast<uint32_t *>(smem + L.x) + static_cast<uint32_t>(warp) * (NB * kRows);
+    bool more_segments = false;
     do {
     if (!(kLate && kMma)) {
         token_fragments();
@@ -1291,7 +1330,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
                 // first contraction of this warp: the previous kernel must be complete and the
                 // activations in place (the decode above needed neither)
                 asm volatile("griddepcontrol.wait;" ::: "memory");
-                if (!kXQ && !mbar_wait(bar0 + 8u * kBarX, 0)) {
+                if (!kXQ && !mbar_wait(bar0 + 8u * kBarX, x_parity)) {
                     if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                     return;
                 }
@@ -1389,7 +1428,29 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl, u
         __syncwarp();
         mbar_arrive_lane0(bar0 + 8u * (kBarRedFull + slot), lane);
     }
-    } while (next_segment());
+    if constexpr (Segs::kHetero) {
+        // Every decoder warp passes every phase of the activations' barrier, a warp without a tile in
+        // this segment included: a warp that skipped one could not tell the phase before from the
+        // phase after by its parity.
+        if (!x_ready && !mbar_wait(bar0 + 8u * kBarX, x_parity)) {
+            if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
+            return;
+        }
+        more_segments = next_segment();
+        if (more_segments) {
+            x_ready = false;
+            x_parity ^= 1u;
+            my_rbl0 = (pl.CS == 1) ? warp / pb.G : 0;
+            g_fixed0 = warp - my_rbl0 * pb.G;
+            my_rbl1 = (pl.CS == 1) ? (warp + pl.NW) / pb.G : 0;
+            g_fixed1 = warp + pl.NW - my_rbl1 * pb.G;
+        }
+    } else {
+        more_segments = next_segment();
+    }
+    } while (more_segments);
+#undef pb
+#undef pl
 }
 
 // One problem, this block's share of its items.
@@ -1436,6 +1497,124 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
                              b - ma.first_block[j], &fo, b);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Phased launch: jobs in dependency order inside ONE launch.  The jobs of phase p may read what the
+// jobs of phase p - 1 wrote (a decoder layer's o projection follows q, k and v; down follows gate
+// and up), so a thread block fetches a job's activations only after every block has finished the
+// phase before it.  Everything that does not depend on the phase before -- the packed weights, their
+// decode -- runs ahead: the producer warp streams the next phase's tiles while the current one is
+// being decoded, and every decoder warp decodes its first tile of the next phase before it waits.
+// Blocks are persistent and at most one per multiprocessor, so all of them are resident together
+// and the wait on the phase counter cannot starve; it is bounded like every other wait here.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxPhases = BITCOS_MAX_PHASES;
+struct PhasedArgs {
+    Problem pr[kMaxJobs];
+    Plan pl[kMaxJobs];                      // every plan with the layout's NW and stages
+    Plan layout;                            // the widest plan: shared-memory layout, barrier counts, block size
+    Problem shape;                          // K = the longest row (layout only)
+    int job_first_block[kMaxJobs];          // a job's range of thread blocks inside its phase
+    int job_blocks[kMaxJobs];
+    int expect[kMaxPhases];                 // thread blocks that have items in the phase
+    int n_phases;
+    unsigned int *sync;                     // device: one arrival counter per phase, zero between launches
+    uint8_t job_of[kMaxPhases][kMaxGrid];   // the job a thread block works on in a phase (0xFF: none)
+};
+
+__device__ __forceinline__ unsigned int load_acquire(const unsigned int *p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// The segments of one thread block of a phased launch: in every phase, its share of one job.
+template <bool XG>
+struct PhasedSegs {
+    typedef ParamView View;
+    static constexpr bool kSingle = false;
+    static constexpr bool kHetero = true;
+    static constexpr bool kDebug = false;
+    static constexpr bool kGroupScales = XG;
+    static constexpr bool kQuantize = false;
+    static constexpr bool kBlend = false;
+    const PhasedArgs *pa;
+    int block;               // blockIdx.x
+    int next_phase;          // phase the next call of next() looks at
+    int phase;               // phase of the current segment
+    int rel_block;           // this block's index inside the current job's range
+    Problem cur_pb;
+    Plan cur_pl;
+    __device__ __forceinline__ const Problem &shape() const { return pa->shape; }
+    __device__ __forceinline__ const Problem *problem_ptr() const { return &cur_pb; }
+    __device__ __forceinline__ const Plan *plan_ptr() const { return &cur_pl; }
+    __device__ __forceinline__ int block_in_job(int) const { return rel_block; }
+    __device__ __forceinline__ bool next(View &, Walk &w) {
+        while (next_phase < pa->n_phases) {
+            const int p = next_phase++;
+            const int j = pa->job_of[p][block];
+            if (j == 0xFF) continue;
+            const int rel = block - pa->job_first_block[j];
+            const Walk wj = make_walk(pa->pl[j], rel, pa->job_blocks[j]);
+            if (wj.count <= 0) continue;
+            cur_pb = pa->pr[j];
+            cur_pl = pa->pl[j];
+            w = wj;
+            phase = p;
+            rel_block = rel;
+            return true;
+        }
+        return false;
+    }
+    // Epilogue warp, before it fetches the current segment's activations: every block that has items
+    // in the phase before must have written its outputs.  false if the wait ran out.
+    __device__ __forceinline__ bool wait_dependency(int lane) const {
+        if (phase == 0) return true;
+        bool ok = true;
+        if (lane == 0) {
+            const unsigned int *ctr = pa->sync + (phase - 1);
+            const unsigned int want = static_cast<unsigned int>(pa->expect[phase - 1]);
+            uint64_t t0 = 0;
+            for (uint32_t i = 0; load_acquire(ctr) < want; ++i) {
+                if ((i & 15u) == 15u) {
+                    const uint64_t now = global_timer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > kWaitLimitNs) {
+                        ok = false;
+                        break;
+                    }
+                }
+            }
+            // what the other blocks wrote, ordered before this block's asynchronous copies
+            asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        return __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+    }
+    // Epilogue warp, after the last output of the current segment: count this block in.  The last
+    // arrival of the last phase leaves every counter zero for the next launch (by then no block
+    // reads an earlier counter any more: each one read it before it arrived here).
+    __device__ __forceinline__ void signal_done(int lane) const {
+        __syncwarp();
+        if (lane != 0) return;
+        __threadfence();
+        const unsigned int old = atomicAdd(pa->sync + phase, 1u);
+        if (phase == pa->n_phases - 1 && old + 1u == static_cast<unsigned int>(pa->expect[phase])) {
+            for (int p = 0; p < pa->n_phases; ++p) pa->sync[p] = 0u;
+        }
+    }
+};
+
+template <int NB, bool XG = false>
+__global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_phased_kernel(const __grid_constant__ PhasedArgs pa) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    PhasedSegs<XG> segs;
+    segs.pa = &pa;
+    segs.block = static_cast<int>(blockIdx.x);
+    segs.next_phase = 0;
+    segs.phase = 0;
+    segs.rel_block = 0;
+    run_segments<kBitcos, NB, 1>(segs, pa.layout, smem, static_cast<int>(blockIdx.x));
+}
+
 // Fills in what differs between the groups of a grouped product; false if the group is empty or
 // names no expert.
 template <int NB>
@@ -1468,11 +1647,13 @@ struct GroupedSegs {
     int grp;                  // group of item lo
     typedef GroupView View;
     static constexpr bool kSingle = false;
+    static constexpr bool kHetero = false;
     static constexpr bool kDebug = true;
     static constexpr bool kGroupScales = false;
     static constexpr bool kQuantize = false;
     static constexpr bool kBlend = false;
     __device__ __forceinline__ const Problem &shape() const { return *base; }
+    __device__ __forceinline__ int block_in_job(int block) const { return block; }
     __device__ __forceinline__ bool next(View &v, Walk &w) {
         while (lo < hi) {
             const int64_t g_lo = static_cast<int64_t>(grp) * ipg;
@@ -2208,7 +2389,102 @@ int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
 }
 }  // namespace
 
+namespace {
+template <int NB>
+int launch_phased(PhasedArgs &pa, int n_jobs, const int *job_phase, cudaStream_t stream) {
+    for (int j = 0; j < n_jobs; ++j)
+        if (static_cast<int64_t>(NB) * pa.pr[j].K > kXResidentBytes) return BITCOS_ERR_SHAPE;
+    int sms = 0, budget = 0;
+    int rc = prepare_kernel<gemv_phased_kernel<NB>>(&sms, &budget);
+    if (rc) return rc;
+    if (sms > kMaxGrid) sms = kMaxGrid;
+    // the layout every job shares: the widest plan, the longest row
+    Plan layout{};
+    layout.tpw = 1;
+    int64_t kmax = 0;
+    int gmax = 0;
+    for (int j = 0; j < n_jobs; ++j) {
+        if (pa.pl[j].NW > layout.NW) layout.NW = pa.pl[j].NW;
+        if (pa.pr[j].K > kmax) kmax = pa.pr[j].K;
+        if (pa.pr[j].G > gmax) gmax = pa.pr[j].G;
+    }
+    layout.stages = choose_stages(kBitcos, layout, gmax, NB, kmax, budget);
+    pa.layout = layout;
+    pa.shape = Problem{};
+    pa.shape.K = kmax;
+    pa.shape.G = gmax;
+    for (int p = 0; p < kMaxPhases; ++p) {
+        pa.expect[p] = 0;
+        for (int b = 0; b < kMaxGrid; ++b) pa.job_of[p][b] = 0xFF;
+    }
+    int grid = 1;
+    for (int p = 0; p < pa.n_phases; ++p) {
+        // the multiprocessors are shared between the phase's jobs in proportion to their item counts
+        int64_t total_items = 0;
+        for (int j = 0; j < n_jobs; ++j)
+            if (job_phase[j] == p) total_items += pa.pl[j].items;
+        int next = 0;
+        for (int j = 0; j < n_jobs; ++j) {
+            if (job_phase[j] != p) continue;
+            int64_t cap = pa.pl[j].items;
+            if (total_items > sms) {
+                cap = pa.pl[j].items * sms / total_items;
+                if (cap < 1) cap = 1;
+            }
+            int blocks = 1;
+            choose_walk(pa.pl[j], static_cast<int>(cap), &blocks);
+            if (next + blocks > kMaxGrid) return BITCOS_ERR_SHAPE;
+            pa.pl[j].NW = layout.NW;
+            pa.pl[j].stages = layout.stages;
+            pa.job_first_block[j] = next;
+            pa.job_blocks[j] = blocks;
+            for (int b = 0; b < blocks; ++b) {
+                pa.job_of[p][next + b] = static_cast<uint8_t>(j);
+                if (make_walk(pa.pl[j], b, blocks).count > 0) ++pa.expect[p];
+            }
+            next += blocks;
+        }
+        if (next > grid) grid = next;
+    }
+    const SmemLayout L = smem_layout(kBitcos, layout, gmax, NB, kmax);
+    if (static_cast<int>(L.total) > budget) return BITCOS_ERR_SHAPE;
+    return launch_pdl(gemv_phased_kernel<NB>, dim3(static_cast<unsigned>(grid)), (layout.NW + 2) * 32, L.total, stream, pa);
+}
+}  // namespace
+
 extern "C" {
+
+int bitcos_gemv_phased(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, void *sync,
+                       void *cuda_stream) {
+    if (!jobs || !job_phase || !sync) return BITCOS_ERR_NULL;
+    if (n_jobs < 1 || n_jobs > kMaxJobs || batch < 1 || batch > 2) return BITCOS_ERR_SHAPE;
+    if (!aligned16(sync)) return BITCOS_ERR_ALIGN;
+    if (job_phase[0] != 0) return BITCOS_ERR_SHAPE;
+    for (int j = 1; j < n_jobs; ++j)
+        if (job_phase[j] < job_phase[j - 1] || job_phase[j] > job_phase[j - 1] + 1) return BITCOS_ERR_SHAPE;
+    if (job_phase[n_jobs - 1] >= kMaxPhases) return BITCOS_ERR_SHAPE;
+    static PhasedArgs pa_storage;      // (large: kept off the stack; calls are serialised by the lock below)
+    static std::mutex lock;
+    std::lock_guard<std::mutex> guard(lock);
+    PhasedArgs &pa = pa_storage;
+    pa.n_phases = job_phase[n_jobs - 1] + 1;
+    pa.sync = static_cast<unsigned int *>(sync);
+    for (int j = 0; j < n_jobs; ++j) {
+        const bitcos_gemv_job &jb = jobs[j];
+        if (!jb.W) return BITCOS_ERR_NULL;
+        const int bad = check_common(kBitcos, jb.W->bitmap, jb.W->signs, jb.W->tile_off, jb.W->scales, jb.W->M, jb.W->K,
+                                     jb.x, jb.x_scale, batch, jb.y, nullptr, jb.workspace, jb.workspace_bytes);
+        if (bad) return bad;
+        for (int i = 0; i < j; ++i)
+            if (jobs[i].workspace == jb.workspace) return BITCOS_ERR_SHAPE;
+        pa.pl[j] = make_plan(jb.W->M, jb.W->K, decoder_warps(batch));
+        fill_problem(pa.pr[j], jb.W->bitmap, jb.W->signs, jb.W->tile_off, jb.W->scales, jb.W->M, jb.W->K, jb.x,
+                     jb.x_scale, batch, jb.y, nullptr, jb.workspace);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (batch == 1) return launch_phased<1>(pa, n_jobs, job_phase, stream);
+    return launch_phased<2>(pa, n_jobs, job_phase, stream);
+}
 
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {
     return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, false);
@@ -2327,6 +2603,39 @@ int bitcos_gemv_multi_host(const bitcos_gemv_host_job *jobs, int n_jobs, int bat
                                         cudaMemcpyDeviceToHost, stream));
         if (rc) return rc;
     }
+    return check_cuda(cudaStreamSynchronize(stream));
+}
+
+int bitcos_gemv_phases_host(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, const void *in_host,
+                            void *in_device, size_t in_bytes, void *out_host, const void *out_device, size_t out_bytes,
+                            void *cuda_stream) {
+    if (!jobs || !job_phase || !in_host || !in_device || !out_host || !out_device) return BITCOS_ERR_NULL;
+    if (n_jobs < 1 || n_jobs > kMaxJobs || in_bytes == 0 || out_bytes == 0) return BITCOS_ERR_SHAPE;
+    if (job_phase[0] != 0) return BITCOS_ERR_SHAPE;
+    for (int j = 1; j < n_jobs; ++j)
+        if (job_phase[j] < job_phase[j - 1] || job_phase[j] > job_phase[j - 1] + 1) return BITCOS_ERR_SHAPE;
+    // every job's activations, scales and outputs must lie inside the two blocks that are copied
+    const uintptr_t in0 = reinterpret_cast<uintptr_t>(in_device), out0 = reinterpret_cast<uintptr_t>(out_device);
+    for (int j = 0; j < n_jobs; ++j) {
+        if (!jobs[j].W || !jobs[j].x || !jobs[j].x_scale || !jobs[j].y) return BITCOS_ERR_NULL;
+        const uintptr_t x = reinterpret_cast<uintptr_t>(jobs[j].x), xs = reinterpret_cast<uintptr_t>(jobs[j].x_scale),
+                        y = reinterpret_cast<uintptr_t>(jobs[j].y);
+        const size_t xb = static_cast<size_t>(batch) * static_cast<size_t>(jobs[j].W->K), yb = static_cast<size_t>(batch) * static_cast<size_t>(jobs[j].W->M) * 4;
+        if (x < in0 || x + xb > in0 + in_bytes || xs < in0 || xs + static_cast<size_t>(batch) * 4 > in0 + in_bytes) return BITCOS_ERR_CAPACITY;
+        if (y < out0 || y + yb > out0 + out_bytes) return BITCOS_ERR_CAPACITY;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int rc = check_cuda(cudaMemcpyAsync(in_device, in_host, in_bytes, cudaMemcpyHostToDevice, stream));
+    if (rc) return rc;
+    for (int first = 0; first < n_jobs;) {
+        int last = first;
+        while (last + 1 < n_jobs && job_phase[last + 1] == job_phase[first]) ++last;
+        rc = bitcos_gemv_multi(jobs + first, last - first + 1, batch, cuda_stream);
+        if (rc) return rc;
+        first = last + 1;
+    }
+    rc = check_cuda(cudaMemcpyAsync(out_host, out_device, out_bytes, cudaMemcpyDeviceToHost, stream));
+    if (rc) return rc;
     return check_cuda(cudaStreamSynchronize(stream));
 }
 
