@@ -422,20 +422,41 @@ int bit2_gemv(const uint32_t *words, const uint16_t *scales_tiled, int64_t M, in
 
 /* Grouped product over selected experts of a mixture-of-experts layer (all experts M x K).
  * The caller lists the P (token, expert) pairs grouped by expert: group i covers pairs
- * group_begin[i] .. group_begin[i+1]-1 (at most 16 per group), all using expert
- * group_expert[i]; pair p reads activation row pair_xrow[p] of x[R][K] and writes y[p][M].
+ * group_begin[i] .. group_begin[i+1]-1 (at most max_group_size <= 16 per group), all using expert
+ * group_expert[i]; pair p reads activation row pair_xrow[p] of x[n_xrows][K] and writes y[p][M].
  * Each listed expert's packed bytes are read once.  No activation function, routing weight
- * or sum over experts is applied.
+ * or sum over experts is applied (the paper runs its mixture-of-experts checkpoints end to end only,
+ * Table I; this is the per-expert product such a layer needs).
  *   experts       device array of bitcos_weights (device pointers inside), n_experts entries
  *   group_expert  device int32 [n_groups];  group_begin  device int32 [n_groups + 1]
- *   pair_xrow     device int32 [P];  x device int8 [R][K];  x_scale device float [R]
- *   y             device float [P][M];  acc_debug NULL or device int32 [P][M][K/128]
- *   workspace     at least n_groups * bitcos_gemv_workspace_bytes(M, K) bytes, zero filled once */
-int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K,
-                        const int32_t *group_expert, const int32_t *group_begin, int n_groups,
-                        const int32_t *pair_xrow, int n_pairs, int max_group_size, const int8_t *x,
-                        const float *x_scale, float *y, int32_t *acc_debug, void *workspace,
-                        size_t workspace_bytes, void *cuda_stream);
+ *   pair_xrow     device int32 [n_pairs];  x device int8 [n_xrows][K];  x_scale device float [n_xrows]
+ *   y             device float [n_pairs][M];  acc_debug NULL or device int32 [n_pairs][M][K/128]
+ *   workspace     at least n_groups * bitcos_gemv_workspace_bytes(M, K) bytes, zero filled once;
+ *                 group i's status word is word 0 of workspace + i * bitcos_gemv_workspace_bytes(M, K)
+ * The routing lists live in device memory (they may come from a router kernel) and are checked on
+ * the device: a group whose pairs fall outside [0, n_pairs), that has more than max_group_size
+ * pairs (rounded up to 1, 2, 4, 8 or 16), that names an expert outside [0, n_experts) or an
+ * activation row outside [0, n_xrows) is skipped whole -- nothing of it is read or written -- and
+ * its status word and word 0 of the workspace (what bitcos_workspace_status reads) are set to 2.
+ * An empty group (group_begin[i+1] <= group_begin[i]) is skipped without a mark. */
+int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                        const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs,
+                        int max_group_size, const int8_t *x, int n_xrows, const float *x_scale, float *y,
+                        int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* The same grouped product from five-trit and 2-bit experts, so that the layout's gain can be
+ * measured on the same chip for the mixture-of-experts shapes too (Section II-A: below a zero
+ * density of 0.375 the five-trit format is the smaller one).  experts[e].bitmap points to the packed
+ * words (trit5_pack / bit2_pack layout), experts[e].scales to the scales in tile order; signs,
+ * tile_off and tile_off_host are not used. */
+int trit5_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                       const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs,
+                       int max_group_size, const int8_t *x, int n_xrows, const float *x_scale, float *y,
+                       int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
+int bit2_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                      const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs,
+                      int max_group_size, const int8_t *x, int n_xrows, const float *x_scale, float *y,
+                      int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 #ifdef __cplusplus
 }

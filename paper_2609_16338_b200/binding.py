@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped",
 ]
 
 
@@ -90,8 +90,9 @@ def load_library():
     L.bitcos_gemv.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, vp, sz, vp]
     for name in ("trit5_gemv", "bit2_gemv"):
         getattr(L, name).argtypes = [vp, vp, i64, i64, vp, vp, C.c_int, vp, vp, vp, sz, vp]
-    L.bitcos_gemv_grouped.argtypes = [vp, C.c_int, i64, i64, vp, vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp, vp,
-                                      vp, sz, vp]
+    for name in ("bitcos_gemv_grouped", "trit5_gemv_grouped", "bit2_gemv_grouped"):
+        getattr(L, name).argtypes = [vp, C.c_int, i64, i64, vp, vp, C.c_int, vp, C.c_int, C.c_int, vp, C.c_int, vp, vp,
+                                     vp, vp, sz, vp]
     L.bitcos_gemv_host_staging_bytes.restype = sz
     L.bitcos_gemv_host_staging_bytes.argtypes = [i64, i64, C.c_int]
     L.bitcos_gemv_host.argtypes = [C.POINTER(_Weights), vp, vp, C.c_int, vp, vp, sz, vp, sz, vp]
@@ -469,13 +470,16 @@ def bit2_gemv(W: DevicePlain, x, x_scale, y=None, acc_debug=None, workspace=None
 class DeviceExperts:
     """Descriptors of E same-shaped BITCOS matrices, copied to the device once."""
 
-    def __init__(self, experts: list[DeviceBitcos]):
+    def __init__(self, experts):
+        """experts: DeviceBitcos matrices, or DevicePlain ones (five-trit / 2-bit) of one format."""
         import torch
         self.experts = experts
         self.M, self.K = experts[0].M, experts[0].K
-        arr = (_Weights * len(experts))(*[e.desc for e in experts])
+        descs = [e.desc if isinstance(e, DeviceBitcos) else
+                 _Weights(e.words.data_ptr(), None, None, e.scales.data_ptr(), e.M, e.K, None) for e in experts]
+        arr = (_Weights * len(experts))(*descs)
         raw = np.frombuffer(bytes(arr), dtype=np.uint8).copy()
-        self.table = torch.from_numpy(raw).to(experts[0].bitmap.device)
+        self.table = torch.from_numpy(raw).to(experts[0].scales.device)
 
 
 def group_pairs(pair_expert, pair_xrow):
@@ -490,9 +494,7 @@ def group_pairs(pair_expert, pair_xrow):
     return order, ge.astype(np.int32), begin, pr_s, int(np.diff(begin).max())
 
 
-def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale,
-                        y=None, acc_debug=None, workspace=None):
-    """Grouped product: pairs listed per expert (device int32 tensors); y is [P, M] in list order."""
+def _grouped(name, E: DeviceExperts, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale, y, acc_debug, workspace):
     import torch
     n_groups, n_pairs = group_expert.numel(), pair_xrow.numel()
     if workspace is None:
@@ -502,12 +504,30 @@ def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, 
     acc = None
     if acc_debug is True:
         acc = torch.empty((n_pairs, E.M, E.K // GROUP), dtype=torch.int32, device=x.device)
-    _check(load_library().bitcos_gemv_grouped(E.table.data_ptr(), len(E.experts), E.M, E.K, group_expert.data_ptr(),
-                                              group_begin.data_ptr(), n_groups, pair_xrow.data_ptr(), n_pairs,
-                                              max_group_size, x.data_ptr(), x_scale.data_ptr(), y.data_ptr(),
-                                              acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
-                                              workspace.numel(), _stream()), "bitcos_gemv_grouped")
+    _check(getattr(load_library(), name)(E.table.data_ptr(), len(E.experts), E.M, E.K, group_expert.data_ptr(),
+                                         group_begin.data_ptr(), n_groups, pair_xrow.data_ptr(), n_pairs,
+                                         max_group_size, x.data_ptr(), x.shape[0], x_scale.data_ptr(), y.data_ptr(),
+                                         acc.data_ptr() if acc is not None else None, workspace.data_ptr(),
+                                         workspace.numel(), _stream()), name)
     return y, acc
+
+
+def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale,
+                        y=None, acc_debug=None, workspace=None):
+    """Grouped product: pairs listed per expert (device int32 tensors); y is [P, M] in list order."""
+    return _grouped("bitcos_gemv_grouped", E, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale, y, acc_debug, workspace)
+
+
+def trit5_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale,
+                       y=None, acc_debug=None, workspace=None):
+    """The grouped product from five-trit experts (DeviceExperts over DevicePlain matrices)."""
+    return _grouped("trit5_gemv_grouped", E, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale, y, acc_debug, workspace)
+
+
+def bit2_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale,
+                      y=None, acc_debug=None, workspace=None):
+    """The grouped product from 2-bit experts (DeviceExperts over DevicePlain matrices)."""
+    return _grouped("bit2_gemv_grouped", E, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale, y, acc_debug, workspace)
 
 
 class MultiJobs:

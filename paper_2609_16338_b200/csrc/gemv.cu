@@ -116,7 +116,37 @@ struct GroupedArgs {
     int n_experts;
     int n_groups;
     int flat;                  // 1: one list of all groups' items, split evenly over the thread blocks
+    int n_pairs;               // length of the pair list (outputs, pair_xrow)
+    int n_xrows;               // rows of x
 };
+
+// A group of a grouped product as its routing lists describe it; ok = false if the lists are
+// malformed for it (its pairs outside the pair list, more tokens than the launch was sized for, an
+// activation row outside x).  Such a group is skipped -- nothing of it is read or written -- and its
+// status word and the launch's (word 0 of the first group's workspace) are set to 2.
+struct GroupDesc {
+    int e, begin, end;
+    bool ok, empty;
+};
+__device__ __forceinline__ GroupDesc read_group(const GroupedArgs &ga, const int32_t *pair_xrow, unsigned int *status0, int grp,
+                                                int nb_max) {
+    GroupDesc d;
+    d.e = __ldg(ga.group_expert + grp);
+    d.begin = __ldg(ga.group_begin + grp);
+    d.end = __ldg(ga.group_begin + grp + 1);
+    d.empty = d.end <= d.begin;
+    d.ok = d.e >= 0 && d.e < ga.n_experts && d.begin >= 0 && d.end <= ga.n_pairs && d.end - d.begin <= nb_max;
+    if (d.ok && !d.empty)
+        for (int i = d.begin; i < d.end; ++i) {
+            const int r = __ldg(pair_xrow + i);
+            if (r < 0 || r >= ga.n_xrows) d.ok = false;
+        }
+    if (!d.ok && !d.empty) {
+        *reinterpret_cast<unsigned int *>(reinterpret_cast<uint8_t *>(status0) + static_cast<size_t>(grp) * ga.ws_stride) = 2u;
+        *status0 = 2u;
+    }
+    return d;
+}
 
 inline int64_t padded_rows(int64_t M) { return (M + kRows - 1) / kRows * kRows; }
 
@@ -520,6 +550,16 @@ __device__ __forceinline__ void issue_item(const Problem &pb, const View &pr, co
     sign_base[s * 4 + 0] = static_cast<uint32_t>(r.nt) | (static_cast<uint32_t>(r.t0 & 3) << 8);
     sign_base[s * 4 + 1] = static_cast<uint32_t>(r.g0);
     sign_base[s * 4 + 2] = static_cast<uint32_t>(r.rb0);
+    const uint32_t x_bytes = pl.x_in_stage ? static_cast<uint32_t>(pr.nb(pb)) * static_cast<uint32_t>(pb.K) : 0u;
+    // (issued after the format's expect_tx below; a grouped launch only)
+    auto copy_x = [&]() {
+        // the activation rows of this group's tokens (from L2): the decoders of a grouped launch
+        // find them next to the weights and need no block-wide staging step per group
+        if (pl.x_in_stage)
+            for (int b = 0; b < pr.nb(pb) && b < 2; ++b)
+                bulk_copy(d_scales + L.scale_cap + L.off_cap + static_cast<uint32_t>(b) * static_cast<uint32_t>(pb.K),
+                          pb.x + static_cast<int64_t>(xrows[b]) * pb.K, static_cast<uint32_t>(pb.K), bar);
+    };
     if (FMT == kBitcos) {
         const uint32_t b_lo = (o_lo >> 7) << 4, b_hi = ((o_hi + 127u) >> 7) << 4;
         const uint32_t sign_bytes = b_hi - b_lo;
@@ -528,15 +568,8 @@ __device__ __forceinline__ void issue_item(const Problem &pb, const View &pr, co
         // the tiles' entry offsets: the 16-byte aligned slice of tile_off that covers t0 .. t0 + nt
         const uint32_t o_first = static_cast<uint32_t>(r.t0 & 3);
         const uint32_t off_bytes = ((o_first + static_cast<uint32_t>(r.nt) + 1u + 3u) & ~3u) * 4u;
-        const uint32_t x_bytes = pl.x_in_stage ? static_cast<uint32_t>(pr.nb(pb)) * static_cast<uint32_t>(pb.K) : 0u;
         mbar_expect_tx(bar, bm_bytes + sign_bytes + scale_bytes + off_bytes + x_bytes);
-        if (pl.x_in_stage) {
-            // the activation rows of this group's tokens (from L2): the decoders of a grouped launch
-            // find them next to the weights and need no block-wide staging step per group
-            for (int b = 0; b < pr.nb(pb) && b < 2; ++b)
-                bulk_copy(d_scales + L.scale_cap + L.off_cap + static_cast<uint32_t>(b) * static_cast<uint32_t>(pb.K),
-                          pb.x + static_cast<int64_t>(xrows[b]) * pb.K, static_cast<uint32_t>(pb.K), bar);
-        }
+        copy_x();
         bulk_copy(d_scales + L.scale_cap, pr.tile_off(pb) + (r.t0 - o_first), off_bytes, bar);
         bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload(pb)) + r.t0 * 512, bm_bytes, bar);
         if (sign_bytes) bulk_copy(d_signs, reinterpret_cast<const uint8_t *>(pr.signs(pb)) + b_lo, sign_bytes, bar);
@@ -548,12 +581,14 @@ __device__ __forceinline__ void issue_item(const Problem &pb, const View &pr, co
         if (pl.CS == 1) w_hi = (r.rb0 + r.nt / pb.G) * WPR;
         else w_hi = r.rb0 * WPR + ((26 * (r.g0 + r.nt) - 1) >> 2) + 1;
         const uint32_t bytes = static_cast<uint32_t>(w_hi - w_lo) * 128u;
-        mbar_expect_tx(bar, bytes + scale_bytes);
+        mbar_expect_tx(bar, bytes + scale_bytes + x_bytes);
+        copy_x();
         bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload(pb)) + w_lo * 128, bytes, bar);
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
     } else {
         const uint32_t bytes = static_cast<uint32_t>(r.nt) * 1024u;
-        mbar_expect_tx(bar, bytes + scale_bytes);
+        mbar_expect_tx(bar, bytes + scale_bytes + x_bytes);
+        copy_x();
         bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload(pb)) + r.t0 * 1024, bytes, bar);
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
     }
@@ -1619,9 +1654,9 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_phased_kernel(c
 // names no expert.
 template <int NB>
 __device__ __forceinline__ bool grouped_problem(Problem &pr, const Problem &base, const GroupedArgs &ga, int grp) {
-    const int e = __ldg(ga.group_expert + grp);
-    const int begin = __ldg(ga.group_begin + grp), end = __ldg(ga.group_begin + grp + 1);
-    if (e < 0 || e >= ga.n_experts || end <= begin) return false;
+    const GroupDesc gd = read_group(ga, base.xrow, base.status, grp, NB);
+    if (!gd.ok || gd.empty) return false;
+    const int e = gd.e, begin = gd.begin, end = gd.end;
     const bitcos_weights wdesc = ga.experts[e];
     pr = base;
     pr.payload = wdesc.bitmap;
@@ -1665,9 +1700,9 @@ struct GroupedSegs {
             w.rem = 0;
             lo = seg_hi;
             const int g = grp++;
-            const int e = __ldg(ga->group_expert + g);
-            const int begin = __ldg(ga->group_begin + g), end = __ldg(ga->group_begin + g + 1);
-            if (e < 0 || e >= ga->n_experts || end <= begin) continue;
+            const GroupDesc gd = read_group(*ga, base->xrow, base->status, g, NB);
+            if (!gd.ok || gd.empty) continue;
+            const int e = gd.e, begin = gd.begin, end = gd.end;
             const bitcos_weights *wd = ga->experts + e;
             v.payload_ = wd->bitmap;
             v.signs_ = wd->signs;
@@ -1689,7 +1724,7 @@ struct GroupedSegs {
 // that crosses from one group to the next keeps its pipeline running (the producer is already
 // copying the next group's weights while the last tiles of this one are decoded).  Otherwise:
 // blockIdx.y = group, and the blocks of a row of the grid share that group's items.
-template <int NB>
+template <int FMT, int NB>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(const __grid_constant__ Problem base, const Plan pl,
                                                                                 const __grid_constant__ GroupedArgs ga) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -1698,7 +1733,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(
     if (!ga.flat) {
         Problem pr;
         if (!grouped_problem<NB>(pr, base, ga, static_cast<int>(blockIdx.y))) return;
-        run_problem<kBitcos, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
+        run_problem<FMT, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                                  static_cast<int>(blockIdx.x));
         return;
     }
@@ -1712,7 +1747,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(
     segs.lo = b * q + (b < rem ? b : rem);
     segs.hi = segs.lo + q + (b < rem ? 1 : 0);
     segs.grp = static_cast<int>(segs.lo / ipg);
-    run_segments<kBitcos, NB, 1>(segs, pl, smem, static_cast<int>(b));
+    run_segments<FMT, NB, 1>(segs, pl, smem, static_cast<int>(b));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -2046,15 +2081,15 @@ int launch_nb(const Problem &pr, const Plan &pl, cudaStream_t stream, const uint
     return launch<FMT, 16, XG>(pr, pl, stream, off_host);
 }
 
-template <int NB>
+template <int FMT, int NB>
 int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int n_groups, cudaStream_t stream) {
     if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * pr.K > kXResidentBytes) return BITCOS_ERR_SHAPE;
     int sms = 0, budget = 0;
-    int rc = prepare_kernel<gemv_grouped_kernel<NB>>(&sms, &budget);
+    int rc = prepare_kernel<gemv_grouped_kernel<FMT, NB>>(&sms, &budget);
     if (rc) return rc;
     Plan plw = pl;
-    plw.stages = choose_stages(kBitcos, pl, pr.G, NB, pr.K, budget);
-    const SmemLayout L = smem_layout(kBitcos, plw, pr.G, NB, pr.K);
+    plw.stages = choose_stages(FMT, pl, pr.G, NB, pr.K, budget);
+    const SmemLayout L = smem_layout(FMT, plw, pr.G, NB, pr.K);
     GroupedArgs gaw = ga;
     gaw.n_groups = n_groups;
     if (pl.CS == 1) {
@@ -2064,9 +2099,9 @@ int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int
         gaw.flat = 1;
         plw.cyclic = 0;
         plw.x_in_stage = NB < kMmaMinBatch ? 1 : 0;
-        plw.stages = choose_stages(kBitcos, plw, pr.G, NB, pr.K, budget);
-        const SmemLayout Lf = smem_layout(kBitcos, plw, pr.G, NB, pr.K);
-        return launch_pdl(gemv_grouped_kernel<NB>, dim3(static_cast<unsigned>(total < sms ? total : sms)), (pl.NW + 2) * 32,
+        plw.stages = choose_stages(FMT, plw, pr.G, NB, pr.K, budget);
+        const SmemLayout Lf = smem_layout(FMT, plw, pr.G, NB, pr.K);
+        return launch_pdl(gemv_grouped_kernel<FMT, NB>, dim3(static_cast<unsigned>(total < sms ? total : sms)), (pl.NW + 2) * 32,
                           Lf.total, stream, pr, plw, gaw);
     }
     // the machine is shared by all groups: spread its multiprocessors over them
@@ -2075,7 +2110,7 @@ int launch_grouped(const Problem &pr, const Plan &pl, const GroupedArgs &ga, int
     int gx = 1;
     choose_walk(plw, per_group, &gx);
     gaw.flat = 0;
-    return launch_pdl(gemv_grouped_kernel<NB>, dim3(gx, n_groups), (pl.NW + 2) * 32, L.total, stream, pr, plw, gaw);
+    return launch_pdl(gemv_grouped_kernel<FMT, NB>, dim3(gx, n_groups), (pl.NW + 2) * 32, L.total, stream, pr, plw, gaw);
 }
 
 // Validates the arguments every product shares; fills nothing.
@@ -2653,15 +2688,18 @@ int bit2_gemv(const uint32_t *words, const uint16_t *scales_tiled, int64_t M, in
                        workspace, workspace_bytes, cuda_stream);
 }
 
-int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K,
-                        const int32_t *group_expert, const int32_t *group_begin, int n_groups,
-                        const int32_t *pair_xrow, int n_pairs, int max_group_size, const int8_t *x,
-                        const float *x_scale, float *y, int32_t *acc_debug, void *workspace,
-                        size_t workspace_bytes, void *cuda_stream) {
+}  // extern "C"
+
+namespace {
+template <int FMT>
+int grouped_common(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                   const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs, int max_group_size,
+                   const int8_t *x, int n_xrows, const float *x_scale, float *y, int32_t *acc_debug, void *workspace,
+                   size_t workspace_bytes, void *cuda_stream) {
     if (!experts || !group_expert || !group_begin || !pair_xrow || !x || !x_scale || !y || !workspace)
         return BITCOS_ERR_NULL;
     if (M < 1 || K < kGroup || K % kGroup != 0 || n_experts < 1 || n_groups < 1 || n_groups > 65535 ||
-        n_pairs < n_groups || max_group_size < 1 || max_group_size > BITCOS_MAX_BATCH)
+        n_pairs < n_groups || n_xrows < 1 || max_group_size < 1 || max_group_size > BITCOS_MAX_BATCH)
         return BITCOS_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(y) || !aligned16(workspace) || (acc_debug && !aligned16(acc_debug)))
         return BITCOS_ERR_ALIGN;
@@ -2680,14 +2718,41 @@ int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M,
     pr.G = static_cast<int>(K / kGroup);
     pr.RB = static_cast<int>(padded_rows(M) / kRows);
     pr.status = static_cast<unsigned int *>(workspace);
-    GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts, n_groups, 0};
+    GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts, n_groups, 0, n_pairs, n_xrows};
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int nbk = nb_bucket(max_group_size, K);
-    if (nbk == 1) return launch_grouped<1>(pr, pl, ga, n_groups, stream);
-    if (nbk == 2) return launch_grouped<2>(pr, pl, ga, n_groups, stream);
-    if (max_group_size <= 4) return launch_grouped<4>(pr, pl, ga, n_groups, stream);
-    if (max_group_size <= 8) return launch_grouped<8>(pr, pl, ga, n_groups, stream);
-    return launch_grouped<16>(pr, pl, ga, n_groups, stream);
+    if (nbk == 1) return launch_grouped<FMT, 1>(pr, pl, ga, n_groups, stream);
+    if (nbk == 2) return launch_grouped<FMT, 2>(pr, pl, ga, n_groups, stream);
+    if (max_group_size <= 4) return launch_grouped<FMT, 4>(pr, pl, ga, n_groups, stream);
+    if (max_group_size <= 8) return launch_grouped<FMT, 8>(pr, pl, ga, n_groups, stream);
+    return launch_grouped<FMT, 16>(pr, pl, ga, n_groups, stream);
+}
+}  // namespace
+
+extern "C" {
+
+int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                        const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs,
+                        int max_group_size, const int8_t *x, int n_xrows, const float *x_scale, float *y,
+                        int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return grouped_common<kBitcos>(experts, n_experts, M, K, group_expert, group_begin, n_groups, pair_xrow, n_pairs,
+                                   max_group_size, x, n_xrows, x_scale, y, acc_debug, workspace, workspace_bytes, cuda_stream);
+}
+
+int trit5_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                       const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs,
+                       int max_group_size, const int8_t *x, int n_xrows, const float *x_scale, float *y,
+                       int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return grouped_common<kTrit5>(experts, n_experts, M, K, group_expert, group_begin, n_groups, pair_xrow, n_pairs,
+                                  max_group_size, x, n_xrows, x_scale, y, acc_debug, workspace, workspace_bytes, cuda_stream);
+}
+
+int bit2_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                      const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs,
+                      int max_group_size, const int8_t *x, int n_xrows, const float *x_scale, float *y,
+                      int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return grouped_common<kBit2>(experts, n_experts, M, K, group_expert, group_begin, n_groups, pair_xrow, n_pairs,
+                                 max_group_size, x, n_xrows, x_scale, y, acc_debug, workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"

@@ -130,7 +130,10 @@ def test_config4_moe_experts(bc, proj):
     base = datagen.config_seed(4, 0 if proj == "gate" else 500)
     Ws = [datagen.trits(base + e, M, K, z) for e in range(E)]
     Ss = [datagen.scales(base + e, M, K) for e in range(E)]
-    experts = bc.DeviceExperts([bc.bitcos_pack(Ws[e], Ss[e]).to_device() for e in range(E)])
+    sts = [bc.scales_tile(Ss[e], M, K) for e in range(E)]
+    formats = (("bitcos", bc.DeviceExperts([bc.bitcos_pack(Ws[e], Ss[e]).to_device() for e in range(E)]), bc.bitcos_gemv_grouped),
+               ("trit5", bc.DeviceExperts([bc.plain_to_device(bc.trit5_pack(Ws[e]), sts[e], M, K) for e in range(E)]), bc.trit5_gemv_grouped),
+               ("bit2", bc.DeviceExperts([bc.plain_to_device(bc.bit2_pack(Ws[e]), sts[e], M, K) for e in range(E)]), bc.bit2_gemv_grouped))
     for tokens in cfg["batches"]:
         ids = datagen.expert_choices(base + tokens, tokens, E, top_k)
         pair_expert = ids.reshape(-1)
@@ -145,7 +148,8 @@ def test_config4_moe_experts(bc, proj):
         order, ge, gb, xr, mx = bc.group_pairs(pair_expert, pair_xrow)
         acc_ref, y_ref, mag = oracle.grouped_dense(Ws, Ss, pair_expert[order], pair_xrow[order], x, xs)
         ws = bc.make_workspace(M, K, copies=len(ge))
-        for rep in range(2):
-            y, acc = bc.bitcos_gemv_grouped(experts, dev(ge), dev(gb), dev(xr), mx, dev(x), dev(xs), acc_debug=True,
-                                            workspace=ws)
-            compare(y, acc, acc_ref, y_ref, mag, f"config 4 {proj} tokens={tokens} rep{rep}")
+        for fmt, experts, f in formats:
+            for rep in range(2):
+                y, acc = f(experts, dev(ge), dev(gb), dev(xr), mx, dev(x), dev(xs), acc_debug=True, workspace=ws)
+                compare(y, acc, acc_ref, y_ref, mag, f"config 4 {proj} tokens={tokens} {fmt} rep{rep}")
+            assert bc.workspace_status(ws) == 0

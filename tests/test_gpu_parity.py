@@ -164,6 +164,49 @@ def test_grouped_many_small_groups(bc):
             check(y, acc, acc_ref, y_ref, mag, f"many groups tokens={tokens} rep{rep}")
 
 
+def test_grouped_malformed_routing_lists_are_skipped(bc):
+    """Routing lists come from device memory (a router's output) and are checked on the device: a
+    group that points outside the pair list, holds more pairs than the launch was sized for, names
+    an expert or an activation row that does not exist is skipped whole -- its outputs keep what
+    they held -- and the status word reads 2; the well-formed groups of the same call are right."""
+    E, M, K, tokens = 6, 96, 512, 4
+    Ws = [datagen.trits(1700 + e, M, K, 0.33) for e in range(E)]
+    Ss = [datagen.scales(1700 + e, M, K) for e in range(E)]
+    experts = bc.DeviceExperts([bc.bitcos_pack(Ws[e], Ss[e]).to_device() for e in range(E)])
+    x, xs = datagen.activations(1700, tokens, K)
+    pair_expert = np.array([0, 0, 2, 3, 3, 5], np.int32)
+    pair_xrow = np.array([0, 1, 2, 0, 3, 1], np.int32)
+    order, ge, gb, xr, mx = bc.group_pairs(pair_expert, pair_xrow)
+    acc_ref, y_ref, mag = oracle.grouped_dense(Ws, Ss, pair_expert[order], pair_xrow[order], x, xs)
+    n_groups = len(ge)
+
+    def run(ge_, gb_, xr_, mx_, bad_group):
+        ws = bc.make_workspace(M, K, copies=n_groups)
+        y = torch.full((len(xr_), M), 777.0, dtype=torch.float32, device="cuda")
+        y, _ = bc.bitcos_gemv_grouped(experts, dev(ge_), dev(gb_), dev(xr_), mx_, dev(x), dev(xs), y=y, workspace=ws)
+        torch.cuda.synchronize()
+        yh = y.cpu().numpy().astype(np.float64)
+        for g in range(n_groups):
+            rows = range(gb[g], gb[g + 1])
+            for r in rows:
+                if g in bad_group:
+                    assert (yh[r] == 777.0).all(), ("skipped group was written", g)
+                else:
+                    assert (np.abs(yh[r] - y_ref[r]) <= REL * mag[r]).all(), ("good group wrong", g)
+        assert bc.workspace_status(ws) == (2 if bad_group else 0)
+
+    run(ge, gb, xr, mx, set())
+    bad = ge.copy(); bad[1] = E + 3                    # an expert that does not exist
+    run(bad, gb, xr, mx, {1})
+    bad = ge.copy(); bad[2] = -1
+    run(bad, gb, xr, mx, {2})
+    bad = xr.copy(); bad[gb[0]] = tokens               # an activation row past the end of x
+    run(ge, gb, bad, mx, {0})
+    bad = xr.copy(); bad[gb[3]] = -5
+    run(ge, gb, bad, mx, {3})
+    run(ge, gb, xr, 1, {0, 2})                         # groups 0 and 2 hold two pairs, the launch was sized for one
+
+
 def test_grouped_down_projection_shape(bc):
     # K = 768 (six groups), per-pair activation rows
     E, M, K = 4, 2048, 768
