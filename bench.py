@@ -39,10 +39,25 @@ METRIC = "bitcos_gemv_us_per_token"
 UNIT = "us"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of all launches of one step, from ncu captures of this
-# command (summaries under profiles/): four launches per step (the default) and seven (--serial /
-# --branches, an earlier capture of the same kernels)
-NCU_DRAM_BYTES_PER_STEP = {4: 15289129, 7: 15627520}
+# roofline.traffic comes from the ncu summary of this command under profiles/: the file carries a line
+#   dram_bytes_per_step = <dram__bytes_read.sum + dram__bytes_write.sum of the launches of one step>  commit = <hash>
+TRAFFIC_PROFILE = os.path.join("profiles", "launch_list_and_dram_traffic_bitnet2b_layer_bench_default.md")
+
+
+def ncu_traffic():
+    """(bytes per step, source) of the default step's DRAM traffic as the committed ncu summary states it;
+    (None, reason) if the summary is missing or carries no figure."""
+    import re
+    path = os.path.join(ROOT, TRAFFIC_PROFILE)
+    try:
+        with open(path) as f:
+            text = f.read()
+    except OSError:
+        return None, f"{TRAFFIC_PROFILE} missing"
+    m = re.search(r"dram_bytes_per_step\s*=\s*(\d+)\s+commit\s*=\s*([0-9a-f]{7,40})", text)
+    if not m:
+        return None, f"{TRAFFIC_PROFILE} carries no dram_bytes_per_step line"
+    return int(m.group(1)), f"{TRAFFIC_PROFILE} (ncu capture at commit {m.group(2)})"
 
 
 def layer_config():
@@ -319,11 +334,8 @@ def run_cuda(args):
     step(0)
     torch.cuda.synchronize()
     if rank == 0:
-        import oracle
-        m = layer[1]
-        _, y_ref, mag = oracle.gemv_dense(m["W"], m["S"], m["x"], m["xs"])
-        err = np.abs(ys[1].cpu().numpy().astype(np.float64) - y_ref)
-        assert (err <= 1e-5 * mag).all(), "bench: bitcos_gemv disagrees with the oracle"
+        for m, y in zip(layer, ys):
+            assert_matches_oracle(y, m["W"], m["S"], m["x"], m["xs"], f"layer pass, {m['name']}")
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -427,16 +439,20 @@ def run_cuda(args):
         host_phases[i % copies].run()
 
     e2e_steps = 0 if args.no_e2e else min(args.steps, 200)
-    e2e_us = float("nan")
+    e2e_us, e2e_chunks = float("nan"), []
     if e2e_steps:
-        for i in range(3):
+        for i in range(10):
             e2e_step(i)
         torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for i in range(e2e_steps):
-            e2e_step(i)
+        # wall clock around chunks of steps (every step ends with its own stream wait); the median chunk
+        # is reported, so that a burst of other work on the host does not decide the figure
+        for c in range(10):
+            t0 = time.perf_counter()
+            for i in range(e2e_steps):
+                e2e_step(c * e2e_steps + i)
+            e2e_chunks.append((time.perf_counter() - t0) / e2e_steps * 1e6)
         torch.cuda.synchronize()
-        e2e_us = (time.perf_counter() - t0) / e2e_steps * 1e6
+        e2e_us = float(np.median(e2e_chunks))
     e2e_us = ranks.max(e2e_us)
     if args.serial or args.branches or args.e2e_per_phase:
         h2d = sum(m["K"] + 4 for m in layer)
@@ -447,6 +463,28 @@ def run_cuda(args):
     if rank != 0:
         ranks.close()
         return
+
+    # ---- every launch of a step on its own: idle GPU, cold L2, events around the one launch ----
+    isolated_us = None
+    phased_us = None
+    if not args.no_detail:
+        flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+        isolated_us = []
+        for gi in range(len(groups)):
+            ts = []
+            for r in range(12):
+                flush_buf.zero_()
+                torch.cuda.synchronize()
+                with torch.cuda.stream(stream):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    bc.bitcos_gemv_multi(multi[r % copies][gi])
+                    b.record(stream)
+                    stream.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3)
+            isolated_us.append(float(np.median(ts)))
+        # the whole layer pass as ONE launch with the dependencies enforced inside it
+        phased_us = graph_time_us(torch, stream, lambda i: bc.bitcos_gemv_phased(phased[i]), copies, launches=copies)
 
     # ---- the same seven products as ONE launch per step (what the launch structure costs) ----
     one_launch_us = None
@@ -468,7 +506,7 @@ def run_cuda(args):
 
     # ---- CPU baseline: the oracle on the host cores, bounded sample ----
     import oracle
-    reps, cpu_us = 0, float("nan")
+    reps, cpu_us, cpu1_us = 0, float("nan"), float("nan")
     if not args.no_cpu_baseline:
         o_packed = oracle_pack_layer(layer)
         t0 = time.perf_counter()
@@ -478,10 +516,19 @@ def run_cuda(args):
             if time.perf_counter() - t0 > 10.0 or reps >= 20:
                 break
         cpu_us = (time.perf_counter() - t0) / reps * 1e6
+        # the same on one thread (two passes)
+        all_threads = oracle.threads()
+        oracle.set_threads(1)
+        t0 = time.perf_counter()
+        for _ in range(2):
+            oracle_layer_pass(layer, o_packed)
+        cpu1_us = (time.perf_counter() - t0) / 2 * 1e6
+        oracle.set_threads(all_threads)
 
     peak, which = measured_peaks()
     us_per_step = ms * 1e3 / args.steps
-    launches_per_step = 7 if (args.serial or args.branches) else len(groups)
+    launches_per_step = 7 if (args.serial or args.branches) else 1 if args.launch == "phased" else len(groups)
+    traffic_step, traffic_src = ncu_traffic()
     n_launch = launches_per_step * args.steps
     achieved = layer_bytes * args.steps / (ms * 1e-3) / 1e9
     line = {
@@ -503,16 +550,18 @@ def run_cuda(args):
         "achieved_gbs": achieved,
         "frac_of_8tbs": achieved / 8000.0,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_DRAM_BYTES_PER_STEP[launches_per_step] / launches_per_step, "peak_source": f"{which} (STREAM-style copy)",
-                     "kernel": "gemv_kernel<bitcos, 1 token>" if launches_per_step == 7 else "gemv_multi_kernel<1 token>",
+                     "traffic": (traffic_step / launches_per_step) if (traffic_step and launches_per_step == 4 and args.launch == "multi") else None,
+                     "traffic_source": traffic_src, "peak_source": f"{which} (STREAM-style copy)",
+                     "kernel": "gemv_kernel<bitcos, 1 token>" if launches_per_step == 7 else "gemv_phased_kernel<1 token>" if launches_per_step == 1 else "gemv_multi_kernel<1 token>",
                      "launches": n_launch,
                      "avg_launch_us": ms * 1e3 / n_launch,
                      "algorithmic_bytes_per_launch": layer_bytes / launches_per_step},
-        "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+        "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "one_thread_us": cpu1_us,
                          "sample": f"{reps} full layer passes (7 GEMVs, 69.5 M weights each): BITCOS decode bit by "
                                    "bit, dense int32 dot per group, double scale-and-sum"},
         "e2e": {"value": whole_job_value(e2e_us, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps,
+                "steps": e2e_steps, "chunks": len(e2e_chunks), "statistic": "median chunk",
+                "us_min": min(e2e_chunks) if e2e_chunks else None, "us_max": max(e2e_chunks) if e2e_chunks else None,
                 "path": ("bitcos_gemv_host per GEMV: pinned x -> device, kernel, y -> pinned host, stream wait"
                          if (args.serial or args.branches) else
                          "bitcos_gemv_multi_host, four calls per step, each: pinned x -> device, launch, y -> pinned host, stream wait"
@@ -526,6 +575,13 @@ def run_cuda(args):
     }
     line["two_term_roofline"] = two_term_roofline(bc, cfg["z"], peak, clocks.get("sm_mhz") or 1965.0)
     if detail is not None:
+        line["isolated_launch_us"] = {"q+k+v": isolated_us[0], "o": isolated_us[1], "gate+up": isolated_us[2], "down": isolated_us[3],
+                                      "note": "one launch on an idle GPU with L2 flushed, CUDA events directly around it "
+                                              "(launch latency included, nothing overlaps)"}
+        line["phased_launch_per_step"] = {
+            "us": phased_us,
+            "note": "bitcos_gemv_phased: the layer pass as one launch, phases q|k|v, o, gate|up, down, the dependency "
+                    "between phases enforced by a device-side counter"}
         line["one_launch_per_step"] = {
             "us": one_launch_us, "gbs": layer_bytes / one_launch_us / 1e3, "frac": layer_bytes / one_launch_us / 1e3 / peak,
             "note": "all seven products of the layer in a single bitcos_gemv_multi launch: possible for independent "
@@ -543,12 +599,14 @@ def run_cuda(args):
         line["shapes"] = detail
         line["batch"] = batch_detail(bc, torch, stream)
         line["activation_quant"] = quant_detail(bc, torch, stream)
-    if args.all_configs:
+    if detail is not None and not args.layer_only:
+        # the other configurations: zero-density sweep, the Qwen3-32B-shaped layer at 1 to 16 tokens,
+        # the grouped mixture-of-experts product
         line["density_sweep"] = sweep_detail(bc, torch, stream)
         line["qwen32b_layer"] = qwen32b_layer_detail(bc, torch, stream)
-        line["device_pack"] = pack_detail(bc, torch)
-    if args.moe or args.all_configs:
         line["moe"] = moe_detail(bc, torch, stream)
+    if args.all_configs:
+        line["device_pack"] = pack_detail(bc, torch)
     print(json.dumps(line))
     ranks.close()
 
@@ -819,6 +877,14 @@ def pack_detail(bc, torch):
     return out
 
 
+def assert_matches_oracle(y, W, S, x, xs, what):
+    """Every table times outputs that were compared with the oracle first (fp32 within 1e-5 of sum|terms|)."""
+    import oracle
+    _, y_ref, mag = oracle.gemv_dense(W, S, x, xs)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref)
+    assert (err <= 1e-5 * mag).all(), f"bench: {what} disagrees with the oracle"
+
+
 def sweep_detail(bc, torch, stream):
     """Zero-density sweep (two matrix shapes, five densities, one token): the three formats on
     identical weights, realised gain against the byte ratio."""
@@ -842,6 +908,9 @@ def sweep_detail(bc, torch, stream):
             for name, (Wd, f) in fmts.items():
                 n_copies = max(2, int(np.ceil(4.2 * L2_BYTES / Wd.payload_bytes())))
                 reps = [Wd] + [Wd.clone() for _ in range(n_copies - 1)]
+                f(reps[-1], xd, xsd, y=y, workspace=ws)
+                torch.cuda.synchronize()
+                assert_matches_oracle(y, W, S, x, xs, f"density sweep {M}x{K} z={z} {name}")
                 us = graph_time_us(torch, stream, lambda i: f(reps[i], xd, xsd, y=y, workspace=ws), n_copies)
                 nbytes = algorithmic_bytes(M, K, packed.nnz, 1, name)
                 row[name] = {"us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak, "bytes": int(nbytes)}
@@ -863,19 +932,21 @@ def qwen32b_layer_detail(bc, torch, stream, z=0.4711):
     peak, _ = measured_peaks()
     shapes = [("q", 8192, 5120), ("k", 1024, 5120), ("v", 1024, 5120), ("o", 5120, 8192), ("gate", 25600, 5120),
               ("up", 25600, 5120), ("down", 5120, 25600)]
-    host = []
+    host, dense = [], []
     for i, (_, M, K) in enumerate(shapes):
         seed = datagen.config_seed(3, i)
-        host.append(bc.bitcos_pack(datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)))
+        dense.append((datagen.trits(seed, M, K, z), datagen.scales(seed, M, K)))
+        host.append(bc.bitcos_pack(*dense[-1]))
     base = [h.to_device() for h in host]
     replicas = [base, [w.clone() for w in base]]
     wss = [bc.make_workspace(M, K) for (_, M, K) in shapes]
     groups = [[0, 1, 2], [3], [4, 5], [6]]
     out = []
     for B in (1, 2, 4, 8, 16):
-        xs_dev = []
+        xs_dev, xs_host = [], []
         for i, (_, M, K) in enumerate(shapes):
             x, xs = datagen.activations(datagen.config_seed(3, i), B, K)
+            xs_host.append((x, xs))
             xs_dev.append((torch.from_numpy(x).cuda(), torch.from_numpy(xs).cuda()))
         ys = [torch.empty((B, M), dtype=torch.float32, device="cuda") for (_, M, K) in shapes]
         multi = [[bc.MultiJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in g]) for g in groups]
@@ -885,6 +956,10 @@ def qwen32b_layer_detail(bc, torch, stream, z=0.4711):
             for mj in multi[i]:
                 bc.bitcos_gemv_multi(mj)
 
+        step(1)
+        torch.cuda.synchronize()
+        for i, (nm, M, K) in enumerate(shapes):
+            assert_matches_oracle(ys[i], dense[i][0], dense[i][1], xs_host[i][0], xs_host[i][1], f"qwen layer {nm} B={B}")
         us = graph_time_us(torch, stream, step, len(replicas), launches=8)
         nbytes = sum(algorithmic_bytes(M, K, h.nnz, B) for (_, M, K), h in zip(shapes, host))
         out.append({"batch": B, "us_per_step": us, "us_per_token": us / B, "gbs": nbytes / us / 1e3,
@@ -937,11 +1012,13 @@ def run_profile_batch(args):
 
 
 def moe_detail(bc, torch, stream, E=128, top_k=8, z=0.3288):
-    """Grouped BITCOS product over the selected experts of a Qwen3-30B-A3B-shaped layer: gate/up
-    (768 x 2048, the token's activations) and down (2048 x 768, one activation row per pair), 1 to 16
-    tokens, expert ids drawn without replacement per token.  The experts of one projection (46 MB
-    packed) would fit in L2, so L2 is flushed before every launch and the routing is redrawn."""
+    """Grouped product over the selected experts of a Qwen3-30B-A3B-shaped layer, the three formats on
+    identical weights: gate/up (768 x 2048, the token's activations) and down (2048 x 768, one activation
+    row per pair), 1 to 16 tokens, expert ids drawn without replacement per token.  The experts of one
+    projection (46 MB packed) would fit in L2, so L2 is flushed before every launch and the routing is
+    redrawn.  Every format's first draw is compared with the oracle before it is timed."""
     import datagen
+    import oracle
     peak, _ = measured_peaks()
 
     def dev(a):
@@ -950,9 +1027,13 @@ def moe_detail(bc, torch, stream, E=128, top_k=8, z=0.3288):
     out = []
     flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
     for name, (M, K) in (("gate/up", (768, 2048)), ("down", (2048, 768))):
-        host = [bc.bitcos_pack(datagen.trits(datagen.config_seed(4, e), M, K, z), datagen.scales(datagen.config_seed(4, e), M, K))
-                for e in range(E)]
-        experts = bc.DeviceExperts([h.to_device() for h in host])
+        Ws = [datagen.trits(datagen.config_seed(4, e), M, K, z) for e in range(E)]
+        Ss = [datagen.scales(datagen.config_seed(4, e), M, K) for e in range(E)]
+        host = [bc.bitcos_pack(Ws[e], Ss[e]) for e in range(E)]
+        sts = [bc.scales_tile(Ss[e], M, K) for e in range(E)]
+        formats = (("bitcos", bc.DeviceExperts([h.to_device() for h in host]), bc.bitcos_gemv_grouped),
+                   ("trit5", bc.DeviceExperts([bc.plain_to_device(bc.trit5_pack(Ws[e]), sts[e], M, K) for e in range(E)]), bc.trit5_gemv_grouped),
+                   ("bit2", bc.DeviceExperts([bc.plain_to_device(bc.bit2_pack(Ws[e]), sts[e], M, K) for e in range(E)]), bc.bit2_gemv_grouped))
         for tokens in (1, 2, 4, 8, 16):
             draws = []
             for d in range(12):
@@ -965,22 +1046,33 @@ def moe_detail(bc, torch, stream, E=128, top_k=8, z=0.3288):
                     pair_xrow = np.arange(tokens * top_k, dtype=np.int32)
                     x, xs = datagen.activations(17, tokens * top_k, K)
                 order, ge, gb, xr, mx = bc.group_pairs(pair_expert, pair_xrow)
-                nbytes = sum(algorithmic_bytes(M, K, host[e].nnz, int(gb[i + 1] - gb[i])) for i, e in enumerate(ge))
-                draws.append((dev(ge), dev(gb), dev(xr), mx, len(ge), nbytes))
+                nb = {f: sum(algorithmic_bytes(M, K, host[e].nnz, int(gb[i + 1] - gb[i]), f) for i, e in enumerate(ge))
+                      for f in ("bitcos", "trit5", "bit2")}
+                draws.append((dev(ge), dev(gb), dev(xr), mx, len(ge), nb, (pair_expert[order], pair_xrow[order])))
             xd, xsd = dev(x), dev(xs)
             ws = bc.make_workspace(M, K, copies=max(d[4] for d in draws))
             y = torch.empty((tokens * top_k, M), dtype=torch.float32, device="cuda")
+            _, y_ref, mag = oracle.grouped_dense(Ws, Ss, draws[0][6][0], draws[0][6][1], x, xs)
+            row = {"projection": name, "M": M, "K": K, "tokens": tokens,
+                   "distinct_experts": float(np.mean([d[4] for d in draws]))}
+            for fmt, experts, f in formats:
+                def launch(i):
+                    ge, gb, xr, mx = draws[i][:4]
+                    f(experts, ge, gb, xr, mx, xd, xsd, y=y, workspace=ws)
 
-            def launch(i):
-                ge, gb, xr, mx, _, _ = draws[i]
-                bc.bitcos_gemv_grouped(experts, ge, gb, xr, mx, xd, xsd, y=y, workspace=ws)
-
-            us = graph_time_flushed_us(torch, stream, launch, len(draws), flush)
-            nbytes = float(np.mean([d[5] for d in draws]))
-            out.append({"projection": name, "M": M, "K": K, "tokens": tokens,
-                        "distinct_experts": float(np.mean([d[4] for d in draws])), "us": us,
-                        "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak})
-        del experts
+                launch(0)
+                torch.cuda.synchronize()
+                err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref)
+                assert (err <= 1e-5 * mag).all(), f"bench: grouped {fmt} {name} tokens={tokens} disagrees with the oracle"
+                us = graph_time_flushed_us(torch, stream, launch, len(draws), flush)
+                nbytes = float(np.mean([d[5][fmt] for d in draws]))
+                row[fmt] = {"us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak, "bytes": nbytes}
+            row["speedup_vs_trit5"] = row["trit5"]["us"] / row["bitcos"]["us"]
+            row["byte_ratio_trit5"] = row["trit5"]["bytes"] / row["bitcos"]["bytes"]
+            row["speedup_vs_bit2"] = row["bit2"]["us"] / row["bitcos"]["us"]
+            row["byte_ratio_bit2"] = row["bit2"]["bytes"] / row["bitcos"]["bytes"]
+            out.append(row)
+        del formats
         torch.cuda.empty_cache()
     return out
 
@@ -1012,9 +1104,9 @@ def main():
                     help="matrix of --profile-batch (default: the batch table's q projection)")
     ap.add_argument("--profile-batch", type=int, default=0, metavar="B",
                     help="only launch bitcos_gemv at batch B on the batch table's matrix, --steps times (for profilers)")
-    ap.add_argument("--all-configs", action="store_true",
-                    help="add the density sweep and the Qwen3-32B-shaped layer at 1-16 tokens (minutes of host-side packing)")
-    ap.add_argument("--moe", action="store_true", help="add the grouped mixture-of-experts table (slow to generate)")
+    ap.add_argument("--layer-only", action="store_true",
+                    help="leave out the tables of the other configurations (density sweep, Qwen3-32B-shaped layer, experts)")
+    ap.add_argument("--all-configs", action="store_true", help="add the device-side packing table")
     args = ap.parse_args()
     if args.profile_batch:
         if args.steps is None:

@@ -102,6 +102,8 @@ def lib():
                                     C.POINTER(C.c_double)]
         L.o_threads.restype = C.c_int
         L.o_threads.argtypes = []
+        L.o_set_threads.restype = None
+        L.o_set_threads.argtypes = [C.c_int]
         _lib = L
     return _lib
 
@@ -416,3 +418,8 @@ def gemv_dense_blend(W, scales, x):
 
 def threads() -> int:
     return int(lib().o_threads())
+
+
+def set_threads(n: int) -> None:
+    """Timing aid: the number of host threads the oracle's loops may use from now on."""
+    lib().o_set_threads(int(n))

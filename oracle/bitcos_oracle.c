@@ -571,3 +571,14 @@ int o_threads(void)
 #endif
     return n;
 }
+
+/* Timing aid only (no arithmetic): limits the number of threads the loops above may use, so that
+ * the same code can be timed on one core and on all of them.  n < 1 is ignored. */
+void o_set_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}

@@ -96,3 +96,20 @@ def test_reference_arm_under_two_ranks_prints_one_line_from_rank_zero():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
     assert line["e2e"] == {"value": line["value"], "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert line["value"] > 0
+
+
+def test_roofline_traffic_comes_from_the_committed_ncu_summary():
+    """bench.py takes roofline.traffic from the ncu summary under profiles/, not from a constant of its
+    own: the summary must exist, carry the figure and the commit it was captured at, and the figure
+    must agree with the step total the summary's own table prints."""
+    import re
+    import bench
+    step, src = bench.ncu_traffic()
+    assert step is not None, src
+    assert "commit" in src
+    with open(os.path.join(bench.ROOT, bench.TRAFFIC_PROFILE)) as f:
+        text = f.read()
+    m = re.search(r"\*\*step\*\*.*?\*\*([\d ]+)\*\* \| \*\*([\d ]+)\*\*", text)
+    assert m, "the summary's table has no step row"
+    assert int(m.group(1).replace(" ", "")) == step
+    assert 1.0 <= step / int(m.group(2).replace(" ", "")) < 1.2        # traffic against algorithmic bytes
