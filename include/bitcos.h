@@ -368,6 +368,18 @@ int bitcos_gemv_phased(const bitcos_gemv_job *jobs, const int *job_phase, int n_
 #define BITCOS_STATIC_WORKSPACE_BYTES (8 * 1024 * 1024)
 int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
                        void *cuda_stream);
+/* The status word of that array (as bitcos_workspace_status for a caller's workspace; waits for the
+ * stream): 0 if the last bitcos_gemv_static call on this device completed normally.  Every
+ * bitcos_gemv_static call clears the word before its kernel, so ask before the next call. */
+int bitcos_gemv_static_status(void *cuda_stream, int *status);
+
+/* Exercises the give-up path of the bounded waits without a fault (every wait inside the kernels is
+ * bounded; Section II of the paper has no counterpart: this is the library's own safety net).  One warp
+ * arms a barrier for bytes that no copy ever delivers, polls it with the kernels' own loop for limit_ns
+ * nanoseconds (1 us .. 100 ms), then sets the status word of `workspace` (device, at least 4 bytes) to 1 and
+ * returns normally, as a product whose copy never arrived would.  waited_ns: NULL or device uint64
+ * receiving the time spent polling.  The context stays usable; bitcos_workspace_status reads the word. */
+int bitcos_wait_probe(void *workspace, uint64_t limit_ns, uint64_t *waited_ns, void *cuda_stream);
 
 /* Host-buffer form of bitcos_gemv for callers whose activations live in host memory: copies
  * x_host[batch][K] and x_scale_host[batch] into `staging`, runs bitcos_gemv, copies

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe",
 ]
 
 
@@ -102,6 +102,8 @@ def load_library():
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_gemv_phased.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp]
     L.bitcos_gemv_phases_host.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp, sz, vp, vp, sz, vp]
+    L.bitcos_gemv_static_status.argtypes = [vp, C.POINTER(C.c_int)]
+    L.bitcos_wait_probe.argtypes = [vp, C.c_uint64, vp, vp]
     L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
     L.bitcos_quantize_activations.argtypes = [vp, C.c_int, i64, C.c_int, vp, vp, vp]
     L.bitcos_gemv_bf16.argtypes = [C.POINTER(_Weights), vp, C.c_int, vp, vp, vp, sz, vp]
@@ -670,6 +672,23 @@ def bitcos_decode_probe_variant(variant: int, W: DeviceBitcos, first_tile: int, 
 
 
 STATIC_WORKSPACE_BYTES = 8 * 1024 * 1024
+
+
+def bitcos_gemv_static_status() -> int:
+    """Status word of the library's built-in scratch array after the last bitcos_gemv_static call (waits for the stream)."""
+    v = C.c_int(-1)
+    _check(load_library().bitcos_gemv_static_status(_stream(), C.byref(v)), "bitcos_gemv_static_status")
+    return int(v.value)
+
+
+def bitcos_wait_probe(workspace, limit_ns: int = 1_000_000):
+    """Lets one bounded wait run out on purpose (no fault): sets the workspace's status word to 1; returns the
+    nanoseconds the kernel spent polling."""
+    import torch
+    waited = torch.zeros(1, dtype=torch.int64, device=workspace.device)
+    _check(load_library().bitcos_wait_probe(workspace.data_ptr(), int(limit_ns), waited.data_ptr(), _stream()), "bitcos_wait_probe")
+    torch.cuda.synchronize()
+    return int(waited.item())
 
 
 def bitcos_gemv_static(W: DeviceBitcos, x, x_scale, y):

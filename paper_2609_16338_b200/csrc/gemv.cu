@@ -299,18 +299,19 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return done;
 }
-// Polls until the phase completes, for at most kWaitLimitNs; false if it gave up.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
+// Polls until the phase completes, for at most limit_ns; false if it gave up.
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
     uint64_t t0 = 0;
     for (uint32_t i = 0;; ++i) {
         if (mbar_try(bar, parity)) return true;
         if ((i & 15u) == 15u) {
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
+            else if (now - t0 > limit_ns) return false;
         }
     }
 }
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) { return mbar_wait_limited(bar, parity, kWaitLimitNs); }
 // Waits for the given phase parity (bounded); the common case, an already completed phase, costs
 // one instruction.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -650,6 +651,7 @@ struct OneSegT {
     typedef ParamView View;
     static constexpr bool kSingle = true;      // never more than one segment
     static constexpr bool kHetero = false;     // all segments share one problem shape and one plan
+    static constexpr bool kListsLate = false;  // (no routing lists)
     static constexpr bool kDebug = DEBUG;      // false: acc_debug is known to be NULL (no code for it)
     static constexpr bool kGroupScales = XG;   // x_scale holds one scale per token AND group: [nb][G]
     static constexpr bool kQuantize = XQ;      // x holds bf16 activations: quantised per group of 128 by the decoder warps
@@ -811,11 +813,24 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
                 xrows[1] = pr.nb(pb) > 1 ? (pr.xrow(pb) ? __ldg(pr.xrow(pb) + 1) : 1) : 0;
             }
         };
+        // A grouped launch reads its routing lists (which may come from the previous kernel in the
+        // stream) to find its first item: the table copy, which depends on nothing, goes out before
+        // the wait for that kernel.
+        bool lut_issued = false;
+        if constexpr (Segs::kListsLate) {
+            if (lane == 0 && FMT != kBit2) {
+                mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
+                bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
+                          bar0 + 8u * kBarLut);
+                lut_issued = true;
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+        }
         bool have = src.next(pr, wk);
         while (have && wk.count <= 0) have = src.next(pr, wk);
         // The lookup table first: it is the largest transfer of the start-up (64 KB from L2) and
         // needs no address arithmetic.
-        if (lane == 0 && have && FMT != kBit2) {
+        if (lane == 0 && have && FMT != kBit2 && !lut_issued) {
             mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
             bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
                       bar0 + 8u * kBarLut);
@@ -827,6 +842,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             issue_loop(1);
         }
         __syncthreads();       // pairs with the barrier the other warps reach after staging the activations
+        if (lane == 0 && !have && lut_issued) mbar_wait(bar0 + 8u * kBarLut, 0);      // no copy may outlive the block
         if (lane != 0 || !have) return;
         if (ok) issue_loop(wk.count);
         while (!Segs::kSingle && ok && src.next(pr, wk)) {
@@ -1568,6 +1584,7 @@ struct PhasedSegs {
     typedef ParamView View;
     static constexpr bool kSingle = false;
     static constexpr bool kHetero = true;
+    static constexpr bool kListsLate = false;
     static constexpr bool kDebug = false;
     static constexpr bool kGroupScales = XG;
     static constexpr bool kQuantize = false;
@@ -1683,6 +1700,7 @@ struct GroupedSegs {
     typedef GroupView View;
     static constexpr bool kSingle = false;
     static constexpr bool kHetero = false;
+    static constexpr bool kListsLate = true;   // the routing lists are read only after the previous kernel has completed
     static constexpr bool kDebug = true;
     static constexpr bool kGroupScales = false;
     static constexpr bool kQuantize = false;
@@ -1728,9 +1746,9 @@ template <int FMT, int NB>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(const __grid_constant__ Problem base, const Plan pl,
                                                                                 const __grid_constant__ GroupedArgs ga) {
     extern __shared__ __align__(128) uint8_t smem[];
-    // the routing lists may come from the previous kernel in the stream
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (!ga.flat) {
+        // the routing lists may come from the previous kernel in the stream
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         Problem pr;
         if (!grouped_problem<NB>(pr, base, ga, static_cast<int>(blockIdx.y))) return;
         run_problem<FMT, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
@@ -1831,6 +1849,31 @@ __global__ void __launch_bounds__((kMaxWarps + 2) * 32, 1) decode_probe_kernel(i
     __syncthreads();
     if (threadIdx.x == 0) cycles[blockIdx.x] = s_max;
     if (total == 0x12345678) *sink = total;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Give-up path of the bounded waits, exercised without a fault: one warp arms an mbarrier for bytes
+// that no copy ever delivers and waits for it with the kernels' own polling loop and a short limit.
+// The wait runs out, the warp sets the workspace's status word exactly as the products do, and the
+// kernel returns normally; the context stays usable.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32, 1) wait_probe_kernel(unsigned int *status, unsigned long long limit_ns, unsigned long long *waited_ns) {
+    __shared__ __align__(8) unsigned long long bar_word;
+    const uint32_t bar = smem_addr(&bar_word);
+    const int lane = threadIdx.x & 31;
+    if (lane == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar, 64);                  // 64 bytes are announced; nothing is ever copied
+    }
+    __syncwarp();
+    const uint64_t t0 = global_timer_ns();
+    const bool ok = mbar_wait_limited(bar, 0, limit_ns);
+    const uint64_t t1 = global_timer_ns();
+    if (!ok && lane == 0) {
+        *status = 1u;
+        if (waited_ns) *waited_ns = t1 - t0;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -2308,7 +2351,8 @@ namespace {
 // cudaGetSymbolAddress; it is not a device address and is never passed to a kernel.
 static __device__ __align__(256) unsigned char g_static_workspace[BITCOS_STATIC_WORKSPACE_BYTES];
 
-// Device address of g_static_workspace on the current device, looked up once per device.
+// Device address of g_static_workspace on the current device, looked up once per device.  (The cache is
+// written without a lock: two threads that race on a device's first call both store the same address.)
 int static_workspace_ptr(void **out) {
     constexpr int kMaxDev = 32;
     static void *cache[kMaxDev];
@@ -2340,6 +2384,10 @@ int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_
     void *ws = nullptr;
     int rc = static_workspace_ptr(&ws);
     if (rc) return rc;
+    // (nothing is enqueued for a call that is going to be refused)
+    rc = check_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_scale, batch, y, nullptr, ws,
+                      BITCOS_STATIC_WORKSPACE_BYTES);
+    if (rc) return rc;
     // The array keeps whatever the last call left.  The status word and the arrival counters must
     // start at zero, so they are cleared on the caller's stream ahead of the kernel (the partial
     // sums behind them are always written before they are read).
@@ -2348,6 +2396,22 @@ int bitcos_gemv_static(const bitcos_weights *W, const int8_t *x, const float *x_
     if (rc) return rc;
     return gemv_common(kBitcos, W->bitmap, W->signs, W->tile_off, W->scales, W->M, W->K, x, x_scale, batch, y,
                        nullptr, ws, BITCOS_STATIC_WORKSPACE_BYTES, cuda_stream, W->tile_off_host);
+}
+
+int bitcos_gemv_static_status(void *cuda_stream, int *status) {
+    if (!status) return BITCOS_ERR_NULL;
+    void *ws = nullptr;
+    const int rc = static_workspace_ptr(&ws);
+    if (rc) return rc;
+    return bitcos_workspace_status(ws, cuda_stream, status);
+}
+
+int bitcos_wait_probe(void *workspace, uint64_t limit_ns, uint64_t *waited_ns, void *cuda_stream) {
+    if (!workspace) return BITCOS_ERR_NULL;
+    if (limit_ns < 1000 || limit_ns > 100ull * 1000 * 1000) return BITCOS_ERR_SHAPE;      // 1 us .. 100 ms
+    wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<unsigned int *>(workspace), limit_ns,
+                                                                        reinterpret_cast<unsigned long long *>(waited_ns));
+    return check_cuda(cudaGetLastError());
 }
 
 int bitcos_quantize_activations(const uint16_t *x_bf16, int batch, int64_t K, int group, int8_t *xq, float *x_scale,
