@@ -641,7 +641,7 @@ def quantised_layer_steps(bc, torch, layer, groups, replicas, ys, wss):
 
 
 def two_term_roofline(bc, z, peak_gbs, sm_mhz, sms=148):
-    """The paper's model T = max(B / beta, gamma) per 32 weights (Section IV-B.1), evaluated on this
+    """The paper's model T = max(B / beta, gamma) per 32 weights (Section III-B.1), evaluated on this
     GPU: gamma = measured cycles per 32 weights per multiprocessor with every operand on chip
     (bitcos_decode_probe, 20 decoder warps), beta = measured HBM bytes per clock per multiprocessor,
     B = bytes per 32 weights including the 16-bit group scale (and tile offsets for BITCOS)."""

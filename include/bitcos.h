@@ -9,7 +9,7 @@
  *              non-zero weight, same order) + entry offsets: 2 - z bits per weight at zero
  *              density z (paper Section II-A, Eq. 1).
  *   five-trit  five ternary digits per byte, 26 bytes per 128 weights (paper Section I).
- *   2-bit      two bits per weight (the paper's baseline format, Section IV).
+ *   2-bit      two bits per weight (the paper's baseline format, Section III).
  *
  *     acc[b][m][g] = sum_{k in group g} W[m][k] * x[b][k]                    (int32, exact)
  *     y[b][m]      = x_scale[b] * sum_g float(scale[m][g]) * float(acc[b][m][g])   (fp32)
@@ -74,7 +74,7 @@ int bitcos_last_cuda_error(void);
 
 /* ---------------------------------------------------------------------------------------
  * Host side: packers (paper Section II-A for BITCOS; Section I for five-trit; the 2-bit
- * format of Section IV).  Synchronous, deterministic; every padding bit and byte written
+ * format of Section III).  Synchronous, deterministic; every padding bit and byte written
  * is zero so that packed buffers can be compared with memcmp.
  * ------------------------------------------------------------------------------------- */
 
@@ -196,7 +196,7 @@ int bitcos_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_st
  * *status == 0 means every call that used the workspace so far completed normally. */
 int bitcos_workspace_status(const void *workspace, void *cuda_stream, int *status);
 
-/* Measurement aid for the paper's two-term roofline (Section IV-B.1, Eq. 6: T = max(B/beta, gamma)):
+/* Measurement aid for the paper's two-term roofline (Section III-B.1, Eq. 6: T = max(B/beta, gamma)):
  * gamma is the cost of the unpack sequence when every operand is already on chip.  Launches
  * `blocks` thread blocks of `warps_per_block` warps (1..22); each warp decodes one synthetic
  * 32 x 128 tile held in shared memory `iters` times with the code the GEMV kernels run (format
@@ -249,7 +249,7 @@ int bitcos_decode_probe_variant(int variant, const uint32_t *bitmap, const uint3
 int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, int batch, float *y,
                 int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
-/* Activation quantiser in front of the product.  Section III-C has the integer contraction
+/* Activation quantiser in front of the product.  Section II-C has the integer contraction
  * quantise the activations to int8 per group of 128 and apply the scales once per group; the
  * paper does not spell the rule out, and this library uses symmetric absmax quantisation, decided
  * in float32:
@@ -265,7 +265,7 @@ int bitcos_gemv(const bitcos_weights *W, const int8_t *x, const float *x_scale, 
 int bitcos_quantize_activations(const uint16_t *x_bf16, int batch, int64_t K, int group, int8_t *xq, float *x_scale,
                                 void *cuda_stream);
 
-/* bitcos_gemv with one activation scale per token and group of 128 (Section III-C):
+/* bitcos_gemv with one activation scale per token and group of 128 (Section II-C):
  *     y[b][m] = sum over groups g of  s[m][g] * x_group_scale[b][g] * (int32 sum over the group)
  *   x_group_scale   device float [batch][K/128], e.g. from bitcos_quantize_activations(group = 128)
  * Everything else as for bitcos_gemv (same accumulators, same workspace rules). */
@@ -288,7 +288,7 @@ int bitcos_gemv_bf16(const bitcos_weights *W, const uint16_t *x_bf16, int batch,
  *     y[b][m] = sum over k of (W[m][k] * s[m][k / 128]) * x[b][k],
  * on the tensor cores (mma.m16n8k16, bf16 operands, fp32 accumulation over each group of 128; the
  * groups are then added in fp32 in the fixed order of the other products).  Every product is exact
- * in fp32; the sums are within 4e-5 of the sum of |terms|.  batch 1..8 (ERR_SHAPE above);
+ * in fp32; the sums are within 2e-5 of the sum of |terms|.  batch 1..8 (ERR_SHAPE above);
  * x_bf16 = device bf16 [batch][K], 16-byte aligned; no accumulator dump.  About twice the cost of
  * the integer product at one token (the decoded weights are expanded to 16 bits on the way to the
  * tensor cores), the same at eight. */

@@ -344,14 +344,14 @@ def grouped_dense(expert_W, expert_scales, pair_expert, pair_xrow, x, xs):
     return np.stack(accs), np.stack(ys), np.stack(mags)
 
 
-# --- activations quantised per group of 128 (Section III-C: the integer contraction) ---------------
+# --- activations quantised per group of 128 (Section II-C: the integer contraction) ---------------
 AMAX_FLOOR = np.float32(2.0 ** -100)
 
 
 def quantize_activations(x, group: int = GROUP):
     """16- or 32-bit float activations [B, K] -> (int8 codes [B, K], float32 scales).
 
-    Section III-C only says that the integer path quantises the activations to int8 per group
+    Section II-C only says that the integer path quantises the activations to int8 per group
     of 128 and applies the scales once per group; the rule below is this build's reading of it
     (symmetric absmax quantisation), taken in float32, the precision the kernel decides in:
 
@@ -378,7 +378,7 @@ def quantize_activations(x, group: int = GROUP):
 
 def dense_y_group_scales(acc, scales, xs_g):
     """y[b, m] = sum over groups g of  s[m, g] * xs_g[b, g] * acc[b, m, g]   in float64
-    (Section III-C: int32 group sums, weight and activation scale applied once per group);
+    (Section II-C: int32 group sums, weight and activation scale applied once per group);
     also the sum of the absolute values of the terms, for the tolerance."""
     acc = np.asarray(acc, np.int64)
     B, M, G = acc.shape

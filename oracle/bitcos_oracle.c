@@ -31,7 +31,7 @@
 #include <omp.h>
 #endif
 
-#define O_GROUP 128      /* reduction elements per scale (Section IV-B.2: group size 128) */
+#define O_GROUP 128      /* reduction elements per scale (Section III-B.2: group size 128) */
 #define O_ROWS 32        /* output rows interleaved in one block, as the paper's 32-row panels */
 
 #define O_OK 0
@@ -42,21 +42,23 @@
 #define O_ERR_CURSOR (-5)
 
 /* ------------------------------------------------------------------------------------
- * Fig. 4: dst := _pdep_u32(a, mask).  For m = 0..31, if mask[m] then dst[m] := a[k++].
- * Bit m of a word is (word >> m) & 1 (LSB first; the figure merely draws bit 0 on the
- * left).
+ * Bit deposit (the operation of Fig. 4): the low bits of `a` are handed out, one by one
+ * and lowest first, to the positions where `mask` has a one; every other bit of the
+ * result is zero.  Written here as a walk over the ones of the mask: take the lowest
+ * one still standing, give it the next bit of `a`, strike it out.  Bit m of a word is
+ * (word >> m) & 1, i.e. LSB first.
  * ---------------------------------------------------------------------------------- */
 uint32_t o_pdep32(uint32_t a, uint32_t mask)
 {
-    uint32_t dst = 0;
-    int k = 0;
-    for (int m = 0; m < 32; ++m) {
-        if ((mask >> m) & 1u) {
-            dst |= ((a >> k) & 1u) << m;
-            k = k + 1;
-        }
+    uint32_t out = 0;
+    uint32_t left = mask;
+    while (left) {
+        uint32_t lowest = left & (~left + 1u);     /* the lowest one of the mask, alone */
+        if (a & 1u) out |= lowest;
+        a >>= 1;
+        left ^= lowest;
     }
-    return dst;
+    return out;
 }
 
 /* Eq. 2: w = p - 2n, with p the presence bit and n the "present and negative" bit. */

@@ -1770,7 +1770,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(
 
 // ---------------------------------------------------------------------------------------------
 // Decode-rate probe: what the paper's roofline calls gamma -- the cost of the unpack sequence when
-// every operand is already on chip (Section IV-B.1, Eq. 6).  Each warp decodes one synthetic tile
+// every operand is already on chip (Section III-B.1, Eq. 6).  Each warp decodes one synthetic tile
 // that sits in shared memory, `iters` times, with the same code the GEMV kernels run (popcounts,
 // prefix sum, sign windows, table lookups, dp4a); nothing is read from global memory inside the
 // timed loop.  cycles[block] receives the block's elapsed clock cycles.

@@ -1,4 +1,4 @@
-"""GPU parity for the quantised-activation front end (Section III-C): the int8 quantiser per
+"""GPU parity for the quantised-activation front end (Section II-C): the int8 quantiser per
 group of 128 / per token, and the product with one activation scale per token and group.
 
 Bar: codes, scales and int32 group accumulators bit-exact (the quantiser decides in float32

@@ -435,7 +435,7 @@ def test_generator_is_counter_based_and_has_the_stated_distribution():
     assert all(len(set(r)) == 8 for r in ids) and ids.min() >= 0 and ids.max() < 128
 
 
-# --- Section III-C: activations quantised per group of 128, scales applied once per group ---------
+# --- Section II-C: activations quantised per group of 128, scales applied once per group ---------
 def _bf16(vals):
     return datagen.bf16_bits_to_f32(datagen.f32_to_bf16_bits(np.asarray(vals, np.float32)))
 
@@ -625,3 +625,40 @@ def test_blend_product_bruteforce_and_cross_checks():
     Wz[1, 200] = -1
     y4, m4 = oracle.gemv_dense_blend(Wz, S, x)
     assert np.array_equal(y4[:, 1], -Sf[1, 1] * x[:, 200]) and not y4[:, [0, 2, 3]].any() and np.array_equal(m4, np.abs(y4))
+
+
+# --- row interleave of the two baseline layouts away from the first row block and the first word -----
+def test_trit5_word_lands_at_the_hand_computed_index_in_a_later_row_block():
+    """Row 70 = row block 2, lane 6; k = 130 = block 1 of the row, trit 2 of that block.  A 256-wide row
+    holds 52 bytes = 13 words (WPR); byte 26 opens block 1 and sits in word 6 at byte position 2.
+    Word q of row 32 rb + r is stored at (rb * WPR + q) * 32 + r = (2 * 13 + 6) * 32 + 6 = 1030.
+    An all-zero block byte is 1 + 3 + 9 + 27 + 81 = 121 (every digit holds trit + 1 = 1, and the 26th
+    byte pads its two unused places with digit 1); trit +1 in digit 2 adds 9: 130."""
+    M, K = 96, 256
+    W = np.zeros((M, K), dtype=np.int8)
+    zero_words = oracle.trit5_pack(W)
+    W[70, 130] = 1
+    words = oracle.trit5_pack(W)
+    assert words.size == 3 * 13 * 32
+    changed = np.flatnonzero(words != zero_words)
+    assert changed.tolist() == [1030]
+    assert int(words[1030]) == 121 | (121 << 8) | (130 << 16) | (121 << 24)
+    assert int(zero_words[1030]) == 121 * 0x01010101
+
+
+def test_bit2_word_lands_at_the_hand_computed_index_in_a_later_row_block():
+    """Row 70 = row block 2, lane 6; k = 130 = word 8 of the row (weight 2 of it), i.e. 16-byte chunk 2,
+    word 0.  Word j of chunk c of row 32 rb + r is stored at ((rb * (K / 64) + c) * 32 + r) * 4 + j
+    = ((2 * 4 + 2) * 32 + 6) * 4 = 1304.  Code = trit + 1, weight i at bits [8 (i % 4) + 2 (i / 4), + 2):
+    weight 2 sits at bits 16..17, where +1 turns code 01 into 10."""
+    M, K = 96, 256
+    W = np.zeros((M, K), dtype=np.int8)
+    zero_words = oracle.bit2_pack(W)
+    assert (zero_words == 0x55555555).all()
+    W[70, 130] = 1
+    words = oracle.bit2_pack(W)
+    changed = np.flatnonzero(words != zero_words)
+    assert changed.tolist() == [1304]
+    assert int(words[1304]) == 0x55565555
+    W[70, 130] = -1
+    assert int(oracle.bit2_pack(W)[1304]) == 0x55545555
