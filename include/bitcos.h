@@ -456,6 +456,33 @@ int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M,
                         int max_group_size, const int8_t *x, int n_xrows, const float *x_scale, float *y,
                         int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Routing with every list on the device, for decode loops whose router runs on the GPU (the paper's
+ * mixture-of-experts checkpoints, Table I, route per token; it gives no kernel for it).
+ *
+ * bitcos_group_pairs_device: the stable grouping by expert that the grouped products expect, done by
+ * one small kernel on the caller's stream.  pair_expert / pair_xrow: device int32 [n_pairs]
+ * (n_pairs <= BITCOS_GROUP_PAIRS_MAX, expert ids in [0, n_experts), n_experts <=
+ * BITCOS_GROUP_EXPERTS_MAX).  Outputs (device): group_expert [min(n_pairs, n_experts)], group_begin
+ * [min(n_pairs, n_experts) + 1], pair_xrow_sorted [n_pairs], order [n_pairs] (sorted pair i is input
+ * pair order[i]: output row i of the grouped product belongs to it), n_groups [1].  Experts ascending,
+ * input order kept inside a group.  A pair with an expert id out of range is left out.
+ *
+ * bitcos_gemv_grouped_lists: bitcos_gemv_grouped with the NUMBER of groups read from device memory
+ * (n_groups_device, as bitcos_group_pairs_device wrote it; values above max_groups are clipped).
+ * max_groups sizes the launch and the workspace (max_groups * bitcos_gemv_workspace_bytes(M, K)).
+ * max_group_size is an upper bound the caller knows without the lists, e.g. the number of tokens when
+ * every token picks distinct experts.  Everything else as for bitcos_gemv_grouped. */
+#define BITCOS_GROUP_PAIRS_MAX 4096
+#define BITCOS_GROUP_EXPERTS_MAX 1024
+int bitcos_group_pairs_device(const int32_t *pair_expert, const int32_t *pair_xrow, int n_pairs, int n_experts,
+                              int32_t *group_expert, int32_t *group_begin, int32_t *pair_xrow_sorted, int32_t *order,
+                              int32_t *n_groups, void *cuda_stream);
+int bitcos_gemv_grouped_lists(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                              const int32_t *group_begin, const int32_t *n_groups_device, int max_groups,
+                              const int32_t *pair_xrow, int n_pairs, int max_group_size, const int8_t *x, int n_xrows,
+                              const float *x_scale, float *y, int32_t *acc_debug, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream);
+
 /* The same grouped product from five-trit and 2-bit experts, so that the layout's gain can be
  * measured on the same chip for the mixture-of-experts shapes too (Section II-A: below a zero
  * density of 0.375 the five-trit format is the smaller one).  experts[e].bitmap points to the packed

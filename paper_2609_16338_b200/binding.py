@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe", "bitcos_group_pairs_device", "bitcos_gemv_grouped_lists",
 ]
 
 
@@ -102,6 +102,9 @@ def load_library():
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
     L.bitcos_gemv_phased.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp]
     L.bitcos_gemv_phases_host.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp, sz, vp, vp, sz, vp]
+    L.bitcos_group_pairs_device.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp]
+    L.bitcos_gemv_grouped_lists.argtypes = [vp, C.c_int, i64, i64, vp, vp, vp, C.c_int, vp, C.c_int, C.c_int, vp, C.c_int,
+                                            vp, vp, vp, vp, sz, vp]
     L.bitcos_gemv_static_status.argtypes = [vp, C.POINTER(C.c_int)]
     L.bitcos_wait_probe.argtypes = [vp, C.c_uint64, vp, vp]
     L.bitcos_gemv_multi_host.argtypes = [C.POINTER(_HostJob), C.c_int, C.c_int, vp]
@@ -518,6 +521,44 @@ def bitcos_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, 
                         y=None, acc_debug=None, workspace=None):
     """Grouped product: pairs listed per expert (device int32 tensors); y is [P, M] in list order."""
     return _grouped("bitcos_gemv_grouped", E, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale, y, acc_debug, workspace)
+
+
+def bitcos_group_pairs_device(pair_expert, pair_xrow, n_experts: int):
+    """Groups (expert, activation row) pairs by expert on the device (device int32 tensors in, device tensors out):
+    returns (group_expert, group_begin, pair_xrow_sorted, order, n_groups), n_groups a one-element device tensor."""
+    import torch
+    P = pair_expert.numel()
+    cap = min(P, n_experts)
+    dev = pair_expert.device
+    ge = torch.zeros(cap, dtype=torch.int32, device=dev)
+    gb = torch.zeros(cap + 1, dtype=torch.int32, device=dev)
+    xr = torch.zeros(P, dtype=torch.int32, device=dev)
+    order = torch.full((P,), -1, dtype=torch.int32, device=dev)
+    ng = torch.zeros(1, dtype=torch.int32, device=dev)
+    _check(load_library().bitcos_group_pairs_device(pair_expert.data_ptr(), pair_xrow.data_ptr(), P, n_experts, ge.data_ptr(),
+                                                    gb.data_ptr(), xr.data_ptr(), order.data_ptr(), ng.data_ptr(), _stream()),
+           "bitcos_group_pairs_device")
+    return ge, gb, xr, order, ng
+
+
+def bitcos_gemv_grouped_lists(E: DeviceExperts, group_expert, group_begin, n_groups_dev, pair_xrow, max_group_size, x, x_scale,
+                              y=None, acc_debug=None, workspace=None):
+    """bitcos_gemv_grouped with the number of groups left on the device (see bitcos_group_pairs_device)."""
+    import torch
+    max_groups, n_pairs = group_expert.numel(), pair_xrow.numel()
+    if workspace is None:
+        workspace = make_workspace(E.M, E.K, x.device, copies=max_groups)
+    if y is None:
+        y = torch.empty((n_pairs, E.M), dtype=torch.float32, device=x.device)
+    acc = None
+    if acc_debug is True:
+        acc = torch.empty((n_pairs, E.M, E.K // GROUP), dtype=torch.int32, device=x.device)
+    _check(load_library().bitcos_gemv_grouped_lists(E.table.data_ptr(), len(E.experts), E.M, E.K, group_expert.data_ptr(),
+                                                    group_begin.data_ptr(), n_groups_dev.data_ptr(), max_groups,
+                                                    pair_xrow.data_ptr(), n_pairs, max_group_size, x.data_ptr(), x.shape[0],
+                                                    x_scale.data_ptr(), y.data_ptr(), acc.data_ptr() if acc is not None else None,
+                                                    workspace.data_ptr(), workspace.numel(), _stream()), "bitcos_gemv_grouped_lists")
+    return y, acc
 
 
 def trit5_gemv_grouped(E: DeviceExperts, group_expert, group_begin, pair_xrow, max_group_size, x, x_scale,

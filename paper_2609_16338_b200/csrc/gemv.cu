@@ -118,6 +118,7 @@ struct GroupedArgs {
     int flat;                  // 1: one list of all groups' items, split evenly over the thread blocks
     int n_pairs;               // length of the pair list (outputs, pair_xrow)
     int n_xrows;               // rows of x
+    const int32_t *n_groups_dev;   // NULL, or device word holding the number of groups (n_groups is then its upper bound)
 };
 
 // A group of a grouped product as its routing lists describe it; ok = false if the lists are
@@ -1746,16 +1747,24 @@ template <int FMT, int NB>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_grouped_kernel(const __grid_constant__ Problem base, const Plan pl,
                                                                                 const __grid_constant__ GroupedArgs ga) {
     extern __shared__ __align__(128) uint8_t smem[];
+    int n_groups = ga.n_groups;
+    if (ga.n_groups_dev) {
+        // the number of groups itself comes from the device (a grouping kernel earlier in the stream)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const int n = __ldg(ga.n_groups_dev);
+        n_groups = n < 0 ? 0 : (n < n_groups ? n : n_groups);
+    }
     if (!ga.flat) {
         // the routing lists may come from the previous kernel in the stream
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (static_cast<int>(blockIdx.y) >= n_groups) return;
         Problem pr;
         if (!grouped_problem<NB>(pr, base, ga, static_cast<int>(blockIdx.y))) return;
         run_problem<FMT, NB>(pr, pl, smem, make_walk(pl, static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x)),
                                  static_cast<int>(blockIdx.x));
         return;
     }
-    const int64_t ipg = pl.items, total = ipg * ga.n_groups;
+    const int64_t ipg = pl.items, total = ipg * n_groups;
     const int64_t nblk = gridDim.x, b = blockIdx.x;
     const int64_t q = total / nblk, rem = total - q * nblk;
     GroupedSegs<NB> segs;
@@ -1873,6 +1882,56 @@ __global__ void __launch_bounds__(32, 1) wait_probe_kernel(unsigned int *status,
     if (!ok && lane == 0) {
         *status = 1u;
         if (waited_ns) *waited_ns = t1 - t0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Routing pairs grouped by expert on the device (a stable counting sort in one thread block), so
+// that a decode loop whose router runs on the GPU never has to bring the pairs to the host: count
+// the pairs of every expert, give every expert that has any a group (experts ascending), place
+// every pair behind the pairs of the same expert that precede it in the input.  A pair whose expert
+// id is out of range is dropped (it gets no group and order -1 is never written for it; its output
+// row is simply not produced).
+// ---------------------------------------------------------------------------------------------
+constexpr int kGroupPairsThreads = 256;
+__global__ void __launch_bounds__(kGroupPairsThreads) group_pairs_kernel(const int32_t *__restrict__ pair_expert,
+                                                                         const int32_t *__restrict__ pair_xrow, int n_pairs, int n_experts,
+                                                                         int32_t *group_expert, int32_t *group_begin,
+                                                                         int32_t *pair_xrow_sorted, int32_t *order, int32_t *n_groups) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    __shared__ int count[BITCOS_GROUP_EXPERTS_MAX];      // pairs per expert, then the expert's first position
+    for (int e = threadIdx.x; e < n_experts; e += kGroupPairsThreads) count[e] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_pairs; i += kGroupPairsThreads) {
+        const int e = pair_expert[i];
+        if (e >= 0 && e < n_experts) atomicAdd(&count[e], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int pos = 0, g = 0;
+        for (int e = 0; e < n_experts; ++e) {
+            const int c = count[e];
+            count[e] = pos;
+            if (c) {
+                group_expert[g] = e;
+                group_begin[g] = pos;
+                ++g;
+            }
+            pos += c;
+        }
+        group_begin[g] = pos;
+        *n_groups = g;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_pairs; i += kGroupPairsThreads) {
+        const int e = pair_expert[i];
+        if (e < 0 || e >= n_experts) continue;
+        int rank = 0;
+        for (int j = 0; j < i; ++j) rank += (pair_expert[j] == e) ? 1 : 0;      // stable: input order inside a group
+        const int at = count[e] + rank;
+        pair_xrow_sorted[at] = pair_xrow[i];
+        order[at] = i;
     }
 }
 
@@ -2759,11 +2818,11 @@ template <int FMT>
 int grouped_common(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
                    const int32_t *group_begin, int n_groups, const int32_t *pair_xrow, int n_pairs, int max_group_size,
                    const int8_t *x, int n_xrows, const float *x_scale, float *y, int32_t *acc_debug, void *workspace,
-                   size_t workspace_bytes, void *cuda_stream) {
+                   size_t workspace_bytes, void *cuda_stream, const int32_t *n_groups_dev = nullptr) {
     if (!experts || !group_expert || !group_begin || !pair_xrow || !x || !x_scale || !y || !workspace)
         return BITCOS_ERR_NULL;
     if (M < 1 || K < kGroup || K % kGroup != 0 || n_experts < 1 || n_groups < 1 || n_groups > 65535 ||
-        n_pairs < n_groups || n_xrows < 1 || max_group_size < 1 || max_group_size > BITCOS_MAX_BATCH)
+        (!n_groups_dev && n_pairs < n_groups) || n_pairs < 1 || n_xrows < 1 || max_group_size < 1 || max_group_size > BITCOS_MAX_BATCH)
         return BITCOS_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(y) || !aligned16(workspace) || (acc_debug && !aligned16(acc_debug)))
         return BITCOS_ERR_ALIGN;
@@ -2782,7 +2841,7 @@ int grouped_common(const bitcos_weights *experts, int n_experts, int64_t M, int6
     pr.G = static_cast<int>(K / kGroup);
     pr.RB = static_cast<int>(padded_rows(M) / kRows);
     pr.status = static_cast<unsigned int *>(workspace);
-    GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts, n_groups, 0, n_pairs, n_xrows};
+    GroupedArgs ga{experts, group_expert, group_begin, stride, n_experts, n_groups, 0, n_pairs, n_xrows, n_groups_dev};
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int nbk = nb_bucket(max_group_size, K);
     if (nbk == 1) return launch_grouped<FMT, 1>(pr, pl, ga, n_groups, stream);
@@ -2801,6 +2860,27 @@ int bitcos_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M,
                         int32_t *acc_debug, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     return grouped_common<kBitcos>(experts, n_experts, M, K, group_expert, group_begin, n_groups, pair_xrow, n_pairs,
                                    max_group_size, x, n_xrows, x_scale, y, acc_debug, workspace, workspace_bytes, cuda_stream);
+}
+
+int bitcos_gemv_grouped_lists(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,
+                              const int32_t *group_begin, const int32_t *n_groups_device, int max_groups,
+                              const int32_t *pair_xrow, int n_pairs, int max_group_size, const int8_t *x, int n_xrows,
+                              const float *x_scale, float *y, int32_t *acc_debug, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream) {
+    if (!n_groups_device) return BITCOS_ERR_NULL;
+    return grouped_common<kBitcos>(experts, n_experts, M, K, group_expert, group_begin, max_groups, pair_xrow, n_pairs,
+                                   max_group_size, x, n_xrows, x_scale, y, acc_debug, workspace, workspace_bytes, cuda_stream,
+                                   n_groups_device);
+}
+
+int bitcos_group_pairs_device(const int32_t *pair_expert, const int32_t *pair_xrow, int n_pairs, int n_experts,
+                              int32_t *group_expert, int32_t *group_begin, int32_t *pair_xrow_sorted, int32_t *order,
+                              int32_t *n_groups, void *cuda_stream) {
+    if (!pair_expert || !pair_xrow || !group_expert || !group_begin || !pair_xrow_sorted || !order || !n_groups)
+        return BITCOS_ERR_NULL;
+    if (n_pairs < 1 || n_pairs > BITCOS_GROUP_PAIRS_MAX || n_experts < 1 || n_experts > BITCOS_GROUP_EXPERTS_MAX) return BITCOS_ERR_SHAPE;
+    return launch_pdl(group_pairs_kernel, dim3(1), kGroupPairsThreads, 0, static_cast<cudaStream_t>(cuda_stream), pair_expert,
+                      pair_xrow, n_pairs, n_experts, group_expert, group_begin, pair_xrow_sorted, order, n_groups);
 }
 
 int trit5_gemv_grouped(const bitcos_weights *experts, int n_experts, int64_t M, int64_t K, const int32_t *group_expert,

@@ -207,6 +207,33 @@ def test_grouped_malformed_routing_lists_are_skipped(bc):
     run(ge, gb, xr, 1, {0, 2})                         # groups 0 and 2 hold two pairs, the launch was sized for one
 
 
+def test_routing_grouped_on_the_device(bc):
+    """The pairs stay on the device: bitcos_group_pairs_device sorts them by expert (stable), and
+    bitcos_gemv_grouped_lists reads the number of groups from device memory.  Same lists as the host
+    grouping, same outputs as the oracle; rows cut into column blocks (K = 6912) and rows in one piece."""
+    for (E, M, K, top_k, tokens) in ((32, 160, 1280, 4, 5), (16, 96, 6912, 3, 2), (128, 768, 2048, 8, 16), (8, 64, 256, 2, 1)):
+        Ws = [datagen.trits(1800 + e, M, K, 0.33) for e in range(E)]
+        Ss = [datagen.scales(1800 + e, M, K) for e in range(E)]
+        experts = bc.DeviceExperts([bc.bitcos_pack(Ws[e], Ss[e]).to_device() for e in range(E)])
+        x, xs = datagen.activations(1800 + tokens, tokens, K)
+        ids = datagen.expert_choices(1800 + tokens, tokens, E, top_k)
+        rng = np.random.default_rng(E)
+        perm = rng.permutation(tokens * top_k)                     # pairs in no particular order
+        pair_expert = ids.reshape(-1)[perm].astype(np.int32)
+        pair_xrow = np.repeat(np.arange(tokens, dtype=np.int32), top_k)[perm]
+        order_h, ge_h, gb_h, xr_h, mx = bc.group_pairs(pair_expert, pair_xrow)
+        ge, gb, xr, order, ng = bc.bitcos_group_pairs_device(dev(pair_expert), dev(pair_xrow), E)
+        torch.cuda.synchronize()
+        n = int(ng.item())
+        assert n == len(ge_h)
+        assert np.array_equal(ge.cpu().numpy()[:n], ge_h) and np.array_equal(gb.cpu().numpy()[:n + 1], gb_h)
+        assert np.array_equal(xr.cpu().numpy(), xr_h) and np.array_equal(order.cpu().numpy(), order_h)
+        acc_ref, y_ref, mag = oracle.grouped_dense(Ws, Ss, pair_expert[order_h], pair_xrow[order_h], x, xs)
+        for rep in range(2):
+            y, acc = bc.bitcos_gemv_grouped_lists(experts, ge, gb, ng, xr, min(tokens, 16), dev(x), dev(xs), acc_debug=True)
+            check(y, acc, acc_ref, y_ref, mag, f"device routing E={E} tokens={tokens} rep{rep}")
+
+
 def test_grouped_down_projection_shape(bc):
     # K = 768 (six groups), per-pair activation rows
     E, M, K = 4, 2048, 768
