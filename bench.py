@@ -288,6 +288,14 @@ def run_cuda(args):
     multi = [[bc.MultiJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in g]) for g in groups]
              for rep in replicas]
 
+    # what each launch asks to be brought into L2: the matrices of the launch after it (the first
+    # launch of the next layer -- the next rotated copy -- after the last)
+    def later(c, gi, d):
+        g = gi + d
+        return [replicas[(c + g // len(groups)) % copies][j] for j in groups[g % len(groups)]]
+    nexts = [[bc.NextWeights([w for d in args.prefetch_depth for w in later(c, gi, d)]) for gi in range(len(groups))]
+             for c in range(copies)]
+
     phases = [p for p, g in enumerate(groups) for _ in g]
     order = [j for g in groups for j in g]
     phased = [bc.PhasedJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in order], phases) for rep in replicas]
@@ -309,8 +317,8 @@ def run_cuda(args):
             bc.bitcos_gemv_phased(phased[i % copies])
             return
         if not args.branches:
-            for mj in multi[i % copies]:
-                bc.bitcos_gemv_multi(mj)
+            for gi, mj in enumerate(multi[i % copies]):
+                bc.bitcos_gemv_multi(mj, next=nexts[i % copies][gi] if args.prefetch and gi in args.prefetch_launches else None)
             return
         cur = torch.cuda.current_stream()
         for sd in sides:
@@ -544,7 +552,11 @@ def run_cuda(args):
                                  "7 launches per step: q|k|v on parallel branches, o, gate|up on parallel branches, down"
                                  if args.branches else
                                  "4 launches per step through bitcos_gemv_multi: q+k+v, o, gate+up, down (GEMVs that "
-                                 "read the same input share a launch)")
+                                 "read the same input share a launch)"
+                                 + ("; launches " + ",".join(str(g + 1) for g in args.prefetch_launches)
+                                    + " of the step also ask for the NEXT launch's packed weights to be brought into L2"
+                                      " (bitcos_gemv_multi_prefetch): every byte still comes from device memory"
+                                      " once per step" if args.prefetch and args.launch == "multi" else ""))
                               + "; programmatic dependent launch between consecutive kernels of a stream"),
                    "replicas": world},
         "achieved_gbs": achieved,
@@ -1090,6 +1102,12 @@ def main():
     ap.add_argument("--launch", default="multi", choices=["multi", "phased"],
                     help="multi: four bitcos_gemv_multi launches per step; phased: the whole layer pass as one "
                          "bitcos_gemv_phased launch (phases q|k|v, o, gate|up, down)")
+    ap.add_argument("--no-prefetch", dest="prefetch", action="store_false",
+                    help="plain bitcos_gemv_multi launches: no launch asks for the next launch's packed weights to be brought into L2")
+    ap.add_argument("--prefetch-launches", type=lambda v: [int(t) for t in v.split(",")], default=[1, 2],
+                    help="with --prefetch: which of the step's four launches carry a request")
+    ap.add_argument("--prefetch-depth", type=lambda v: [int(t) for t in v.split(",")], default=[1],
+                    help="with --prefetch: which later launches' weights a launch asks for (1 = the next one)")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA graphs (for profilers)")
     ap.add_argument("--e2e-per-phase", action="store_true",
                     help="end-to-end leg through four bitcos_gemv_multi_host calls per step instead of one bitcos_gemv_phases_host call")

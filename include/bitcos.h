@@ -313,6 +313,19 @@ typedef struct bitcos_gemv_job {
     size_t workspace_bytes;
 } bitcos_gemv_job;
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
+/* bitcos_gemv_multi, which in passing asks for the packed arrays of `next` (host array of n_next
+ * pointers to host structs of device pointers, n_next <= 7; may be 0) to be brought into the
+ * level-2 cache: the matrices a LATER launch multiplies by (the next products of the layer, the
+ * first of the next layer).  Every thread block requests its share of each array once its own first
+ * copies are under way; nothing waits for the requests and nothing is written, so results are
+ * those of bitcos_gemv_multi whatever `next` holds.  The sign vector of a matrix is only requested
+ * if its descriptor carries tile_off_host (its length is not known otherwise).  The paper reads
+ * weights from memory as the product reaches them (Section II-D); this hint has no counterpart
+ * there.  It pays when the launches of a decode step are short: the later launch then starts from
+ * L2 instead of device memory.  Errors as bitcos_gemv_multi, plus BITCOS_ERR_NULL / BITCOS_ERR_SHAPE
+ * for a malformed `next`. */
+int bitcos_gemv_multi_prefetch(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *next,
+                               int n_next, void *cuda_stream);
 /* The same with one activation scale per token and group of 128 (see bitcos_gemv_group_scales):
  * every job's x_scale points to device float [batch][K/128]. */
 int bitcos_gemv_multi_group_scales(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe", "bitcos_group_pairs_device", "bitcos_gemv_grouped_lists",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe", "bitcos_group_pairs_device", "bitcos_gemv_grouped_lists", "bitcos_gemv_multi_prefetch",
 ]
 
 
@@ -100,6 +100,7 @@ def load_library():
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.bitcos_decode_probe_variant.argtypes = [C.c_int, vp, vp, sz, vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp]
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
+    L.bitcos_gemv_multi_prefetch.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, C.POINTER(C.c_void_p), C.c_int, vp]
     L.bitcos_gemv_phased.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp]
     L.bitcos_gemv_phases_host.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp, sz, vp, vp, sz, vp]
     L.bitcos_group_pairs_device.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp]
@@ -583,11 +584,25 @@ class MultiJobs:
                                              y.data_ptr(), ws.data_ptr(), ws.numel()) for (W, x, xs, y, ws) in jobs])
 
 
-def bitcos_gemv_multi(jobs):
+class NextWeights:
+    """The `next` argument of bitcos_gemv_multi_prefetch, built once: the matrices some later launch multiplies by."""
+
+    def __init__(self, weights):
+        self.keep = list(weights)
+        self.arr = (C.c_void_p * len(self.keep))(*[C.addressof(W.desc) for W in self.keep])
+
+
+def bitcos_gemv_multi(jobs, next=None):
     """Up to eight (BITCOS_MAX_JOBS) independent BITCOS products in one launch; `jobs` is a MultiJobs or a list of
-    (W, x, x_scale, y, workspace) tuples with a common batch size."""
+    (W, x, x_scale, y, workspace) tuples with a common batch size.  `next` (a NextWeights or a list of DeviceBitcos):
+    matrices a later launch will read, which this launch asks to be brought into L2 (bitcos_gemv_multi_prefetch)."""
     mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
-    _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")
+    if next is None:
+        _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")
+    else:
+        nw = next if isinstance(next, NextWeights) else NextWeights(next)
+        _check(load_library().bitcos_gemv_multi_prefetch(mj.arr, len(mj.arr), mj.batch, nw.arr, len(nw.keep), _stream()),
+               "bitcos_gemv_multi_prefetch")
     return [j[3] for j in mj.keep]
 
 

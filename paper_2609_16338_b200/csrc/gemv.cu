@@ -108,6 +108,16 @@ struct FirstOff {
     int walks;                 // 1: first / count are filled in
 };
 
+// Arrays some LATER launch will read (the packed weights of the next products of a layer): every
+// thread block asks for its 1 / gridDim.x share of each to be brought into L2 once its own first
+// copies are on their way, so that the later launch starts from L2 instead of device memory.
+constexpr int kMaxPrefetch = 28;
+struct PrefetchList {
+    const uint8_t *ptr[kMaxPrefetch];
+    uint32_t bytes[kMaxPrefetch];     // multiples of 16
+    int n;
+};
+
 struct GroupedArgs {
     const bitcos_weights *experts;
     const int32_t *group_expert;
@@ -283,6 +293,11 @@ __device__ __forceinline__ void bulk_copy(uint32_t dst, const void *src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
+}
+// Asks for a range of global memory to be brought into L2 (no destination, nothing to wait for);
+// the address and the size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
@@ -671,6 +686,18 @@ struct OneSegT {
     }
 };
 
+// This block's share of the arrays a later launch will read, requested into L2: entries first,
+// first + step, ...
+__device__ __forceinline__ void prefetch_share(const PrefetchList *pf, int first, int step) {
+    const uint32_t nblk = gridDim.x, bid = blockIdx.x;
+    for (int i = first; i < pf->n; i += step) {
+        const uint32_t total = pf->bytes[i];
+        const uint32_t chunk = ((total / 16u + nblk - 1u) / nblk) * 16u;
+        const uint32_t off = bid * chunk;
+        if (off < total) bulk_prefetch_l2(pf->ptr[i] + off, total - off < chunk ? total - off : chunk);
+    }
+}
+
 // Warp roles: warps 0 .. NW-1 decode one tile per item each; warp NW feeds the stage ring with
 // bulk copies; warp NW+1 adds the decoders' partial sums in a fixed order and writes the
 // outputs (and runs the cross-block protocol).  The roles meet only through mbarriers, every
@@ -679,7 +706,7 @@ struct OneSegT {
 // one's items; the stage ring, the partial-sum slots and their barriers run on across them.
 template <int FMT, int NB, int TPW, typename Segs>
 __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in, uint8_t *smem, int block,
-                                             const FirstOff *fo = nullptr, int fo_index = 0) {
+                                             const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // The problem and the plan of the segment a warp role is working on.  The plain and the grouped
     // launches have one shape and one plan for all their segments.  A phased launch (kHetero) moves
@@ -844,6 +871,12 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         }
         __syncthreads();       // pairs with the barrier the other warps reach after staging the activations
         if (lane == 0 && !have && lut_issued) mbar_wait(bar0 + 8u * kBarLut, 0);      // no copy may outlive the block
+        // The hint for a later launch goes out behind this block's own first copies (as many as the
+        // ring holds): measured, requests issued before them or from another warp gain less.
+        if (pf && lane == 0) {
+            if (have && ok) issue_loop(wk.count < pl.stages ? wk.count : pl.stages);
+            prefetch_share(pf, 0, 1);
+        }
         if (lane != 0 || !have) return;
         if (ok) issue_loop(wk.count);
         while (!Segs::kSingle && ok && src.next(pr, wk)) {
@@ -1508,12 +1541,12 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
 // One problem, this block's share of its items.
 template <int FMT, int NB, bool DEBUG = true, int TPW = 1, bool XG = false, bool XQ = false, bool BL = false>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
-                                            const FirstOff *fo = nullptr, int fo_index = 0) {
+                                            const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr) {
     OneSegT<DEBUG, XG, XQ, BL> one;
     one.pr = &pr;
     one.wk = wk;
     one.used = false;
-    run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index);
+    run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index, pf);
 }
 
 template <int FMT, int NB, int TPW = 1, bool XG = false, bool XQ = false, bool BL = false>
@@ -1533,6 +1566,7 @@ struct MultiArgs {
     Plan pl[kMaxJobs];
     int first_block[kMaxJobs + 1];
     int n;
+    PrefetchList pf;
 };
 
 template <int NB, int TPW = 1, bool XQ = false, bool XG = false>
@@ -1546,7 +1580,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     const Problem pr = ma.pr[j];
     // (the multi launch has no accumulator dump)
     run_problem<kBitcos, NB, false, TPW, XG, XQ>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
-                             b - ma.first_block[j], &fo, b);
+                             b - ma.first_block[j], &fo, b, ma.pf.n ? &ma.pf : nullptr);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -2502,12 +2536,31 @@ namespace {
 // bf16 = true: every job's x holds 16-bit activations (x_scale is not used) and the decoder warps
 // quantise them per group of 128; one or two tokens.
 int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream, bool bf16,
-                      bool group_scales = false) {
+                      bool group_scales = false, const bitcos_weights *const *next = nullptr, int n_next = 0) {
     if (!jobs) return BITCOS_ERR_NULL;
     if (n_jobs < 1 || n_jobs > kMaxJobs) return BITCOS_ERR_SHAPE;
     if (bf16 && batch > 2) return BITCOS_ERR_SHAPE;
+    if (n_next < 0 || n_next * 4 > kMaxPrefetch || (n_next > 0 && !next)) return BITCOS_ERR_SHAPE;
     MultiArgs ma{};
     ma.n = n_jobs;
+    for (int i = 0; i < n_next; ++i) {
+        const bitcos_weights *w = next[i];
+        if (!w || !w->bitmap || !w->signs || !w->tile_off || !w->scales) return BITCOS_ERR_NULL;
+        if (w->M < 1 || w->K < kGroup || w->K % kGroup) return BITCOS_ERR_SHAPE;
+        const uint64_t tiles = static_cast<uint64_t>(padded_rows(w->M) / kRows) * static_cast<uint64_t>(w->K / kGroup);
+        auto add = [&](const void *p, uint64_t bytes) {
+            bytes &= ~static_cast<uint64_t>(15);
+            if (bytes > 0xFFFFFFF0ull) bytes = 0xFFFFFFF0ull;
+            if (!bytes || (reinterpret_cast<uintptr_t>(p) & 15)) return;
+            ma.pf.ptr[ma.pf.n] = static_cast<const uint8_t *>(p);
+            ma.pf.bytes[ma.pf.n++] = static_cast<uint32_t>(bytes);
+        };
+        add(w->bitmap, tiles * 512);
+        add(w->scales, tiles * kRows * sizeof(uint16_t));
+        add(w->tile_off, (tiles + 1) * sizeof(uint32_t));
+        // the length of the sign vector is only known from the host copy of the entry offsets
+        if (w->tile_off_host) add(w->signs, (static_cast<uint64_t>(w->tile_off_host[tiles]) + 31) / 32 * 4);
+    }
     for (int j = 0; j < n_jobs; ++j) {
         bitcos_gemv_job jb = jobs[j];
         if (!jb.W) return BITCOS_ERR_NULL;
@@ -2642,6 +2695,11 @@ int bitcos_gemv_phased(const bitcos_gemv_job *jobs, const int *job_phase, int n_
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (batch == 1) return launch_phased<1>(pa, n_jobs, job_phase, stream);
     return launch_phased<2>(pa, n_jobs, job_phase, stream);
+}
+
+int bitcos_gemv_multi_prefetch(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *next,
+                               int n_next, void *cuda_stream) {
+    return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, false, false, next, n_next);
 }
 
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {

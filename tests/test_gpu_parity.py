@@ -276,6 +276,49 @@ def test_multi_launch_matches_separate_products(bc, B):
         assert torch.equal(y1, y)
 
 
+def test_multi_launch_with_l2_request_for_later_matrices(bc):
+    """bitcos_gemv_multi_prefetch: the launch also asks for other matrices' packed arrays to be brought into
+    L2.  Whatever `next` holds (large, tiny, without the host copy of the entry offsets, the launch's own
+    matrices, seven entries), the results are those of the oracle and of bitcos_gemv_multi bit for bit; a
+    malformed `next` is refused before anything is launched."""
+    shapes = [(2560, 2560), (640, 2560), (96, 6912), (33, 256)]
+    jobs, refs, plain = [], [], []
+    for i, (M, K) in enumerate(shapes):
+        W, S = datagen.trits(650 + i, M, K, 0.4219), datagen.scales(650 + i, M, K)
+        x, xs = datagen.activations(650 + i, 1, K)
+        refs.append(oracle.gemv_dense(W, S, x, xs))
+        y = torch.full((1, M), float("nan"), dtype=torch.float32, device="cuda")
+        jobs.append((bc.bitcos_pack(W, S).to_device(), dev(x), dev(xs), y, bc.make_workspace(M, K)))
+    bc.bitcos_gemv_multi(jobs)
+    torch.cuda.synchronize()
+    plain = [j[3].clone() for j in jobs]
+    later = [bc.bitcos_pack(datagen.trits(660 + i, M, K, 0.4219), datagen.scales(660 + i, M, K)).to_device()
+             for i, (M, K) in enumerate([(6912, 2560), (2560, 6912), (32, 128), (70, 384)])]
+    nexts = [later[:1], later, [w.without_host_offsets() for w in later], [j[0] for j in jobs],
+             (later + later)[:7], []]
+    for n_jobs in (4, 1):
+        for nx in nexts:
+            for j in jobs:
+                j[3].fill_(float("nan"))
+            bc.bitcos_gemv_multi(jobs[:n_jobs], next=nx)
+            for (Wd, _, _, y, ws), (acc_ref, y_ref, mag), y0 in zip(jobs[:n_jobs], refs, plain):
+                check(y, None, acc_ref, y_ref, mag, f"prefetch {len(nx)} later matrices, {Wd.M}x{Wd.K}")
+                assert torch.equal(y, y0)
+                assert bc.workspace_status(ws) == 0
+    # a following product reads what was requested: still the oracle's numbers
+    M, K = 6912, 2560
+    W, S = datagen.trits(660, M, K, 0.4219), datagen.scales(660, M, K)
+    x, xs = datagen.activations(670, 1, K)
+    bc.bitcos_gemv_multi(jobs, next=later[:1])
+    y, acc = bc.bitcos_gemv(later[0], dev(x), dev(xs), acc_debug=True)
+    check(y, acc, *oracle.gemv_dense(W, S, x, xs), "product after the request")
+    with pytest.raises(RuntimeError):
+        bc.bitcos_gemv_multi(jobs, next=(later + later))         # eight entries: more than the launch carries
+    L = bc.load_library()
+    mj = bc.MultiJobs(jobs)
+    assert L.bitcos_gemv_multi_prefetch(mj.arr, len(mj.arr), 1, None, 1, None) != 0
+
+
 def test_host_copy_of_entry_offsets_changes_nothing(bc):
     """With a host copy of tile_off the launch passes each block's first entry offsets by value;
     without it the kernel loads them.  Same results, bit for bit, and both match the oracle."""
