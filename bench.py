@@ -295,6 +295,8 @@ def run_cuda(args):
         return [replicas[(c + g // len(groups)) % copies][j] for j in groups[g % len(groups)]]
     nexts = [[bc.NextWeights([w for d in args.prefetch_depth for w in later(c, gi, d)]) for gi in range(len(groups))]
              for c in range(copies)]
+    # ... and what each launch is told runs directly before it (shapes only)
+    prevs = [bc.NextWeights([base[j] for j in groups[gi - 1]]) for gi in range(len(groups))]
 
     phases = [p for p, g in enumerate(groups) for _ in g]
     order = [j for g in groups for j in g]
@@ -318,7 +320,8 @@ def run_cuda(args):
             return
         if not args.branches:
             for gi, mj in enumerate(multi[i % copies]):
-                bc.bitcos_gemv_multi(mj, next=nexts[i % copies][gi] if args.prefetch and gi in args.prefetch_launches else None)
+                bc.bitcos_gemv_multi(mj, next=nexts[i % copies][gi] if args.prefetch and gi in args.prefetch_launches else None,
+                                     prev=prevs[gi] if args.chain_hint else None)
             return
         cur = torch.cuda.current_stream()
         for sd in sides:
@@ -555,7 +558,7 @@ def run_cuda(args):
                                  "read the same input share a launch)"
                                  + ("; launches " + ",".join(str(g + 1) for g in args.prefetch_launches)
                                     + " of the step also ask for the NEXT launch's packed weights to be brought into L2"
-                                      " (bitcos_gemv_multi_prefetch): every byte still comes from device memory"
+                                      " (bitcos_gemv_multi_chained): every byte still comes from device memory"
                                       " once per step" if args.prefetch and args.launch == "multi" else ""))
                               + "; programmatic dependent launch between consecutive kernels of a stream"),
                    "replicas": world},
@@ -1104,6 +1107,9 @@ def main():
                          "bitcos_gemv_phased launch (phases q|k|v, o, gate|up, down)")
     ap.add_argument("--no-prefetch", dest="prefetch", action="store_false",
                     help="plain bitcos_gemv_multi launches: no launch asks for the next launch's packed weights to be brought into L2")
+    ap.add_argument("--no-chain-hint", dest="chain_hint", action="store_false",
+                    help="launches are not told which launch runs directly before them (no uneven split between "
+                         "thread blocks that start at once and thread blocks that start late)")
     ap.add_argument("--prefetch-launches", type=lambda v: [int(t) for t in v.split(",")], default=[1, 2],
                     help="with --prefetch: which of the step's four launches carry a request")
     ap.add_argument("--prefetch-depth", type=lambda v: [int(t) for t in v.split(",")], default=[1],

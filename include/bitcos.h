@@ -313,19 +313,30 @@ typedef struct bitcos_gemv_job {
     size_t workspace_bytes;
 } bitcos_gemv_job;
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);
-/* bitcos_gemv_multi, which in passing asks for the packed arrays of `next` (host array of n_next
- * pointers to host structs of device pointers, n_next <= 7; may be 0) to be brought into the
- * level-2 cache: the matrices a LATER launch multiplies by (the next products of the layer, the
- * first of the next layer).  Every thread block requests its share of each array once its own first
- * copies are under way; nothing waits for the requests and nothing is written, so results are
- * those of bitcos_gemv_multi whatever `next` holds.  The sign vector of a matrix is only requested
- * if its descriptor carries tile_off_host (its length is not known otherwise).  The paper reads
- * weights from memory as the product reaches them (Section II-D); this hint has no counterpart
- * there.  It pays when the launches of a decode step are short: the later launch then starts from
- * L2 instead of device memory.  Errors as bitcos_gemv_multi, plus BITCOS_ERR_NULL / BITCOS_ERR_SHAPE
- * for a malformed `next`. */
-int bitcos_gemv_multi_prefetch(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *next,
-                               int n_next, void *cuda_stream);
+/* bitcos_gemv_multi for a launch inside a fixed sequence of launches (the products of a decoder
+ * layer, token after token), told what runs directly before it and what comes after it in the
+ * stream.  Both are hints: results are those of bitcos_gemv_multi, bit for bit, whatever they hold.
+ * The paper reads weights from memory as the product reaches them and has one product at a time
+ * (Section II-D); neither hint has a counterpart there.
+ *   next, n_next   matrices a LATER launch multiplies by (host array of pointers to host structs of
+ *                  device pointers, n_next <= 7, may be 0): every thread block asks for its share of
+ *                  their packed arrays to be brought into the level-2 cache once its own first copies
+ *                  are under way.  Nothing waits for the requests and nothing is written.  The sign
+ *                  vector of a matrix is only requested if its descriptor carries tile_off_host (its
+ *                  length is not known otherwise).  Pays when launches are short: the later launch
+ *                  starts from L2 instead of device memory.
+ *   prev, n_prev   the matrices of the launch directly BEFORE this one in the stream (only M and K
+ *                  are read; n_prev <= BITCOS_MAX_JOBS, may be 0 = unknown), same batch.  Kernels of
+ *                  this library start before their predecessor has finished (see "stream ordering"),
+ *                  but only on multiprocessors it has left free; the thread blocks that have to wait
+ *                  for one go through their start-up late and fall about two work items behind.  Knowing
+ *                  how many blocks the previous launch runs, this launch hands the blocks that start at
+ *                  once correspondingly more items.  Only applied when every job's rows fit one work item
+ *                  (K <= 2560 at up to eight tokens), where the split cannot touch any sum.  A wrong
+ *                  hint costs time (an uneven split), never correctness.
+ * Errors as bitcos_gemv_multi, plus BITCOS_ERR_NULL / BITCOS_ERR_SHAPE for a malformed list. */
+int bitcos_gemv_multi_chained(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *prev,
+                              int n_prev, const bitcos_weights *const *next, int n_next, void *cuda_stream);
 /* The same with one activation scale per token and group of 128 (see bitcos_gemv_group_scales):
  * every job's x_scale points to device float [batch][K/128]. */
 int bitcos_gemv_multi_group_scales(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);

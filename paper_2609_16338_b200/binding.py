@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe", "bitcos_group_pairs_device", "bitcos_gemv_grouped_lists", "bitcos_gemv_multi_prefetch",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe", "bitcos_group_pairs_device", "bitcos_gemv_grouped_lists", "bitcos_gemv_multi_chained",
 ]
 
 
@@ -100,7 +100,8 @@ def load_library():
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.bitcos_decode_probe_variant.argtypes = [C.c_int, vp, vp, sz, vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp]
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
-    L.bitcos_gemv_multi_prefetch.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, C.POINTER(C.c_void_p), C.c_int, vp]
+    L.bitcos_gemv_multi_chained.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, C.POINTER(C.c_void_p), C.c_int,
+                                            C.POINTER(C.c_void_p), C.c_int, vp]
     L.bitcos_gemv_phased.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp]
     L.bitcos_gemv_phases_host.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp, sz, vp, vp, sz, vp]
     L.bitcos_group_pairs_device.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp]
@@ -585,24 +586,28 @@ class MultiJobs:
 
 
 class NextWeights:
-    """The `next` argument of bitcos_gemv_multi_prefetch, built once: the matrices some later launch multiplies by."""
+    """A `prev` or `next` argument of bitcos_gemv_multi_chained, built once: the matrices of the launch before,
+    or of a later launch."""
 
     def __init__(self, weights):
         self.keep = list(weights)
         self.arr = (C.c_void_p * len(self.keep))(*[C.addressof(W.desc) for W in self.keep])
 
 
-def bitcos_gemv_multi(jobs, next=None):
+def bitcos_gemv_multi(jobs, next=None, prev=None):
     """Up to eight (BITCOS_MAX_JOBS) independent BITCOS products in one launch; `jobs` is a MultiJobs or a list of
-    (W, x, x_scale, y, workspace) tuples with a common batch size.  `next` (a NextWeights or a list of DeviceBitcos):
-    matrices a later launch will read, which this launch asks to be brought into L2 (bitcos_gemv_multi_prefetch)."""
+    (W, x, x_scale, y, workspace) tuples with a common batch size.  Hints for a launch inside a fixed sequence
+    (bitcos_gemv_multi_chained; each a NextWeights or a list of DeviceBitcos): `next` = matrices a later launch
+    will read, which this launch asks to be brought into L2; `prev` = the matrices of the launch directly before
+    this one in the stream, from which the launch works out how many of its blocks will start late."""
     mj = jobs if isinstance(jobs, MultiJobs) else MultiJobs(jobs)
-    if next is None:
+    if next is None and prev is None:
         _check(load_library().bitcos_gemv_multi(mj.arr, len(mj.arr), mj.batch, _stream()), "bitcos_gemv_multi")
     else:
-        nw = next if isinstance(next, NextWeights) else NextWeights(next)
-        _check(load_library().bitcos_gemv_multi_prefetch(mj.arr, len(mj.arr), mj.batch, nw.arr, len(nw.keep), _stream()),
-               "bitcos_gemv_multi_prefetch")
+        nw = next if isinstance(next, NextWeights) else NextWeights(next or [])
+        pw = prev if isinstance(prev, NextWeights) else NextWeights(prev or [])
+        _check(load_library().bitcos_gemv_multi_chained(mj.arr, len(mj.arr), mj.batch, pw.arr, len(pw.keep), nw.arr,
+                                                        len(nw.keep), _stream()), "bitcos_gemv_multi_chained")
     return [j[3] for j in mj.keep]
 
 

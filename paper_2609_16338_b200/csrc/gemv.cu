@@ -116,7 +116,32 @@ struct PrefetchList {
     const uint8_t *ptr[kMaxPrefetch];
     uint32_t bytes[kMaxPrefetch];     // multiples of 16
     int n;
+#ifdef BITCOS_TIMELINE
+    unsigned long long *tl;           // debug build: 16 time stamps per thread block of this launch
+#endif
 };
+#ifdef BITCOS_TIMELINE
+#define BITCOS_TLP(src, i)                                                                                              \
+    do {                                                                                                                \
+        if constexpr (Segs::kHetero)                                                                                    \
+            if ((src).pa->tl) (src).pa->tl[static_cast<size_t>(blockIdx.x) * 32 + (src).phase * 6 + (i)] = global_timer_ns(); \
+    } while (0)
+#else
+#define BITCOS_TLP(src, i) \
+    do {                   \
+    } while (0)
+#endif
+// Debug build (-DBITCOS_TIMELINE): where a thread block of the multi launch spends its time.
+#ifdef BITCOS_TIMELINE
+#define BITCOS_TL(i, v)                                                                   \
+    do {                                                                                  \
+        if (pf && pf->tl) pf->tl[static_cast<size_t>(blockIdx.x) * 32 + (i)] = (v);      \
+    } while (0)
+#else
+#define BITCOS_TL(i, v) \
+    do {                \
+    } while (0)
+#endif
 
 struct GroupedArgs {
     const bitcos_weights *experts;
@@ -555,7 +580,13 @@ struct GroupView {
 template <int FMT, typename View>
 __device__ __forceinline__ void issue_item(const Problem &pb, const View &pr, const Plan &pl, const ItemRange &r,
                                            const SmemLayout &L, uint8_t *smem, int s, uint32_t *sign_base, uint32_t o_lo,
-                                           uint32_t o_hi, const int (&xrows)[2]) {
+                                           uint32_t o_hi, const int (&xrows)[2], unsigned long long *tl = nullptr) {
+#ifdef BITCOS_TIMELINE
+#define BITCOS_TLI(i) do { if (tl) tl[i] = clock64(); } while (0)
+#else
+#define BITCOS_TLI(i) do { } while (0)
+#endif
+    BITCOS_TLI(21);
     uint8_t *stage = smem + L.stage + static_cast<uint32_t>(s) * L.stage_bytes;
     const uint32_t bar = smem_addr(smem + L.bar) + 8u * static_cast<uint32_t>(s);
     const uint32_t d_payload = smem_addr(stage);
@@ -585,12 +616,18 @@ __device__ __forceinline__ void issue_item(const Problem &pb, const View &pr, co
         // the tiles' entry offsets: the 16-byte aligned slice of tile_off that covers t0 .. t0 + nt
         const uint32_t o_first = static_cast<uint32_t>(r.t0 & 3);
         const uint32_t off_bytes = ((o_first + static_cast<uint32_t>(r.nt) + 1u + 3u) & ~3u) * 4u;
+        BITCOS_TLI(22);
         mbar_expect_tx(bar, bm_bytes + sign_bytes + scale_bytes + off_bytes + x_bytes);
+        BITCOS_TLI(23);
         copy_x();
         bulk_copy(d_scales + L.scale_cap, pr.tile_off(pb) + (r.t0 - o_first), off_bytes, bar);
+        BITCOS_TLI(24);
         bulk_copy(d_payload, reinterpret_cast<const uint8_t *>(pr.payload(pb)) + r.t0 * 512, bm_bytes, bar);
+        BITCOS_TLI(25);
         if (sign_bytes) bulk_copy(d_signs, reinterpret_cast<const uint8_t *>(pr.signs(pb)) + b_lo, sign_bytes, bar);
+        BITCOS_TLI(26);
         bulk_copy(d_scales, g_scales, scale_bytes, bar);
+        BITCOS_TLI(27);
     } else if (FMT == kTrit5) {
         const int64_t WPR = (26 * static_cast<int64_t>(pb.G) + 3) / 4;
         const int64_t w_lo = r.rb0 * WPR + ((26 * r.g0) >> 2);
@@ -708,6 +745,7 @@ template <int FMT, int NB, int TPW, typename Segs>
 __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in, uint8_t *smem, int block,
                                              const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (static_cast<int>(threadIdx.x) == pl_in.NW * 32) BITCOS_TL(16, clock64());
     // The problem and the plan of the segment a warp role is working on.  The plain and the grouped
     // launches have one shape and one plan for all their segments.  A phased launch (kHetero) moves
     // from job to job: only what the shared-memory layout and the barrier counts need -- the widest
@@ -754,6 +792,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
     // It also sets the barriers up, so that the first copies are in flight before anything else
     // happens in the block.
     if (warp == pl.NW) {
+        if (lane == 0) {
+            BITCOS_TL(13, clock64());
+            BITCOS_TL(0, global_timer_ns());
+            BITCOS_TL(17, clock64());
+        }
         // All 33 barrier slots at once, one per lane (slots of unused stages included): slots
         // kBarEmpty .. kBarRedFull + 7 count the decoder warps, the others one arrival.  Every
         // barrier is initialised and fenced before the first asynchronous copy is issued.
@@ -766,6 +809,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the other lanes' barriers, seen by this lane's copies
+        if (lane == 0) BITCOS_TL(14, clock64());
         // The first copies go out before the block-wide barrier below, while the other warps are
         // still fetching the activations.
         // Entry offsets are requested two items before they are needed (r0 = item k, r1 = item
@@ -807,7 +851,12 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
+#ifdef BITCOS_TIMELINE
+                issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows,
+                                (kk == 0 && pf && pf->tl) ? pf->tl + static_cast<size_t>(blockIdx.x) * 32 : nullptr);
+#else
                 issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows);
+#endif
                 r0 = r1; lo0 = lo1; hi0 = hi1;
                 r1 = r2; lo1 = lo2; hi1 = hi2;
                 if (++ps == pl.stages) {
@@ -863,13 +912,17 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             bulk_copy(smem_addr(smem + L.lut), FMT == kBitcos ? g_bitcos_lut.v : g_trit5_lut.v, kLutBytes,
                       bar0 + 8u * kBarLut);
         }
+        if (lane == 0) BITCOS_TL(15, clock64());
         // Only the first item goes out before the block-wide barrier: issuing a bulk copy costs this
         // thread on the order of a hundred nanoseconds, and the other warps wait at that barrier.
         if (lane == 0 && have) {
             prime(true);
+            BITCOS_TL(18, clock64());
             issue_loop(1);
         }
+        if (lane == 0) BITCOS_TL(2, clock64());
         __syncthreads();       // pairs with the barrier the other warps reach after staging the activations
+        if (lane == 0) BITCOS_TL(12, clock64());
         if (lane == 0 && !have && lut_issued) mbar_wait(bar0 + 8u * kBarLut, 0);      // no copy may outlive the block
         // The hint for a later launch goes out behind this block's own first copies (as many as the
         // ring holds): measured, requests issued before them or from another warp gain less.
@@ -957,6 +1010,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         };
         if (kLate) {
             asm volatile("griddepcontrol.wait;" ::: "memory");
+            if (lane == 0) BITCOS_TL(8, clock64());
             if (!Segs::kHetero) fetch_x();
         }
         float run[NB];          // running sum of the current row block over this block's items
@@ -1048,6 +1102,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
                 if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                 return;
             }
+            if (lane == 0) BITCOS_TLP(src, 0);
             fetch_x();
         }
         n_pend = 0;
@@ -1122,9 +1177,14 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         }
         for (int i = 0; i < n_pend; ++i) finish_share<NB, kXG>(pb, pl, xr, pend[i], lane);
         if constexpr (Segs::kHetero) src.signal_done(lane);      // this block's outputs of the phase are written
+        if (lane == 0) BITCOS_TLP(src, 5);
         have = next_segment();
         if (have && !Segs::kHetero) token_rows();
         } while (have);
+        if (lane == 0) {
+            BITCOS_TL(9, clock64());
+            BITCOS_TL(11, global_timer_ns());
+        }
         return;
     }
 
@@ -1144,6 +1204,8 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             return;
         }
     }
+    if (warp == 0 && lane == 0) BITCOS_TL(3, clock64());
+    bool tl_first = true;
     constexpr int RS = red_slots(NB);
     constexpr bool kMma = NB >= kMmaMinBatch;          // contraction on the tensor cores
     constexpr int NH = NB > 8 ? 2 : 1;                 // 8-token halves of the batch
@@ -1241,6 +1303,8 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
             return;
         }
+        if (tl_first && warp == 0 && lane == 0) BITCOS_TL(4, clock64());
+        if (tl_first && warp == 0 && lane == 0) BITCOS_TLP(src, 1);
         const uint4 d = desc[s];
         const int nt = static_cast<int>(d.x & 0xFFu);
         const int slot = kk & rs_mask;
@@ -1414,12 +1478,16 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             if (kEarly && !x_ready) {
                 // first contraction of this warp: the previous kernel must be complete and the
                 // activations in place (the decode above needed neither)
+                if (tl_first && warp == 0 && lane == 0) BITCOS_TL(5, clock64());
+                if (tl_first && warp == 0 && lane == 0) BITCOS_TLP(src, 2);
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 if (!kXQ && !mbar_wait(bar0 + 8u * kBarX, x_parity)) {
                     if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                     return;
                 }
                 x_ready = true;
+                if (tl_first && warp == 0 && lane == 0) BITCOS_TL(6, clock64());
+                if (tl_first && warp == 0 && lane == 0) BITCOS_TLP(src, 3);
             }
             if (kXQ && g != q_g) {
                 // 16-bit activations: this warp quantises the group its tile multiplies (four values
@@ -1512,7 +1580,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         }
         __syncwarp();
         mbar_arrive_lane0(bar0 + 8u * (kBarRedFull + slot), lane);
+        if (tl_first && warp == 0 && lane == 0) BITCOS_TL(7, clock64());
+        tl_first = false;
     }
+    if (warp == 0 && lane == 0) BITCOS_TL(10, clock64());
+    if (warp == 0 && lane == 0) BITCOS_TLP(src, 4);
     if constexpr (Segs::kHetero) {
         // Every decoder warp passes every phase of the activations' barrier, a warp without a tile in
         // this segment included: a warp that skipped one could not tell the phase before from the
@@ -1522,6 +1594,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             return;
         }
         more_segments = next_segment();
+        tl_first = true;
         if (more_segments) {
             x_ready = false;
             x_parity ^= 1u;
@@ -1566,6 +1639,12 @@ struct MultiArgs {
     Plan pl[kMaxJobs];
     int first_block[kMaxJobs + 1];
     int n;
+    // mapped = 1: block b works on job job_of[b] as that job's block number rank[b] of nblk[job]
+    // (the jobs' blocks interleaved); 0: job j owns blocks first_block[j] .. first_block[j + 1] - 1
+    int mapped;
+    int nblk[kMaxJobs];
+    uint8_t job_of[kMaxGrid];
+    uint8_t rank[kMaxGrid];
     PrefetchList pf;
 };
 
@@ -1574,13 +1653,33 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
                                                                               const __grid_constant__ FirstOff fo) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b = static_cast<int>(blockIdx.x);
-    int j = 0;
-    while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
+#ifdef BITCOS_TIMELINE
+    if (threadIdx.x == 0 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 1] = clock64();
+#endif
+    int j = 0, bj, nbj;
+    if (ma.mapped) {
+        j = ma.job_of[b];
+        bj = ma.rank[b];
+        nbj = ma.nblk[j];
+    } else {
+        while (j + 1 < ma.n && b >= ma.first_block[j + 1]) ++j;
+        bj = b - ma.first_block[j];
+        nbj = ma.first_block[j + 1] - ma.first_block[j];
+    }
     const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
     const Problem pr = ma.pr[j];
     // (the multi launch has no accumulator dump)
-    run_problem<kBitcos, NB, false, TPW, XG, XQ>(pr, pl, smem, block_walk(fo, b, pl, b - ma.first_block[j], ma.first_block[j + 1] - ma.first_block[j]),
-                             b - ma.first_block[j], &fo, b, ma.pf.n ? &ma.pf : nullptr);
+#ifdef BITCOS_TIMELINE
+    if (static_cast<int>(threadIdx.x) == pl.NW * 32 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 20] = clock64();
+#endif
+    run_problem<kBitcos, NB, false, TPW, XG, XQ>(pr, pl, smem, block_walk(fo, b, pl, bj, nbj),
+                             bj, &fo, b,
+#ifdef BITCOS_TIMELINE
+                             &ma.pf
+#else
+                             ma.pf.n ? &ma.pf : nullptr
+#endif
+    );
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1605,7 +1704,11 @@ struct PhasedArgs {
     int n_phases;
     unsigned int *sync;                     // device: one arrival counter per phase, zero between launches
     uint8_t job_of[kMaxPhases][kMaxGrid];   // the job a thread block works on in a phase (0xFF: none)
+#ifdef BITCOS_TIMELINE
+    unsigned long long *tl;
+#endif
 };
+
 
 __device__ __forceinline__ unsigned int load_acquire(const unsigned int *p) {
     unsigned int v;
@@ -2039,6 +2142,8 @@ inline int choose_stages(int fmt, const Plan &pl, int G, int nb, int64_t K, int 
 inline int small_launch_cap(int64_t items, int sms) {
     if (items > sms) return sms;
     const int cap = sms * 46 / 100;
+    static const char *env = std::getenv("BITCOS_SMALL_FULL");
+    if ((!env || env[0] != '0') && items <= sms - cap) return static_cast<int>(items);
     return cap < 1 ? 1 : cap;
 }
 
@@ -2143,60 +2248,166 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     return launch_pdl(gemv_kernel<FMT, NB, 1, XG, XQ, BL>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
-template <int NB, bool XQ = false, bool XG = false>
-int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_host) {
-    for (int j = 0; j < ma.n; ++j)
-        if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * ma.pr[j].K > kXResidentBytes) return BITCOS_ERR_SHAPE;
-    int sms = 0, budget = 0;
-    int rc = prepare_kernel<gemv_multi_kernel<NB, 1, XQ, XG>>(&sms, &budget);
-    if (rc) return rc;
-    // share the multiprocessors between the problems in proportion to their item counts
+// Grids of a multi launch: whether it runs two tiles per decoder warp, and each job's plan, walk
+// and number of thread blocks (the multiprocessors shared between the jobs in proportion to their
+// item counts).  Returns the total number of blocks.
+inline int plan_multi(MultiArgs &ma, int nb_template, int sms, bool *two_out, int *grids) {
     int64_t total_items = 0;
     for (int j = 0; j < ma.n; ++j) total_items += ma.pl[j].items;
     // enough items altogether: every problem with two tiles per decoder warp
     Plan all{};
     all.items = total_items;
-    const bool two = wants_two_tiles(all, NB, sms);
-    if constexpr (NB < kMmaMinBatch) {
-        if (two) {
-            rc = prepare_kernel<gemv_multi_kernel<NB, 2, XQ, XG>>(&sms, &budget);
-            if (rc) return rc;
-            total_items = 0;
-            for (int j = 0; j < ma.n; ++j) {
-                ma.pl[j] = make_plan(ma.pr[j].M, ma.pr[j].K, decoder_warps(NB), 2);
-                total_items += ma.pl[j].items;
-            }
+    const bool two = wants_two_tiles(all, nb_template, sms);
+    if (two) {
+        total_items = 0;
+        for (int j = 0; j < ma.n; ++j) {
+            ma.pl[j] = make_plan(ma.pr[j].M, ma.pr[j].K, decoder_warps(nb_template), 2);
+            total_items += ma.pl[j].items;
         }
     }
+    *two_out = two;
     sms = small_launch_cap(total_items, sms);
-    int nw = 0;
-    uint32_t smem = 0;
     int next = 0;
-    FirstOff fo;
-    fo.valid = 1;
-    fo.walks = 1;
-    for (int j = 0; j < ma.n; ++j) fo.valid = (fo.valid && off_host[j]) ? 1 : 0;
     for (int j = 0; j < ma.n; ++j) {
         int64_t cap = ma.pl[j].items;
         if (total_items > sms) {
             cap = ma.pl[j].items * sms / total_items;
             if (cap < 1) cap = 1;
         }
-        int grid = 1;
-        choose_walk(ma.pl[j], static_cast<int>(cap), &grid);
+        choose_walk(ma.pl[j], static_cast<int>(cap), &grids[j]);
+        next += grids[j];
+    }
+    return next;
+}
+
+// A launch whose first `early` thread blocks (of `grid`) find a free multiprocessor at once while
+// the others have to wait for the blocks of the kernel before it to leave: by the time a late
+// block has gone through its start-up, an early one -- which did all of that, first decode
+// included, while it waited for its dependency -- is about kLateLagItems items ahead.  So early
+// blocks take that many items more.  Only for jobs whose items are whole row blocks (nothing is
+// shared between thread blocks, so the split has no influence on any sum).  counts[r] = items of
+// the job's block number r; its early blocks come first.
+constexpr int kLateLagItems = 2;
+inline void skewed_counts(int64_t items, int n_early, int n_late, int *counts) {
+    const int n = n_early + n_late;
+    int64_t a = (items + static_cast<int64_t>(n_late) * kLateLagItems + n - 1) / n;
+    if (a < 1) a = 1;
+    int64_t sum = 0;
+    for (int r = 0; r < n; ++r) {
+        int64_t c = r < n_early ? a : a - kLateLagItems;
+        if (c < 0) c = 0;
+        counts[r] = static_cast<int>(c);
+        sum += c;
+    }
+    // too many by rounding: taken back one at a time, from the last block backwards
+    for (int r = n - 1; sum > items; r = (r == 0 ? n - 1 : r - 1))
+        if (counts[r] > 0) {
+            --counts[r];
+            --sum;
+        }
+    for (int r = 0; sum < items; r = (r + 1) % n) {       // (too few: only when a - lag was cut at zero)
+        ++counts[r];
+        ++sum;
+    }
+}
+
+// busy_sms: multiprocessors the caller expects the kernel before this one in the stream to hold on
+// to when this launch's blocks are scheduled (0: unknown or none).
+template <int NB, bool XQ = false, bool XG = false>
+int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_host, int busy_sms = 0) {
+    for (int j = 0; j < ma.n; ++j)
+        if (NB < kMmaMinBatch && static_cast<int64_t>(NB) * ma.pr[j].K > kXResidentBytes) return BITCOS_ERR_SHAPE;
+    int sms = 0, budget = 0;
+    int rc = prepare_kernel<gemv_multi_kernel<NB, 1, XQ, XG>>(&sms, &budget);
+    if (rc) return rc;
+    bool two = false;
+    int grids[kMaxJobs];
+    const int total = plan_multi(ma, NB, sms, &two, grids);
+    if constexpr (NB < kMmaMinBatch) {
+        if (two) {
+            rc = prepare_kernel<gemv_multi_kernel<NB, 2, XQ, XG>>(&sms, &budget);
+            if (rc) return rc;
+        }
+    }
+    int nw = 0;
+    uint32_t smem = 0;
+    FirstOff fo;
+    fo.valid = 1;
+    fo.walks = 1;
+    for (int j = 0; j < ma.n; ++j) fo.valid = (fo.valid && off_host[j]) ? 1 : 0;
+    for (int j = 0; j < ma.n; ++j) {
         ma.pl[j].stages = choose_stages(kBitcos, ma.pl[j], ma.pr[j].G, NB, ma.pr[j].K, budget);
         const SmemLayout L = smem_layout(kBitcos, ma.pl[j], ma.pr[j].G, NB, ma.pr[j].K);
         if (L.total > smem) smem = L.total;
         if (ma.pl[j].NW > nw) nw = ma.pl[j].NW;
-        ma.first_block[j] = next;
-        fill_first_off(fo, next, fo.valid ? off_host[j] : nullptr, ma.pr[j], ma.pl[j], grid);
-        next += grid;
     }
-    ma.first_block[ma.n] = next;
+    // late starters: only when part of the grid starts early and part late, and every job's items are whole rows
+    int early = sms - busy_sms;
+    bool skew = busy_sms > 0 && early > 0 && early < total && total <= kMaxGrid && !two;
+    for (int j = 0; j < ma.n; ++j) skew = skew && ma.pl[j].CS == 1 && ma.pl[j].items >= grids[j];
+    if (!skew) {
+        int next = 0;
+        for (int j = 0; j < ma.n; ++j) {
+            ma.first_block[j] = next;
+            fill_first_off(fo, next, fo.valid ? off_host[j] : nullptr, ma.pr[j], ma.pl[j], grids[j]);
+            next += grids[j];
+        }
+        ma.first_block[ma.n] = next;
+        ma.mapped = 0;
+    } else {
+        // early blocks are dealt to the jobs in proportion to their grids, job after job, then the late ones
+        int ne[kMaxJobs], given = 0;
+        for (int j = 0; j < ma.n; ++j) {
+            ne[j] = static_cast<int>(static_cast<int64_t>(early) * grids[j] / total);
+            given += ne[j];
+        }
+        for (int j = 0; given < early; j = (j + 1) % ma.n)
+            if (ne[j] < grids[j]) {
+                ++ne[j];
+                ++given;
+            }
+        int b = 0;
+        for (int pass = 0; pass < 2; ++pass)
+            for (int j = 0; j < ma.n; ++j) {
+                const int r0 = pass ? ne[j] : 0, r1 = pass ? grids[j] : ne[j];
+                for (int r = r0; r < r1; ++r, ++b) {
+                    ma.job_of[b] = static_cast<uint8_t>(j);
+                    ma.rank[b] = static_cast<uint8_t>(r);
+                }
+            }
+        // the walks: contiguous ranges of the job's items, early blocks first
+        b = 0;
+        int counts[kMaxJobs][kMaxGrid], firsts[kMaxJobs][kMaxGrid];
+        for (int j = 0; j < ma.n; ++j) {
+            ma.nblk[j] = grids[j];
+            ma.pl[j].cyclic = 0;
+            skewed_counts(ma.pl[j].items, ne[j], grids[j] - ne[j], counts[j]);
+            int first = 0;
+            for (int r = 0; r < grids[j]; ++r) {
+                firsts[j][r] = first;
+                first += counts[j][r];
+            }
+        }
+        for (b = 0; b < total; ++b) {
+            const int j = ma.job_of[b], r = ma.rank[b];
+            fo.first[b] = firsts[j][r];
+            fo.count[b] = counts[j][r];
+            fo.lo[b] = fo.hi[b] = 0;
+            if (fo.valid && fo.count[b] > 0) {
+                ItemIter it;
+                it.init(ma.pl[j], fo.first[b]);
+                const ItemRange ir = item_range(ma.pr[j], ma.pl[j], it.c, it.cs);
+                fo.lo[b] = off_host[j][ir.t0];
+                fo.hi[b] = off_host[j][ir.t0 + ir.nt];
+            }
+        }
+        ma.first_block[ma.n] = total;
+        ma.mapped = 1;
+    }
     if constexpr (NB < kMmaMinBatch) {
-        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ, XG>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
+        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo);
     }
-    return launch_pdl(gemv_multi_kernel<NB, 1, XQ, XG>, dim3(next), (nw + 2) * 32, smem, stream, ma, fo);
+    return launch_pdl(gemv_multi_kernel<NB, 1, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo);
 }
 
 // Which instantiation serves a batch: 1, 2, 4, 8 or 16 tokens.  The one- and two-token paths read
@@ -2535,14 +2746,47 @@ int bitcos_gemv_group_scales(const bitcos_weights *W, const int8_t *x, const flo
 namespace {
 // bf16 = true: every job's x holds 16-bit activations (x_scale is not used) and the decoder warps
 // quantise them per group of 128; one or two tokens.
+#ifdef BITCOS_TIMELINE
+unsigned long long *g_tl_buf = nullptr;
+int g_tl_slots = 0, g_tl_next = 0;
+#endif
+
 int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream, bool bf16,
-                      bool group_scales = false, const bitcos_weights *const *next = nullptr, int n_next = 0) {
+                      bool group_scales = false, const bitcos_weights *const *next = nullptr, int n_next = 0,
+                      const bitcos_weights *const *prev = nullptr, int n_prev = 0) {
     if (!jobs) return BITCOS_ERR_NULL;
     if (n_jobs < 1 || n_jobs > kMaxJobs) return BITCOS_ERR_SHAPE;
     if (bf16 && batch > 2) return BITCOS_ERR_SHAPE;
     if (n_next < 0 || n_next * 4 > kMaxPrefetch || (n_next > 0 && !next)) return BITCOS_ERR_SHAPE;
+    if (n_prev < 0 || n_prev > kMaxJobs || (n_prev > 0 && !prev)) return BITCOS_ERR_SHAPE;
+    // thread blocks of the launch the caller says runs directly before this one (same batch)
+    int busy = 0;
+    if (n_prev > 0) {
+        MultiArgs pm{};
+        pm.n = n_prev;
+        int64_t kprev = 0;
+        for (int i = 0; i < n_prev; ++i) {
+            const bitcos_weights *w = prev[i];
+            if (!w) return BITCOS_ERR_NULL;
+            if (w->M < 1 || w->K < kGroup || w->K % kGroup) return BITCOS_ERR_SHAPE;
+            pm.pl[i] = make_plan(w->M, w->K, decoder_warps(batch));
+            pm.pr[i].M = w->M;
+            pm.pr[i].K = w->K;
+            kprev = w->K > kprev ? w->K : kprev;
+        }
+        int dev = 0, sms = 0;
+        int rc = check_cuda(cudaGetDevice(&dev));
+        if (!rc) rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        if (rc) return rc;
+        bool two = false;
+        int grids[kMaxJobs];
+        busy = plan_multi(pm, nb_bucket(batch, kprev), sms, &two, grids);
+    }
     MultiArgs ma{};
     ma.n = n_jobs;
+#ifdef BITCOS_TIMELINE
+    if (g_tl_buf) ma.pf.tl = g_tl_buf + static_cast<size_t>(g_tl_next++ % g_tl_slots) * kMaxGrid * 32;
+#endif
     for (int i = 0; i < n_next; ++i) {
         const bitcos_weights *w = next[i];
         if (!w || !w->bitmap || !w->signs || !w->tile_off || !w->scales) return BITCOS_ERR_NULL;
@@ -2592,11 +2836,11 @@ int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
         if (batch <= 8) return launch_multi<8, false, true>(ma, stream, off_host);
         return launch_multi<16, false, true>(ma, stream, off_host);
     }
-    if (nbk == 1) return launch_multi<1>(ma, stream, off_host);
-    if (nbk == 2) return launch_multi<2>(ma, stream, off_host);
-    if (batch <= 4) return launch_multi<4>(ma, stream, off_host);
-    if (batch <= 8) return launch_multi<8>(ma, stream, off_host);
-    return launch_multi<16>(ma, stream, off_host);
+    if (nbk == 1) return launch_multi<1>(ma, stream, off_host, busy);
+    if (nbk == 2) return launch_multi<2>(ma, stream, off_host, busy);
+    if (batch <= 4) return launch_multi<4>(ma, stream, off_host, busy);
+    if (batch <= 8) return launch_multi<8>(ma, stream, off_host, busy);
+    return launch_multi<16>(ma, stream, off_host, busy);
 }
 }  // namespace
 
@@ -2680,6 +2924,9 @@ int bitcos_gemv_phased(const bitcos_gemv_job *jobs, const int *job_phase, int n_
     PhasedArgs &pa = pa_storage;
     pa.n_phases = job_phase[n_jobs - 1] + 1;
     pa.sync = static_cast<unsigned int *>(sync);
+#ifdef BITCOS_TIMELINE
+    pa.tl = g_tl_buf ? g_tl_buf + static_cast<size_t>(g_tl_next++ % g_tl_slots) * kMaxGrid * 32 : nullptr;
+#endif
     for (int j = 0; j < n_jobs; ++j) {
         const bitcos_gemv_job &jb = jobs[j];
         if (!jb.W) return BITCOS_ERR_NULL;
@@ -2697,9 +2944,18 @@ int bitcos_gemv_phased(const bitcos_gemv_job *jobs, const int *job_phase, int n_
     return launch_phased<2>(pa, n_jobs, job_phase, stream);
 }
 
-int bitcos_gemv_multi_prefetch(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *next,
-                               int n_next, void *cuda_stream) {
-    return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, false, false, next, n_next);
+#ifdef BITCOS_TIMELINE
+// Debug build only: device buffer of slots x 160 blocks x 16 stamps; every multi launch takes the next slot.
+void bitcos_debug_timeline(unsigned long long *buf, int slots) {
+    g_tl_buf = buf;
+    g_tl_slots = slots;
+    g_tl_next = 0;
+}
+#endif
+
+int bitcos_gemv_multi_chained(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *prev,
+                              int n_prev, const bitcos_weights *const *next, int n_next, void *cuda_stream) {
+    return gemv_multi_common(jobs, n_jobs, batch, cuda_stream, false, false, next, n_next, prev, n_prev);
 }
 
 int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream) {

@@ -277,7 +277,7 @@ def test_multi_launch_matches_separate_products(bc, B):
 
 
 def test_multi_launch_with_l2_request_for_later_matrices(bc):
-    """bitcos_gemv_multi_prefetch: the launch also asks for other matrices' packed arrays to be brought into
+    """bitcos_gemv_multi_chained, `next`: the launch also asks for other matrices' packed arrays to be brought into
     L2.  Whatever `next` holds (large, tiny, without the host copy of the entry offsets, the launch's own
     matrices, seven entries), the results are those of the oracle and of bitcos_gemv_multi bit for bit; a
     malformed `next` is refused before anything is launched."""
@@ -316,7 +316,47 @@ def test_multi_launch_with_l2_request_for_later_matrices(bc):
         bc.bitcos_gemv_multi(jobs, next=(later + later))         # eight entries: more than the launch carries
     L = bc.load_library()
     mj = bc.MultiJobs(jobs)
-    assert L.bitcos_gemv_multi_prefetch(mj.arr, len(mj.arr), 1, None, 1, None) != 0
+    assert L.bitcos_gemv_multi_chained(mj.arr, len(mj.arr), 1, None, 0, None, 1, None) != 0
+    assert L.bitcos_gemv_multi_chained(mj.arr, len(mj.arr), 1, None, 1, None, 0, None) != 0
+
+
+def test_multi_launch_told_what_runs_before_it(bc):
+    """bitcos_gemv_multi_chained, `prev`: the launch hands the blocks it expects to start at once more work items
+    than the ones it expects to start late, and interleaves the jobs' blocks.  Every output still matches the
+    oracle and bitcos_gemv_multi bit for bit: for previous launches of every size (a few blocks, about half the
+    chip -- the case that changes the split --, the whole chip), for jobs whose rows are cut into column blocks
+    (hint not applied) and for jobs with fewer items than blocks."""
+    cases = {
+        "gate+up": [(6912, 2560), (6912, 2560)],
+        "three": [(2560, 2560), (4000, 2560), (1333, 1280)],
+        "cut rows": [(2560, 6912), (2560, 2560)],
+        "small": [(640, 2560), (96, 128)],
+    }
+    prevs = {"few blocks": [(320, 2560)], "half the chip": [(2560, 2560)], "more than half": [(3000, 2560)],
+             "whole chip": [(6912, 2560), (6912, 2560)], "tiny": [(32, 128)]}
+    prev_w = {k: [bc.bitcos_pack(datagen.trits(690 + i, M, K, 0.4219), datagen.scales(690 + i, M, K)).to_device()
+                  for i, (M, K) in enumerate(v)] for k, v in prevs.items()}
+    for name, shapes in cases.items():
+        for B in (1, 2, 5):
+            jobs, refs = [], []
+            for i, (M, K) in enumerate(shapes):
+                W, S = datagen.trits(680 + i, M, K, 0.4219), datagen.scales(680 + i, M, K)
+                x, xs = datagen.activations(680 + i + 10 * B, B, K)
+                refs.append(oracle.gemv_dense(W, S, x, xs))
+                y = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
+                jobs.append((bc.bitcos_pack(W, S).to_device(), dev(x), dev(xs), y, bc.make_workspace(M, K)))
+            bc.bitcos_gemv_multi(jobs)
+            torch.cuda.synchronize()
+            plain = [j[3].clone() for j in jobs]
+            for pname, pw in prev_w.items():
+                for rep in range(2):
+                    for j in jobs:
+                        j[3].fill_(float("nan"))
+                    bc.bitcos_gemv_multi(jobs, prev=pw, next=[jobs[0][0]] if rep else None)
+                    for (Wd, _, _, y, ws), (acc_ref, y_ref, mag), y0 in zip(jobs, refs, plain):
+                        check(y, None, acc_ref, y_ref, mag, f"{name} B={B} after {pname}, {Wd.M}x{Wd.K}")
+                        assert torch.equal(y, y0), f"{name} B={B} after {pname}"
+                        assert bc.workspace_status(ws) == 0
 
 
 def test_host_copy_of_entry_offsets_changes_nothing(bc):
