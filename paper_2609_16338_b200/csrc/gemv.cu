@@ -735,9 +735,9 @@ __device__ __forceinline__ void prefetch_share(const PrefetchList *pf, int first
     }
 }
 
-// Warp roles: warps 0 .. NW-1 decode one tile per item each; warp NW feeds the stage ring with
-// bulk copies; warp NW+1 adds the decoders' partial sums in a fixed order and writes the
-// outputs (and runs the cross-block protocol).  The roles meet only through mbarriers, every
+// Warp roles: warps 0 .. NW-1 decode one tile per item each; warp NW adds the decoders' partial
+// sums in a fixed order and writes the outputs (and runs the cross-block protocol); the block's
+// LAST warp (known without reading a kernel argument) feeds the stage ring with bulk copies.  The roles meet only through mbarriers, every
 // wait is bounded, and there is no block-wide barrier inside the loop.
 // `segs` yields the problems this block works on, one after the other, with its share of each
 // one's items; the stage ring, the partial-sum slots and their barriers run on across them.
@@ -745,7 +745,8 @@ template <int FMT, int NB, int TPW, typename Segs>
 __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in, uint8_t *smem, int block,
                                              const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (static_cast<int>(threadIdx.x) == pl_in.NW * 32) BITCOS_TL(16, clock64());
+    const int prod_warp = static_cast<int>(blockDim.x >> 5) - 1;      // the producer: always the block's last warp
+    if (static_cast<int>(threadIdx.x) == prod_warp * 32) BITCOS_TL(16, clock64());
     // The problem and the plan of the segment a warp role is working on.  The plain and the grouped
     // launches have one shape and one plan for all their segments.  A phased launch (kHetero) moves
     // from job to job: only what the shared-memory layout and the barrier counts need -- the widest
@@ -783,7 +784,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
 
     // A block launched wider than this problem needs (several problems in one launch): the spare
     // warps only take part in the one block-wide barrier.
-    if (warp >= pl.NW + 2) {
+    if (warp > pl.NW && warp < prod_warp) {
         __syncthreads();
         return;
     }
@@ -791,7 +792,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
     // ------------------------------------------------------------------ producer warp
     // It also sets the barriers up, so that the first copies are in flight before anything else
     // happens in the block.
-    if (warp == pl.NW) {
+    if (warp == prod_warp) {
         if (lane == 0) {
             BITCOS_TL(13, clock64());
             BITCOS_TL(0, global_timer_ns());
@@ -806,7 +807,6 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         if (lane == 0) mbar_init(bar0 + 8u * kBarLut, 1);
         if (lane == 1) mbar_init(bar0 + 8u * kBarX, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the other lanes' barriers, seen by this lane's copies
         if (lane == 0) BITCOS_TL(14, clock64());
@@ -834,15 +834,26 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             lo = __ldg(pr.tile_off(pb) + r.t0);
             hi = __ldg(pr.tile_off(pb) + r.t0 + r.nt);
         };
+        auto second_item = [&]() {
+            if (wk.count > 1) {
+                it2.next(pl, wk);
+                r1 = item_range(pb, pl, it2.c, it2.cs);
+                offsets(r1, lo1, hi1);
+            }
+        };
         auto issue_loop = [&](int k_end) {
             for (int k = k0; k < k_end; ++k, ++kk) {
                 const int s = ps;
                 uint32_t lo2 = 0, hi2 = 0;
-                if (k + 2 < wk.count) {
-                    it2.next(pl, wk);
-                    r2 = item_range(pb, pl, it2.c, it2.cs);
-                    offsets(r2, lo2, hi2);
-                }
+                // (the block's very first item goes out before anything is worked out for the items after it)
+                auto look_ahead = [&]() {
+                    if (k + 2 < wk.count) {
+                        it2.next(pl, wk);
+                        r2 = item_range(pb, pl, it2.c, it2.cs);
+                        offsets(r2, lo2, hi2);
+                    }
+                };
+                if (kk != 0) look_ahead();
                 if (kk >= pl.stages) {
                     if (!mbar_wait(bar0 + 8u * (kBarEmpty + s), pphase)) {
                         if (pr.status(pb)) *pr.status(pb) = 1u;
@@ -857,6 +868,10 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
 #else
                 issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows);
 #endif
+                if (kk == 0) {
+                    second_item();
+                    look_ahead();
+                }
                 r0 = r1; lo0 = lo1; hi0 = hi1;
                 r1 = r2; lo1 = lo2; hi1 = hi2;
                 if (++ps == pl.stages) {
@@ -866,7 +881,8 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             }
             k0 = k_end;
         };
-        // first item(s) of a segment: ranges and entry offsets of items 0 and 1
+        // first item(s) of a segment: ranges and entry offsets of items 0 and 1 (the block's first
+        // segment: of item 0 only; item 1 follows once item 0 is on its way)
         auto prime = [&](bool first_segment) {
             k0 = 0;
             it2.init(pl, wk.first);
@@ -880,11 +896,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
                     hi0 = __ldg(pr.tile_off(pb) + r0.t0 + r0.nt);
                 }
             }
-            if (wk.count > 1) {
-                it2.next(pl, wk);
-                r1 = item_range(pb, pl, it2.c, it2.cs);
-                offsets(r1, lo1, hi1);
-            }
+            if (!first_segment) second_item();
             if (pl.x_in_stage) {
                 xrows[0] = pr.xrow(pb) ? __ldg(pr.xrow(pb)) : 0;
                 xrows[1] = pr.nb(pb) > 1 ? (pr.xrow(pb) ? __ldg(pr.xrow(pb) + 1) : 1) : 0;
@@ -981,8 +993,8 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
     if (x_resident && have && !kEarly) {
         int4 *xs = reinterpret_cast<int4 *>(smem + L.x);
         const int per_tok = static_cast<int>(pb.K / 16);
-        const int nthr = (pl.NW + 2) * 32 - 32;              // all warps but the producer
-        const int tid = warp < pl.NW ? threadIdx.x : threadIdx.x - 32;
+        const int nthr = (pl.NW + 1) * 32;                   // the decoder warps and the epilogue warp
+        const int tid = threadIdx.x;
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             if (b < pr.nb(pb)) {
@@ -995,7 +1007,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
     if (!have) return;
 
     // ------------------------------------------------------------------ epilogue warp
-    if (warp == pl.NW + 1) {
+    if (warp == pl.NW) {
         // the segment's activations into shared memory: one bulk copy per token (one or two tokens)
         auto fetch_x = [&]() {
             token_rows();
@@ -1654,7 +1666,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     extern __shared__ __align__(128) uint8_t smem[];
     const int b = static_cast<int>(blockIdx.x);
 #ifdef BITCOS_TIMELINE
-    if (threadIdx.x == 0 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 1] = clock64();
+    if (threadIdx.x == blockDim.x - 32 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 1] = clock64();
 #endif
     int j = 0, bj, nbj;
     if (ma.mapped) {
@@ -1670,7 +1682,7 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     const Problem pr = ma.pr[j];
     // (the multi launch has no accumulator dump)
 #ifdef BITCOS_TIMELINE
-    if (static_cast<int>(threadIdx.x) == pl.NW * 32 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 20] = clock64();
+    if (threadIdx.x == blockDim.x - 32 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 20] = clock64();
 #endif
     run_problem<kBitcos, NB, false, TPW, XG, XQ>(pr, pl, smem, block_walk(fo, b, pl, bj, nbj),
                              bj, &fo, b,
