@@ -131,6 +131,23 @@ struct PrefetchList {
     do {                   \
     } while (0)
 #endif
+// What the producer warp needs to send a thread block's first copies on their way, worked out on
+// the host for every block of a multi launch: with it the block's first tiles and its lookup table
+// are requested a few hundred cycles after the block starts, before any of the block's own address
+// arithmetic (arguments, layout, walk, item ranges), which then runs while the data is in flight.
+struct FirstCopies {
+    const void *src[4];      // entry offsets, bitmap, sign bits, scales of the block's first item
+    uint32_t bytes[4];       // (bytes[2] may be 0: an item without a nonzero weight)
+    uint32_t dst[4];         // byte offsets inside the block's shared memory
+    uint32_t desc[4];        // the item's descriptor for the decoder warps (see issue_item)
+    uint32_t desc_off;       // where it goes
+    uint32_t bar;            // byte offset of the barrier region
+};
+struct FirstCopiesTable {
+    FirstCopies c[kMaxGrid];
+    int valid;
+};
+
 // Debug build (-DBITCOS_TIMELINE): where a thread block of the multi launch spends its time.
 #ifdef BITCOS_TIMELINE
 #define BITCOS_TL(i, v)                                                                   \
@@ -735,6 +752,9 @@ __device__ __forceinline__ void prefetch_share(const PrefetchList *pf, int first
     }
 }
 
+#ifndef BITCOS_TRIGGER_ONE
+#define BITCOS_TRIGGER_ONE 1
+#endif
 // Warp roles: warps 0 .. NW-1 decode one tile per item each; warp NW adds the decoders' partial
 // sums in a fixed order and writes the outputs (and runs the cross-block protocol); the block's
 // LAST warp (known without reading a kernel argument) feeds the stage ring with bulk copies.  The roles meet only through mbarriers, every
@@ -743,7 +763,10 @@ __device__ __forceinline__ void prefetch_share(const PrefetchList *pf, int first
 // one's items; the stage ring, the partial-sum slots and their barriers run on across them.
 template <int FMT, int NB, int TPW, typename Segs>
 __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in, uint8_t *smem, int block,
-                                             const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr) {
+                                             const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr,
+                                             bool first_sent = false) {
+    // first_sent: the caller has already initialised the barriers of stage 0 and of the lookup table
+    // and issued the table's copy and the copies of this block's first item (send_first_copies)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int prod_warp = static_cast<int>(blockDim.x >> 5) - 1;      // the producer: always the block's last warp
     if (static_cast<int>(threadIdx.x) == prod_warp * 32) BITCOS_TL(16, clock64());
@@ -780,7 +803,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
     // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as
     // every block of this one got here; whatever it reads from us it reads after its own
     // griddepcontrol.wait.
+#if BITCOS_TRIGGER_ONE
+    if (warp == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // (once per block is enough)
+#else
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
 
     // A block launched wider than this problem needs (several problems in one launch): the spare
     // warps only take part in the one block-wide barrier.
@@ -803,8 +830,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         // barrier is initialised and fenced before the first asynchronous copy is issued.
         static_assert(kBarFull == 0 && kBarEmpty == 8 && kBarRedFull == 16 && kBarRedEmpty == 24 && kBarLut == 32,
                       "one barrier slot per lane, plus the table's");
-        mbar_init(bar0 + 8u * static_cast<uint32_t>(lane), (lane >= kBarEmpty && lane < kBarRedEmpty) ? pl.NW : 1);
-        if (lane == 0) mbar_init(bar0 + 8u * kBarLut, 1);
+        if (!(first_sent && lane == kBarFull))
+            mbar_init(bar0 + 8u * static_cast<uint32_t>(lane), (lane >= kBarEmpty && lane < kBarRedEmpty) ? pl.NW : 1);
+        if (lane == 0 && !first_sent) mbar_init(bar0 + 8u * kBarLut, 1);
         if (lane == 1) mbar_init(bar0 + 8u * kBarX, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         __syncwarp();
@@ -862,12 +890,14 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
+                if (!(first_sent && kk == 0)) {
 #ifdef BITCOS_TIMELINE
-                issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows,
-                                (kk == 0 && pf && pf->tl) ? pf->tl + static_cast<size_t>(blockIdx.x) * 32 : nullptr);
+                    issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows,
+                                    (kk == 0 && pf && pf->tl) ? pf->tl + static_cast<size_t>(blockIdx.x) * 32 : nullptr);
 #else
-                issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows);
+                    issue_item<FMT>(pb, pr, pl, r0, L, smem, s, sign_base, lo0, hi0, xrows);
 #endif
+                }
                 if (kk == 0) {
                     second_item();
                     look_ahead();
@@ -905,7 +935,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         // A grouped launch reads its routing lists (which may come from the previous kernel in the
         // stream) to find its first item: the table copy, which depends on nothing, goes out before
         // the wait for that kernel.
-        bool lut_issued = false;
+        bool lut_issued = first_sent;
         if constexpr (Segs::kListsLate) {
             if (lane == 0 && FMT != kBit2) {
                 mbar_expect_tx(bar0 + 8u * kBarLut, kLutBytes);
@@ -927,7 +957,9 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         if (lane == 0) BITCOS_TL(15, clock64());
         // Only the first item goes out before the block-wide barrier: issuing a bulk copy costs this
         // thread on the order of a hundred nanoseconds, and the other warps wait at that barrier.
-        if (lane == 0 && have) {
+        // (first item already sent by the kernel's first instructions: its bookkeeping waits until
+        // the other warps have been let through the block-wide barrier)
+        if (lane == 0 && have && !first_sent) {
             prime(true);
             BITCOS_TL(18, clock64());
             issue_loop(1);
@@ -935,7 +967,11 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         if (lane == 0) BITCOS_TL(2, clock64());
         __syncthreads();       // pairs with the barrier the other warps reach after staging the activations
         if (lane == 0) BITCOS_TL(12, clock64());
-        if (lane == 0 && !have && lut_issued) mbar_wait(bar0 + 8u * kBarLut, 0);      // no copy may outlive the block
+        if (lane == 0 && have && first_sent) {
+            prime(true);
+            issue_loop(1);
+        }
+        if (lane == 0 && !have && lut_issued && !first_sent) mbar_wait(bar0 + 8u * kBarLut, 0);      // no copy may outlive the block
         // The hint for a later launch goes out behind this block's own first copies (as many as the
         // ring holds): measured, requests issued before them or from another warp gain less.
         if (pf && lane == 0) {
@@ -1626,12 +1662,13 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
 // One problem, this block's share of its items.
 template <int FMT, int NB, bool DEBUG = true, int TPW = 1, bool XG = false, bool XQ = false, bool BL = false>
 __device__ __forceinline__ void run_problem(const Problem &pr, const Plan &pl, uint8_t *smem, const Walk &wk, int block,
-                                            const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr) {
+                                            const FirstOff *fo = nullptr, int fo_index = 0, const PrefetchList *pf = nullptr,
+                                            bool first_sent = false) {
     OneSegT<DEBUG, XG, XQ, BL> one;
     one.pr = &pr;
     one.wk = wk;
     one.used = false;
-    run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index, pf);
+    run_segments<FMT, NB, TPW>(one, pl, smem, block, fo, fo_index, pf, first_sent);
 }
 
 template <int FMT, int NB, int TPW = 1, bool XG = false, bool XQ = false, bool BL = false>
@@ -1662,9 +1699,29 @@ struct MultiArgs {
 
 template <int NB, int TPW = 1, bool XQ = false, bool XG = false>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma,
-                                                                              const __grid_constant__ FirstOff fo) {
+                                                                              const __grid_constant__ FirstOff fo,
+                                                                              const __grid_constant__ FirstCopiesTable fc) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b = static_cast<int>(blockIdx.x);
+    // The block's first copies, from the host's table: before anything else is read or worked out.
+    const bool first_sent = fc.valid != 0 && fc.c[b].bytes[1] != 0;
+    if (first_sent && threadIdx.x == blockDim.x - 32) {
+        const FirstCopies &c = fc.c[b];
+        const uint32_t base = smem_addr(smem);
+        const uint32_t bar_full = base + c.bar + 8u * kBarFull, bar_lut = base + c.bar + 8u * kBarLut;
+        mbar_init(bar_full, 1);
+        mbar_init(bar_lut, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // (the descriptor before the arrival below, which publishes it to the decoder warps)
+        *reinterpret_cast<uint4 *>(smem + c.desc_off) = make_uint4(c.desc[0], c.desc[1], c.desc[2], c.desc[3]);
+        mbar_expect_tx(bar_full, c.bytes[0] + c.bytes[1] + c.bytes[2] + c.bytes[3]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (i != 2 || c.bytes[2]) bulk_copy(base + c.dst[i], c.src[i], c.bytes[i], bar_full);
+        mbar_expect_tx(bar_lut, kLutBytes);
+        bulk_copy(base, g_bitcos_lut.v, kLutBytes, bar_lut);
+    }
 #ifdef BITCOS_TIMELINE
     if (threadIdx.x == blockDim.x - 32 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 1] = clock64();
 #endif
@@ -1680,18 +1737,19 @@ __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(co
     }
     const Plan pl = ma.pl[j];      // by value: read through the run-time index once, not at every use
     const Problem pr = ma.pr[j];
+    const Walk wk0 = block_walk(fo, b, pl, bj, nbj);
     // (the multi launch has no accumulator dump)
 #ifdef BITCOS_TIMELINE
     if (threadIdx.x == blockDim.x - 32 && ma.pf.tl) ma.pf.tl[static_cast<size_t>(blockIdx.x) * 32 + 20] = clock64();
 #endif
-    run_problem<kBitcos, NB, false, TPW, XG, XQ>(pr, pl, smem, block_walk(fo, b, pl, bj, nbj),
+    run_problem<kBitcos, NB, false, TPW, XG, XQ>(pr, pl, smem, wk0,
                              bj, &fo, b,
 #ifdef BITCOS_TIMELINE
                              &ma.pf
 #else
                              ma.pf.n ? &ma.pf : nullptr
 #endif
-    );
+                             , first_sent);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -2260,6 +2318,36 @@ int launch(const Problem &pr, const Plan &pl_in, cudaStream_t stream, const uint
     return launch_pdl(gemv_kernel<FMT, NB, 1, XG, XQ, BL>, dim3(grid), (pl.NW + 2) * 32, L.total, stream, pr, plw, fo);
 }
 
+// The copies of a thread block's first item, as issue_item<kBitcos> would issue them into stage 0
+// (first = the block's first item, o_lo / o_hi = entry offsets of its first tile and of the tile
+// after its last).
+inline void fill_first_copies(FirstCopies &c, const Problem &pr, const Plan &pl, const SmemLayout &L, int first, uint32_t o_lo,
+                              uint32_t o_hi) {
+    ItemIter it;
+    it.init(pl, first);
+    const ItemRange r = item_range(pr, pl, it.c, it.cs);
+    const uint32_t b_lo = (o_lo >> 7) << 4, b_hi = ((o_hi + 127u) >> 7) << 4;
+    const uint32_t o_first = static_cast<uint32_t>(r.t0 & 3);
+    c.src[0] = pr.tile_off + (r.t0 - o_first);
+    c.bytes[0] = ((o_first + static_cast<uint32_t>(r.nt) + 1u + 3u) & ~3u) * 4u;
+    c.src[1] = reinterpret_cast<const uint8_t *>(pr.payload) + r.t0 * 512;
+    c.bytes[1] = static_cast<uint32_t>(r.nt) * 512u;
+    c.src[2] = reinterpret_cast<const uint8_t *>(pr.signs) + b_lo;
+    c.bytes[2] = b_hi - b_lo;
+    c.src[3] = reinterpret_cast<const uint8_t *>(pr.scales) + r.t0 * 64;
+    c.bytes[3] = static_cast<uint32_t>(r.nt) * 64u;
+    c.dst[1] = L.stage;
+    c.dst[2] = c.dst[1] + L.payload_cap;
+    c.dst[3] = c.dst[2] + L.sign_cap;
+    c.dst[0] = c.dst[3] + L.scale_cap;
+    c.desc[0] = static_cast<uint32_t>(r.nt) | (o_first << 8);
+    c.desc[1] = static_cast<uint32_t>(r.g0);
+    c.desc[2] = static_cast<uint32_t>(r.rb0);
+    c.desc[3] = b_lo * 8u;
+    c.desc_off = L.bar + 384u;
+    c.bar = L.bar;
+}
+
 // Grids of a multi launch: whether it runs two tiles per decoder warp, and each job's plan, walk
 // and number of thread blocks (the multiprocessors shared between the jobs in proportion to their
 // item counts).  Returns the total number of blocks.
@@ -2416,10 +2504,31 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
         ma.first_block[ma.n] = total;
         ma.mapped = 1;
     }
-    if constexpr (NB < kMmaMinBatch) {
-        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo);
+    // every block's first copies, when the entry offsets are known on the host
+    static thread_local FirstCopiesTable fc;
+    static const char *fc_env = std::getenv("BITCOS_FIRST_COPIES");
+    fc.valid = 0;
+    if (fo.valid && fo.walks && total <= kMaxGrid && !(fc_env && fc_env[0] == '0')) {
+        fc.valid = 1;
+        int jb = 0;
+        for (int b = 0; b < total; ++b) {
+            int j;
+            if (ma.mapped) {
+                j = ma.job_of[b];
+            } else {
+                while (jb + 1 < ma.n && b >= ma.first_block[jb + 1]) ++jb;
+                j = jb;
+            }
+            fc.c[b] = FirstCopies{};
+            if (fo.count[b] <= 0) continue;
+            const SmemLayout L = smem_layout(kBitcos, ma.pl[j], ma.pr[j].G, NB, ma.pr[j].K);
+            fill_first_copies(fc.c[b], ma.pr[j], ma.pl[j], L, fo.first[b], fo.lo[b], fo.hi[b]);
+        }
     }
-    return launch_pdl(gemv_multi_kernel<NB, 1, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo);
+    if constexpr (NB < kMmaMinBatch) {
+        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo, fc);
+    }
+    return launch_pdl(gemv_multi_kernel<NB, 1, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo, fc);
 }
 
 // Which instantiation serves a batch: 1, 2, 4, 8 or 16 tokens.  The one- and two-token paths read
