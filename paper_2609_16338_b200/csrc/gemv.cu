@@ -34,7 +34,11 @@
 
 #include <cstdint>
 #include <cstdlib>
+#include <algorithm>
+#include <cstring>
 #include <mutex>
+#include <utility>
+#include <vector>
 
 namespace {
 
@@ -2251,6 +2255,16 @@ int launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cu
     return check_cuda(cudaLaunchKernelEx(&cfg, kernel, args...));
 }
 
+// While a launch sequence is being recorded for replay (bitcos_gemv_phases_host), every value a
+// plan takes from a host copy of tile_off is noted here, so that a replay can make sure that the
+// values it was built from are still there.
+thread_local std::vector<std::pair<const uint32_t *, uint32_t>> *g_offset_log = nullptr;
+inline uint32_t host_offset(const uint32_t *off_host, int64_t i) {
+    const uint32_t v = off_host[i];
+    if (g_offset_log) g_offset_log->emplace_back(off_host + i, v);
+    return v;
+}
+
 // Fills fo.lo / fo.hi [base .. base + grid) from a host copy of tile_off: the sign-vector range of
 // the first item of each of the `grid` thread blocks that share the problem.
 void fill_first_off(FirstOff &fo, int base, const uint32_t *off_host, const Problem &pr, const Plan &pl, int grid) {
@@ -2273,8 +2287,8 @@ void fill_first_off(FirstOff &fo, int base, const uint32_t *off_host, const Prob
         ItemIter it;
         it.init(pl, wk.first);
         const ItemRange r = item_range(pr, pl, it.c, it.cs);
-        fo.lo[base + b] = off_host[r.t0];
-        fo.hi[base + b] = off_host[r.t0 + r.nt];
+        fo.lo[base + b] = host_offset(off_host, r.t0);
+        fo.hi[base + b] = host_offset(off_host, r.t0 + r.nt);
     }
 }
 
@@ -2497,8 +2511,8 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
                 ItemIter it;
                 it.init(ma.pl[j], fo.first[b]);
                 const ItemRange ir = item_range(ma.pr[j], ma.pl[j], it.c, it.cs);
-                fo.lo[b] = off_host[j][ir.t0];
-                fo.hi[b] = off_host[j][ir.t0 + ir.nt];
+                fo.lo[b] = host_offset(off_host[j], ir.t0);
+                fo.hi[b] = host_offset(off_host[j], ir.t0 + ir.nt);
             }
         }
         ma.first_block[ma.n] = total;
@@ -2924,7 +2938,8 @@ int gemv_multi_common(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
         add(w->scales, tiles * kRows * sizeof(uint16_t));
         add(w->tile_off, (tiles + 1) * sizeof(uint32_t));
         // the length of the sign vector is only known from the host copy of the entry offsets
-        if (w->tile_off_host) add(w->signs, (static_cast<uint64_t>(w->tile_off_host[tiles]) + 31) / 32 * 4);
+        if (w->tile_off_host)
+            add(w->signs, (static_cast<uint64_t>(host_offset(w->tile_off_host, static_cast<int64_t>(tiles))) + 31) / 32 * 4);
     }
     for (int j = 0; j < n_jobs; ++j) {
         bitcos_gemv_job jb = jobs[j];
@@ -3199,6 +3214,175 @@ int bitcos_gemv_multi_host(const bitcos_gemv_host_job *jobs, int n_jobs, int bat
     return check_cuda(cudaStreamSynchronize(stream));
 }
 
+}  // extern "C"
+
+namespace {
+// The work of bitcos_gemv_phases_host on a stream: copy in, one launch per phase (each told which
+// launch runs before it and which comes after it), copy out.
+int host_step_enqueue(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, const void *in_host,
+                      void *in_device, size_t in_bytes, void *out_host, const void *out_device, size_t out_bytes,
+                      cudaStream_t stream) {
+    int rc = check_cuda(cudaMemcpyAsync(in_device, in_host, in_bytes, cudaMemcpyHostToDevice, stream));
+    if (rc) return rc;
+    const bitcos_weights *w[kMaxJobs];
+    for (int j = 0; j < n_jobs; ++j) w[j] = jobs[j].W;
+    int prev_first = 0, prev_n = 0;
+    for (int first = 0; first < n_jobs;) {
+        int last = first;
+        while (last + 1 < n_jobs && job_phase[last + 1] == job_phase[first]) ++last;
+        int next_n = 0;
+        while (last + 1 + next_n < n_jobs && job_phase[last + 1 + next_n] == job_phase[last + 1] && next_n < kMaxPrefetch / 4) ++next_n;
+        rc = bitcos_gemv_multi_chained(jobs + first, last - first + 1, batch, w + prev_first, prev_n, w + last + 1, next_n, stream);
+        if (rc) return rc;
+        prev_first = first;
+        prev_n = last - first + 1;
+        first = last + 1;
+    }
+    return check_cuda(cudaMemcpyAsync(out_host, out_device, out_bytes, cudaMemcpyDeviceToHost, stream));
+}
+
+// Recorded steps.  A record is keyed by everything the enqueued work depends on, by value: the job
+// list, the descriptors behind it, the blocks and their sizes, the device; and it remembers every
+// entry offset its plans took from the host copies of tile_off, which a replay compares with what
+// is there now (packed arrays in device memory may change freely between calls: the kernels read
+// them when they run).  Anything that does not match is simply enqueued directly.
+struct alignas(8) HostStepKey {
+    int n_jobs, batch, device, pad;
+    int phase[kMaxJobs];
+    bitcos_gemv_job jobs[kMaxJobs];
+    bitcos_weights w[kMaxJobs];
+    const void *in_host, *out_device;
+    void *in_device, *out_host;
+    size_t in_bytes, out_bytes;
+};
+struct HostStepRecord {
+    HostStepKey key;
+    uint64_t hash = 0;
+    std::vector<std::pair<const uint32_t *, uint32_t>> offsets;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    uint64_t last_use = 0;
+    int seen = 0;          // calls with this key so far
+    bool failed = false;   // recording did not work for this key: never tried again
+};
+constexpr int kHostStepRecords = 64;
+HostStepRecord g_host_steps[kHostStepRecords];
+std::mutex g_host_steps_lock;
+uint64_t g_host_steps_clock = 0;
+cudaStream_t g_record_stream = nullptr;
+
+void host_step_key(HostStepKey &k, const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, const void *in_host,
+                   void *in_device, size_t in_bytes, void *out_host, const void *out_device, size_t out_bytes) {
+    std::memset(&k, 0, sizeof(k));
+    k.n_jobs = n_jobs;
+    k.batch = batch;
+    cudaGetDevice(&k.device);
+    for (int j = 0; j < n_jobs; ++j) {
+        k.phase[j] = job_phase[j];
+        std::memcpy(&k.jobs[j], &jobs[j], sizeof(bitcos_gemv_job));
+        std::memcpy(&k.w[j], jobs[j].W, sizeof(bitcos_weights));
+    }
+    k.in_host = in_host;
+    k.in_device = in_device;
+    k.in_bytes = in_bytes;
+    k.out_host = out_host;
+    k.out_device = out_device;
+    k.out_bytes = out_bytes;
+}
+
+// true: the step was launched on `stream` as a recorded graph.  false: the caller enqueues it directly
+// (first sight of these arguments, a stale record, or recording is not possible).
+bool host_step_replay(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, const void *in_host,
+                      void *in_device, size_t in_bytes, void *out_host, const void *out_device, size_t out_bytes,
+                      cudaStream_t stream) {
+    static const char *env = std::getenv("BITCOS_HOST_GRAPH");
+    if (env && env[0] == '0') return false;
+    static thread_local HostStepKey key;
+    host_step_key(key, jobs, job_phase, n_jobs, batch, in_host, in_device, in_bytes, out_host, out_device, out_bytes);
+    uint64_t hash = 1469598103934665603ull;      // (FNV-1a over the key's words: only to skip most comparisons)
+    {
+        const uint64_t *kw = reinterpret_cast<const uint64_t *>(&key);
+        for (size_t i = 0; i < sizeof(key) / 8; ++i) hash = (hash ^ kw[i]) * 1099511628211ull;
+    }
+    std::lock_guard<std::mutex> guard(g_host_steps_lock);
+    HostStepRecord *rec = nullptr, *oldest = &g_host_steps[0];
+    for (HostStepRecord &r : g_host_steps) {
+        if (r.seen && r.hash == hash && std::memcmp(&r.key, &key, sizeof(key)) == 0) rec = &r;
+        if (r.last_use < oldest->last_use) oldest = &r;
+    }
+    if (!rec) {
+        // first sight: remember the arguments (in the least recently used slot), enqueue directly this time
+        rec = oldest;
+        if (rec->exec) cudaGraphExecDestroy(rec->exec);
+        if (rec->graph) cudaGraphDestroy(rec->graph);
+        rec->exec = nullptr;
+        rec->graph = nullptr;
+        rec->offsets.clear();
+        rec->key = key;
+        rec->hash = hash;
+        rec->seen = 1;
+        rec->failed = false;
+        rec->last_use = ++g_host_steps_clock;
+        return false;
+    }
+    rec->last_use = ++g_host_steps_clock;
+    if (rec->failed) return false;
+    if (rec->exec) {
+        for (const auto &o : rec->offsets)
+            if (*o.first != o.second) {        // the host copy of the entry offsets changed under the same descriptor
+                cudaGraphExecDestroy(rec->exec);
+                cudaGraphDestroy(rec->graph);
+                rec->exec = nullptr;
+                rec->graph = nullptr;
+                rec->offsets.clear();
+                rec->seen = 1;
+                return false;
+            }
+        return cudaGraphLaunch(rec->exec, stream) == cudaSuccess;
+    }
+    // second sight: record the step on a stream of the library's own (nothing runs), then replay it
+    ++rec->seen;
+    cudaPointerAttributes ai{}, ao{};
+    if (cudaPointerGetAttributes(&ai, in_host) != cudaSuccess || cudaPointerGetAttributes(&ao, out_host) != cudaSuccess ||
+        ai.type != cudaMemoryTypeHost || ao.type != cudaMemoryTypeHost) {
+        cudaGetLastError();
+        rec->failed = true;       // pageable host blocks: their copies are not recorded
+        return false;
+    }
+    if (!g_record_stream && cudaStreamCreateWithFlags(&g_record_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        cudaGetLastError();
+        rec->failed = true;
+        return false;
+    }
+    if (cudaStreamBeginCapture(g_record_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        rec->failed = true;
+        return false;
+    }
+    g_offset_log = &rec->offsets;
+    const int rc = host_step_enqueue(jobs, job_phase, n_jobs, batch, in_host, in_device, in_bytes, out_host, out_device, out_bytes,
+                                     g_record_stream);
+    g_offset_log = nullptr;
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(g_record_stream, &graph);
+    if (rc || ce != cudaSuccess || !graph || cudaGraphInstantiate(&rec->exec, graph, 0) != cudaSuccess) {
+        cudaGetLastError();
+        if (graph) cudaGraphDestroy(graph);
+        rec->exec = nullptr;
+        rec->offsets.clear();
+        rec->failed = true;
+        return false;
+    }
+    rec->graph = graph;
+    // (neighbouring blocks share entry offsets: every address once)
+    std::sort(rec->offsets.begin(), rec->offsets.end());
+    rec->offsets.erase(std::unique(rec->offsets.begin(), rec->offsets.end()), rec->offsets.end());
+    return cudaGraphLaunch(rec->exec, stream) == cudaSuccess;
+}
+}  // namespace
+
+extern "C" {
+
 int bitcos_gemv_phases_host(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, const void *in_host,
                             void *in_device, size_t in_bytes, void *out_host, const void *out_device, size_t out_bytes,
                             void *cuda_stream) {
@@ -3218,16 +3402,12 @@ int bitcos_gemv_phases_host(const bitcos_gemv_job *jobs, const int *job_phase, i
         if (y < out0 || y + yb > out0 + out_bytes) return BITCOS_ERR_CAPACITY;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    int rc = check_cuda(cudaMemcpyAsync(in_device, in_host, in_bytes, cudaMemcpyHostToDevice, stream));
-    if (rc) return rc;
-    for (int first = 0; first < n_jobs;) {
-        int last = first;
-        while (last + 1 < n_jobs && job_phase[last + 1] == job_phase[first]) ++last;
-        rc = bitcos_gemv_multi(jobs + first, last - first + 1, batch, cuda_stream);
-        if (rc) return rc;
-        first = last + 1;
-    }
-    rc = check_cuda(cudaMemcpyAsync(out_host, out_device, out_bytes, cudaMemcpyDeviceToHost, stream));
+    // A step that was seen before, argument for argument, is replayed as one CUDA graph (one call
+    // into the driver instead of six); the first time round the work is enqueued directly.
+    if (host_step_replay(jobs, job_phase, n_jobs, batch, in_host, in_device, in_bytes, out_host, out_device, out_bytes, stream))
+        return check_cuda(cudaStreamSynchronize(stream));
+    const int rc = host_step_enqueue(jobs, job_phase, n_jobs, batch, in_host, in_device, in_bytes, out_host, out_device,
+                                     out_bytes, stream);
     if (rc) return rc;
     return check_cuda(cudaStreamSynchronize(stream));
 }

@@ -125,7 +125,8 @@ def test_phases_from_host_buffers_in_one_call(bc):
         W, S = datagen.trits(4300 + i, M, K, 0.4219), datagen.scales(4300 + i, M, K)
         mats.append((W, S, bc.bitcos_pack(W, S).to_device(), bc.make_workspace(M, K)))
     hp = bc.HostPhases([(m[2], m[3]) for m in mats], LAYER_PHASES, batch=B)
-    for rep in range(2):
+    # (the first call enqueues the step directly, the second records it, from the third on it is replayed)
+    for rep in range(5):
         refs = []
         for i, (W, S, Wd, ws) in enumerate(mats):
             x, xs = datagen.activations(4300 + 10 * rep + i, B, Wd.K)
@@ -138,3 +139,45 @@ def test_phases_from_host_buffers_in_one_call(bc):
             y_dev, _ = bc.bitcos_gemv(mats[i][2], dev(hp.x[i].copy()), dev(hp.x_scale[i].copy()), workspace=mats[i][3])
             torch.cuda.synchronize()
             assert np.array_equal(y_dev.cpu().numpy(), ys[i])
+
+
+def test_recorded_host_step_follows_weights_repacked_in_place(bc):
+    """A step seen before is replayed as a recorded graph.  The record holds entry offsets taken from the
+    host copy of tile_off; when different weights are packed into the SAME buffers (same descriptor, new
+    offsets), the next call must notice and still return the new product."""
+    B = 1
+    shapes = [(640, 2560), (320, 1280)]
+    Wh = [datagen.trits(4400 + i, M, K, 0.4219) for i, (M, K) in enumerate(shapes)]
+    Sh = [datagen.scales(4400 + i, M, K) for i, (M, K) in enumerate(shapes)]
+    packs = [bc.bitcos_pack(W, S) for W, S in zip(Wh, Sh)]
+    devs = [p.to_device() for p in packs]
+    hp = bc.HostPhases([(d, bc.make_workspace(M, K)) for d, (M, K) in zip(devs, shapes)], [0, 1], batch=B)
+
+    def check(tag):
+        for rep in range(4):
+            refs = []
+            for i, (M, K) in enumerate(shapes):
+                x, xs = datagen.activations(4400 + 7 * rep + i, B, K)
+                hp.x[i][:] = x
+                hp.x_scale[i][:] = xs
+                refs.append(oracle.gemv_dense(Wh[i], Sh[i], x, xs))
+            ys = hp.run()
+            for i, (acc_ref, y_ref, mag) in enumerate(refs):
+                assert (np.abs(ys[i].astype(np.float64) - y_ref) <= REL * mag).all(), (tag, rep, i)
+
+    check("first weights")
+    # new weights of another density into the same device arrays and the same host copy of the entry offsets
+    for i, (M, K) in enumerate(shapes):
+        Wh[i] = datagen.trits(4500 + i, M, K, 0.6)
+        Sh[i] = datagen.scales(4500 + i, M, K)
+        p2 = bc.bitcos_pack(Wh[i], Sh[i])
+        d = devs[i]
+        assert p2.signs.size <= d.signs.numel()          # fewer nonzero weights than before: the sign vector fits
+        off = p2.tile_off_buf if p2.tile_off_buf is not None else p2.tile_off
+        d.bitmap.copy_(torch.from_numpy(p2.bitmap.view(np.int32)))
+        d.signs[:p2.signs.size].copy_(torch.from_numpy(p2.signs.view(np.int32)))
+        d.tile_off[:off.size].copy_(torch.from_numpy(off.view(np.int32)))
+        d.scales.copy_(torch.from_numpy(p2.scales.view(np.int16)))
+        d.tile_off_host[:] = p2.tile_off
+    torch.cuda.synchronize()
+    check("weights repacked in place")
