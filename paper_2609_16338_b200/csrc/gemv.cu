@@ -37,6 +37,7 @@
 #include <algorithm>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 #include <utility>
 #include <vector>
 
@@ -150,6 +151,20 @@ struct FirstCopies {
 struct FirstCopiesTable {
     FirstCopies c[kMaxGrid];
     int valid;
+};
+// (the table is 14 KB of kernel arguments: free when the launch is recorded into a CUDA graph, whose
+// arguments are staged once, but about 4 us of launch latency on a plain stream launch, which therefore
+// goes without it)
+struct NoFirstCopies {
+    int valid;
+};
+template <typename T>
+struct first_copy {
+    __device__ static bool sent(const T &, int) { return false; }
+};
+template <>
+struct first_copy<FirstCopiesTable> {
+    __device__ static bool sent(const FirstCopiesTable &t, int b) { return t.valid != 0 && t.c[b].bytes[1] != 0; }
 };
 
 // Debug build (-DBITCOS_TIMELINE): where a thread block of the multi launch spends its time.
@@ -1701,14 +1716,15 @@ struct MultiArgs {
     PrefetchList pf;
 };
 
-template <int NB, int TPW = 1, bool XQ = false, bool XG = false>
+template <int NB, int TPW = 1, bool XQ = false, bool XG = false, typename FC = NoFirstCopies>
 __global__ void __launch_bounds__(max_block_threads(NB), 1) gemv_multi_kernel(const __grid_constant__ MultiArgs ma,
                                                                               const __grid_constant__ FirstOff fo,
-                                                                              const __grid_constant__ FirstCopiesTable fc) {
+                                                                              const __grid_constant__ FC fc) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b = static_cast<int>(blockIdx.x);
     // The block's first copies, from the host's table: before anything else is read or worked out.
-    const bool first_sent = fc.valid != 0 && fc.c[b].bytes[1] != 0;
+    const bool first_sent = first_copy<FC>::sent(fc, b);
+    if constexpr (std::is_same<FC, FirstCopiesTable>::value)
     if (first_sent && threadIdx.x == blockDim.x - 32) {
         const FirstCopies &c = fc.c[b];
         const uint32_t base = smem_addr(smem);
@@ -2434,6 +2450,11 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     int sms = 0, budget = 0;
     int rc = prepare_kernel<gemv_multi_kernel<NB, 1, XQ, XG>>(&sms, &budget);
     if (rc) return rc;
+    if constexpr (!XQ && !XG && NB <= 2) {
+        // (the variant that is only launched while a graph is being recorded is set up here, on whichever call comes first)
+        rc = prepare_kernel<gemv_multi_kernel<NB, 1, false, false, FirstCopiesTable>>(&sms, &budget);
+        if (rc) return rc;
+    }
     bool two = false;
     int grids[kMaxJobs];
     const int total = plan_multi(ma, NB, sms, &two, grids);
@@ -2520,9 +2541,16 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
     }
     // every block's first copies, when the entry offsets are known on the host
     static thread_local FirstCopiesTable fc;
-    static const char *fc_env = std::getenv("BITCOS_FIRST_COPIES");
+    static const char *fc_env = std::getenv("BITCOS_FIRST_COPIES");      // 0: never, 1: also on plain stream launches (A/B runs)
     fc.valid = 0;
-    if (fo.valid && fo.walks && total <= kMaxGrid && !(fc_env && fc_env[0] == '0')) {
+    bool recording = false;
+    {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cs) == cudaSuccess) recording = cs == cudaStreamCaptureStatusActive;
+        else cudaGetLastError();
+    }
+    const bool with_table = !XQ && !XG && NB <= 2 && !two && (recording || (fc_env && fc_env[0] == '1')) && !(fc_env && fc_env[0] == '0');
+    if (with_table && fo.valid && fo.walks && total <= kMaxGrid) {
         fc.valid = 1;
         int jb = 0;
         for (int b = 0; b < total; ++b) {
@@ -2539,10 +2567,16 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
             fill_first_copies(fc.c[b], ma.pr[j], ma.pl[j], L, fo.first[b], fo.lo[b], fo.hi[b]);
         }
     }
-    if constexpr (NB < kMmaMinBatch) {
-        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo, fc);
+    if constexpr (!XQ && !XG && NB <= 2) {
+        if (fc.valid) {
+            return launch_pdl(gemv_multi_kernel<NB, 1, false, false, FirstCopiesTable>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo, fc);
+        }
     }
-    return launch_pdl(gemv_multi_kernel<NB, 1, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo, fc);
+    const NoFirstCopies none{0};
+    if constexpr (NB < kMmaMinBatch) {
+        if (two) return launch_pdl(gemv_multi_kernel<NB, 2, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo, none);
+    }
+    return launch_pdl(gemv_multi_kernel<NB, 1, XQ, XG>, dim3(total), (nw + 2) * 32, smem, stream, ma, fo, none);
 }
 
 // Which instantiation serves a batch: 1, 2, 4, 8 or 16 tokens.  The one- and two-token paths read

@@ -112,4 +112,6 @@ def test_roofline_traffic_comes_from_the_committed_ncu_summary():
     m = re.search(r"\*\*step\*\*.*?\*\*([\d ]+)\*\* \| \*\*([\d ]+)\*\*", text)
     assert m, "the summary's table has no step row"
     assert int(m.group(1).replace(" ", "")) == step
-    assert 1.0 <= step / int(m.group(2).replace(" ", "")) < 1.2        # traffic against algorithmic bytes
+    # traffic against algorithmic bytes: a little below 1 when the activations, outputs and the lookup table
+    # (part of the algorithmic figure) are served from L2, above 1 if anything were fetched twice
+    assert 0.97 <= step / int(m.group(2).replace(" ", "")) < 1.2
