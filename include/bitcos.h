@@ -439,9 +439,18 @@ int bitcos_gemv_multi_host(const bitcos_gemv_host_job *jobs, int n_jobs, int bat
  * job's x and x_scale out inside one device block `in_device` (and the same bytes, at the same
  * offsets, inside the host block `in_host`), and every job's y inside one device block
  * `out_device`; jobs[] holds the DEVICE addresses, as for bitcos_gemv_multi.  The call copies
- * in_host -> in_device (in_bytes), runs one bitcos_gemv_multi launch per phase (job_phase as for
- * bitcos_gemv_phased), copies out_device -> out_host (out_bytes) and waits for the stream, so
- * out_host is valid on return.  Pinned host blocks keep the two copies asynchronous until the wait.
+ * in_host -> in_device (in_bytes), runs one launch per phase (job_phase as for bitcos_gemv_phased;
+ * each launch is told its neighbours as by bitcos_gemv_multi_chained), copies out_device ->
+ * out_host (out_bytes) and waits for the stream, so out_host is valid on return.  Pinned host
+ * blocks keep the two copies asynchronous until the wait.
+ * Replay: the second call with the same arguments (every pointer, size and descriptor field
+ * compared by value) records the step as a CUDA graph on a stream of the library's own; that call and
+ * the following ones launch the graph on `cuda_stream` (one driver call instead of six).  The record
+ * holds the entry offsets its launch plans read from the descriptors' tile_off_host; every replay
+ * compares them with the host arrays' current contents and falls back to enqueueing directly if
+ * they differ, so matrices re-packed into the same buffers are handled; the packed arrays in device
+ * memory are read when the kernels run and may change freely.  Up to 64 argument sets are kept
+ * (least recently used replaced).  Pageable host blocks are never recorded.  Thread safe.
  * ERR_CAPACITY if a job's x, x_scale or y lies outside its block.  The paper has no counterpart (it
  * measures resident activations). */
 int bitcos_gemv_phases_host(const bitcos_gemv_job *jobs, const int *job_phase, int n_jobs, int batch, const void *in_host,
