@@ -359,6 +359,54 @@ def test_multi_launch_told_what_runs_before_it(bc):
                         assert bc.workspace_status(ws) == 0
 
 
+@pytest.mark.parametrize("B", [1, 2, 3])
+def test_multi_launch_recorded_into_a_graph(bc, B):
+    """Recorded into a CUDA graph, a multi launch of one or two tokens carries a host-made table of every
+    block's first copies, which the kernel issues with its first instructions (a plain stream launch goes
+    without it).  Replayed, the outputs are those of the oracle and of the plain launch bit for bit: layer
+    shapes, ragged row counts, rows cut into column blocks, a job with a single tile, jobs with and
+    without the host copy of the entry offsets, with and without the sequence hints, several replays."""
+    sets = {
+        "gate+up": [(6912, 2560), (6912, 2560)],
+        "q+k+v": [(2560, 2560), (640, 2560), (640, 2560)],
+        "down": [(2560, 6912)],
+        "ragged": [(1000, 512), (33, 2560), (32, 128), (70, 384)],
+        "two tiles per warp": [(25600, 2560), (12000, 2560)],
+    }
+    side = torch.cuda.Stream()
+    for name, shapes in sets.items():
+        jobs, refs = [], []
+        for i, (M, K) in enumerate(shapes):
+            W, S = datagen.trits(720 + i, M, K, 0.4219), datagen.scales(720 + i, M, K)
+            x, xs = datagen.activations(720 + i + 10 * B, B, K)
+            refs.append(oracle.gemv_dense(W, S, x, xs))
+            y = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
+            Wd = bc.bitcos_pack(W, S).to_device()
+            jobs.append((Wd, dev(x), dev(xs), y, bc.make_workspace(M, K)))
+        bc.bitcos_gemv_multi(jobs)
+        torch.cuda.synchronize()
+        plain = [j[3].clone() for j in jobs]
+        variants = [("no hints", jobs, None, None), ("hints", jobs, [jobs[0][0]], [jobs[-1][0]])]
+        if name == "ragged":
+            mixed = [(j[0].without_host_offsets() if i == 1 else j[0],) + j[1:] for i, j in enumerate(jobs)]
+            variants.append(("one job without host offsets", mixed, None, None))
+        for tag, js, prev, nxt in variants:
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    bc.bitcos_gemv_multi(js, prev=prev, next=nxt)
+                for rep in range(3):
+                    for j in jobs:
+                        j[3].fill_(float("nan"))
+                    g.replay()
+                    side.synchronize()
+                    for (Wd, _, _, y, ws), (acc_ref, y_ref, mag), y0 in zip(jobs, refs, plain):
+                        check(y, None, acc_ref, y_ref, mag, f"recorded {name} B={B} {tag} rep{rep} {Wd.M}x{Wd.K}")
+                        assert torch.equal(y, y0), f"recorded {name} B={B} {tag} rep{rep}"
+                        assert bc.workspace_status(ws) == 0
+            del g
+
+
 def test_host_copy_of_entry_offsets_changes_nothing(bc):
     """With a host copy of tile_off the launch passes each block's first entry offsets by value;
     without it the kernel loads them.  Same results, bit for bit, and both match the oracle."""
