@@ -584,7 +584,8 @@ def run_cuda(args):
                          "bitcos_gemv_multi_host, four calls per step, each: pinned x -> device, launch, y -> pinned host, stream wait"
                          if args.e2e_per_phase else
                          "bitcos_gemv_phases_host, one call per step: one pinned block with all activations -> device, "
-                         "four launches (q+k+v, o, gate+up, down), all outputs -> one pinned block, one stream wait")},
+                         "four launches (q+k+v, o, gate+up, down), all outputs -> one pinned block, one stream wait; "
+                         "the library replays a step it has seen before as a recorded CUDA graph")},
         "gpu_launches": n_launch,
         "timing": {"replays": len(replay_ms), "steps_per_replay": args.steps, "statistic": "median replay",
                    "us_per_step_min": ms_min * 1e3 / args.steps, "us_per_step_max": ms_max * 1e3 / args.steps},
