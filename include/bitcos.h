@@ -337,6 +337,22 @@ int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
  * Errors as bitcos_gemv_multi, plus BITCOS_ERR_NULL / BITCOS_ERR_SHAPE for a malformed list. */
 int bitcos_gemv_multi_chained(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *prev,
                               int n_prev, const bitcos_weights *const *next, int n_next, void *cuda_stream);
+/* How a multi launch would hand its work to thread blocks, without launching anything (needs no
+ * GPU): for tests and for callers who want to see the split.  M, K: the jobs' shapes (host arrays of
+ * n_jobs); multiprocessors: of the device the launch is meant for; busy_multiprocessors: thread
+ * blocks of the launch before it (what bitcos_gemv_multi_chained works out from `prev`), 0 = none.
+ * Work is counted in items: a job's rows are cut into row blocks of 32 and, when a row is too long
+ * for one item, into job_column_blocks[j] column blocks; item i of job j is column block
+ * i % job_column_blocks[j] of chunk i / job_column_blocks[j] (a chunk = job_tiles_per_item[j] tiles'
+ * worth of whole row blocks, or one row block).  Outputs (host): n_blocks; for every block its job,
+ * its first item and its number of items (block_* hold `capacity` entries; ERR_CAPACITY if fewer than
+ * n_blocks); per job the number of items, tiles per item, column blocks, and the chunk stride: 1 = the
+ * block's items are consecutive; s > 1 = after the last column block of a chunk the block moves on
+ * s chunks (blocks take chunks round robin). */
+int bitcos_gemv_multi_plan(const int64_t *M, const int64_t *K, int n_jobs, int batch, int multiprocessors,
+                           int busy_multiprocessors, int capacity, int *block_job, int *block_first_item, int *block_items,
+                           int *job_items, int *job_tiles_per_item, int *job_column_blocks, int *job_chunk_stride,
+                           int *n_blocks);
 /* The same with one activation scale per token and group of 128 (see bitcos_gemv_group_scales):
  * every job's x_scale points to device float [batch][K/128]. */
 int bitcos_gemv_multi_group_scales(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *cuda_stream);

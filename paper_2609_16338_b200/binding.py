@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "bitcos_gemv_host_staging_bytes", "bitcos_gemv_host", "bitcos_gemv_static", "bitcos_decode_probe", "bitcos_gemv_multi",
     "bitcos_gemv_multi_host", "bitcos_quantize_activations", "bitcos_gemv_group_scales",
     "bitcos_choose_format", "bitcos_count_nnz_device", "bitcos_pack_device", "bitcos_gemv_bf16", "bitcos_gemv_multi_bf16",
-    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe", "bitcos_group_pairs_device", "bitcos_gemv_grouped_lists", "bitcos_gemv_multi_chained",
+    "bitcos_gemv_multi_group_scales", "bitcos_gemv_blend_bf16", "bitcos_decode_probe_variant", "bitcos_gemv_phased", "bitcos_gemv_phases_host", "trit5_gemv_grouped", "bit2_gemv_grouped", "bitcos_gemv_static_status", "bitcos_wait_probe", "bitcos_group_pairs_device", "bitcos_gemv_grouped_lists", "bitcos_gemv_multi_chained", "bitcos_gemv_multi_plan",
 ]
 
 
@@ -100,6 +100,9 @@ def load_library():
     L.bitcos_decode_probe.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.bitcos_decode_probe_variant.argtypes = [C.c_int, vp, vp, sz, vp, C.c_int, vp, C.c_int, C.c_int, vp, vp, vp]
     L.bitcos_gemv_multi.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, vp]
+    pi = C.POINTER(C.c_int)
+    L.bitcos_gemv_multi_plan.argtypes = [C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                         pi, pi, pi, pi, pi, pi, pi, pi]
     L.bitcos_gemv_multi_chained.argtypes = [C.POINTER(_Job), C.c_int, C.c_int, C.POINTER(C.c_void_p), C.c_int,
                                             C.POINTER(C.c_void_p), C.c_int, vp]
     L.bitcos_gemv_phased.argtypes = [C.POINTER(_Job), C.POINTER(C.c_int), C.c_int, C.c_int, vp, vp]
@@ -592,6 +595,25 @@ class NextWeights:
     def __init__(self, weights):
         self.keep = list(weights)
         self.arr = (C.c_void_p * len(self.keep))(*[C.addressof(W.desc) for W in self.keep])
+
+
+def bitcos_gemv_multi_plan(shapes, batch=1, multiprocessors=148, busy_multiprocessors=0):
+    """The split of a multi launch over thread blocks (host only): shapes = [(M, K)].  Returns a dict with
+    per-block arrays job / first_item / items and per-job arrays items / tiles_per_item / column_blocks /
+    chunk_stride."""
+    L = load_library()
+    n = len(shapes)
+    M = (C.c_int64 * n)(*[int(s[0]) for s in shapes])
+    K = (C.c_int64 * n)(*[int(s[1]) for s in shapes])
+    cap = 256
+    blk = [(C.c_int * cap)() for _ in range(3)]
+    job = [(C.c_int * n)() for _ in range(4)]
+    nb = C.c_int(0)
+    _check(L.bitcos_gemv_multi_plan(M, K, n, batch, multiprocessors, busy_multiprocessors, cap, *blk, *job, C.byref(nb)),
+           "bitcos_gemv_multi_plan")
+    keys_b, keys_j = ("job", "first_item", "items"), ("items", "tiles_per_item", "column_blocks", "chunk_stride")
+    return {"n_blocks": nb.value, "block": {k: list(a[:nb.value]) for k, a in zip(keys_b, blk)},
+            "per_job": {k: list(a) for k, a in zip(keys_j, job)}}
 
 
 def bitcos_gemv_multi(jobs, next=None, prev=None):

@@ -2441,6 +2441,55 @@ inline void skewed_counts(int64_t items, int n_early, int n_late, int *counts) {
     }
 }
 
+// Whether a launch's blocks are split into early and late ones, and if so the split: block b works on
+// job job_of[b] as that job's block number rank[b] and takes count[b] items from item first[b] of the job
+// (early blocks are dealt to the jobs in proportion to their grids, job after job, then the late ones;
+// inside a job, contiguous ranges of its items, early blocks first).
+inline bool skewed_assignment(MultiArgs &ma, const int *grids, int total, bool two, int sms, int busy_sms, int *first, int *count) {
+    // late starters: only when part of the grid starts early and part late, and every job's items are whole rows
+    const int early = sms - busy_sms;
+    bool skew = busy_sms > 0 && early > 0 && early < total && total <= kMaxGrid && !two;
+    for (int j = 0; j < ma.n; ++j) skew = skew && ma.pl[j].CS == 1 && ma.pl[j].items >= grids[j];
+    if (!skew) return false;
+    int ne[kMaxJobs], given = 0;
+    for (int j = 0; j < ma.n; ++j) {
+        ne[j] = static_cast<int>(static_cast<int64_t>(early) * grids[j] / total);
+        given += ne[j];
+    }
+    for (int j = 0; given < early; j = (j + 1) % ma.n)
+        if (ne[j] < grids[j]) {
+            ++ne[j];
+            ++given;
+        }
+    int b = 0;
+    for (int pass = 0; pass < 2; ++pass)
+        for (int j = 0; j < ma.n; ++j) {
+            const int r0 = pass ? ne[j] : 0, r1 = pass ? grids[j] : ne[j];
+            for (int r = r0; r < r1; ++r, ++b) {
+                ma.job_of[b] = static_cast<uint8_t>(j);
+                ma.rank[b] = static_cast<uint8_t>(r);
+            }
+        }
+    static thread_local int counts[kMaxJobs][kMaxGrid], firsts[kMaxJobs][kMaxGrid];
+    for (int j = 0; j < ma.n; ++j) {
+        ma.nblk[j] = grids[j];
+        ma.pl[j].cyclic = 0;
+        skewed_counts(ma.pl[j].items, ne[j], grids[j] - ne[j], counts[j]);
+        int f = 0;
+        for (int r = 0; r < grids[j]; ++r) {
+            firsts[j][r] = f;
+            f += counts[j][r];
+        }
+    }
+    for (b = 0; b < total; ++b) {
+        first[b] = firsts[ma.job_of[b]][ma.rank[b]];
+        count[b] = counts[ma.job_of[b]][ma.rank[b]];
+    }
+    ma.first_block[ma.n] = total;
+    ma.mapped = 1;
+    return true;
+}
+
 // busy_sms: multiprocessors the caller expects the kernel before this one in the stream to hold on
 // to when this launch's blocks are scheduled (0: unknown or none).
 template <int NB, bool XQ = false, bool XG = false>
@@ -2476,11 +2525,7 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
         if (L.total > smem) smem = L.total;
         if (ma.pl[j].NW > nw) nw = ma.pl[j].NW;
     }
-    // late starters: only when part of the grid starts early and part late, and every job's items are whole rows
-    int early = sms - busy_sms;
-    bool skew = busy_sms > 0 && early > 0 && early < total && total <= kMaxGrid && !two;
-    for (int j = 0; j < ma.n; ++j) skew = skew && ma.pl[j].CS == 1 && ma.pl[j].items >= grids[j];
-    if (!skew) {
+    if (!skewed_assignment(ma, grids, total, two, sms, busy_sms, fo.first, fo.count)) {
         int next = 0;
         for (int j = 0; j < ma.n; ++j) {
             ma.first_block[j] = next;
@@ -2490,43 +2535,8 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
         ma.first_block[ma.n] = next;
         ma.mapped = 0;
     } else {
-        // early blocks are dealt to the jobs in proportion to their grids, job after job, then the late ones
-        int ne[kMaxJobs], given = 0;
-        for (int j = 0; j < ma.n; ++j) {
-            ne[j] = static_cast<int>(static_cast<int64_t>(early) * grids[j] / total);
-            given += ne[j];
-        }
-        for (int j = 0; given < early; j = (j + 1) % ma.n)
-            if (ne[j] < grids[j]) {
-                ++ne[j];
-                ++given;
-            }
-        int b = 0;
-        for (int pass = 0; pass < 2; ++pass)
-            for (int j = 0; j < ma.n; ++j) {
-                const int r0 = pass ? ne[j] : 0, r1 = pass ? grids[j] : ne[j];
-                for (int r = r0; r < r1; ++r, ++b) {
-                    ma.job_of[b] = static_cast<uint8_t>(j);
-                    ma.rank[b] = static_cast<uint8_t>(r);
-                }
-            }
-        // the walks: contiguous ranges of the job's items, early blocks first
-        b = 0;
-        int counts[kMaxJobs][kMaxGrid], firsts[kMaxJobs][kMaxGrid];
-        for (int j = 0; j < ma.n; ++j) {
-            ma.nblk[j] = grids[j];
-            ma.pl[j].cyclic = 0;
-            skewed_counts(ma.pl[j].items, ne[j], grids[j] - ne[j], counts[j]);
-            int first = 0;
-            for (int r = 0; r < grids[j]; ++r) {
-                firsts[j][r] = first;
-                first += counts[j][r];
-            }
-        }
-        for (b = 0; b < total; ++b) {
-            const int j = ma.job_of[b], r = ma.rank[b];
-            fo.first[b] = firsts[j][r];
-            fo.count[b] = counts[j][r];
+        for (int b = 0; b < total; ++b) {
+            const int j = ma.job_of[b];
             fo.lo[b] = fo.hi[b] = 0;
             if (fo.valid && fo.count[b] > 0) {
                 ItemIter it;
@@ -2536,8 +2546,6 @@ int launch_multi(MultiArgs &ma, cudaStream_t stream, const uint32_t *const *off_
                 fo.hi[b] = host_offset(off_host[j], ir.t0 + ir.nt);
             }
         }
-        ma.first_block[ma.n] = total;
-        ma.mapped = 1;
     }
     // every block's first copies, when the entry offsets are known on the host
     static thread_local FirstCopiesTable fc;
@@ -3122,6 +3130,60 @@ void bitcos_debug_timeline(unsigned long long *buf, int slots) {
     g_tl_next = 0;
 }
 #endif
+
+int bitcos_gemv_multi_plan(const int64_t *M, const int64_t *K, int n_jobs, int batch, int multiprocessors,
+                           int busy_multiprocessors, int capacity, int *block_job, int *block_first_item, int *block_items,
+                           int *job_items, int *job_tiles_per_item, int *job_column_blocks, int *job_chunk_stride,
+                           int *n_blocks) {
+    if (!M || !K || !block_job || !block_first_item || !block_items || !job_items || !job_tiles_per_item ||
+        !job_column_blocks || !job_chunk_stride || !n_blocks)
+        return BITCOS_ERR_NULL;
+    if (n_jobs < 1 || n_jobs > kMaxJobs || batch < 1 || batch > BITCOS_MAX_BATCH || multiprocessors < 1 ||
+        multiprocessors > kMaxGrid || busy_multiprocessors < 0)
+        return BITCOS_ERR_SHAPE;
+    static thread_local MultiArgs ma;
+    ma = MultiArgs{};
+    ma.n = n_jobs;
+    int64_t kmax = 0;
+    for (int j = 0; j < n_jobs; ++j) {
+        if (M[j] < 1 || K[j] < kGroup || K[j] % kGroup) return BITCOS_ERR_SHAPE;
+        ma.pl[j] = make_plan(M[j], K[j], decoder_warps(batch));
+        ma.pr[j].M = M[j];
+        ma.pr[j].K = K[j];
+        ma.pr[j].G = static_cast<int>(K[j] / kGroup);
+        ma.pr[j].RB = static_cast<int>(padded_rows(M[j]) / kRows);
+        kmax = K[j] > kmax ? K[j] : kmax;
+    }
+    bool two = false;
+    int grids[kMaxJobs];
+    const int total = plan_multi(ma, nb_bucket(batch, kmax), multiprocessors, &two, grids);
+    if (total > capacity) return BITCOS_ERR_CAPACITY;
+    static thread_local int first[kMaxGrid], count[kMaxGrid];
+    if (skewed_assignment(ma, grids, total, two, multiprocessors, busy_multiprocessors, first, count)) {
+        for (int b = 0; b < total; ++b) {
+            block_job[b] = ma.job_of[b];
+            block_first_item[b] = first[b];
+            block_items[b] = count[b];
+        }
+    } else {
+        int b = 0;
+        for (int j = 0; j < n_jobs; ++j)
+            for (int r = 0; r < grids[j]; ++r, ++b) {
+                const Walk w = make_walk(ma.pl[j], r, grids[j]);
+                block_job[b] = j;
+                block_first_item[b] = w.first;
+                block_items[b] = w.count;
+            }
+    }
+    for (int j = 0; j < n_jobs; ++j) {
+        job_items[j] = static_cast<int>(ma.pl[j].items);
+        job_tiles_per_item[j] = ma.pl[j].NW * ma.pl[j].tpw;
+        job_column_blocks[j] = ma.pl[j].CS;
+        job_chunk_stride[j] = ma.pl[j].cyclic ? grids[j] : 1;
+    }
+    *n_blocks = total;
+    return BITCOS_OK;
+}
 
 int bitcos_gemv_multi_chained(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *prev,
                               int n_prev, const bitcos_weights *const *next, int n_next, void *cuda_stream) {
