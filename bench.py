@@ -561,7 +561,9 @@ def run_cuda(args):
                                  + ("; launches " + ",".join(str(g + 1) for g in args.prefetch_launches)
                                     + " of the step also ask for the NEXT launch's packed weights to be brought into L2"
                                       " (bitcos_gemv_multi_chained): every byte still comes from device memory"
-                                      " once per step" if args.prefetch and args.launch == "multi" else ""))
+                                      " once per step" if args.prefetch and args.launch == "multi" else "")
+                                 + ("; every launch is told which launch runs directly before it (blocks that start late take"
+                                    " fewer work items; results unchanged)" if args.chain_hint and args.launch == "multi" else ""))
                               + "; programmatic dependent launch between consecutive kernels of a stream"),
                    "replicas": world},
         "achieved_gbs": achieved,
