@@ -407,6 +407,44 @@ def test_multi_launch_recorded_into_a_graph(bc, B):
             del g
 
 
+@pytest.mark.parametrize("B", [1, 2])
+def test_single_launches_recorded_into_a_graph(bc, B):
+    """The single-matrix products of all three formats recorded into a CUDA graph, two launches back to back (the
+    second starts under the first): accumulators bit for bit, outputs as the plain launch.  Layer shapes, ragged row counts, rows cut into column blocks (K = 6912, 12288), a single
+    tile, BITCOS with and without the host copy of the entry offsets."""
+    side = torch.cuda.Stream()
+    for (M, K) in ((2560, 2560), (640, 2560), (2560, 6912), (1000, 512), (33, 12288), (32, 128), (70, 384), (4096, 1280)):
+        W, S = datagen.trits(760 + M, M, K, 0.4219), datagen.scales(760 + M, M, K)
+        x, xs = datagen.activations(760 + K + B, B, K)
+        acc_ref, y_ref, mag = oracle.gemv_dense(W, S, x, xs)
+        xd, xsd = dev(x), dev(xs)
+        st = bc.scales_tile(S, M, K)
+        Wb = bc.bitcos_pack(W, S).to_device()
+        cases = [("bitcos", Wb, bc.bitcos_gemv), ("bitcos without host offsets", Wb.without_host_offsets(), bc.bitcos_gemv),
+                 ("trit5", bc.plain_to_device(bc.trit5_pack(W), st, M, K), bc.trit5_gemv),
+                 ("bit2", bc.plain_to_device(bc.bit2_pack(W), st, M, K), bc.bit2_gemv)]
+        ws = bc.make_workspace(M, K)
+        for fmt, Wd, f in cases:
+            y0, _ = f(Wd, xd, xsd, workspace=ws)
+            torch.cuda.synchronize()
+            y = torch.full((B, M), float("nan"), dtype=torch.float32, device="cuda")
+            acc = torch.full((B, M, K // 128), -1, dtype=torch.int32, device="cuda")
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    f(Wd, xd, xsd, y=y, acc_debug=acc, workspace=ws)
+                    f(Wd, xd, xsd, y=y, acc_debug=acc, workspace=ws)      # twice in a row: the second starts under the first
+                for rep in range(2):
+                    y.fill_(float("nan"))
+                    acc.fill_(-1)
+                    g.replay()
+                    side.synchronize()
+                    check(y, acc, acc_ref, y_ref, mag, f"recorded {fmt} {M}x{K} B={B} rep{rep}")
+                    assert torch.equal(y, y0), f"recorded {fmt} {M}x{K} B={B}"
+                    assert bc.workspace_status(ws) == 0
+            del g
+
+
 def test_host_copy_of_entry_offsets_changes_nothing(bc):
     """With a host copy of tile_off the launch passes each block's first entry offsets by value;
     without it the kernel loads them.  Same results, bit for bit, and both match the oracle."""
