@@ -686,7 +686,7 @@ __device__ __forceinline__ void issue_item(const Problem &pb, const View &pr, co
 
 // mbarrier slots inside the `bar` region (8 bytes each)
 constexpr int kBarFull = 0;                       // [stages] stage filled by the copy engine
-constexpr int kBarEmpty = kMaxStages;             // [stages] stage released by all decoder warps
+constexpr int kBarEmpty = kMaxStages;             // [stages] stage released (by the epilogue warp, once all decoder warps have posted the item's sums)
 constexpr int kBarRedFull = 2 * kMaxStages;       // [slots] partial sums of an item written by all decoder warps
 constexpr int kBarRedEmpty = 2 * kMaxStages + 8;  // [slots] partial sums consumed by the epilogue warp
 constexpr int kBarLut = 2 * kMaxStages + 16;      // lookup table arrived
@@ -845,12 +845,12 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
             BITCOS_TL(17, clock64());
         }
         // All 33 barrier slots at once, one per lane (slots of unused stages included): slots
-        // kBarEmpty .. kBarRedFull + 7 count the decoder warps, the others one arrival.  Every
+        // kBarRedFull .. kBarRedFull + 7 count the decoder warps, the others one arrival.  Every
         // barrier is initialised and fenced before the first asynchronous copy is issued.
         static_assert(kBarFull == 0 && kBarEmpty == 8 && kBarRedFull == 16 && kBarRedEmpty == 24 && kBarLut == 32,
                       "one barrier slot per lane, plus the table's");
         if (!(first_sent && lane == kBarFull))
-            mbar_init(bar0 + 8u * static_cast<uint32_t>(lane), (lane >= kBarEmpty && lane < kBarRedEmpty) ? pl.NW : 1);
+            mbar_init(bar0 + 8u * static_cast<uint32_t>(lane), (lane >= kBarRedFull && lane < kBarRedEmpty) ? pl.NW : 1);
         if (lane == 0 && !first_sent) mbar_init(bar0 + 8u * kBarLut, 1);
         if (lane == 1) mbar_init(bar0 + 8u * kBarX, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1093,6 +1093,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
         int n_pend = 0;
         ItemIter it;
         int kk = 0;             // items consumed so far, over all segments
+        int es = 0;             // stage of the item the epilogue looks at next
         constexpr int RS = red_slots(NB);
         // sum of n <= 20 partial sums of token b, spaced NB * 32 floats apart: all loads are issued
         // before the first addition, and the additions always follow the same tree
@@ -1185,6 +1186,10 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
                 if (lane == 0 && pr.status(pb)) *pr.status(pb) = 1u;
                 return;
             }
+            // every decoder warp has posted this item's sums, so none of them reads its stage any more:
+            // one arrival per item hands the stage back to the producer
+            if (lane == 0) mbar_arrive(bar0 + 8u * (kBarEmpty + es));
+            if (++es == pl.stages) es = 0;
             const float *rs = red + slot * red_slot;
             if (pl.CS == 1) {
                 // whole row blocks: one output per row.  The sums are formed first, the slot is
@@ -1610,9 +1615,7 @@ __device__ __forceinline__ void run_segments(const Segs &segs, const Plan &pl_in
                 if (!kMma) rd_lane0[slot * red_slot + (t_off * NB + b) * kRows] = ysum[b];
         }
         }
-        // the stage has been read: hand it back to the producer
-        __syncwarp();
-        mbar_arrive_lane0(full_bar + 8u * kBarEmpty, lane);
+        // (the stage goes back to the producer when the epilogue warp has seen this item's partial sums)
         stage += L.stage_bytes;
         full_bar += 8u;
         if (++s == pl.stages) {
