@@ -181,3 +181,42 @@ def test_recorded_host_step_follows_weights_repacked_in_place(bc):
         d.tile_off_host[:] = p2.tile_off
     torch.cuda.synchronize()
     check("weights repacked in place")
+
+
+def test_host_steps_from_two_threads(bc):
+    """bitcos_gemv_phases_host from two host threads at once, each with its own matrices, blocks and stream (the
+    records of seen steps are shared between threads, recording happens on one stream of the library's own)."""
+    import threading
+    B = 1
+    shapes = [(640, 2560), (96, 1280)]
+    errors = []
+
+    def worker(t):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            Wh = [datagen.trits(4600 + 10 * t + i, M, K, 0.4219) for i, (M, K) in enumerate(shapes)]
+            Sh = [datagen.scales(4600 + 10 * t + i, M, K) for i, (M, K) in enumerate(shapes)]
+            devs = [bc.bitcos_pack(W, S).to_device() for W, S in zip(Wh, Sh)]
+            hp = bc.HostPhases([(d, bc.make_workspace(M, K)) for d, (M, K) in zip(devs, shapes)], [0, 1], batch=B)
+            with torch.cuda.stream(stream):
+                for rep in range(12):
+                    refs = []
+                    for i, (M, K) in enumerate(shapes):
+                        x, xs = datagen.activations(4600 + 100 * t + 7 * rep + i, B, K)
+                        hp.x[i][:] = x
+                        hp.x_scale[i][:] = xs
+                        refs.append(oracle.gemv_dense(Wh[i], Sh[i], x, xs))
+                    ys = hp.run()
+                    for i, (acc_ref, y_ref, mag) in enumerate(refs):
+                        if not (np.abs(ys[i].astype(np.float64) - y_ref) <= REL * mag).all():
+                            errors.append((t, rep, i))
+        except Exception as e:          # noqa: BLE001 (reported to the main thread)
+            errors.append((t, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(2)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors
