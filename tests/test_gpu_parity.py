@@ -445,6 +445,46 @@ def test_single_launches_recorded_into_a_graph(bc, B):
             del g
 
 
+def test_recorded_chained_launches_random(bc):
+    """Sixty random multi launches (one to five jobs of mixed shapes, one to three tokens, random `prev` and `next`
+    lists) recorded into CUDA graphs: every output bit for bit that of the plain single-matrix product, which the
+    other tests hold against the oracle."""
+    rng = np.random.default_rng(7)
+    side = torch.cuda.Stream()
+    pool = {}
+
+    def mat(M, K):
+        if (M, K) not in pool:
+            z = float(rng.choice([0.3, 0.4219, 0.6]))
+            pool[(M, K)] = bc.bitcos_pack(datagen.trits(M * 7 + K, M, K, z), datagen.scales(M + K, M, K)).to_device()
+        return pool[(M, K)]
+
+    Ms, Ks = [32, 33, 640, 1000, 2560, 4000, 6912, 70], [128, 384, 1280, 2560, 5120, 6912]
+    for it in range(60):
+        n, B = int(rng.integers(1, 6)), int(rng.choice([1, 2, 3]))
+        jobs, plain = [], []
+        for _ in range(n):
+            Wd = mat(int(rng.choice(Ms)), int(rng.choice(Ks)))
+            x, xs = datagen.activations(it * 10 + Wd.M + Wd.K, B, Wd.K)
+            xd, xsd, ws = dev(x), dev(xs), bc.make_workspace(Wd.M, Wd.K)
+            y0, _ = bc.bitcos_gemv(Wd, xd, xsd, workspace=ws)
+            jobs.append((Wd, xd, xsd, torch.full((B, Wd.M), float("nan"), dtype=torch.float32, device="cuda"), ws))
+            plain.append(y0)
+        torch.cuda.synchronize()
+        prev = [mat(int(rng.choice(Ms)), int(rng.choice(Ks))) for _ in range(int(rng.integers(0, 4)))] or None
+        nxt = [mat(int(rng.choice(Ms)), int(rng.choice(Ks))) for _ in range(int(rng.integers(0, 4)))] or None
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                bc.bitcos_gemv_multi(jobs, prev=prev, next=nxt)
+            g.replay()
+            side.synchronize()
+        for (Wd, _, _, y, ws), y0 in zip(jobs, plain):
+            assert torch.equal(y, y0), (it, [(j[0].M, j[0].K) for j in jobs], B)
+            assert bc.workspace_status(ws) == 0
+        del g
+
+
 def test_host_copy_of_entry_offsets_changes_nothing(bc):
     """With a host copy of tile_off the launch passes each block's first entry offsets by value;
     without it the kernel loads them.  Same results, bit for bit, and both match the oracle."""
