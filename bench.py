@@ -972,18 +972,24 @@ def qwen32b_layer_detail(bc, torch, stream, z=0.4711):
         multi = [[bc.MultiJobs([(rep[j], xs_dev[j][0], xs_dev[j][1], ys[j], wss[j]) for j in g]) for g in groups]
                  for rep in replicas]
 
-        def step(i):
-            for mj in multi[i]:
-                bc.bitcos_gemv_multi(mj)
+        # every launch is told which launch runs before it and which matrices the next one reads (as in the headline)
+        prevs = [bc.NextWeights([base[j] for j in groups[gi - 1]]) for gi in range(len(groups))]
+        nexts = [[bc.NextWeights([replicas[(c + (gi + 1) // len(groups)) % len(replicas)][j] for j in groups[(gi + 1) % len(groups)]])
+                  for gi in range(len(groups))] for c in range(len(replicas))]
+
+        def step(i, hints=True):
+            for gi, mj in enumerate(multi[i]):
+                bc.bitcos_gemv_multi(mj, prev=prevs[gi] if hints else None, next=nexts[i][gi] if hints else None)
 
         step(1)
         torch.cuda.synchronize()
         for i, (nm, M, K) in enumerate(shapes):
             assert_matches_oracle(ys[i], dense[i][0], dense[i][1], xs_host[i][0], xs_host[i][1], f"qwen layer {nm} B={B}")
         us = graph_time_us(torch, stream, step, len(replicas), launches=8)
+        us_plain = graph_time_us(torch, stream, lambda i: step(i, False), len(replicas), launches=8)
         nbytes = sum(algorithmic_bytes(M, K, h.nnz, B) for (_, M, K), h in zip(shapes, host))
         out.append({"batch": B, "us_per_step": us, "us_per_token": us / B, "gbs": nbytes / us / 1e3,
-                    "frac": nbytes / us / 1e3 / peak, "bytes": int(nbytes)})
+                    "frac": nbytes / us / 1e3 / peak, "bytes": int(nbytes), "us_per_step_without_hints": us_plain})
     return out
 
 

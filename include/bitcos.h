@@ -324,7 +324,9 @@ int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
  *                  are under way.  Nothing waits for the requests and nothing is written.  The sign
  *                  vector of a matrix is only requested if its descriptor carries tile_off_host (its
  *                  length is not known otherwise).  Pays when launches are short: the later launch
- *                  starts from L2 instead of device memory.
+ *                  starts from L2 instead of device memory.  A request for more than
+ *                  BITCOS_PREFETCH_MAX_BYTES in total is ignored (it would only compete with the
+ *                  launch's own reads).
  *   prev, n_prev   the matrices of the launch directly BEFORE this one in the stream (only M and K
  *                  are read; n_prev <= BITCOS_MAX_JOBS, may be 0 = unknown), same batch.  Kernels of
  *                  this library start before their predecessor has finished (see "stream ordering"),
@@ -335,6 +337,7 @@ int bitcos_gemv_multi(const bitcos_gemv_job *jobs, int n_jobs, int batch, void *
  *                  (K <= 2560 at up to eight tokens), where the split cannot touch any sum.  A wrong
  *                  hint costs time (an uneven split), never correctness.
  * Errors as bitcos_gemv_multi, plus BITCOS_ERR_NULL / BITCOS_ERR_SHAPE for a malformed list. */
+#define BITCOS_PREFETCH_MAX_BYTES (8u << 20)
 int bitcos_gemv_multi_chained(const bitcos_gemv_job *jobs, int n_jobs, int batch, const bitcos_weights *const *prev,
                               int n_prev, const bitcos_weights *const *next, int n_next, void *cuda_stream);
 /* How a multi launch would hand its work to thread blocks, without launching anything (needs no
